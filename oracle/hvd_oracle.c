@@ -1,0 +1,358 @@
+/*
+ * CPU oracle for the per-step path of Hybrid Verified Decoding.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition of what
+ * the CUDA library must compute.  It shares no code, header, table or helper
+ * with the CUDA path, and the CUDA path never calls it.  Only the tests, the
+ * smoke check and the benchmark's CPU-baseline leg load it.
+ *
+ * Every function works on host pointers.  Requests are independent; the
+ * batch entry points may spread requests over `nthreads` POSIX threads (a
+ * plain parallel-for over b, nothing else is parallel).
+ *
+ * What is pinned by the CPU tests (brute-force enumeration on tiny inputs,
+ * constructed cases, invariants, library special cases):
+ *   - longest suffix match length, its count and the draft      (Sec. 3.2)
+ *   - MLP score closed forms and the >= rule                    (Sec. 3.3, 3.4)
+ *   - first-maximum argmax, accepted length, committed block    (Sec. 3.1, label eq. of Sec. 3.3)
+ * Parity unpinned by the paper (the paper is silent; self-consistency only):
+ *   - most-recent-occurrence tie-break among equally long matches,
+ *   - the exact formulas of the eight payoff features (the paper names only
+ *     feature groups, App. B table "Payoff predictor feature groups"),
+ *   - the layout of the recent-history summary h.
+ */
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef struct {
+    uint32_t sel_bits; /* bit j = 1 if the cache draft was selected j steps ago */
+    uint32_t pad;
+    uint64_t acc_ring; /* byte j = accepted length j steps ago */
+} oracle_req_state;
+
+enum { ORACLE_REQ_OK = 0, ORACLE_REQ_CAPACITY = 1, ORACLE_REQ_BAD_LEN = 2 };
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+enum { ORACLE_N_FEATURES = 8 };
+
+/* ------------------------------------------------------------------ */
+/* parallel-for over requests                                          */
+/* ------------------------------------------------------------------ */
+typedef void (*req_fn)(int32_t b, void* arg);
+typedef struct {
+    req_fn fn;
+    void* arg;
+    int32_t B, tid, nthreads;
+} worker_t;
+
+static void* worker_main(void* p) {
+    worker_t* w = (worker_t*)p;
+    for (int32_t b = w->tid; b < w->B; b += w->nthreads) w->fn(b, w->arg);
+    return NULL;
+}
+
+static void for_each_request(int32_t B, int32_t nthreads, req_fn fn, void* arg) {
+    if (nthreads > B) nthreads = B;
+    if (nthreads <= 1) {
+        for (int32_t b = 0; b < B; ++b) fn(b, arg);
+        return;
+    }
+    pthread_t* th = (pthread_t*)malloc(sizeof(pthread_t) * (size_t)nthreads);
+    worker_t* ws = (worker_t*)malloc(sizeof(worker_t) * (size_t)nthreads);
+    for (int32_t t = 0; t < nthreads; ++t) {
+        ws[t].fn = fn; ws[t].arg = arg; ws[t].B = B; ws[t].tid = t; ws[t].nthreads = nthreads;
+        pthread_create(&th[t], NULL, worker_main, &ws[t]);
+    }
+    for (int32_t t = 0; t < nthreads; ++t) pthread_join(th[t], NULL);
+    free(ws);
+    free(th);
+}
+
+/* ------------------------------------------------------------------ */
+/* Step 1: cache draft = continuation of the longest suffix match      */
+/* (Sec. 3.2; suffix-cache limits from the "Drafting configuration"    */
+/* table: depth l_max, draft cap K, speculative factor and offset).    */
+/* ------------------------------------------------------------------ */
+void oracle_lookup_one(const int32_t* h, int32_t n, int32_t K, int32_t k_cap, int32_t l_max,
+                       int32_t min_match, float spec_factor, float spec_offset,
+                       int32_t* draft /*[k_cap]*/, int32_t* draft_len, int32_t* match_len,
+                       int32_t* match_pos, int32_t* match_cnt) {
+    int32_t best_L = 0, best_e = -1, cnt = 0;
+    if (K < 0) K = 0;
+    if (K > k_cap) K = k_cap;
+    /* e = index of the first continuation token of a candidate occurrence.
+       e = n would be the suffix matching itself and is left out. */
+    for (int32_t e = 1; e <= n - 1; ++e) {
+        int32_t l = 0;
+        while (l < l_max && l < e && h[e - 1 - l] == h[n - 1 - l]) ++l;
+        if (l > best_L) {
+            best_L = l; best_e = e; cnt = 1;
+        } else if (l == best_L && l > 0) {
+            best_e = e; /* the latest occurrence wins among equals */
+            ++cnt;
+        }
+    }
+    for (int32_t j = 0; j < k_cap; ++j) draft[j] = -1;
+    if (best_L < min_match || best_L == 0) {
+        *match_len = 0; *match_pos = -1; *match_cnt = 0; *draft_len = 0;
+        return;
+    }
+    int32_t cap = K;
+    if (spec_factor > 0.0f) {
+        float prod = spec_factor * (float)best_L; /* two roundings: multiply, then add */
+        float lim = prod + spec_offset;
+        cap = (int32_t)floorf(lim);
+        if (cap < 0) cap = 0;
+    }
+    int32_t d = K;
+    if (cap < d) d = cap;
+    if (n - best_e < d) d = n - best_e;
+    for (int32_t j = 0; j < d; ++j) draft[j] = h[best_e + j];
+    *match_len = best_L; *match_pos = best_e; *match_cnt = cnt; *draft_len = d;
+}
+
+typedef struct {
+    const int32_t* hist; const int64_t* hist_off; const int32_t* hist_cap; const int32_t* hist_len;
+    const int32_t* K; int32_t k_cap, l_max, min_match; float spec_factor, spec_offset;
+    int32_t *draft, *draft_len, *match_len, *match_pos, *match_cnt;
+} lookup_args;
+
+static void lookup_req(int32_t b, void* p) {
+    lookup_args* a = (lookup_args*)p;
+    int32_t n = a->hist_len[b];
+    if (n < 0 || n > a->hist_cap[b]) n = 0; /* unusable length: behaves as an empty history */
+    oracle_lookup_one(a->hist + a->hist_off[b], n, a->K[b], a->k_cap, a->l_max, a->min_match,
+                      a->spec_factor, a->spec_offset, a->draft + (int64_t)b * a->k_cap,
+                      a->draft_len + b, a->match_len + b, a->match_pos + b, a->match_cnt + b);
+}
+
+void oracle_lookup(int32_t B, const int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                   const int32_t* hist_len, const int32_t* K, int32_t k_cap, int32_t l_max,
+                   int32_t min_match, float spec_factor, float spec_offset, int32_t* draft,
+                   int32_t* draft_len, int32_t* match_len, int32_t* match_pos, int32_t* match_cnt,
+                   int32_t nthreads) {
+    lookup_args a = {hist, hist_off, hist_cap, hist_len, K, k_cap, l_max, min_match, spec_factor,
+                     spec_offset, draft, draft_len, match_len, match_pos, match_cnt};
+    for_each_request(B, nthreads, lookup_req, &a);
+}
+
+/* ------------------------------------------------------------------ */
+/* Step 2: payoff features (Sec. 3.3; App. B feature-group table).     */
+/* Every operation is an exact integer->float conversion or a single   */
+/* correctly rounded IEEE operation.                                   */
+/* ------------------------------------------------------------------ */
+static int32_t bit_width_u32(uint32_t x) {
+    int32_t w = 0;
+    while (x) { ++w; x >>= 1; }
+    return w;
+}
+
+void oracle_features_one(int32_t n, int32_t prompt_len, oracle_req_state st, int32_t draft_len,
+                         int32_t match_len, int32_t match_pos, int32_t match_cnt, float* phi /*[8]*/) {
+    if (n < 0) n = 0;
+    if (prompt_len < 0) prompt_len = 0;
+    if (match_cnt < 0) match_cnt = 0;
+    /* cache match group */
+    phi[0] = (float)match_len;
+    phi[1] = (float)draft_len;
+    phi[2] = (float)bit_width_u32((uint32_t)match_cnt);
+    phi[3] = (match_pos < 0 || n == 0) ? 0.0f : (float)(n - match_pos) / (float)n;
+    /* decode state group */
+    phi[4] = (float)bit_width_u32((uint32_t)prompt_len);
+    phi[5] = (n == 0) ? 0.0f : (float)(n - prompt_len) / (float)n;
+    /* recent history group: last 8 steps */
+    int32_t sel_count = 0;
+    for (int j = 0; j < 8; ++j) sel_count += (int32_t)((st.sel_bits >> j) & 1u);
+    phi[6] = (float)sel_count / 8.0f;
+    int32_t acc_sum = 0;
+    for (int j = 0; j < 8; ++j) acc_sum += (int32_t)((st.acc_ring >> (8 * j)) & 0xFFu);
+    phi[7] = (float)acc_sum / 8.0f;
+}
+
+/* ------------------------------------------------------------------ */
+/* Step 3: payoff score y = g_theta(phi) and the rule y >= tau          */
+/* (Sec. 3.3 predictor; Sec. 3.4 selection equation; Algorithm 1).     */
+/* One hidden ReLU layer; fp32 with a fixed left-to-right fused         */
+/* multiply-add chain, plus an fp64 evaluation of the same network.    */
+/* ------------------------------------------------------------------ */
+float oracle_mlp_f32(const float* phi, int32_t F, int32_t H, const float* W1 /*[H,F]*/,
+                     const float* b1, const float* W2, float b2) {
+    float y = b2;
+    for (int32_t j = 0; j < H; ++j) {
+        float acc = b1[j];
+        for (int32_t i = 0; i < F; ++i) acc = fmaf(W1[(int64_t)j * F + i], phi[i], acc);
+        float hid = acc > 0.0f ? acc : 0.0f;
+        y = fmaf(W2[j], hid, y);
+    }
+    return y;
+}
+
+double oracle_mlp_f64(const float* phi, int32_t F, int32_t H, const float* W1, const float* b1,
+                      const float* W2, float b2) {
+    double y = (double)b2;
+    for (int32_t j = 0; j < H; ++j) {
+        double acc = (double)b1[j];
+        for (int32_t i = 0; i < F; ++i) acc += (double)W1[(int64_t)j * F + i] * (double)phi[i];
+        double hid = acc > 0.0 ? acc : 0.0;
+        y += (double)W2[j] * hid;
+    }
+    return y;
+}
+
+typedef struct {
+    const int32_t *hist_len, *prompt_len; const oracle_req_state* state; const int32_t* K;
+    const int32_t *draft, *draft_len, *match_len, *match_pos, *match_cnt;
+    const int32_t *model_draft, *model_len; int32_t k_cap, H;
+    const float *W1, *b1, *W2; float b2, tau;
+    float *features, *score; double* score64; int32_t *select, *sel_draft, *sel_len;
+} score_args;
+
+static void score_req(int32_t b, void* p) {
+    score_args* a = (score_args*)p;
+    float phi[ORACLE_N_FEATURES];
+    int32_t kc = a->k_cap;
+    int32_t K = a->K[b];
+    if (K < 0) K = 0;
+    if (K > kc) K = kc;
+    int32_t d = a->draft_len[b];
+    if (d < 0) d = 0;
+    if (d > kc) d = kc;
+    oracle_features_one(a->hist_len[b], a->prompt_len[b], a->state[b], d, a->match_len[b],
+                        a->match_pos[b], a->match_cnt[b], phi);
+    if (a->features) memcpy(a->features + (int64_t)b * ORACLE_N_FEATURES, phi, sizeof(phi));
+    float y = oracle_mlp_f32(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->W2, a->b2);
+    a->score[b] = y;
+    if (a->score64) a->score64[b] = oracle_mlp_f64(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->W2, a->b2);
+    /* cache draft is verified iff it exists and its predicted payoff reaches the threshold */
+    int32_t sel = (d > 0 && y >= a->tau) ? 1 : 0;
+    a->select[b] = sel;
+    int32_t* out = a->sel_draft + (int64_t)b * kc;
+    for (int32_t j = 0; j < kc; ++j) out[j] = -1;
+    if (sel) {
+        for (int32_t j = 0; j < d; ++j) out[j] = a->draft[(int64_t)b * kc + j];
+        a->sel_len[b] = d;
+    } else {
+        int32_t m = 0;
+        if (a->model_draft && a->model_len) {
+            m = a->model_len[b];
+            if (m < 0) m = 0;
+            if (m > K) m = K;
+            for (int32_t j = 0; j < m; ++j) out[j] = a->model_draft[(int64_t)b * kc + j];
+        }
+        a->sel_len[b] = m;
+    }
+}
+
+void oracle_score_select(int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
+                         const oracle_req_state* state, const int32_t* K, const int32_t* draft,
+                         const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
+                         const int32_t* match_cnt, const int32_t* model_draft, const int32_t* model_len,
+                         int32_t k_cap, int32_t H, const float* W1, const float* b1, const float* W2,
+                         float b2, float tau, float* features, float* score, double* score64,
+                         int32_t* select, int32_t* sel_draft, int32_t* sel_len, int32_t nthreads) {
+    score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
+                    model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
+                    select, sel_draft, sel_len};
+    for_each_request(B, nthreads, score_req, &a);
+}
+
+/* ------------------------------------------------------------------ */
+/* Step 4: greedy verification and commit (Sec. 3.1 Verify; Sec. 3.4;  */
+/* Algorithm 1 verify/append/update lines; accepted length = the label */
+/* equation of Sec. 3.3).                                              */
+/* ------------------------------------------------------------------ */
+static float widen_bf16(uint16_t u) {
+    uint32_t bits = (uint32_t)u << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+/* index of the first maximum: scan ascending, replace only on strictly greater */
+int32_t oracle_argmax_row(const void* row, int32_t dtype, int64_t V) {
+    int64_t best = 0;
+    if (dtype == ORACLE_BF16) {
+        const uint16_t* r = (const uint16_t*)row;
+        float bv = widen_bf16(r[0]);
+        for (int64_t v = 1; v < V; ++v) {
+            float x = widen_bf16(r[v]);
+            if (x > bv) { bv = x; best = v; }
+        }
+    } else {
+        const float* r = (const float*)row;
+        float bv = r[0];
+        for (int64_t v = 1; v < V; ++v) {
+            if (r[v] > bv) { bv = r[v]; best = v; }
+        }
+    }
+    return (int32_t)best;
+}
+
+typedef struct {
+    const void* logits; int32_t dtype; int64_t V; const int64_t* row_off; int32_t k_uniform;
+    const int32_t *sel_draft, *sel_len, *select; int32_t k_cap;
+    int32_t* hist; const int64_t* hist_off; const int32_t* hist_cap; int32_t* hist_len;
+    oracle_req_state* state;
+    int32_t *accepted, *committed, *n_commit, *target_tok, *status;
+} verify_args;
+
+static void verify_req(int32_t b, void* p) {
+    verify_args* a = (verify_args*)p;
+    int32_t kc = a->k_cap;
+    int64_t r0 = a->row_off ? a->row_off[b] : (int64_t)b * (a->k_uniform + 1);
+    int64_t r1 = a->row_off ? a->row_off[b + 1] : r0 + (a->k_uniform + 1);
+    int64_t rows = r1 - r0;
+    size_t elt = a->dtype == ORACLE_BF16 ? 2 : 4;
+    int32_t* z = a->committed + (int64_t)b * (kc + 1);
+    for (int32_t j = 0; j <= kc; ++j) z[j] = -1;
+    if (a->target_tok)
+        for (int64_t i = 0; i < rows; ++i) a->target_tok[r0 + i] = -1;
+    int32_t n = a->hist_len[b];
+    if (n < 0 || n > a->hist_cap[b] || rows <= 0) {
+        a->status[b] = ORACLE_REQ_BAD_LEN; a->accepted[b] = 0; a->n_commit[b] = 0;
+        return;
+    }
+    int32_t m = a->sel_len[b];
+    if (m < 0) m = 0;
+    if (m > kc) m = kc;
+    if (m > rows - 1) m = (int32_t)(rows - 1);
+    int32_t t[65 + 1];
+    for (int32_t i = 0; i <= m; ++i) {
+        const char* row = (const char*)a->logits + (size_t)(r0 + i) * (size_t)a->V * elt;
+        t[i] = oracle_argmax_row(row, a->dtype, a->V);
+        if (a->target_tok) a->target_tok[r0 + i] = t[i];
+    }
+    const int32_t* d = a->sel_draft + (int64_t)b * kc;
+    int32_t acc = 0;
+    while (acc < m && d[acc] == t[acc]) ++acc;
+    for (int32_t j = 0; j < acc; ++j) z[j] = d[j];
+    z[acc] = t[acc]; /* the target's own token after the accepted prefix: always committed */
+    int32_t room = a->hist_cap[b] - n;
+    int32_t w = acc + 1;
+    int32_t st = ORACLE_REQ_OK;
+    if (w > room) { w = room; st = ORACLE_REQ_CAPACITY; }
+    int32_t* h = a->hist + a->hist_off[b];
+    for (int32_t j = 0; j < w; ++j) h[n + j] = z[j];
+    a->hist_len[b] = n + w;
+    a->n_commit[b] = w;
+    a->accepted[b] = acc;
+    a->status[b] = st;
+    oracle_req_state s = a->state[b];
+    s.sel_bits = (s.sel_bits << 1) | (uint32_t)(a->select[b] ? 1 : 0);
+    s.acc_ring = (s.acc_ring << 8) | (uint64_t)(uint8_t)acc;
+    a->state[b] = s;
+}
+
+void oracle_verify_commit(int32_t B, const void* logits, int32_t dtype, int64_t V,
+                          const int64_t* row_off, int32_t k_uniform, const int32_t* sel_draft,
+                          const int32_t* sel_len, const int32_t* select, int32_t k_cap, int32_t* hist,
+                          const int64_t* hist_off, const int32_t* hist_cap, int32_t* hist_len,
+                          oracle_req_state* state, int32_t* accepted, int32_t* committed,
+                          int32_t* n_commit, int32_t* target_tok, int32_t* status, int32_t nthreads) {
+    verify_args a = {logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, select, k_cap, hist,
+                     hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, target_tok,
+                     status};
+    for_each_request(B, nthreads, verify_req, &a);
+}

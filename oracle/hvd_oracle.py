@@ -1,0 +1,179 @@
+"""ctypes front end of the CPU oracle (test infrastructure only).
+
+Loads ``libhvd_oracle.so`` built from ``hvd_oracle.c`` and exposes the three
+steps on numpy arrays.  Nothing here is imported by the CUDA package; only the
+tests, the smoke check and the benchmark's CPU-baseline leg use it.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "hvd_oracle.c")
+_LIB = os.path.join(_HERE, "libhvd_oracle.so")
+
+F32, BF16 = 0, 1
+REQ_OK, REQ_CAPACITY, REQ_BAD_LEN = 0, 1, 2
+N_FEATURES = 8
+
+STATE_DTYPE = np.dtype([("sel_bits", "<u4"), ("pad", "<u4"), ("acc_ring", "<u8")])
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc; contraction off so every fp32 step rounds as written."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fPIC", "-shared", "-pthread",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.oracle_argmax_row.restype = C.c_int32
+        _lib.oracle_mlp_f32.restype = C.c_float
+        _lib.oracle_mlp_f64.restype = C.c_double
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+@dataclass
+class LookupOut:
+    draft: np.ndarray
+    draft_len: np.ndarray
+    match_len: np.ndarray
+    match_pos: np.ndarray
+    match_cnt: np.ndarray
+
+
+def lookup(hist, hist_off, hist_cap, hist_len, K, *, k_cap, l_max=64, min_match=2,
+           spec_factor=1.0, spec_offset=0.0, nthreads=1) -> LookupOut:
+    B = len(hist_len)
+    hist = _i32(hist); hist_len = _i32(hist_len); hist_cap = _i32(hist_cap); K = _i32(K)
+    hist_off = np.ascontiguousarray(hist_off, dtype=np.int64)
+    out = LookupOut(np.empty((B, k_cap), np.int32), np.empty(B, np.int32), np.empty(B, np.int32),
+                    np.empty(B, np.int32), np.empty(B, np.int32))
+    lib().oracle_lookup(C.c_int32(B), _p(hist), _p(hist_off), _p(hist_cap), _p(hist_len), _p(K),
+                        C.c_int32(k_cap), C.c_int32(l_max), C.c_int32(min_match),
+                        C.c_float(spec_factor), C.c_float(spec_offset), _p(out.draft),
+                        _p(out.draft_len), _p(out.match_len), _p(out.match_pos), _p(out.match_cnt),
+                        C.c_int32(nthreads))
+    return out
+
+
+@dataclass
+class ScoreOut:
+    features: np.ndarray
+    score: np.ndarray
+    score64: np.ndarray
+    select: np.ndarray
+    sel_draft: np.ndarray
+    sel_len: np.ndarray
+
+
+def score_select(hist_len, prompt_len, state, K, lk: LookupOut, model_draft, model_len, *, k_cap,
+                 W1, b1, W2, b2, tau, nthreads=1) -> ScoreOut:
+    B = len(hist_len)
+    H = int(np.asarray(W2).shape[0])
+    W1 = np.ascontiguousarray(W1, np.float32); b1 = np.ascontiguousarray(b1, np.float32)
+    W2 = np.ascontiguousarray(W2, np.float32)
+    assert W1.shape == (H, N_FEATURES)
+    state = np.ascontiguousarray(state, dtype=STATE_DTYPE)
+    hist_len = _i32(hist_len); prompt_len = _i32(prompt_len); K = _i32(K)
+    md = None if model_draft is None else _i32(model_draft)
+    ml = None if model_len is None else _i32(model_len)
+    out = ScoreOut(np.empty((B, N_FEATURES), np.float32), np.empty(B, np.float32),
+                   np.empty(B, np.float64), np.empty(B, np.int32), np.empty((B, k_cap), np.int32),
+                   np.empty(B, np.int32))
+    lib().oracle_score_select(C.c_int32(B), _p(hist_len), _p(prompt_len), _p(state), _p(K),
+                              _p(_i32(lk.draft)), _p(_i32(lk.draft_len)), _p(_i32(lk.match_len)),
+                              _p(_i32(lk.match_pos)), _p(_i32(lk.match_cnt)), _p(md), _p(ml),
+                              C.c_int32(k_cap), C.c_int32(H), _p(W1), _p(b1), _p(W2), C.c_float(b2),
+                              C.c_float(tau), _p(out.features), _p(out.score), _p(out.score64),
+                              _p(out.select), _p(out.sel_draft), _p(out.sel_len), C.c_int32(nthreads))
+    return out
+
+
+@dataclass
+class VerifyOut:
+    accepted: np.ndarray
+    committed: np.ndarray
+    n_commit: np.ndarray
+    target_tok: np.ndarray
+    status: np.ndarray
+
+
+def verify_commit(logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, select, *, k_cap, hist,
+                  hist_off, hist_cap, hist_len, state, nthreads=1) -> VerifyOut:
+    """`hist`, `hist_len` and `state` are updated IN PLACE (they must be writable, contiguous
+    int32 / int32 / STATE_DTYPE arrays).  `logits` is a contiguous float32 array (dtype F32) or a
+    uint16 array of bfloat16 bit patterns (dtype BF16), rows of V."""
+    B = len(hist_len)
+    assert hist.dtype == np.int32 and hist.flags.c_contiguous and hist.flags.writeable
+    assert hist_len.dtype == np.int32 and hist_len.flags.c_contiguous
+    assert state.dtype == STATE_DTYPE and state.flags.c_contiguous
+    assert logits.flags.c_contiguous
+    assert logits.dtype == (np.float32 if dtype == F32 else np.uint16)
+    hist_off = np.ascontiguousarray(hist_off, dtype=np.int64)
+    hist_cap = _i32(hist_cap)
+    if row_off is not None:
+        row_off = np.ascontiguousarray(row_off, dtype=np.int64)
+        total_rows = int(row_off[B])
+    else:
+        total_rows = B * (k_uniform + 1)
+    assert logits.size >= total_rows * V
+    out = VerifyOut(np.empty(B, np.int32), np.empty((B, k_cap + 1), np.int32), np.empty(B, np.int32),
+                    np.empty(total_rows, np.int32), np.empty(B, np.int32))
+    lib().oracle_verify_commit(C.c_int32(B), _p(logits), C.c_int32(dtype), C.c_int64(V), _p(row_off),
+                               C.c_int32(k_uniform), _p(_i32(sel_draft)), _p(_i32(sel_len)),
+                               _p(_i32(select)), C.c_int32(k_cap), _p(hist), _p(hist_off),
+                               _p(hist_cap), _p(hist_len), _p(state), _p(out.accepted),
+                               _p(out.committed), _p(out.n_commit), _p(out.target_tok),
+                               _p(out.status), C.c_int32(nthreads))
+    return out
+
+
+def argmax_row(row: np.ndarray, dtype: int) -> int:
+    row = np.ascontiguousarray(row)
+    return int(lib().oracle_argmax_row(_p(row), C.c_int32(dtype), C.c_int64(row.size)))
+
+
+def mlp_f32(phi, W1, b1, W2, b2) -> float:
+    phi = np.ascontiguousarray(phi, np.float32); W1 = np.ascontiguousarray(W1, np.float32)
+    b1 = np.ascontiguousarray(b1, np.float32); W2 = np.ascontiguousarray(W2, np.float32)
+    return float(lib().oracle_mlp_f32(_p(phi), C.c_int32(phi.size), C.c_int32(W2.size), _p(W1), _p(b1),
+                                      _p(W2), C.c_float(b2)))
+
+
+def mlp_f64(phi, W1, b1, W2, b2) -> float:
+    phi = np.ascontiguousarray(phi, np.float32); W1 = np.ascontiguousarray(W1, np.float32)
+    b1 = np.ascontiguousarray(b1, np.float32); W2 = np.ascontiguousarray(W2, np.float32)
+    return float(lib().oracle_mlp_f64(_p(phi), C.c_int32(phi.size), C.c_int32(W2.size), _p(W1), _p(b1),
+                                      _p(W2), C.c_float(b2)))
+
+
+def features_one(n, prompt_len, sel_bits, acc_ring, draft_len, match_len, match_pos, match_cnt):
+    class St(C.Structure):
+        _fields_ = [("sel_bits", C.c_uint32), ("pad", C.c_uint32), ("acc_ring", C.c_uint64)]
+    phi = np.empty(N_FEATURES, np.float32)
+    lib().oracle_features_one(C.c_int32(n), C.c_int32(prompt_len), St(sel_bits, 0, acc_ring),
+                              C.c_int32(draft_len), C.c_int32(match_len), C.c_int32(match_pos),
+                              C.c_int32(match_cnt), _p(phi))
+    return phi
