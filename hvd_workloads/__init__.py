@@ -251,23 +251,6 @@ def make_requests(w: Workload) -> Requests:
                 h[n - T:n] = h[e0 - T:e0]
         hists.append(h)
     cap = (n_all + 4 * (K_all + 1)).astype(np.int64)
-    # layout: [guard][slab, start aligned to 32 words = 128 B][guard] ...
-    off = np.empty(B, np.int64)
-    p = 0
-    for b in range(B):
-        p += GUARD_WORDS
-        p = (p + 31) // 32 * 32
-        off[b] = p
-        p += int(cap[b])
-    p += GUARD_WORDS
-    total = (p + 31) // 32 * 32
-    hist = np.full(total, GUARD_VALUE, np.int32)
-    guard = np.ones(total, bool)
-    for b in range(B):
-        o, c, n = int(off[b]), int(cap[b]), int(n_all[b])
-        hist[o:o + c] = FREE_VALUE
-        hist[o:o + n] = hists[b]
-        guard[o:o + c] = False
     u = r_state.uniform(0.25, 0.9, B)
     prompt_len = np.floor(n_all * u).astype(np.int32)
     state = np.zeros(B, STATE_DTYPE)
@@ -279,11 +262,42 @@ def make_requests(w: Workload) -> Requests:
     model_draft = np.full((B, w.k_cap), -1, np.int32)
     for b in range(B):
         model_draft[b, :int(K_all[b])] = r_model.integers(0, w.V, int(K_all[b]))
-    model_len = K_all.astype(np.int32)
+    return pack_requests(hists, K_all, cap, prompt_len, state, model_draft, K_all.astype(np.int32))
+
+
+def pack_requests(hists, K, cap, prompt_len, state, model_draft, model_len, hist_len=None,
+                  misalign=None) -> Requests:
+    """Lays token lists out as guarded slabs: [64 canary words][slab, start aligned to 128 bytes]...
+    `hist_len` may override the true lengths (to build invalid requests); `misalign[b]` shifts slab
+    b by that many words off the 128-byte boundary."""
+    B = len(hists)
+    K = np.asarray(K, np.int64)
+    cap = np.asarray(cap, np.int64)
+    off = np.empty(B, np.int64)
+    p = 0
+    for b in range(B):
+        p += GUARD_WORDS
+        p = (p + 31) // 32 * 32
+        if misalign is not None:
+            p += int(misalign[b])
+        off[b] = p
+        p += int(cap[b])
+    p += GUARD_WORDS
+    total = (p + 31) // 32 * 32
+    hist = np.full(total, GUARD_VALUE, np.int32)
+    guard = np.ones(total, bool)
+    for b in range(B):
+        o, c, n = int(off[b]), int(cap[b]), len(hists[b])
+        hist[o:o + c] = FREE_VALUE
+        hist[o:o + n] = hists[b]
+        guard[o:o + c] = False
     row_off = np.zeros(B + 1, np.int64)
-    row_off[1:] = np.cumsum(K_all + 1)
-    return Requests(hist, off, cap.astype(np.int32), n_all.astype(np.int32), K_all.astype(np.int32),
-                    prompt_len, state, model_draft, model_len, row_off, guard)
+    row_off[1:] = np.cumsum(K + 1)
+    n_all = np.asarray([len(h) for h in hists], np.int32) if hist_len is None else np.asarray(hist_len, np.int32)
+    return Requests(hist, off, cap.astype(np.int32), n_all, K.astype(np.int32),
+                    np.asarray(prompt_len, np.int32), np.ascontiguousarray(state, STATE_DTYPE),
+                    np.ascontiguousarray(model_draft, np.int32), np.asarray(model_len, np.int32),
+                    row_off, guard)
 
 
 def make_predictor(w: Workload):

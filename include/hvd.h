@@ -1,0 +1,180 @@
+/*
+ * hvd.h -- C ABI of the B200 (sm_100a) library for the per-step path of
+ * Hybrid Verified Decoding: cache-draft lookup, payoff scoring and draft
+ * selection, greedy verification and commit.
+ *
+ * One decoding cycle (Algorithm 1 of the paper) maps to three calls:
+ *
+ *     d_c          <- D_C(x; C)                      hvd_lookup
+ *     phi, y       <- Phi(x, d_c, C, h), g_theta     hvd_score_select
+ *     d            <- d_c if y >= tau else D_m(x)    hvd_score_select
+ *     (target forward on x || d: the caller's job, gives the logits)
+ *     a, z         <- Verify(x, d; M)                hvd_verify_commit
+ *     x <- x || z, update C and h                    hvd_verify_commit
+ *
+ * Conventions
+ *  - Unless an argument is marked HOST, every pointer is a DEVICE pointer owned
+ *    by the caller.  The library never frees caller memory and keeps no
+ *    reference to it after the call returns.
+ *  - Device entry points only enqueue work on `stream` (a cudaStream_t passed
+ *    as void*, NULL = default stream) and never synchronise.
+ *  - Errors the host can see (NULL pointer, sizes outside the limits given at
+ *    hvd_create, unknown dtype, misaligned base pointer) are returned at once
+ *    and nothing is enqueued.  Data-dependent problems are reported per
+ *    request in `status[b]` by the device; nothing is ever written out of
+ *    bounds and no kernel traps or waits on another.
+ *  - A context belongs to one device.  Calls on one context must not overlap
+ *    on the GPU (they share the context's scratch memory): use one stream per
+ *    context, or one context per concurrent stream.
+ *  - Token histories are ragged: request b owns the slab
+ *    hist[hist_off[b] .. hist_off[b] + hist_cap[b]) of which the first
+ *    hist_len[b] tokens are valid (prompt followed by committed tokens).
+ */
+#ifndef HVD_H
+#define HVD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define HVD_API __attribute__((visibility("default")))
+#else
+#define HVD_API
+#endif
+
+typedef struct hvd_ctx hvd_ctx;
+
+typedef enum {
+    HVD_OK = 0,
+    HVD_ERR_INVALID_ARG = 1,
+    HVD_ERR_CUDA = 2,
+    HVD_ERR_UNSUPPORTED = 3,
+    HVD_ERR_ALLOC = 4
+} hvd_status;
+
+typedef enum { HVD_F32 = 0, HVD_BF16 = 1 } hvd_dtype;
+
+/* written per request, on the device, by hvd_verify_commit */
+typedef enum {
+    HVD_REQ_OK = 0,
+    HVD_REQ_CAPACITY = 1, /* slab too small: commit clamped to the free space */
+    HVD_REQ_BAD_LEN = 2   /* hist_len outside [0, hist_cap] or no logits rows: request skipped */
+} hvd_req_status;
+
+/* Recent-history summary h of one request (Sec. 3.3; Algorithm 1 "update C and h").
+   bit j of sel_bits = 1 if the cache draft was verified j steps ago;
+   byte j of acc_ring = accepted length j steps ago. */
+typedef struct {
+    uint32_t sel_bits;
+    uint32_t pad;
+    uint64_t acc_ring;
+} hvd_req_state;
+
+enum { HVD_N_FEATURES = 8, HVD_MAX_K = 64, HVD_MAX_L = 64, HVD_MAX_HIDDEN = 256 };
+
+typedef struct {
+    int32_t max_batch;    /* largest B of any call, 1..8192 */
+    int32_t k_cap;        /* row length of every draft array, 1..64 (suffix cache "maximum draft tokens") */
+    int32_t l_max;        /* longest suffix match looked for, 1..64 (suffix cache "maximum tree depth") */
+    int32_t min_match;    /* shorter matches count as no match, >= 1 */
+    float spec_factor;    /* draft_len <= floor(spec_factor*match_len + spec_offset); <= 0 disables the limit */
+    float spec_offset;    /* ("maximum speculative factor / offset" of the suffix cache: 1.0 / 0.0) */
+    int32_t hidden;       /* hidden units of the payoff MLP, 1..256 */
+    int32_t max_hist_len; /* largest hist_len of any request */
+    int64_t max_rows;     /* largest total number of logits rows of any call */
+    int64_t max_vocab;    /* largest V of any call */
+} hvd_config;
+
+/* Creates a context on the current CUDA device and allocates its scratch
+   memory (a few MB; sized from cfg).  *out is NULL on failure. */
+HVD_API hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg);
+HVD_API hvd_status hvd_destroy(hvd_ctx* ctx);
+HVD_API const char* hvd_status_string(hvd_status s);
+/* text of the last error recorded on this context ("" if none) */
+HVD_API const char* hvd_last_error(const hvd_ctx* ctx);
+
+/* Payoff predictor g_theta (Sec. 3.3): y = b2 + sum_j W2[j] * relu(b1[j] + sum_i W1[j][i] * phi[i]),
+   fp32, accumulated left to right with fused multiply-adds, and the threshold tau of Sec. 3.4.
+   W1 [hidden, 8] row-major, b1 [hidden], W2 [hidden]: HOST pointers, copied before returning. */
+HVD_API hvd_status hvd_set_predictor(hvd_ctx* ctx, const float* W1, const float* b1, const float* W2,
+                             float b2, float tau, void* stream);
+
+/*
+ * Cache-based drafting D_C (Sec. 3.2), with the request's own history as the cache.
+ * For every request: among the positions e in [1, n-1], find the longest l <= l_max such that
+ * hist[e-l .. e) equals the last l tokens hist[n-l .. n)  (n = hist_len[b]; e = n, the suffix
+ * itself, is left out; occurrences may overlap the suffix).
+ *   match_len[b] = that l (0 if it is shorter than min_match)
+ *   match_pos[b] = the largest e reaching it (-1 if none): the most recent occurrence
+ *   match_cnt[b] = how many e reach it (lengths are capped at l_max before counting)
+ *   draft[b, 0..d) = hist[e .. e+d),  d = draft_len[b] = min(K[b], floor(spec_factor*l + spec_offset), n - e);
+ *   draft[b, d..k_cap) = -1
+ * K[b] is clamped to [0, k_cap].  A request whose hist_len is outside [0, min(hist_cap, n_max)]
+ * is treated as an empty history (no match).
+ *
+ * hist      int32, 16-byte aligned base; slabs should start on 16-byte boundaries (any start works)
+ * hist_off  int64 [B], hist_cap int32 [B], hist_len int32 [B], K int32 [B]
+ * n_max     HOST value: upper bound on hist_len[b] of this call (sizes the launch), <= max_hist_len
+ * outputs   draft int32 [B, k_cap]; draft_len, match_len, match_pos, match_cnt int32 [B]
+ */
+HVD_API hvd_status hvd_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                      const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
+                      int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
+                      int32_t* match_pos, int32_t* match_cnt, void* stream);
+
+/*
+ * Payoff features Phi, predictor g_theta and the selection rule (Sec. 3.3, Sec. 3.4, App. B):
+ *   phi0 = match_len, phi1 = draft_len, phi2 = bit_width(match_cnt),
+ *   phi3 = (n - match_pos) / n (0 without a match),
+ *   phi4 = bit_width(prompt_len), phi5 = (n - prompt_len) / n (0 for n = 0),
+ *   phi6 = popcount(sel_bits & 0xFF) / 8, phi7 = (sum of the 8 bytes of acc_ring) / 8,
+ *   score = g_theta(phi);   select = 1 (verify the cache draft) iff draft_len > 0 and score >= tau,
+ *   sel_draft/sel_len = the cache draft if select, else the first min(model_len, K) model tokens.
+ * model_draft [B, k_cap] / model_len [B] may both be NULL (no model drafter: empty draft).
+ * features [B, 8] may be NULL.  Outputs: score fp32 [B], select int32 [B], sel_draft int32
+ * [B, k_cap] (-1 beyond sel_len), sel_len int32 [B].  Needs hvd_set_predictor first.
+ */
+HVD_API hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
+                            const int32_t* prompt_len, const hvd_req_state* state, const int32_t* K,
+                            const int32_t* draft, const int32_t* draft_len, const int32_t* match_len,
+                            const int32_t* match_pos, const int32_t* match_cnt,
+                            const int32_t* model_draft, const int32_t* model_len, float* features,
+                            float* score, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
+                            void* stream);
+
+/*
+ * Greedy verification and commit (Sec. 3.1 Verify; Sec. 3.4; Algorithm 1; the accepted length is
+ * the label equation of Sec. 3.3).  Request b owns logits rows [r0, r1): r0 = row_off[b],
+ * r1 = row_off[b+1], or r0 = b*(k_uniform+1), r1 = r0 + k_uniform + 1 when row_off is NULL.  Row r
+ * holds V values of `dtype`, densely packed at logits + r*V.  Row r0+i is the target model's
+ * output after the prefix extended by the first i draft tokens.  With m = min(sel_len[b], r1-r0-1):
+ *   t_i = argmax of row r0+i, i = 0..m   (lowest index among equal maxima; -0.0 equals +0.0; the
+ *         logits must not contain NaN)
+ *   a   = largest l <= m with sel_draft[b, j] == t_j for all j < l         -> accepted[b]
+ *   z   = sel_draft[b, 0..a) followed by t_a  (always a+1 tokens)          -> committed[b, 0..a], -1 after
+ *   the first w = min(a+1, hist_cap - n) tokens of z are appended to the history,
+ *   hist_len[b] += w, n_commit[b] = w, status[b] = HVD_REQ_CAPACITY if w < a+1;
+ *   state[b].sel_bits = sel_bits << 1 | select[b];  state[b].acc_ring = acc_ring << 8 | a.
+ * Rows beyond m are not read.  target_tok (may be NULL) receives t_i for the rows read, -1 for
+ * the others.
+ *
+ * logits     16-byte aligned base recommended (any alignment of the element type works)
+ * total_rows HOST value: number of rows in `logits` (= row_off[B]); <= max_rows
+ * in/out     hist, hist_len [B], state [B];   outputs accepted, n_commit, status int32 [B],
+ *            committed int32 [B, k_cap+1], target_tok int32 [total_rows] or NULL
+ */
+HVD_API hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                             const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                             const int32_t* sel_draft, const int32_t* sel_len, const int32_t* select,
+                             int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                             int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                             int32_t* committed, int32_t* n_commit, int32_t* target_tok,
+                             int32_t* status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HVD_H */

@@ -58,9 +58,10 @@ def verify_commit(w, rq, sc, logits_np, nthreads=1):
                            hist_len=rq.hist_len, state=rq.state, nthreads=nthreads)
 
 
-def prepare(w: W.Workload, device="cpu", nthreads=None, salt: int = 0) -> Inputs:
+def prepare(w: W.Workload, device="cpu", nthreads=None, salt: int = 0, rq: W.Requests = None) -> Inputs:
+    """Seeded inputs for one step.  `rq` replaces the generated requests (hand-built edge cases)."""
     nthreads = nthreads or host_threads()
-    rq = W.make_requests(w)
+    rq = W.make_requests(w) if rq is None else rq
     W1, b1, W2, b2, tau = W.make_predictor(w)
     lk = lookup(w, rq, nthreads)
     sc = score_select(w, rq, lk, W1, b1, W2, b2, tau, nthreads)
@@ -68,7 +69,7 @@ def prepare(w: W.Workload, device="cpu", nthreads=None, salt: int = 0) -> Inputs
         tau = W.calibrate_tau(sc.score, lk.draft_len > 0, w.calibrate_cache_frac)
         sc = score_select(w, rq, lk, W1, b1, W2, b2, tau, nthreads)
     A = W.make_agreement(w, sc.sel_len)
-    logits = W.make_logits(w, int(rq.row_off[-1]), device=device, salt=salt)
+    logits = W.make_logits(w, max(int(rq.row_off[-1]), 1), device=device, salt=salt)
     strict = W.plant_agreement(w, logits, rq.row_off, sc.sel_draft, sc.sel_len, A, salt=salt)
     return Inputs(w, rq, W1, b1, W2, b2, tau, A, strict, logits, W.logits_to_numpy(logits))
 

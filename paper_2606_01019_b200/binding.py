@@ -1,0 +1,149 @@
+"""ctypes binding of the C ABI declared in ``include/hvd.h``: same names, marshalling only.
+
+Tensors are torch CUDA tensors (device memory and streams are all torch is used for); each method
+passes raw device pointers and the current CUDA stream to the library.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+REQ_OK, REQ_CAPACITY, REQ_BAD_LEN = 0, 1, 2
+N_FEATURES = 8
+STATE_DTYPE = np.dtype([("sel_bits", "<u4"), ("pad", "<u4"), ("acc_ring", "<u8")])
+
+_vp, _i32, _i64, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+
+
+class HvdError(RuntimeError):
+    pass
+
+
+class HvdConfig(C.Structure):
+    _fields_ = [("max_batch", _i32), ("k_cap", _i32), ("l_max", _i32), ("min_match", _i32),
+                ("spec_factor", _f32), ("spec_offset", _f32), ("hidden", _i32),
+                ("max_hist_len", _i32), ("max_rows", _i64), ("max_vocab", _i64)]
+
+
+_SIGNATURES = {
+    "hvd_create": (_i32, [C.POINTER(_vp), C.POINTER(HvdConfig)]),
+    "hvd_destroy": (_i32, [_vp]),
+    "hvd_status_string": (C.c_char_p, [_i32]),
+    "hvd_last_error": (C.c_char_p, [_vp]),
+    "hvd_set_predictor": (_i32, [_vp, _vp, _vp, _vp, _f32, _f32, _vp]),
+    "hvd_lookup": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
+    "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
+}
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def exported_symbols():
+    return sorted(_SIGNATURES)
+
+
+def load_library(build: bool = True):
+    """Loads (building first if the sources are newer) the shared library.  Fails loudly if it
+    cannot be built or loaded: there is no other implementation to fall back to."""
+    global _lib
+    if _lib is None:
+        if build:
+            _build.build()
+        if not os.path.exists(_build.LIB):
+            raise HvdError(f"{_build.LIB} is missing: run paper_2606_01019_b200/build.py")
+        lib = C.CDLL(_build.LIB)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream():
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Context:
+    """One library context on the current CUDA device (see ``hvd_create``)."""
+
+    def __init__(self, *, max_batch, k_cap, max_hist_len, max_rows, max_vocab, l_max=64, min_match=2,
+                 spec_factor=1.0, spec_offset=0.0, hidden=32):
+        import torch
+        if not torch.cuda.is_available():
+            raise HvdError("no CUDA device: the HVD path runs only in its sm_100a kernels")
+        self._lib = load_library()
+        self.cfg = HvdConfig(max_batch, k_cap, l_max, min_match, spec_factor, spec_offset, hidden,
+                             max_hist_len, max_rows, max_vocab)
+        self._h = _vp()
+        st = self._lib.hvd_create(C.byref(self._h), C.byref(self.cfg))
+        if st != 0:
+            raise HvdError(f"hvd_create: {self._lib.hvd_status_string(st).decode()}")
+        self.k_cap = k_cap
+        self.hidden = hidden
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.hvd_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st, what):
+        if st != 0:
+            raise HvdError(f"{what}: {self._lib.hvd_status_string(st).decode()}: "
+                           f"{self._lib.hvd_last_error(self._h).decode()}")
+
+    def hvd_set_predictor(self, W1, b1, W2, b2, tau):
+        W1 = np.ascontiguousarray(W1, np.float32); b1 = np.ascontiguousarray(b1, np.float32)
+        W2 = np.ascontiguousarray(W2, np.float32)
+        if W1.shape != (self.hidden, N_FEATURES) or b1.shape != (self.hidden,) or W2.shape != (self.hidden,):
+            raise HvdError("hvd_set_predictor: weight shapes do not match the context")
+        self._check(self._lib.hvd_set_predictor(self._h, W1.ctypes.data, b1.ctypes.data, W2.ctypes.data,
+                                                float(b2), float(tau), _stream()), "hvd_set_predictor")
+
+    def hvd_lookup(self, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len, match_len,
+                   match_pos, match_cnt):
+        self._check(self._lib.hvd_lookup(self._h, B, _ptr(hist), _ptr(hist_off), _ptr(hist_cap),
+                                         _ptr(hist_len), _ptr(K), n_max, _ptr(draft), _ptr(draft_len),
+                                         _ptr(match_len), _ptr(match_pos), _ptr(match_cnt), _stream()),
+                    "hvd_lookup")
+
+    def hvd_score_select(self, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
+                         match_cnt, model_draft, model_len, features, score, select, sel_draft, sel_len):
+        self._check(self._lib.hvd_score_select(self._h, B, _ptr(hist_len), _ptr(prompt_len), _ptr(state),
+                                               _ptr(K), _ptr(draft), _ptr(draft_len), _ptr(match_len),
+                                               _ptr(match_pos), _ptr(match_cnt), _ptr(model_draft),
+                                               _ptr(model_len), _ptr(features), _ptr(score), _ptr(select),
+                                               _ptr(sel_draft), _ptr(sel_len), _stream()),
+                    "hvd_score_select")
+
+    def hvd_verify_commit(self, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
+                          select, hist, hist_off, hist_cap, hist_len, state, accepted, committed,
+                          n_commit, target_tok, status):
+        self._check(self._lib.hvd_verify_commit(self._h, B, _ptr(logits), dtype, V, _ptr(row_off),
+                                                k_uniform, total_rows, _ptr(sel_draft), _ptr(sel_len),
+                                                _ptr(select), _ptr(hist), _ptr(hist_off), _ptr(hist_cap),
+                                                _ptr(hist_len), _ptr(state), _ptr(accepted),
+                                                _ptr(committed), _ptr(n_commit), _ptr(target_tok),
+                                                _ptr(status), _stream()),
+                    "hvd_verify_commit")

@@ -1,0 +1,193 @@
+// C ABI of the library: context management, argument checks, kernel launches.
+#include <new>
+
+#include "hvd_internal.cuh"
+
+using namespace hvd;
+
+namespace {
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+void release(hvd_ctx* c) {
+    if (!c) return;
+    cudaFree(c->d_W1); cudaFree(c->d_b1); cudaFree(c->d_W2);
+    cudaFree(c->lk_partial); cudaFree(c->lk_cnt);
+    cudaFree(c->vf_partial); cudaFree(c->vf_cnt); cudaFree(c->vf_ctrl);
+    delete c;
+}
+
+template <typename P>
+cudaError_t alloc_zero(P** p, size_t bytes) {
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes);
+    if (e != cudaSuccess) return e;
+    return cudaMemset(*p, 0, bytes);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* hvd_status_string(hvd_status s) {
+    switch (s) {
+        case HVD_OK: return "HVD_OK";
+        case HVD_ERR_INVALID_ARG: return "HVD_ERR_INVALID_ARG";
+        case HVD_ERR_CUDA: return "HVD_ERR_CUDA";
+        case HVD_ERR_UNSUPPORTED: return "HVD_ERR_UNSUPPORTED";
+        case HVD_ERR_ALLOC: return "HVD_ERR_ALLOC";
+    }
+    return "HVD_ERR_UNKNOWN";
+}
+
+const char* hvd_last_error(const hvd_ctx* ctx) { return ctx ? ctx->last_error : ""; }
+
+hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
+    if (!out) return HVD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!cfg) return HVD_ERR_INVALID_ARG;
+    if (cfg->max_batch < 1 || cfg->max_batch > 8192) return HVD_ERR_INVALID_ARG;
+    if (cfg->k_cap < 1 || cfg->k_cap > HVD_MAX_K) return HVD_ERR_INVALID_ARG;
+    if (cfg->l_max < 1 || cfg->l_max > HVD_MAX_L) return HVD_ERR_INVALID_ARG;
+    if (cfg->min_match < 1) return HVD_ERR_INVALID_ARG;
+    if (cfg->hidden < 1 || cfg->hidden > HVD_MAX_HIDDEN) return HVD_ERR_INVALID_ARG;
+    if (cfg->max_hist_len < 1) return HVD_ERR_INVALID_ARG;
+    if (cfg->max_rows < 1 || cfg->max_vocab < 1 || cfg->max_vocab > 0x7fffffffLL) return HVD_ERR_INVALID_ARG;
+    if (!(cfg->spec_factor == cfg->spec_factor) || !(cfg->spec_offset == cfg->spec_offset)) return HVD_ERR_INVALID_ARG;
+
+    hvd_ctx* c = new (std::nothrow) hvd_ctx();
+    if (!c) return HVD_ERR_ALLOC;
+    c->cfg = *cfg;
+    c->last_error[0] = 0;
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (e != cudaSuccess) { delete c; return HVD_ERR_CUDA; }
+
+    c->lk_max_chunks = (int)(((int64_t)cfg->max_hist_len + 3 + kLookupMinChunk - 1) / kLookupMinChunk);
+    // work items per row for the narrowest element (4 bytes): an upper bound for every dtype
+    c->vf_max_seg = (cfg->max_vocab * 4 / 16 + kVerifyVecPerItem - 1) / kVerifyVecPerItem;
+    if (c->vf_max_seg < 1) c->vf_max_seg = 1;
+    if (cfg->max_rows * c->vf_max_seg >= 0x7fffffffLL) { delete c; return HVD_ERR_INVALID_ARG; }
+
+    const size_t H = (size_t)cfg->hidden;
+    bool ok = true;
+    ok = ok && alloc_zero(&c->d_W1, H * HVD_N_FEATURES * sizeof(float)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->d_b1, H * sizeof(float)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->d_W2, H * sizeof(float)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->lk_partial, (size_t)cfg->max_batch * c->lk_max_chunks * sizeof(LookupPartial)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->lk_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->vf_partial, (size_t)cfg->max_rows * c->vf_max_seg * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->vf_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->vf_ctrl, sizeof(Ctrl)) == cudaSuccess;
+    if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) { (void)cudaGetLastError(); release(c); return HVD_ERR_ALLOC; }
+
+    const size_t smem = verify_dyn_smem(cfg->max_batch);
+    c->vf_blocks_per_sm[0] = verify_occupancy(HVD_F32, smem);
+    c->vf_blocks_per_sm[1] = verify_occupancy(HVD_BF16, smem);
+    if (c->vf_blocks_per_sm[0] < 1 || c->vf_blocks_per_sm[1] < 1) { release(c); return HVD_ERR_UNSUPPORTED; }
+    c->has_predictor = false;
+    *out = c;
+    return HVD_OK;
+}
+
+hvd_status hvd_destroy(hvd_ctx* ctx) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    release(ctx);
+    return HVD_OK;
+}
+
+hvd_status hvd_set_predictor(hvd_ctx* ctx, const float* W1, const float* b1, const float* W2,
+                             float b2, float tau, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (!W1 || !b1 || !W2) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_predictor: NULL weights");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t H = (size_t)ctx->cfg.hidden;
+    HVD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_W1, W1, H * HVD_N_FEATURES * sizeof(float), cudaMemcpyHostToDevice, st));
+    HVD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_b1, b1, H * sizeof(float), cudaMemcpyHostToDevice, st));
+    HVD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_W2, W2, H * sizeof(float), cudaMemcpyHostToDevice, st));
+    HVD_CUDA_TRY(ctx, cudaStreamSynchronize(st));  // the host arrays may be reused as soon as we return
+    ctx->b2 = b2;
+    ctx->tau = tau;
+    ctx->has_predictor = true;
+    return HVD_OK;
+}
+
+hvd_status hvd_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                      const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
+                      int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
+                      int32_t* match_pos, int32_t* match_cnt, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: B outside [1, max_batch]");
+    if (!hist || !hist_off || !hist_cap || !hist_len || !K || !draft || !draft_len || !match_len ||
+        !match_pos || !match_cnt)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: NULL pointer");
+    if (!aligned(hist, 16)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: hist must be 16-byte aligned");
+    if (n_max < 0 || n_max > ctx->cfg.max_hist_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max outside [0, max_hist_len]");
+    return launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
+                         match_len, match_pos, match_cnt, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
+                            const int32_t* prompt_len, const hvd_req_state* state, const int32_t* K,
+                            const int32_t* draft, const int32_t* draft_len, const int32_t* match_len,
+                            const int32_t* match_pos, const int32_t* match_cnt,
+                            const int32_t* model_draft, const int32_t* model_len, float* features,
+                            float* score, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
+                            void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select: B outside [1, max_batch]");
+    if (!ctx->has_predictor) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select: call hvd_set_predictor first");
+    if (!hist_len || !prompt_len || !state || !K || !draft || !draft_len || !match_len || !match_pos ||
+        !match_cnt || !score || !select || !sel_draft || !sel_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select: NULL pointer");
+    if ((model_draft == nullptr) != (model_len == nullptr))
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select: model_draft and model_len go together");
+    if (!aligned(state, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select: state must be 8-byte aligned");
+    return launch_score_select(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len,
+                               match_pos, match_cnt, model_draft, model_len, features, score, select,
+                               sel_draft, sel_len, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                             const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                             const int32_t* sel_draft, const int32_t* sel_len, const int32_t* select,
+                             int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                             int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                             int32_t* committed, int32_t* n_commit, int32_t* target_tok,
+                             int32_t* status, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: B outside [1, max_batch]");
+    if (dtype != HVD_F32 && dtype != HVD_BF16) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: unknown dtype");
+    if (V < 1 || V > ctx->cfg.max_vocab) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: V outside [1, max_vocab]");
+    if (!logits || !sel_draft || !sel_len || !select || !hist || !hist_off || !hist_cap || !hist_len ||
+        !state || !accepted || !committed || !n_commit || !status)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: NULL pointer");
+    const size_t esz = dtype == HVD_F32 ? 4 : 2;
+    if (!aligned(logits, esz)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: logits not aligned to its element type");
+    if (!aligned(state, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: state must be 8-byte aligned");
+    if (!row_off) {
+        if (k_uniform < 0 || k_uniform > ctx->cfg.k_cap)
+            return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: k_uniform outside [0, k_cap]");
+        if (total_rows != (int64_t)B * (k_uniform + 1))
+            return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: total_rows != B*(k_uniform+1)");
+    }
+    if (total_rows < 1 || total_rows > ctx->cfg.max_rows)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: total_rows outside [1, max_rows]");
+
+    VerifyArgs a;
+    a.B = B; a.logits = logits; a.V = V; a.row_off = row_off; a.k_uniform = k_uniform;
+    a.sel_draft = sel_draft; a.sel_len = sel_len; a.select = select;
+    a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.state = state;
+    a.accepted = accepted; a.committed = committed; a.n_commit = n_commit; a.target_tok = target_tok;
+    a.status = status; a.k_cap = ctx->cfg.k_cap;
+    a.partial = ctx->vf_partial; a.req_cnt = ctx->vf_cnt; a.ctrl = ctx->vf_ctrl;
+    const int64_t vec_per_row = V * (int64_t)esz / 16;
+    int64_t n_seg = (vec_per_row + kVerifyVecPerItem - 1) / kVerifyVecPerItem;
+    if (n_seg < 1) n_seg = 1;
+    if (n_seg > ctx->vf_max_seg) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: V exceeds the scratch sized at create");
+    a.n_seg = (int32_t)n_seg;
+    return launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

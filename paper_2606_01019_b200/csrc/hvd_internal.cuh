@@ -1,0 +1,119 @@
+// Internal declarations shared by the translation units of the CUDA library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "hvd.h"
+
+namespace hvd {
+
+// One partial result of the history scan: best match seen by one chunk of one request.
+struct LookupPartial {
+    unsigned long long key;  // (match length << 32) | position of the first continuation token
+    uint32_t cnt;            // positions in the chunk reaching that length
+    uint32_t pad;
+};
+
+constexpr int kLookupThreads = 256;
+constexpr int kLookupTokPerVec = 4;
+constexpr int kLookupMinChunk = kLookupThreads * kLookupTokPerVec;  // tokens, one 128-bit load per thread
+
+constexpr int kVerifyThreads = 256;
+constexpr int kVerifyUnroll = 8;                                   // 128-bit loads in flight per thread
+constexpr int kVerifyVecPerItem = kVerifyThreads * kVerifyUnroll;  // 32 KB of logits per work item
+
+struct Ctrl {
+    uint32_t next_item;      // dynamic work counter of the verify kernel (zero at rest)
+    uint32_t blocks_exited;  // blocks that left the verify work loop (zero at rest)
+};
+
+}  // namespace hvd
+
+struct hvd_ctx {
+    hvd_config cfg;
+    int device;
+    int num_sms;
+    // predictor
+    float* d_W1;
+    float* d_b1;
+    float* d_W2;
+    float b2, tau;
+    bool has_predictor;
+    // lookup scratch
+    hvd::LookupPartial* lk_partial;  // [max_batch, lk_max_chunks]
+    uint32_t* lk_cnt;                // [max_batch], zero at rest
+    int lk_max_chunks;
+    // verify scratch
+    unsigned long long* vf_partial;  // [max_rows, vf_max_seg]
+    uint32_t* vf_cnt;                // [max_batch], zero at rest
+    hvd::Ctrl* vf_ctrl;              // zero at rest
+    int64_t vf_max_seg;
+    int vf_blocks_per_sm[2];         // per dtype
+    char last_error[256];
+};
+
+namespace hvd {
+
+inline hvd_status fail(hvd_ctx* ctx, hvd_status s, const char* msg) {
+    if (ctx) snprintf(ctx->last_error, sizeof(ctx->last_error), "%s", msg);
+    return s;
+}
+
+inline hvd_status cuda_fail(hvd_ctx* ctx, cudaError_t e, const char* where) {
+    if (ctx) snprintf(ctx->last_error, sizeof(ctx->last_error), "%s: %s", where, cudaGetErrorString(e));
+    return HVD_ERR_CUDA;
+}
+
+#define HVD_CUDA_TRY(ctx, call)                                          \
+    do {                                                                 \
+        cudaError_t e_ = (call);                                         \
+        if (e_ != cudaSuccess) return hvd::cuda_fail((ctx), e_, #call);  \
+    } while (0)
+
+hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                         const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
+                         int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
+                         int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream);
+
+hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
+                               const int32_t* prompt_len, const hvd_req_state* state, const int32_t* K,
+                               const int32_t* draft, const int32_t* draft_len, const int32_t* match_len,
+                               const int32_t* match_pos, const int32_t* match_cnt,
+                               const int32_t* model_draft, const int32_t* model_len, float* features,
+                               float* score, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
+                               cudaStream_t stream);
+
+struct VerifyArgs {
+    int32_t B;
+    const void* logits;
+    int64_t V;
+    const int64_t* row_off;
+    int32_t k_uniform;
+    const int32_t* sel_draft;
+    const int32_t* sel_len;
+    const int32_t* select;
+    int32_t* hist;
+    const int64_t* hist_off;
+    const int32_t* hist_cap;
+    int32_t* hist_len;
+    hvd_req_state* state;
+    int32_t* accepted;
+    int32_t* committed;
+    int32_t* n_commit;
+    int32_t* target_tok;
+    int32_t* status;
+    int32_t k_cap;
+    // scratch
+    unsigned long long* partial;
+    uint32_t* req_cnt;
+    Ctrl* ctrl;
+    int32_t n_seg;  // work items per row
+};
+
+hvd_status launch_verify(hvd_ctx* ctx, const VerifyArgs& a, hvd_dtype dtype, cudaStream_t stream);
+int verify_occupancy(hvd_dtype dtype, size_t dyn_smem);
+size_t verify_dyn_smem(int32_t B);
+
+}  // namespace hvd

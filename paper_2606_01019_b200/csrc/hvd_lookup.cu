@@ -1,0 +1,254 @@
+// Cache-draft lookup (Sec. 3.2): longest match of the history's own suffix inside the history.
+//
+// The history of a request is cut into chunks; one CTA scans one chunk with 128-bit loads, looking
+// for the last token of the history.  Every hit is a candidate end position; the warp that found it
+// extends the match backwards cooperatively (one compared token per lane, ballot + find-first-set
+// gives the match length).  Each CTA leaves one partial (best length, latest position, count) in
+// the context's scratch; the CTA that arrives last for a request combines the partials, applies the
+// minimum-length and draft-length rules and copies the draft.  No CTA waits for another.
+#include "hvd_internal.cuh"
+
+namespace hvd {
+namespace {
+
+struct LookupArgs {
+    const int32_t* hist;
+    const int64_t* hist_off;
+    const int32_t* hist_cap;
+    const int32_t* hist_len;
+    const int32_t* K;
+    int32_t n_max;
+    int32_t* draft;
+    int32_t* draft_len;
+    int32_t* match_len;
+    int32_t* match_pos;
+    int32_t* match_cnt;
+    LookupPartial* partial;
+    uint32_t* req_cnt;
+    int32_t max_chunks;
+    int32_t k_cap, l_max, min_match;
+    float spec_factor, spec_offset;
+};
+
+struct Best {
+    unsigned long long key;  // (L << 32) | e ; 0 = nothing found
+    uint32_t cnt;
+};
+
+__device__ __forceinline__ Best combine(Best a, Best b) {
+    const uint32_t la = (uint32_t)(a.key >> 32), lb = (uint32_t)(b.key >> 32);
+    if (la > lb) return a;
+    if (lb > la) return b;
+    Best r;
+    r.key = a.key > b.key ? a.key : b.key;
+    r.cnt = a.cnt + b.cnt;
+    return r;
+}
+
+__device__ __forceinline__ Best warp_combine(Best v) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        Best o;
+        o.key = __shfl_xor_sync(0xffffffffu, v.key, off);
+        o.cnt = __shfl_xor_sync(0xffffffffu, v.cnt, off);
+        v = combine(v, o);
+    }
+    return v;
+}
+
+__device__ __forceinline__ int4 ld_hist(const int4* p) {
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+template <int ITER>
+__global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs a) {
+    const int b = blockIdx.y;
+    const int chunk = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+
+    int n = a.hist_len[b];
+    if (n < 0 || n > a.hist_cap[b] || n > a.n_max) n = 0;  // unusable length: empty history
+    const int32_t* __restrict__ slab = a.hist + a.hist_off[b];
+    // 128-bit loads run on the 16-byte grid; `mis` tokens of the first vector lie before the slab
+    const int mis = (int)((reinterpret_cast<uintptr_t>(slab) >> 2) & 3);
+    constexpr int CHUNK = kLookupMinChunk * ITER;  // tokens of the aligned grid per CTA
+    // candidate positions p (index of the matched copy's last token) are 0 .. n-2
+    const int g_end = (n >= 2) ? (n - 1 + mis) : 0;  // exclusive end on the aligned grid
+    const int n_chunks = (g_end + CHUNK - 1) / CHUNK;
+
+    if (n_chunks == 0) {
+        if (chunk == 0 && warp == 0) {
+            for (int j = lane; j < a.k_cap; j += 32) a.draft[(int64_t)b * a.k_cap + j] = -1;
+            if (lane == 0) {
+                a.draft_len[b] = 0; a.match_len[b] = 0; a.match_pos[b] = -1; a.match_cnt[b] = 0;
+            }
+        }
+        return;
+    }
+    if (chunk >= n_chunks) return;
+
+    const int4* __restrict__ vbase = reinterpret_cast<const int4*>(slab - mis);
+    const int v0 = chunk * (CHUNK / 4);
+
+    int4 x[ITER];
+#pragma unroll
+    for (int i = 0; i < ITER; ++i) {
+        const int v = v0 + i * kLookupThreads + tid;
+        if (4 * v < g_end) x[i] = ld_hist(vbase + v);
+        else x[i] = make_int4(0, 0, 0, 0);
+    }
+    // query: the history's own tail.  q0 = last token; lane j keeps the tokens 1+j and 33+j back.
+    const int32_t q0 = slab[n - 1];
+    const int32_t qa = (1 + lane <= n - 1) ? slab[n - 2 - lane] : 0;
+    const int32_t qb = (33 + lane <= n - 1) ? slab[n - 34 - lane] : 0;
+
+    Best best;  // identical in all lanes of a warp
+    best.key = 0; best.cnt = 0;
+
+#pragma unroll
+    for (int i = 0; i < ITER; ++i) {
+        const int p0 = 4 * (v0 + i * kLookupThreads + tid) - mis;  // position of x[i].x
+        uint32_t m = 0;
+        m |= (x[i].x == q0 && p0 + 0 >= 0 && p0 + 0 <= n - 2) ? 1u : 0u;
+        m |= (x[i].y == q0 && p0 + 1 >= 0 && p0 + 1 <= n - 2) ? 2u : 0u;
+        m |= (x[i].z == q0 && p0 + 2 >= 0 && p0 + 2 <= n - 2) ? 4u : 0u;
+        m |= (x[i].w == q0 && p0 + 3 >= 0 && p0 + 3 <= n - 2) ? 8u : 0u;
+        uint32_t hits = __ballot_sync(0xffffffffu, m != 0);
+        while (hits) {
+            const int src = __ffs(hits) - 1;
+            hits &= hits - 1;
+            uint32_t ms = __shfl_sync(0xffffffffu, m, src);
+            const int ps = __shfl_sync(0xffffffffu, p0, src);
+            while (ms) {
+                const int k = __ffs(ms) - 1;
+                ms &= ms - 1;
+                const int p = ps + k;
+                // match length of the copy ending at p (>= 1 already); limit: l_max and the slab start
+                const int cap = min(a.l_max, p + 1);
+                int l = lane + 1;
+                bool eq = (l < cap) && (slab[p - l] == qa);
+                uint32_t mm = __ballot_sync(0xffffffffu, !eq);
+                int L;
+                if (mm != 0) {
+                    L = __ffs(mm);  // first failing lane j: lengths 1..j hold, so L = 1 + j
+                } else {
+                    l = lane + 33;
+                    eq = (l < cap) && (slab[p - l] == qb);
+                    mm = __ballot_sync(0xffffffffu, !eq);  // lane 31 (l = 64) always fails
+                    L = 32 + __ffs(mm);
+                }
+                Best c;
+                c.key = ((unsigned long long)(uint32_t)L << 32) | (uint32_t)(p + 1);
+                c.cnt = 1;
+                best = combine(best, c);
+            }
+        }
+    }
+
+    __shared__ unsigned long long s_key[kLookupThreads / 32];
+    __shared__ uint32_t s_cnt[kLookupThreads / 32];
+    if (lane == 0) { s_key[warp] = best.key; s_cnt[warp] = best.cnt; }
+    __syncthreads();
+    if (warp != 0) return;
+
+    Best r;
+    r.key = lane < kLookupThreads / 32 ? s_key[lane] : 0ull;
+    r.cnt = lane < kLookupThreads / 32 ? s_cnt[lane] : 0u;
+    r = warp_combine(r);
+
+    uint32_t last = 0;
+    if (lane == 0) {
+        if (n_chunks > 1) {
+            LookupPartial* slot = a.partial + (int64_t)b * a.max_chunks + chunk;
+            slot->key = r.key; slot->cnt = r.cnt;
+            __threadfence();
+            const uint32_t old = atomicAdd(a.req_cnt + b, 1u);
+            last = (old + 1 == (uint32_t)n_chunks) ? 1u : 0u;
+        } else {
+            last = 1;
+        }
+    }
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+
+    if (n_chunks > 1) {
+        __threadfence();
+        Best t; t.key = 0; t.cnt = 0;
+        const LookupPartial* slots = a.partial + (int64_t)b * a.max_chunks;
+        for (int c = lane; c < n_chunks; c += 32) {
+            Best o;
+            o.key = __ldcg(&slots[c].key);
+            o.cnt = __ldcg(&slots[c].cnt);
+            t = combine(t, o);
+        }
+        r = warp_combine(t);
+        if (lane == 0) a.req_cnt[b] = 0;  // scratch is zero at rest
+    }
+
+    int L = (int)(r.key >> 32);
+    int e = (int)(uint32_t)(r.key & 0xffffffffu);
+    int cnt = (int)r.cnt;
+    int d = 0;
+    if (L < a.min_match || L == 0) {
+        L = 0; e = -1; cnt = 0;
+    } else {
+        int K = a.K[b];
+        K = max(0, min(K, a.k_cap));
+        int lim = K;
+        if (a.spec_factor > 0.0f) {
+            // two separately rounded operations, as written: multiply, then add
+            const float f = __fadd_rn(__fmul_rn(a.spec_factor, (float)L), a.spec_offset);
+            lim = max(0, (int)floorf(f));
+        }
+        d = min(min(K, lim), n - e);
+    }
+    for (int j = lane; j < a.k_cap; j += 32)
+        a.draft[(int64_t)b * a.k_cap + j] = (j < d) ? slab[e + j] : -1;
+    if (lane == 0) {
+        a.draft_len[b] = d; a.match_len[b] = L; a.match_pos[b] = e; a.match_cnt[b] = cnt;
+    }
+}
+
+}  // namespace
+
+hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                         const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
+                         int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
+                         int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream) {
+    LookupArgs a;
+    a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.K = K;
+    a.n_max = n_max;
+    a.draft = draft; a.draft_len = draft_len; a.match_len = match_len; a.match_pos = match_pos;
+    a.match_cnt = match_cnt;
+    a.partial = ctx->lk_partial; a.req_cnt = ctx->lk_cnt; a.max_chunks = ctx->lk_max_chunks;
+    a.k_cap = ctx->cfg.k_cap; a.l_max = ctx->cfg.l_max; a.min_match = ctx->cfg.min_match;
+    a.spec_factor = ctx->cfg.spec_factor; a.spec_offset = ctx->cfg.spec_offset;
+
+    // aligned-grid tokens to cover: n_max - 1 candidates plus up to 3 tokens of misalignment
+    const int64_t span = (int64_t)(n_max > 1 ? n_max - 1 : 1) + 3;
+    // pick the loads per thread so that the grid is about two resident waves at most
+    const int64_t resident = (int64_t)ctx->num_sms * (2048 / kLookupThreads);
+    int iter = 1;
+    while (iter < 8 && ((span + (int64_t)kLookupMinChunk * iter - 1) / ((int64_t)kLookupMinChunk * iter)) * B > 2 * resident)
+        iter *= 2;
+    const int64_t chunk = (int64_t)kLookupMinChunk * iter;
+    const int64_t chunks = (span + chunk - 1) / chunk;
+    if (chunks > ctx->lk_max_chunks) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max exceeds max_hist_len");
+    dim3 grid((unsigned)chunks, (unsigned)B);
+    switch (iter) {
+        case 1: lookup_kernel<1><<<grid, kLookupThreads, 0, stream>>>(a); break;
+        case 2: lookup_kernel<2><<<grid, kLookupThreads, 0, stream>>>(a); break;
+        case 4: lookup_kernel<4><<<grid, kLookupThreads, 0, stream>>>(a); break;
+        default: lookup_kernel<8><<<grid, kLookupThreads, 0, stream>>>(a); break;
+    }
+    HVD_CUDA_TRY(ctx, cudaGetLastError());
+    return HVD_OK;
+}
+
+}  // namespace hvd

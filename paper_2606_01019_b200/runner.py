@@ -1,0 +1,78 @@
+"""Device-side plumbing for one request batch: uploads host arrays into torch CUDA tensors, holds
+the output tensors, and calls the three library entry points.  No step of the method is computed
+here; every call goes to the CUDA library."""
+from __future__ import annotations
+
+import numpy as np
+
+from .binding import BF16, F32, STATE_DTYPE, Context
+
+
+class DeviceBatch:
+    def __init__(self, ctx: Context, *, hist, hist_off, hist_cap, hist_len, K, prompt_len, state,
+                 model_draft, model_len, row_off, V, dtype, uniform_rows=False, device="cuda"):
+        import torch
+        self.torch = torch
+        self.ctx = ctx
+        self.dev = torch.device(device)
+        self.B = int(len(hist_len))
+        self.V = int(V)
+        self.dtype = F32 if dtype in ("f32", F32) else BF16
+        kc = ctx.k_cap
+        up = lambda a, dt: torch.as_tensor(np.ascontiguousarray(a, dt), device=self.dev)
+        self.hist = up(hist, np.int32)
+        self.hist_off = up(hist_off, np.int64)
+        self.hist_cap = up(hist_cap, np.int32)
+        self.hist_len = up(hist_len, np.int32)
+        self.K = up(K, np.int32)
+        self.prompt_len = up(prompt_len, np.int32)
+        self.state = torch.as_tensor(np.ascontiguousarray(state, STATE_DTYPE).view(np.int64).reshape(self.B, 2),
+                                     device=self.dev)
+        self.model_draft = None if model_draft is None else up(model_draft, np.int32)
+        self.model_len = None if model_len is None else up(model_len, np.int32)
+        self.total_rows = int(row_off[-1])
+        self.k_uniform = int(row_off[1] - row_off[0]) - 1 if uniform_rows else 0
+        self.row_off = None if uniform_rows else up(row_off, np.int64)
+        self.n_max = int(max(0, np.max(hist_cap))) if len(hist_cap) else 0
+        B = self.B
+        i32 = lambda *s: torch.full(s, -12345, dtype=torch.int32, device=self.dev)
+        self.draft, self.draft_len = i32(B, kc), i32(B)
+        self.match_len, self.match_pos, self.match_cnt = i32(B), i32(B), i32(B)
+        self.features = torch.full((B, 8), float("nan"), dtype=torch.float32, device=self.dev)
+        self.score = torch.full((B,), float("nan"), dtype=torch.float32, device=self.dev)
+        self.select, self.sel_draft, self.sel_len = i32(B), i32(B, kc), i32(B)
+        self.accepted, self.committed, self.n_commit = i32(B), i32(B, kc + 1), i32(B)
+        self.target_tok, self.status = i32(max(self.total_rows, 1)), i32(B)
+
+    def lookup(self):
+        self.ctx.hvd_lookup(self.B, self.hist, self.hist_off, self.hist_cap, self.hist_len, self.K,
+                            self.n_max, self.draft, self.draft_len, self.match_len, self.match_pos,
+                            self.match_cnt)
+
+    def score_select(self):
+        self.ctx.hvd_score_select(self.B, self.hist_len, self.prompt_len, self.state, self.K, self.draft,
+                                  self.draft_len, self.match_len, self.match_pos, self.match_cnt,
+                                  self.model_draft, self.model_len, self.features, self.score,
+                                  self.select, self.sel_draft, self.sel_len)
+
+    def verify_commit(self, logits, target_tok=True):
+        self.ctx.hvd_verify_commit(self.B, logits, self.dtype, self.V, self.row_off, self.k_uniform,
+                                   self.total_rows, self.sel_draft, self.sel_len, self.select, self.hist,
+                                   self.hist_off, self.hist_cap, self.hist_len, self.state,
+                                   self.accepted, self.committed, self.n_commit,
+                                   self.target_tok if target_tok else None, self.status)
+
+    def step(self, logits, target_tok=True):
+        self.lookup()
+        self.score_select()
+        self.verify_commit(logits, target_tok)
+
+    def download(self) -> dict:
+        """Host copies of every output and in/out array (synchronises)."""
+        names = ["draft", "draft_len", "match_len", "match_pos", "match_cnt", "features", "score",
+                 "select", "sel_draft", "sel_len", "accepted", "committed", "n_commit", "target_tok",
+                 "status", "hist", "hist_len"]
+        out = {k: getattr(self, k).cpu().numpy() for k in names}
+        out["target_tok"] = out["target_tok"][:self.total_rows]
+        out["state"] = self.state.cpu().numpy().reshape(-1).view(STATE_DTYPE)
+        return out

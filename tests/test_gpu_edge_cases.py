@@ -1,0 +1,221 @@
+"""GPU parity on the degenerate and adversarial shapes of the path."""
+import numpy as np
+import pytest
+
+import hvd_workloads as W
+from oracle import hvd_oracle as O
+from oracle import pipeline as P
+from tests import gpu_helpers as G
+
+pytestmark = pytest.mark.gpu
+
+
+def hand_requests(w, hists, K, cap_extra=None, hist_len=None, model_len=None, misalign=None, seed=0,
+                  model_draft=None):
+    rng = np.random.default_rng(seed)
+    B = len(hists)
+    K = np.asarray(K, np.int64)
+    n = np.asarray([len(h) for h in hists], np.int64)
+    extra = 4 * (K + 1) if cap_extra is None else np.asarray(cap_extra, np.int64)
+    cap = n + extra
+    prompt_len = np.floor(n * rng.uniform(0.0, 1.0, B)).astype(np.int32)
+    state = np.zeros(B, W.STATE_DTYPE)
+    state["sel_bits"] = rng.integers(0, 2**32, B, dtype=np.uint64).astype(np.uint32)
+    state["acc_ring"] = rng.integers(0, 2**63, B, dtype=np.uint64)
+    if model_draft is None:
+        model_draft = rng.integers(0, w.V, (B, w.k_cap)).astype(np.int32)
+    if model_len is None:
+        model_len = K
+    return W.pack_requests([np.asarray(h, np.int32) for h in hists], K, cap, prompt_len, state, model_draft,
+                           model_len, hist_len=hist_len, misalign=misalign)
+
+
+def small(V=997, k_cap=8, dtype="bf16", **kw):
+    return W.CONFIGS["C2"].scaled(V=V, k_cap=k_cap, K=k_cap, dtype=dtype, calibrate_cache_frac=0.5, **kw)
+
+
+def run(w, rq, **kw):
+    inp = P.prepare(w.scaled(B=rq.B), device="cuda", rq=rq)
+    return G.run_and_compare(inp, **kw), inp
+
+
+def test_tiny_histories():
+    w = small()
+    rng = np.random.default_rng(3)
+    hists = []
+    for n in (0, 1, 2, 3, 4, 5, 63, 64, 65, 66, 127, 128, 129, 1023, 1024, 1025, 1026, 1027, 2050):
+        hists.append(rng.integers(0, 3, n))                 # tiny vocabulary: matches everywhere
+        hists.append(rng.integers(0, w.V, n))               # large vocabulary: rarely any match
+    rq = hand_requests(w, hists, [8] * len(hists))
+    (g, out, _), _ = run(w, rq)
+    assert (out.lk.match_len > 0).sum() > 10
+
+
+def test_draft_caps_k0_k1_k64():
+    w = small(k_cap=64)
+    rng = np.random.default_rng(4)
+    base = rng.integers(0, 5, 3000)
+    hists = [base[: 2000 + 17 * i] for i in range(12)]
+    K = [0, 1, 64, 0, 1, 64, 2, 63, 33, 32, 31, 64]
+    rq = hand_requests(w, hists, K)
+    run(w, rq)
+
+
+def test_all_equal_and_periodic_histories():
+    w = small()
+    hists = [[7] * 300, [7] * 64, [7] * 65, [7] * 66, [1, 2] * 200, [1, 2, 3] * 150, [1, 2] * 31 + [1],
+             [5] * 2, [5] * 3, [4, 4, 9] * 400 + [4]]
+    rq = hand_requests(w, hists, [8] * len(hists))
+    (g, out, _), _ = run(w, rq)
+    assert tuple(int(x[0]) for x in (out.lk.match_len, out.lk.match_pos, out.lk.match_cnt, out.lk.draft_len)) == (64, 299, 236, 1)
+
+
+def test_match_touching_slab_start_and_end():
+    w = small(V=50021)
+    rng = np.random.default_rng(5)
+    hs = []
+    for L in (2, 5, 64, 70):
+        h = rng.permutation(40000)[:1500].astype(np.int64) + 5
+        h[-L:] = h[:L]                       # only match ends at e = L: touches index 0
+        hs.append(h)
+        h = rng.permutation(40000)[:1500].astype(np.int64) + 5
+        h[-3:] = h[-3]                       # x x x: longest match (2) ends at e = n-1, a one-token draft
+        hs.append(h)
+    rq = hand_requests(w, hs, [8] * len(hs))
+    (g, out, _), _ = run(w, rq)
+    assert out.lk.match_pos[0] == 2 and out.lk.match_len[4] == 64
+    assert out.lk.match_pos[1] == 1499 and out.lk.draft_len[1] == 1
+
+
+@pytest.mark.parametrize("mis", [1, 2, 3])
+def test_misaligned_slabs(mis):
+    w = small()
+    rng = np.random.default_rng(6)
+    hists = [rng.integers(0, 4, n) for n in (10, 100, 1024, 1025, 3000, 4099)]
+    rq = hand_requests(w, hists, [8] * len(hists), misalign=[mis, (mis + 1) % 4, mis, 0, mis, mis])
+    run(w, rq)
+
+
+def test_capacity_edges_and_bad_lengths():
+    w = small()
+    rng = np.random.default_rng(7)
+    hists = [rng.integers(0, 3, 500) for _ in range(12)]
+    extra = [9, 5, 4, 3, 2, 1, 0, 9, 9, 9, 9, 0]
+    hist_len = [500, 500, 500, 500, 500, 500, 500, -1, 510, 2**31 - 1, 500, 500]
+    rq = hand_requests(w, hists, [8] * 12, cap_extra=extra, hist_len=hist_len)
+    (g, out, _), _ = run(w, rq)
+    assert (out.vf.status == O.REQ_BAD_LEN).sum() == 3
+    assert (out.vf.status == O.REQ_CAPACITY).sum() >= 1
+
+
+def test_model_draft_clamp_and_out_of_vocab_tokens():
+    w = small(k_cap=16)
+    rng = np.random.default_rng(8)
+    hists = [rng.integers(0, w.V, 800) for _ in range(10)]          # hardly any cache draft: model path
+    K = [4, 8, 16, 0, 3, 16, 16, 1, 2, 5]
+    md = rng.integers(0, w.V, (10, 16)).astype(np.int32)
+    md[5, 3] = -1; md[6, 0] = w.V; md[2, 15] = 2**31 - 1
+    rq = hand_requests(w, hists, K, model_len=[9, 8, 16, 5, 0, 16, 16, 1, 40, -3], model_draft=md)
+    (g, out, _), _ = run(w.scaled(calibrate_cache_frac=None), rq)
+    assert (out.sc.select == 0).all()
+
+
+def test_no_model_drafter():
+    """model_draft = NULL: requests whose cache draft is not selected verify an empty draft."""
+    w = W.CONFIGS["C1"]
+    inp = P.prepare(w, device="cuda")
+    rq = inp.rq.copy()
+    rq.model_len[:] = 0
+    inp2 = P.prepare(w, device="cuda", rq=rq)
+    ctx = G.make_ctx(w, rq)
+    ctx.hvd_set_predictor(inp2.W1, inp2.b1, inp2.W2, inp2.b2, inp2.tau)
+    batch = G.make_batch(ctx, w, inp2.rq.copy())
+    batch.model_draft = None
+    batch.model_len = None
+    G.run_and_compare(inp2, ctx=ctx, batch=batch, rq=inp2.rq.copy())
+    ctx.close()
+
+
+@pytest.mark.parametrize("V,dtype", [(1, "bf16"), (7, "bf16"), (8, "bf16"), (9, "bf16"), (15, "bf16"), (17, "bf16"),
+                                     (1, "f32"), (3, "f32"), (4, "f32"), (5, "f32"), (32000, "f32"),
+                                     (8193 * 8, "bf16"), (16384 * 8 + 3, "bf16"), (151936, "bf16")])
+def test_vocab_sizes(V, dtype):
+    w = small(V=V, dtype=dtype, k_cap=4)
+    rng = np.random.default_rng(V)
+    hists = [rng.integers(0, min(V, 3), 200 + 13 * i) for i in range(6)]
+    rq = hand_requests(w, hists, [4, 3, 2, 1, 0, 4])
+    run(w, rq)
+
+
+def test_constructed_argmax_ties_on_device():
+    """Whole rows of equal values, +-0, +inf duplicates, maxima in the first and last slot, and a
+    duplicate maximum straddling two work items."""
+    import torch
+    w = small(V=40000, k_cap=8)
+    rng = np.random.default_rng(9)
+    hists = [rng.integers(0, w.V, 300) for _ in range(9)]
+    rq = hand_requests(w, hists, [8] * 9)
+    inp = P.prepare(w.scaled(B=9, calibrate_cache_frac=None), device="cuda", rq=rq)
+    lg = inp.logits
+    r = rq.row_off
+    lg[r[0]:r[1]] = 1.5                                   # all equal -> token 0
+    lg[r[1]:r[2]] = -0.0; lg[r[1], 17] = 0.0              # -0 == +0 -> token 0
+    lg[r[2]:r[3]] = -5.0; lg[r[2], 39999] = 3.0           # maximum in the last slot
+    lg[r[3]:r[4]] = -5.0; lg[r[3], 0] = 3.0               # maximum in the first slot
+    lg[r[4], 16383] = float("inf"); lg[r[4], 16384] = float("inf")     # equal maxima across items
+    lg[r[5], 30000] = 40.0; lg[r[5], 20] = 40.0           # equal maxima far apart
+    lg[r[6]:r[7]] = float("-inf")                         # nothing but -inf -> token 0
+    lg[r[7]:r[8]] = -0.0                                  # nothing but -0
+    inp.logits_np = W.logits_to_numpy(lg)
+    g, out, _ = G.run_and_compare(inp)
+    t = out.vf.target_tok
+    assert t[r[0]] == 0 and t[r[1]] == 0 and t[r[2]] == 39999 and t[r[3]] == 0
+    assert t[r[4]] == 16383 and t[r[5]] == 20 and t[r[6]] == 0 and t[r[7]] == 0
+
+
+def test_batch_of_one_and_full_context_batch():
+    w = small()
+    rng = np.random.default_rng(10)
+    rq = hand_requests(w, [rng.integers(0, 3, 777)], [8])
+    run(w, rq)
+    hists = [rng.integers(0, 4, int(n)) for n in rng.integers(0, 600, 700)]
+    rq = hand_requests(w, hists, rng.integers(0, 9, 700))
+    run(w, rq)
+
+
+def test_two_calls_with_different_shapes_share_a_context():
+    """A context sized for the larger call serves a smaller one afterwards (scratch at rest)."""
+    w = small()
+    rng = np.random.default_rng(11)
+    big = hand_requests(w, [rng.integers(0, 4, 5000) for _ in range(20)], [8] * 20)
+    sm = hand_requests(w, [rng.integers(0, 4, 100) for _ in range(3)], [8] * 3)
+    ctx = G.make_ctx(w, big)
+    for rq in (big, sm, big):
+        inp = P.prepare(w.scaled(B=rq.B), device="cuda", rq=rq.copy())
+        G.run_and_compare(inp, ctx=ctx)
+    ctx.close()
+
+
+def test_host_side_argument_errors():
+    import paper_2606_01019_b200 as H
+    w = small()
+    rng = np.random.default_rng(12)
+    rq = hand_requests(w, [rng.integers(0, 4, 100) for _ in range(3)], [8] * 3)
+    ctx = G.make_ctx(w, rq)
+    b = G.make_batch(ctx, w, rq)
+    with pytest.raises(H.HvdError, match="hvd_set_predictor first"):
+        b.score_select()
+    with pytest.raises(H.HvdError, match="B outside"):
+        ctx.hvd_lookup(4, b.hist, b.hist_off, b.hist_cap, b.hist_len, b.K, b.n_max, b.draft, b.draft_len,
+                       b.match_len, b.match_pos, b.match_cnt)
+    with pytest.raises(H.HvdError, match="NULL"):
+        ctx.hvd_lookup(3, None, b.hist_off, b.hist_cap, b.hist_len, b.K, b.n_max, b.draft, b.draft_len,
+                       b.match_len, b.match_pos, b.match_cnt)
+    with pytest.raises(H.HvdError, match="n_max"):
+        ctx.hvd_lookup(3, b.hist, b.hist_off, b.hist_cap, b.hist_len, b.K, 10**6, b.draft, b.draft_len,
+                       b.match_len, b.match_pos, b.match_cnt)
+    with pytest.raises(H.HvdError):
+        H.Context(max_batch=0, k_cap=8, max_hist_len=10, max_rows=10, max_vocab=10)
+    with pytest.raises(H.HvdError):
+        H.Context(max_batch=4, k_cap=65, max_hist_len=10, max_rows=10, max_vocab=10)
+    ctx.close()

@@ -1,0 +1,70 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Integer results bit-exact; fp32 scores within 1e-5 relative."""
+import numpy as np
+import pytest
+
+import hvd_workloads as W
+from oracle import hvd_oracle as O
+from oracle import pipeline as P
+from tests import gpu_helpers as G
+
+pytestmark = pytest.mark.gpu
+
+
+def test_c1_full():
+    inp = P.prepare(W.CONFIGS["C1"], device="cuda")
+    g, out, _ = G.run_and_compare(inp)
+    assert (g["accepted"] == inp.A)[inp.strict].all()
+    assert g["select"].sum() > 0
+
+
+def test_c1_uniform_row_layout():
+    inp = P.prepare(W.CONFIGS["C1"], device="cuda")
+    G.run_and_compare(inp, uniform_rows=True)
+
+
+@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5"])
+def test_full_size_configs(name):
+    """Every request, row and token of the full-size workloads, in the launch configuration the
+    benchmark uses (same context limits, same entry points)."""
+    inp = P.prepare(W.CONFIGS[name], device="cuda")
+    g, out, _ = G.run_and_compare(inp)
+    assert (g["accepted"] == inp.A)[inp.strict].all()
+    sel = g["select"]
+    assert 0 < sel.sum() < len(sel)                       # both draft sources in play
+    assert (g["status"] == O.REQ_OK).all()
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("C2", dict(B=7, n=5000, V=20011)),                    # odd V: rows not 16-byte multiples (bf16)
+    ("C2", dict(B=5, n=3000, V=9)),
+    ("C1", dict(B=3, n=700, V=4099)),                      # fp32, odd V
+    ("C1", dict(B=3, n=700, V=1)),
+    ("C1", dict(B=2, n=300, V=7)),
+    ("C2", dict(B=3, n=1500, V=8)),
+    ("C3", dict(B=9, n=2500, V=151936)),
+    ("C5", dict(B=40, n=(16, 3000), V=32003)),
+])
+def test_scaled_shapes(name, kw):
+    inp = P.prepare(W.CONFIGS[name].scaled(**kw), device="cuda")
+    G.run_and_compare(inp)
+
+
+def test_multi_step_loop_and_scratch_reuse():
+    """Eight chained steps on one context and one device batch: histories keep growing, the
+    scratch memory must be back at rest after every call."""
+    for name, kw in (("C1", {}), ("C2", dict(B=16, n=4096, V=50021))):
+        w = W.CONFIGS[name].scaled(**kw)
+        inp = P.prepare(w, device="cuda")
+        rq = inp.rq.copy()
+        batch = None
+        ctx = G.make_ctx(w, rq)
+        ctx.hvd_set_predictor(inp.W1, inp.b1, inp.W2, inp.b2, inp.tau)
+        for s in range(8):
+            logits = W.make_logits(w, int(rq.row_off[-1]), device="cuda", salt=50 + s)
+            if batch is None:
+                batch = G.make_batch(ctx, w, rq)
+            g, out, batch = G.run_and_compare(inp, ctx=ctx, logits=logits, logits_np=W.logits_to_numpy(logits),
+                                              rq=rq, batch=batch)
+        assert (rq.hist_len > inp.rq.hist_len).all()
+        ctx.close()
