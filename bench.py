@@ -1,0 +1,488 @@
+#!/usr/bin/env python
+"""Benchmark of the HVD per-step path (lookup -> score/select -> verify/commit) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--impl b200|reference]
+
+One step = one pass of the whole path over one batch of seeded synthetic input.  Prints ONE JSON
+line.  With N > 1 (launched by torch.distributed.run) every rank runs its own copy of the batch:
+requests are independent, so the path shards with no collective on the data path ("weak" scaling);
+only the timing is reduced (max over ranks).
+
+Timed region: K steps captured in one CUDA graph (3 kernel launches per step), bracketed by a
+barrier + synchronize, timed with CUDA events on the launching stream.  Consecutive steps use
+rotating copies of the big inputs (histories, logits) so that nothing a step reads is left in L2
+by an earlier step, and every step gets pristine per-step lengths/state.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "HVD select+verify steps/s"
+UNIT = "steps/s"
+L2_BYTES = 126 * 2**20
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one verify_commit launch on this workload, from
+# the ncu capture summarised under profiles/ (None until captured for a workload)
+NCU_VERIFY_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", default="C2")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--mode", default="graph", choices=["graph", "stream"])
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-kernel-events", action="store_true",
+                    help="leave the per-kernel event records out of the timed graph")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ----------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
+               0x100: "display_clock_setting", 0x10: "sync_boost"}
+
+    def __init__(self, device_index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self.stop_flag = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as e:  # pragma: no cover
+            self.err = repr(e)
+
+    def sample(self):
+        nv = self.nv
+        mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+        try:
+            bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+        except Exception:
+            bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+        self.samples.append(mhz)
+        for bit, name in self.REASONS.items():
+            if bits & bit:
+                self.reasons.add(name)
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self.stop_flag.is_set():
+            try:
+                self.sample()
+            except Exception:
+                break
+            time.sleep(self.period)
+
+    def summary(self, window: str):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "window": window}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples), "window": window}
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+# ----------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import hvd_workloads as W
+    from oracle import pipeline as P
+    w = W.CONFIGS[args.config]
+    cores = P.host_threads()
+    inp = P.prepare(w, device="cpu", nthreads=cores)
+    # one full step to size the per-step sample
+    rq = inp.rq.copy()
+    t0 = time.perf_counter()
+    P.step(inp, rq, nthreads=cores)
+    t_full = time.perf_counter() - t0
+    budget = 150.0
+    B_s = w.B
+    if (args.steps + args.warmup) * t_full > budget:
+        B_s = max(1, int(w.B * budget / ((args.steps + args.warmup) * t_full)))
+    sub = inp
+    if B_s < w.B:
+        # a bounded sample: the first B_s requests of the batch (own history slabs, own logits rows)
+        rows = int(inp.rq.row_off[B_s])
+        keep = slice(0, B_s)
+        sub = P.Inputs(w, W.subset_requests(inp.rq, 0, B_s), inp.W1, inp.b1, inp.W2, inp.b2, inp.tau,
+                       inp.A[keep], inp.strict[keep], inp.logits[:rows], inp.logits_np[:rows])
+    times, committed = [], 0
+    for i in range(args.warmup + args.steps):
+        rq = sub.rq.copy()
+        t0 = time.perf_counter()
+        out = P.step(sub, rq, nthreads=cores)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt)
+            committed += int(out.vf.n_commit.sum())
+    total = float(np.sum(times))
+    frac = B_s / w.B
+    value = args.steps * frac / total
+    sample = (f"{B_s} of {w.B} requests of {w.name} per step (whole-batch-equivalent steps/s = sampled "
+              f"steps/s x {frac:.4f})" if B_s < w.B else f"the whole {w.name} batch every step")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps / frac,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
+            "data": "synthetic", "config": workload_config(w, args.gpus),
+            "tokens_per_s": committed / total,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, n_gpus, extra=None):
+    cfg = {"workload": f"{w.name}: batch {w.B}, histories {w.n} tokens, vocab {w.V}, K {w.K}, {w.dtype} logits",
+           "requests_per_gpu": w.B, "parallelism": f"requests sharded over {n_gpus} GPU(s), no collective"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+# ----------------------------------------------------------------------------------------------
+# the CUDA path
+# ----------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import hvd_workloads as W
+    import paper_2606_01019_b200 as H
+    from paper_2606_01019_b200.sharding import max_over_ranks
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the HVD path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = W.CONFIGS[args.config]
+    K_steps, W_steps = args.steps, args.warmup
+    n_slots = K_steps + W_steps
+    peak_gbs, peak_kind = measured_peak()
+
+    # ---- inputs: the product path itself produces the drafts the logits are planted on ----------
+    rq = W.make_requests(w)
+    W1, b1, W2, b2, tau = W.make_predictor(w)
+    B, kc = rq.B, w.k_cap
+    total_rows = int(rq.row_off[-1])
+    ctx = H.Context(max_batch=B, k_cap=kc, max_hist_len=int(rq.hist_cap.max()), max_rows=total_rows,
+                    max_vocab=w.V, l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
+    ctx.hvd_set_predictor(W1, b1, W2, b2, tau)
+    up = lambda a, dt: torch.as_tensor(np.ascontiguousarray(a, dt), device=dev)
+    hist0 = up(rq.hist, np.int32)
+    hist_off, hist_cap, Kt = up(rq.hist_off, np.int64), up(rq.hist_cap, np.int32), up(rq.K, np.int32)
+    hist_len0, prompt_len = up(rq.hist_len, np.int32), up(rq.prompt_len, np.int32)
+    state0 = torch.as_tensor(rq.state.view(np.int64).reshape(B, 2), device=dev)
+    model_draft, model_len = up(rq.model_draft, np.int32), up(rq.model_len, np.int32)
+    row_off = up(rq.row_off, np.int64)
+    n_max = int(rq.hist_cap.max())
+    i32 = lambda *s: torch.zeros(s, dtype=torch.int32, device=dev)
+    draft, draft_len, match_len, match_pos, match_cnt = i32(B, kc), i32(B), i32(B), i32(B), i32(B)
+    score = torch.zeros(B, dtype=torch.float32, device=dev)
+    select, sel_draft, sel_len = i32(B), i32(B, kc), i32(B)
+    accepted, committed, n_commit, status = i32(B), i32(B, kc + 1), i32(B), i32(B)
+
+    def lookup(hist, hist_len):
+        ctx.hvd_lookup(B, hist, hist_off, hist_cap, hist_len, Kt, n_max, draft, draft_len, match_len,
+                       match_pos, match_cnt)
+
+    def score_select(hist_len, state):
+        ctx.hvd_score_select(B, hist_len, prompt_len, state, Kt, draft, draft_len, match_len, match_pos,
+                             match_cnt, model_draft, model_len, None, score, select, sel_draft, sel_len)
+
+    dtype = H.F32 if w.dtype == "f32" else H.BF16
+
+    def verify(logits, hist, hist_len, state):
+        ctx.hvd_verify_commit(B, logits, dtype, w.V, row_off, 0, total_rows, sel_draft, sel_len, select, hist,
+                              hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, None, status)
+
+    lookup(hist0, hist_len0)
+    score_select(hist_len0, state0)
+    if w.calibrate_cache_frac is not None:
+        torch.cuda.synchronize()
+        tau = W.calibrate_tau(score.cpu().numpy(), draft_len.cpu().numpy() > 0, w.calibrate_cache_frac)
+        ctx.hvd_set_predictor(W1, b1, W2, b2, tau)
+        score_select(hist_len0, state0)
+    torch.cuda.synchronize()
+    sel_len_h = sel_len.cpu().numpy()
+    sel_draft_h = sel_draft.cpu().numpy()
+    A = W.make_agreement(w, sel_len_h)
+    logits0 = W.make_logits(w, total_rows, device=dev)
+    W.plant_agreement(w, logits0, rq.row_off, sel_draft_h, sel_len_h, A)
+
+    # ---- rotating copies of the big inputs, pristine per-step small arrays ------------------------
+    foot = hist0.numel() * 4 + logits0.numel() * logits0.element_size()
+    R = int(max(2, -(-4 * L2_BYTES // foot)))
+    hists = [hist0] + [hist0.clone() for _ in range(R - 1)]
+    logits = [logits0] + [logits0.clone() for _ in range(R - 1)]
+    hist_len_steps = hist_len0.repeat(n_slots, 1).contiguous()
+    state_steps = state0.repeat(n_slots, 1, 1).contiguous()
+    hist_len_pristine, state_pristine = hist_len_steps.clone(), state_steps.clone()
+
+    def restore():
+        hist_len_steps.copy_(hist_len_pristine)
+        state_steps.copy_(state_pristine)
+
+    def step(slot, events=None):
+        r = slot % R
+        hl, st = hist_len_steps[slot], state_steps[slot]
+        if events is not None:
+            events[0].record()
+        lookup(hists[r], hl)
+        if events is not None:
+            events[1].record()
+        score_select(hl, st)
+        if events is not None:
+            events[2].record()
+        verify(logits[r], hists[r], hl, st)
+        if events is not None:
+            events[3].record()
+
+    # ---- warm-up (eager), then the timed K steps --------------------------------------------------
+    for s in range(W_steps):
+        step(s)
+    torch.cuda.synchronize()
+    use_events = not args.no_kernel_events
+    mode = args.mode
+    kernel_events = None
+    graph = None
+    stream = torch.cuda.Stream(device=dev)
+    if mode == "graph":
+        try:
+            if use_events:
+                kernel_events = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(4)]
+                                 for _ in range(K_steps)]
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                graph.capture_begin()
+                for s in range(K_steps):
+                    step(W_steps + s, kernel_events[s] if kernel_events else None)
+                graph.capture_end()
+            torch.cuda.synchronize()
+            with torch.cuda.stream(stream):
+                graph.replay()               # untimed: instantiation and upload costs
+            torch.cuda.synchronize()
+            restore()
+        except Exception as e:  # pragma: no cover
+            sys.stderr.write(f"bench.py: graph capture failed ({e!r}); timing plain stream launches\n")
+            mode, graph, kernel_events = "stream", None, None
+            torch.cuda.synchronize()
+            restore()
+    if mode == "stream" and use_events:
+        kernel_events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K_steps)]
+
+    sampler = ClockSampler(local)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    with torch.cuda.stream(stream):
+        ev0.record()
+        if graph is not None:
+            graph.replay()
+        else:
+            for s in range(K_steps):
+                step(W_steps + s, kernel_events[s] if kernel_events else None)
+        ev1.record()
+    barrier()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    window = "timed region"
+    # results of the timed steps (every step does the same work on identical copies)
+    n_commit_h = n_commit.cpu().numpy()
+    accepted_h = accepted.cpu().numpy()
+    select_h = select.cpu().numpy()
+    status_h = status.cpu().numpy()
+    sel_len_after = sel_len.cpu().numpy()
+    if len(sampler.samples) < 5 and graph is not None:
+        # region too short for the sampler: keep the same graph running, untimed, while sampling
+        window = "timed region + untimed repeats of the same graph"
+        t_end = time.time() + 0.3
+        while time.time() < t_end:
+            restore()
+            with torch.cuda.stream(stream):
+                graph.replay()
+            torch.cuda.synchronize()
+    sampler.stop_flag.set()
+    sampler.join(timeout=2)
+
+    kt = None
+    if kernel_events:
+        try:
+            d = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in kernel_events])
+            kt = {"lookup_us": 1e3 * float(d[:, 0].mean()), "score_select_us": 1e3 * float(d[:, 1].mean()),
+                  "verify_commit_us": 1e3 * float(d[:, 2].mean()),
+                  "verify_commit_us_median": 1e3 * float(np.median(d[:, 2])),
+                  "lookup_us_median": 1e3 * float(np.median(d[:, 0]))}
+        except Exception as e:  # pragma: no cover
+            sys.stderr.write(f"bench.py: per-kernel events unavailable ({e!r})\n")
+
+    elapsed_ms = max_over_ranks(elapsed_ms, dev)
+    steps_per_s = world * K_steps / (elapsed_ms * 1e-3)
+    tokens_per_step = int(n_commit_h.sum())
+    assert (status_h == 0).all(), "a request reported a capacity or length problem"
+
+    # ---- roofline of the dominant kernel (verify/commit): algorithmic bytes = needed rows x V x elt ----
+    verify_bytes = int((sel_len_after.astype(np.int64) + 1).sum()) * w.V * w.elt
+    lookup_bytes = int(rq.hist_len.astype(np.int64).sum()) * 4
+    roofline = {"bound": "hbm", "kernel": "verify_commit_kernel", "achieved": None, "peak": peak_gbs, "unit": "GB/s",
+                "frac": None, "traffic": NCU_VERIFY_TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind,
+                "algorithmic_bytes_per_launch": verify_bytes}
+    roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel", "achieved": None, "peak": peak_gbs, "unit": "GB/s",
+                       "frac": None, "traffic": None, "peak_kind": peak_kind,
+                       "algorithmic_bytes_per_launch": lookup_bytes}
+    if kt:
+        roofline["achieved"] = verify_bytes / (kt["verify_commit_us"] * 1e-6) / 1e9
+        roofline["frac"] = roofline["achieved"] / peak_gbs
+        roofline["frac_of_8000_nominal"] = roofline["achieved"] / 8000.0
+        roofline_lookup["achieved"] = lookup_bytes / (kt["lookup_us"] * 1e-6) / 1e9
+        roofline_lookup["frac"] = roofline_lookup["achieved"] / peak_gbs
+        roofline_lookup["frac_of_8000_nominal"] = roofline_lookup["achieved"] / 8000.0
+
+    # ---- end to end through the host-buffer entry point --------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        E = max(1, min(args.e2e_steps, K_steps))
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        h_hist, h_off, h_cap = pin(rq.hist), pin(rq.hist_off), pin(rq.hist_cap)
+        h_len, h_K, h_pl = pin(rq.hist_len), pin(rq.K), pin(rq.prompt_len)
+        h_state = pin(rq.state.view(np.int64).reshape(B, 2))
+        h_md, h_ml, h_ro = pin(rq.model_draft), pin(rq.model_len), pin(rq.row_off)
+        h_logits = torch.empty(logits0.shape, dtype=logits0.dtype, pin_memory=True)
+        h_logits.copy_(logits0)
+        hz = lambda *s: torch.zeros(s, dtype=torch.int32).pin_memory()
+        o_score = torch.zeros(B, dtype=torch.float32).pin_memory()
+        o_sel, o_sd, o_sl, o_acc, o_com, o_nc, o_st = hz(B), hz(B, kc), hz(B), hz(B), hz(B, kc + 1), hz(B), hz(B)
+        len0, st0 = h_len.clone(), h_state.clone()
+
+        def host_step():
+            h_len.copy_(len0)
+            h_state.copy_(st0)
+            ctx.hvd_step_host(B=B, n_max=n_max, hist=h_hist, hist_off=h_off, hist_cap=h_cap, hist_len=h_len,
+                              K=h_K, prompt_len=h_pl, state=h_state, model_draft=h_md, model_len=h_ml,
+                              logits=h_logits, dtype=dtype, V=w.V, row_off=h_ro, k_uniform=0,
+                              total_rows=total_rows, score=o_score, select=o_sel, sel_draft=o_sd,
+                              sel_len=o_sl, accepted=o_acc, committed=o_com, n_commit=o_nc, status=o_st)
+
+        for _ in range(3):
+            host_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(E):
+            host_step()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        dt = max_over_ranks(dt, dev)
+        assert (o_acc.numpy() == accepted_h).all() and (o_nc.numpy() == n_commit_h).all()
+        small = B * (8 + 4 * 5 + 16) + (B + 1) * 8 + B * kc * 4
+        h2d = int(h_hist.numel() * 4 + h_logits.numel() * h_logits.element_size() + small)
+        d2h = int(B * 4 * 7 + B * kc * 4 + B * (kc + 1) * 4 + B * 16)
+        e2e = {"value": world * E / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "steps": E, "ms_per_step": 1e3 * dt / E, "tokens_per_s": world * E * tokens_per_step / dt,
+               "api": "hvd_step_host (pinned host buffers)"}
+
+    # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ----------
+    cpu_baseline = None
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        from oracle import pipeline as P
+        cores = P.host_threads()
+        logits_np = W.logits_to_numpy(logits0)
+        inp = P.Inputs(w, rq, W1, b1, W2, b2, tau, A, np.ones(B, bool), None, logits_np)
+        times, out = [], None
+        t_begin = time.perf_counter()
+        while len(times) < 5 or (time.perf_counter() - t_begin < 10.0 and len(times) < 200):
+            rq_c = rq.copy()
+            t0 = time.perf_counter()
+            out = P.step(inp, rq_c, nthreads=cores)
+            times.append(time.perf_counter() - t0)
+        med = float(np.median(times))
+        same = bool((out.vf.accepted == accepted_h).all() and (out.vf.n_commit == n_commit_h).all()
+                    and (out.sc.select == select_h).all())
+        cpu_baseline = {"value": 1.0 / med, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"the whole {w.name} batch ({B} requests, {total_rows} logits rows), "
+                                  f"median of {len(times)} repetitions",
+                        "ms_per_step": 1e3 * med, "tokens_per_s": tokens_per_step / med,
+                        "agrees_with_gpu_step": same}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": steps_per_s, "unit": UNIT, "n_gpus": world, "steps": K_steps,
+                "warmup": W_steps, "ms_per_step": elapsed_ms / K_steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+                "config": workload_config(w, world, {
+                    "cold_cache": f"{R} rotating copies of histories+logits ({foot / 2**20:.0f} MiB each, "
+                                  f"L2 is 126 MiB); inputs per step exceed L2",
+                    "launch": f"{mode}: {K_steps} steps x 3 kernels in one CUDA graph" if graph is not None
+                              else "stream: 3 kernel launches per step",
+                    "kernel_events_in_timed_region": bool(kernel_events), "tau": tau}),
+                "tokens_per_s": world * K_steps * tokens_per_step / (elapsed_ms * 1e-3),
+                "tokens_per_step": tokens_per_step,
+                "mean_accepted": float(accepted_h.mean()), "cache_selected_frac": float(select_h.mean()),
+                "kernel_us": kt, "roofline": roofline, "roofline_lookup": roofline_lookup,
+                "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": 3 * K_steps,
+                "clocks": sampler.summary(window)}
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -300,6 +300,16 @@ def pack_requests(hists, K, cap, prompt_len, state, model_draft, model_len, hist
                     row_off, guard)
 
 
+def subset_requests(rq: Requests, lo: int, hi: int) -> Requests:
+    """Requests [lo, hi) of a batch.  The flat history array is shared (offsets stay valid); logits
+    row offsets are rebased to the first kept row, so pass logits[row_off[lo]:row_off[hi]] along."""
+    keep = slice(lo, hi)
+    return Requests(rq.hist, rq.hist_off[keep].copy(), rq.hist_cap[keep].copy(), rq.hist_len[keep].copy(),
+                    rq.K[keep].copy(), rq.prompt_len[keep].copy(), rq.state[keep].copy(),
+                    rq.model_draft[keep].copy(), rq.model_len[keep].copy(),
+                    rq.row_off[lo:hi + 1] - rq.row_off[lo], rq.guard_mask)
+
+
 def make_predictor(w: Workload):
     """W1 [H,8], b1 [H], W2 [H] ~ N(0, 0.1^2) fp32 drawn in that order; b2 and tau from the config."""
     rng = _rng(w.index, S_WEIGHTS)

@@ -174,6 +174,48 @@ HVD_API hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits
                              int32_t* committed, int32_t* n_commit, int32_t* target_tok,
                              int32_t* status, void* stream);
 
+/*
+ * The same decoding cycle with HOST buffers: one call copies the step's inputs to the device,
+ * runs hvd_lookup, hvd_score_select and hvd_verify_commit there, copies the results back, waits
+ * for the stream, and appends the committed tokens to the host histories.  Every pointer in the
+ * struct is a HOST pointer (pinned memory makes the copies asynchronous and faster; pageable
+ * memory works).  Arrays have the shapes documented at the three device entry points.
+ * The context keeps a device staging area that it (re)allocates when a call needs more than any
+ * earlier one (a synchronous cudaMalloc: not for use inside stream capture).  This entry point
+ * synchronises `stream` before returning.
+ */
+typedef struct {
+    int32_t B;
+    int32_t n_max;            /* upper bound on hist_len[b] */
+    int64_t hist_words;       /* length of the hist array in int32 words (all slabs) */
+    int32_t* hist;            /* in/out: committed tokens are appended */
+    const int64_t* hist_off;  /* [B] */
+    const int32_t* hist_cap;  /* [B] */
+    int32_t* hist_len;        /* [B] in/out */
+    const int32_t* K;         /* [B] */
+    const int32_t* prompt_len; /* [B] */
+    hvd_req_state* state;     /* [B] in/out */
+    const int32_t* model_draft; /* [B, k_cap] or NULL */
+    const int32_t* model_len; /* [B] or NULL */
+    const void* logits;       /* [total_rows, V] of dtype */
+    int32_t dtype;            /* hvd_dtype */
+    int32_t k_uniform;        /* used when row_off is NULL */
+    int64_t V;
+    const int64_t* row_off;   /* [B+1] or NULL */
+    int64_t total_rows;
+    /* outputs */
+    float* score;             /* [B] */
+    int32_t* select;          /* [B] */
+    int32_t* sel_draft;       /* [B, k_cap] */
+    int32_t* sel_len;         /* [B] */
+    int32_t* accepted;        /* [B] */
+    int32_t* committed;       /* [B, k_cap+1] */
+    int32_t* n_commit;        /* [B] */
+    int32_t* status;          /* [B] */
+} hvd_host_step_args;
+
+HVD_API hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

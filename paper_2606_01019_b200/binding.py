@@ -30,6 +30,15 @@ class HvdConfig(C.Structure):
                 ("max_hist_len", _i32), ("max_rows", _i64), ("max_vocab", _i64)]
 
 
+class HvdHostStepArgs(C.Structure):
+    _fields_ = [("B", _i32), ("n_max", _i32), ("hist_words", _i64), ("hist", _vp), ("hist_off", _vp),
+                ("hist_cap", _vp), ("hist_len", _vp), ("K", _vp), ("prompt_len", _vp), ("state", _vp),
+                ("model_draft", _vp), ("model_len", _vp), ("logits", _vp), ("dtype", _i32),
+                ("k_uniform", _i32), ("V", _i64), ("row_off", _vp), ("total_rows", _i64),
+                ("score", _vp), ("select", _vp), ("sel_draft", _vp), ("sel_len", _vp), ("accepted", _vp),
+                ("committed", _vp), ("n_commit", _vp), ("status", _vp)]
+
+
 _SIGNATURES = {
     "hvd_create": (_i32, [C.POINTER(_vp), C.POINTER(HvdConfig)]),
     "hvd_destroy": (_i32, [_vp]),
@@ -39,6 +48,7 @@ _SIGNATURES = {
     "hvd_lookup": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
+    "hvd_step_host": (_i32, [_vp, C.POINTER(HvdHostStepArgs), _vp]),
 }
 
 _lib = None
@@ -72,6 +82,13 @@ def load_library(build: bool = True):
 
 def _ptr(t):
     return None if t is None else t.data_ptr()
+
+
+def _hptr(a):
+    """Address of a host array: a torch CPU tensor (pinned or not) or a numpy array."""
+    if a is None:
+        return None
+    return a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data
 
 
 def _stream():
@@ -147,3 +164,16 @@ class Context:
                                                 _ptr(committed), _ptr(n_commit), _ptr(target_tok),
                                                 _ptr(status), _stream()),
                     "hvd_verify_commit")
+
+    def hvd_step_host(self, *, B, n_max, hist, hist_off, hist_cap, hist_len, K, prompt_len, state,
+                      model_draft, model_len, logits, dtype, V, row_off, k_uniform, total_rows, score,
+                      select, sel_draft, sel_len, accepted, committed, n_commit, status):
+        """All arrays are HOST arrays (torch CPU tensors, ideally pinned, or numpy arrays)."""
+        hist_words = hist.numel() if hasattr(hist, "numel") else hist.size
+        args = HvdHostStepArgs(B, n_max, hist_words, _hptr(hist), _hptr(hist_off), _hptr(hist_cap),
+                               _hptr(hist_len), _hptr(K), _hptr(prompt_len), _hptr(state),
+                               _hptr(model_draft), _hptr(model_len), _hptr(logits), dtype, k_uniform, V,
+                               _hptr(row_off), total_rows, _hptr(score), _hptr(select), _hptr(sel_draft),
+                               _hptr(sel_len), _hptr(accepted), _hptr(committed), _hptr(n_commit),
+                               _hptr(status))
+        self._check(self._lib.hvd_step_host(self._h, C.byref(args), _stream()), "hvd_step_host")

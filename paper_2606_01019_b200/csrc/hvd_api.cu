@@ -14,6 +14,7 @@ void release(hvd_ctx* c) {
     cudaFree(c->d_W1); cudaFree(c->d_b1); cudaFree(c->d_W2);
     cudaFree(c->lk_partial); cudaFree(c->lk_cnt);
     cudaFree(c->vf_partial); cudaFree(c->vf_cnt); cudaFree(c->vf_ctrl);
+    cudaFree(c->host_ws);
     delete c;
 }
 
@@ -86,6 +87,8 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->vf_blocks_per_sm[1] = verify_occupancy(HVD_BF16, smem);
     if (c->vf_blocks_per_sm[0] < 1 || c->vf_blocks_per_sm[1] < 1) { release(c); return HVD_ERR_UNSUPPORTED; }
     c->has_predictor = false;
+    c->host_ws = nullptr;
+    c->host_ws_bytes = 0;
     *out = c;
     return HVD_OK;
 }

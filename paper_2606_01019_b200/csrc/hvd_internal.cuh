@@ -51,6 +51,9 @@ struct hvd_ctx {
     hvd::Ctrl* vf_ctrl;              // zero at rest
     int64_t vf_max_seg;
     int vf_blocks_per_sm[2];         // per dtype
+    // device staging of the host-buffer entry point (grown on demand)
+    char* host_ws;
+    size_t host_ws_bytes;
     char last_error[256];
 };
 

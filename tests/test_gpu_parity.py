@@ -68,3 +68,36 @@ def test_multi_step_loop_and_scratch_reuse():
                                               rq=rq, batch=batch)
         assert (rq.hist_len > inp.rq.hist_len).all()
         ctx.close()
+
+
+def test_host_buffer_entry_point():
+    """hvd_step_host: same step with host arrays in and out (copies inside the call)."""
+    import paper_2606_01019_b200 as H
+    for name, kw in (("C1", {}), ("C5", dict(B=24, n=(64, 3000), V=20011))):
+        w = W.CONFIGS[name].scaled(**kw)
+        inp = P.prepare(w, device="cpu")
+        rq_g, rq_o = inp.rq.copy(), inp.rq.copy()
+        ctx = G.make_ctx(w, rq_g)
+        ctx.hvd_set_predictor(inp.W1, inp.b1, inp.W2, inp.b2, inp.tau)
+        B, kc = rq_g.B, w.k_cap
+        o = dict(score=np.zeros(B, np.float32), select=np.zeros(B, np.int32), sel_draft=np.zeros((B, kc), np.int32),
+                 sel_len=np.zeros(B, np.int32), accepted=np.zeros(B, np.int32),
+                 committed=np.zeros((B, kc + 1), np.int32), n_commit=np.zeros(B, np.int32),
+                 status=np.zeros(B, np.int32))
+        for rep in range(2):       # second call: staging area reused, histories have grown
+            ctx.hvd_step_host(B=B, n_max=int(rq_g.hist_cap.max()), hist=rq_g.hist, hist_off=rq_g.hist_off,
+                              hist_cap=rq_g.hist_cap, hist_len=rq_g.hist_len, K=rq_g.K, prompt_len=rq_g.prompt_len,
+                              state=rq_g.state, model_draft=rq_g.model_draft, model_len=rq_g.model_len,
+                              logits=inp.logits_np, dtype=H.F32 if w.dtype == "f32" else H.BF16, V=w.V,
+                              row_off=rq_g.row_off, k_uniform=0, total_rows=int(rq_g.row_off[-1]), **o)
+            out = P.step(inp, rq_o)
+            G.assert_equal("score", o["score"], out.sc.score)
+            for k in ("select", "sel_draft", "sel_len"):
+                G.assert_equal(k, o[k], getattr(out.sc, k))
+            for k in ("accepted", "committed", "n_commit", "status"):
+                G.assert_equal(k, o[k], getattr(out.vf, k))
+            G.assert_equal("hist", rq_g.hist, rq_o.hist)
+            G.assert_equal("hist_len", rq_g.hist_len, rq_o.hist_len)
+            G.assert_equal("acc_ring", rq_g.state["acc_ring"], rq_o.state["acc_ring"])
+            G.assert_equal("sel_bits", rq_g.state["sel_bits"], rq_o.state["sel_bits"])
+        ctx.close()
