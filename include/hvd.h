@@ -96,6 +96,10 @@ HVD_API const char* hvd_status_string(hvd_status s);
 /* text of the last error recorded on this context ("" if none) */
 HVD_API const char* hvd_last_error(const hvd_ctx* ctx);
 
+/* Device-side status of the context: *code = 0 if every kernel ran to completion, 1 if a kernel
+   gave up a bounded wait (its outputs are then incomplete).  Waits for the device (HOST pointer). */
+HVD_API hvd_status hvd_device_status(hvd_ctx* ctx, int32_t* code);
+
 /* Payoff predictor g_theta (Sec. 3.3): y = b2 + sum_j W2[j] * relu(b1[j] + sum_i W1[j][i] * phi[i]),
    fp32, accumulated left to right with fused multiply-adds, and the threshold tau of Sec. 3.4.
    W1 [hidden, 8] row-major, b1 [hidden], W2 [hidden]: HOST pointers, copied before returning. */

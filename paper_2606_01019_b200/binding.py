@@ -44,6 +44,7 @@ _SIGNATURES = {
     "hvd_destroy": (_i32, [_vp]),
     "hvd_status_string": (C.c_char_p, [_i32]),
     "hvd_last_error": (C.c_char_p, [_vp]),
+    "hvd_device_status": (_i32, [_vp, C.POINTER(_i32)]),
     "hvd_set_predictor": (_i32, [_vp, _vp, _vp, _vp, _f32, _f32, _vp]),
     "hvd_lookup": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
@@ -129,6 +130,11 @@ class Context:
         if st != 0:
             raise HvdError(f"{what}: {self._lib.hvd_status_string(st).decode()}: "
                            f"{self._lib.hvd_last_error(self._h).decode()}")
+
+    def hvd_device_status(self) -> int:
+        code = _i32(0)
+        self._check(self._lib.hvd_device_status(self._h, C.byref(code)), "hvd_device_status")
+        return int(code.value)
 
     def hvd_set_predictor(self, W1, b1, W2, b2, tau):
         W1 = np.ascontiguousarray(W1, np.float32); b1 = np.ascontiguousarray(b1, np.float32)

@@ -9,7 +9,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
-LIB = os.path.join(PKG, "libhvd_b200.so")
+LIB = os.environ.get("HVD_B200_LIB") or os.path.join(PKG, "libhvd_b200.so")
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--shared"]
@@ -27,13 +27,17 @@ def stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, defines=()) -> str:
+    """`defines` adds -D flags (compile-time tunables of the kernels)."""
+    if os.environ.get("HVD_B200_LIB") and os.path.exists(LIB) and not force:
+        return LIB       # an explicitly chosen library is used as it is
     if not (force or stale()):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += [f"-D{d}" for d in defines]
     cmd += ["-o", LIB, *sources()]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:

@@ -1,4 +1,6 @@
 // C ABI of the library: context management, argument checks, kernel launches.
+#include <stdlib.h>
+
 #include <new>
 
 #include "hvd_internal.cuh"
@@ -13,7 +15,7 @@ void release(hvd_ctx* c) {
     if (!c) return;
     cudaFree(c->d_W1); cudaFree(c->d_b1); cudaFree(c->d_W2);
     cudaFree(c->lk_partial); cudaFree(c->lk_cnt);
-    cudaFree(c->vf_partial); cudaFree(c->vf_cnt); cudaFree(c->vf_ctrl);
+    cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
     delete c;
 }
@@ -64,10 +66,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     if (e != cudaSuccess) { delete c; return HVD_ERR_CUDA; }
 
     c->lk_max_chunks = (int)(((int64_t)cfg->max_hist_len + 3 + kLookupMinChunk - 1) / kLookupMinChunk);
-    // work items per row for the narrowest element (4 bytes): an upper bound for every dtype
-    c->vf_max_seg = (cfg->max_vocab * 4 / 16 + kVerifyVecPerItem - 1) / kVerifyVecPerItem;
-    if (c->vf_max_seg < 1) c->vf_max_seg = 1;
-    if (cfg->max_rows * c->vf_max_seg >= 0x7fffffffLL) { delete c; return HVD_ERR_INVALID_ARG; }
+    if (cfg->max_rows >= 0x7fffffffLL) { delete c; return HVD_ERR_INVALID_ARG; }
 
     const size_t H = (size_t)cfg->hidden;
     bool ok = true;
@@ -76,9 +75,9 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->d_W2, H * sizeof(float)) == cudaSuccess;
     ok = ok && alloc_zero(&c->lk_partial, (size_t)cfg->max_batch * c->lk_max_chunks * sizeof(LookupPartial)) == cudaSuccess;
     ok = ok && alloc_zero(&c->lk_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
-    ok = ok && alloc_zero(&c->vf_partial, (size_t)cfg->max_rows * c->vf_max_seg * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && alloc_zero(&c->vf_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
-    ok = ok && alloc_zero(&c->vf_ctrl, sizeof(Ctrl)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->vf_row_key, (size_t)cfg->max_rows * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->vf_next_unit, (size_t)kVerifyQueues * 32 * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->dev_error, sizeof(int)) == cudaSuccess;
     if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); release(c); return HVD_ERR_ALLOC; }
 
@@ -89,13 +88,35 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->has_predictor = false;
     c->host_ws = nullptr;
     c->host_ws_bytes = 0;
+#ifdef HVD_TRACE
+    c->trace_words = (size_t)c->num_sms * 64 * 8;
+    alloc_zero(&c->trace, c->trace_words * 8);
+#endif
     *out = c;
     return HVD_OK;
 }
 
 hvd_status hvd_destroy(hvd_ctx* ctx) {
     if (!ctx) return HVD_ERR_INVALID_ARG;
+#ifdef HVD_TRACE
+    if (const char* path = getenv("HVD_TRACE_FILE")) {
+        unsigned long long* h = (unsigned long long*)malloc(ctx->trace_words * 8);
+        cudaDeviceSynchronize();
+        cudaMemcpy(h, ctx->trace, ctx->trace_words * 8, cudaMemcpyDeviceToHost);
+        if (FILE* f = fopen(path, "wb")) { fwrite(h, 8, ctx->trace_words, f); fclose(f); }
+        free(h);
+    }
+    cudaFree(ctx->trace);
+#endif
     release(ctx);
+    return HVD_OK;
+}
+
+hvd_status hvd_device_status(hvd_ctx* ctx, int32_t* code) {
+    if (!ctx || !code) return HVD_ERR_INVALID_ARG;
+    int v = 0;
+    HVD_CUDA_TRY(ctx, cudaMemcpy(&v, ctx->dev_error, sizeof(int), cudaMemcpyDeviceToHost));
+    *code = v;
     return HVD_OK;
 }
 
@@ -184,12 +205,12 @@ hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dt
     a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.state = state;
     a.accepted = accepted; a.committed = committed; a.n_commit = n_commit; a.target_tok = target_tok;
     a.status = status; a.k_cap = ctx->cfg.k_cap;
-    a.partial = ctx->vf_partial; a.req_cnt = ctx->vf_cnt; a.ctrl = ctx->vf_ctrl;
-    const int64_t vec_per_row = V * (int64_t)esz / 16;
-    int64_t n_seg = (vec_per_row + kVerifyVecPerItem - 1) / kVerifyVecPerItem;
-    if (n_seg < 1) n_seg = 1;
-    if (n_seg > ctx->vf_max_seg) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: V exceeds the scratch sized at create");
-    a.n_seg = (int32_t)n_seg;
+    
+#ifdef HVD_TRACE
+    a.trace = ctx->trace;
+#endif
+    a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error;
+    a.row_key = ctx->vf_row_key; a.total_rows = total_rows;
     return launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
 }
 

@@ -20,14 +20,27 @@ constexpr int kLookupThreads = 256;
 constexpr int kLookupTokPerVec = 4;
 constexpr int kLookupMinChunk = kLookupThreads * kLookupTokPerVec;  // tokens, one 128-bit load per thread
 
-constexpr int kVerifyThreads = 256;
-constexpr int kVerifyUnroll = 8;                                   // 128-bit loads in flight per thread
-constexpr int kVerifyVecPerItem = kVerifyThreads * kVerifyUnroll;  // 32 KB of logits per work item
+// tunables of the verify kernel (overridable at compile time for experiments)
+#ifndef HVD_VERIFY_THREADS
+#define HVD_VERIFY_THREADS 256
+#endif
+#ifndef HVD_VERIFY_UNROLL
+#define HVD_VERIFY_UNROLL 8
+#endif
+#ifndef HVD_VERIFY_MIN_BLOCKS
+#define HVD_VERIFY_MIN_BLOCKS 4
+#endif
+constexpr int kVerifyThreads = HVD_VERIFY_THREADS;
+constexpr int kVerifyUnroll = HVD_VERIFY_UNROLL;      // 128-bit loads in flight per lane
+#ifndef HVD_VERIFY_UNIT_BATCHES
+#define HVD_VERIFY_UNIT_BATCHES 2
+#endif
+constexpr int kVerifyUnitBatches = HVD_VERIFY_UNIT_BATCHES;  // 4 KB batches per unit drawn by a warp
+#ifndef HVD_VERIFY_QUEUES
+#define HVD_VERIFY_QUEUES 4
+#endif
+constexpr int kVerifyQueues = HVD_VERIFY_QUEUES;  // unit counters
 
-struct Ctrl {
-    uint32_t next_item;      // dynamic work counter of the verify kernel (zero at rest)
-    uint32_t blocks_exited;  // blocks that left the verify work loop (zero at rest)
-};
 
 }  // namespace hvd
 
@@ -46,14 +59,17 @@ struct hvd_ctx {
     uint32_t* lk_cnt;                // [max_batch], zero at rest
     int lk_max_chunks;
     // verify scratch
-    unsigned long long* vf_partial;  // [max_rows, vf_max_seg]
-    uint32_t* vf_cnt;                // [max_batch], zero at rest
-    hvd::Ctrl* vf_ctrl;              // zero at rest
-    int64_t vf_max_seg;
+    unsigned long long* vf_row_key;  // [max_rows], zero at rest
+    uint32_t* vf_next_unit;          // zero at rest
+    int* dev_error;                  // device status word
     int vf_blocks_per_sm[2];         // per dtype
     // device staging of the host-buffer entry point (grown on demand)
     char* host_ws;
     size_t host_ws_bytes;
+#ifdef HVD_TRACE
+    unsigned long long* trace;  // [num_sms * 64 warps * 8] last verify launch, dumped by hvd_destroy
+    size_t trace_words;
+#endif
     char last_error[256];
 };
 
@@ -109,13 +125,17 @@ struct VerifyArgs {
     int32_t* status;
     int32_t k_cap;
     // scratch
-    unsigned long long* partial;
-    uint32_t* req_cnt;
-    Ctrl* ctrl;
-    int32_t n_seg;  // work items per row
+    unsigned long long* row_key;  // [total_rows] (value, ~index) key per logits row, zero at rest
+    int64_t total_rows;
+    uint32_t* next_unit;   // unit counter, zero at rest
+    int* dev_error;        // device status word (no kernel sets it at present)
+    int32_t n_batch_row;   // 4 KB batches per row
+#ifdef HVD_TRACE
+    unsigned long long* trace;  // per-warp timeline (debug builds only)
+#endif
 };
 
-hvd_status launch_verify(hvd_ctx* ctx, const VerifyArgs& a, hvd_dtype dtype, cudaStream_t stream);
+hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream);
 int verify_occupancy(hvd_dtype dtype, size_t dyn_smem);
 size_t verify_dyn_smem(int32_t B);
 

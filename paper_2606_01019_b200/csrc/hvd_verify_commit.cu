@@ -1,12 +1,27 @@
-// Greedy verification and commit (Sec. 3.1 Verify, Sec. 3.4, Algorithm 1).
+// Greedy verification and commit (Sec. 3.1 Verify, Sec. 3.4, Algorithm 1), as two kernels.
 //
-// The step is a bandwidth-bound stream over the logits rows that are actually needed
-// (rows 0..sel_len of each request).  Those rows are cut into work items of kVerifyVecPerItem
-// 128-bit vectors (32 KB); persistent CTAs draw items from a counter, so SMs that get less DRAM
-// bandwidth simply take fewer items.  Per item every thread issues all its loads at once, keeps a
-// packed running maximum, and the CTA reduces (value, lowest index) to one 64-bit key that it
-// leaves in scratch.  The CTA that delivers the last item of a request turns the keys into target
-// tokens, compares them with the draft, and commits.  No CTA waits for another.
+// verify_stream_kernel: a bandwidth-bound stream over the logits rows that are actually needed
+// (rows 0..sel_len of each request).  Under that stream every other global access takes
+// microseconds, so the streaming warps touch global memory for nothing but the logits, one
+// counter fetch that is issued two units before its answer is needed, and fire-and-forget atomic
+// maxima:
+//  * Phase 0 (once per CTA): the number of needed rows per request, its prefix over requests and
+//    the first logits row of each request go to shared memory.  The needed rows, laid end to
+//    end, are cut into batches of 32*kVerifyUnroll 128-bit vectors (4 KB: what one warp loads with
+//    all its loads in flight) and into units of kVerifyUnitBatches batches.
+//  * Warps draw units from kVerifyQueues global counters (unit numbers interleaved over the
+//    queues; one counter cannot serve more than one fetch per ~1.5 ns under load), so SMs that
+//    get less DRAM bandwidth take fewer units (per-SM rates differ by up to 2x on this part, and
+//    static splits lose a third of the bandwidth to the slowest SMs).  A warp whose queue runs
+//    dry tries the next queue once.
+//  * A lane keeps, for each of its packed element slots, the running maximum and the load that
+//    raised it (three instructions per two bf16 logits); one warp reduction per batch gives the
+//    exact (maximum, lowest index), which is folded into the row's 64-bit key in global scratch
+//    with an atomic max whose result nobody waits for.
+// verify_commit_kernel: one warp per request reads the row keys (the kernel boundary orders them
+// after every atomic), turns them into target tokens, compares them with the draft, commits, and
+// puts the scratch back to zero.
+// No warp waits for another.
 #include <cuda_bf16.h>
 
 #include "hvd_internal.cuh"
@@ -15,10 +30,18 @@ namespace hvd {
 namespace {
 
 constexpr int T = kVerifyThreads;
+constexpr int NW = T / 32;
 constexpr int U = kVerifyUnroll;
+constexpr int UB = kVerifyUnitBatches;
+constexpr int Q = kVerifyQueues;
+constexpr int kQueueStride = 32;  // counters sit on separate 128-byte lines
+static_assert(NW % Q == 0, "every CTA must serve every queue equally");
+constexpr int kBatchVec = 32 * U;  // vectors a warp loads per batch
 constexpr uint32_t kFull = 0xffffffffu;
+static_assert(U <= 8, "the load number must fit the packed 16-bit tracking");
 
-// order-preserving map float -> uint32 with -0.0 folded onto +0.0
+// order-preserving map float -> uint32 with -0.0 folded onto +0.0 (0 is never produced by a
+// non-NaN value, so 0 can stand for "nothing")
 __device__ __forceinline__ uint32_t ord32(float f) {
     uint32_t b = __float_as_uint(f);
     if ((b << 1) == 0) b = 0;
@@ -33,100 +56,135 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     return v;
 }
 
+// Per-lane argmax over the (up to) U vectors of one batch.  best(): order key of the maximum and
+// the offset, inside the batch, of its first occurrence: (load u * 32 + lane) * kPerVec + k.
 template <typename E>
-struct Elem;
+struct Tracker;
 
 template <>
-struct Elem<float> {
+struct Tracker<float> {
     static constexpr int kPerVec = 4;
-    static constexpr uint32_t kFillWord = 0xff800000u;  // -inf
+    float v[4];
+    int u[4];
     __device__ static __forceinline__ float scalar(const void* row, int64_t i) {
         return static_cast<const float*>(row)[i];
     }
-    __device__ static __forceinline__ float get(const uint4& v, int k) {
-        const uint32_t w = k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w;
-        return __uint_as_float(w);
+    __device__ __forceinline__ void init(const uint4& x) {
+        v[0] = __uint_as_float(x.x); v[1] = __uint_as_float(x.y);
+        v[2] = __uint_as_float(x.z); v[3] = __uint_as_float(x.w);
+        u[0] = u[1] = u[2] = u[3] = 0;
     }
-    // maximum of the U vectors held by one thread
-    __device__ static __forceinline__ float thread_max(const uint4 (&x)[U]) {
-        float m0 = __uint_as_float(x[0].x), m1 = __uint_as_float(x[0].y);
-        float m2 = __uint_as_float(x[0].z), m3 = __uint_as_float(x[0].w);
+    __device__ __forceinline__ void fold(const uint4& x, int load) {
+        const float y[4] = {__uint_as_float(x.x), __uint_as_float(x.y), __uint_as_float(x.z), __uint_as_float(x.w)};
 #pragma unroll
-        for (int u = 1; u < U; ++u) {
-            m0 = fmaxf(m0, __uint_as_float(x[u].x)); m1 = fmaxf(m1, __uint_as_float(x[u].y));
-            m2 = fmaxf(m2, __uint_as_float(x[u].z)); m3 = fmaxf(m3, __uint_as_float(x[u].w));
+        for (int k = 0; k < 4; ++k)
+            if (y[k] > v[k]) { v[k] = y[k]; u[k] = load; }
+    }
+    __device__ __forceinline__ void best(int lane, uint32_t& ord, uint32_t& off) const {
+        ord = 0u; off = 0xffffffffu;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t o = ord32(v[k]);
+            const uint32_t f = (uint32_t)((u[k] * 32 + lane) * 4 + k);
+            if (o > ord || (o == ord && f < off)) { ord = o; off = f; }
         }
-        return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     }
 };
 
 template <>
-struct Elem<__nv_bfloat16> {
+struct Tracker<__nv_bfloat16> {
     static constexpr int kPerVec = 8;
-    static constexpr uint32_t kFillWord = 0xff80ff80u;  // two bf16 -inf
+    uint32_t v[4];  // packed maxima: element 2c in the low half of v[c], 2c+1 in the high half
+    uint32_t u[4];  // packed load numbers, same layout
     __device__ static __forceinline__ float scalar(const void* row, int64_t i) {
-        return __uint_as_float((uint32_t)static_cast<const uint16_t*>(row)[i] << 16);
-    }
-    __device__ static __forceinline__ float get(const uint4& v, int k) {
-        const uint32_t w = (k >> 1) == 0 ? v.x : (k >> 1) == 1 ? v.y : (k >> 1) == 2 ? v.z : v.w;
-        return __uint_as_float((k & 1) ? (w & 0xffff0000u) : (w << 16));  // widening is exact
+        return __uint_as_float((uint32_t)static_cast<const uint16_t*>(row)[i] << 16);  // widening is exact
     }
     __device__ static __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
         uint32_t d;
         asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
         return d;
     }
-    __device__ static __forceinline__ float thread_max(const uint4 (&x)[U]) {
-        uint32_t m0 = x[0].x, m1 = x[0].y, m2 = x[0].z, m3 = x[0].w;
+    __device__ static __forceinline__ uint32_t gt2(uint32_t a, uint32_t b) {  // 0xffff per half with a > b
+        uint32_t d;
+        asm("set.gt.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+        return d;
+    }
+    __device__ __forceinline__ void init(const uint4& x) {
+        v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+        u[0] = u[1] = u[2] = u[3] = 0u;
+    }
+    __device__ __forceinline__ void fold(const uint4& x, int load) {
+        const uint32_t y[4] = {x.x, x.y, x.z, x.w};
+        const uint32_t tag = (uint32_t)load * 0x00010001u;
 #pragma unroll
-        for (int u = 1; u < U; ++u) {
-            m0 = max2(m0, x[u].x); m1 = max2(m1, x[u].y);
-            m2 = max2(m2, x[u].z); m3 = max2(m3, x[u].w);
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t m = gt2(y[c], v[c]);
+            v[c] = max2(v[c], y[c]);
+            u[c] = (u[c] & ~m) | (tag & m);
         }
-        const uint32_t m = max2(max2(m0, m1), max2(m2, m3));
-        return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
+    }
+    __device__ __forceinline__ void best(int lane, uint32_t& ord, uint32_t& off) const {
+        ord = 0u; off = 0xffffffffu;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t bits = h ? (v[c] & 0xffff0000u) : (v[c] << 16);
+                const uint32_t load = h ? (u[c] >> 16) : (u[c] & 0xffffu);
+                const uint32_t o = ord32(__uint_as_float(bits));
+                const uint32_t f = (load * 32u + (uint32_t)lane) * 8u + (uint32_t)(2 * c + h);
+                if (o > ord || (o == ord && f < off)) { ord = o; off = f; }
+            }
+        }
     }
 };
 
-// number of needed rows of request b (0 = request skipped) and its first logits row
-__device__ __forceinline__ int needed_rows(const VerifyArgs& a, int b, int64_t* r0_out) {
-    int64_t r0, r1;
-    if (a.row_off) { r0 = a.row_off[b]; r1 = a.row_off[b + 1]; }
-    else { r0 = (int64_t)b * (a.k_uniform + 1); r1 = r0 + a.k_uniform + 1; }
-    *r0_out = r0;
+struct Req {
+    int64_t r0, r1;  // logits rows of the request
+    int nr;          // rows needed = sel_len + 1 (0: request skipped)
+};
+
+__device__ __forceinline__ Req load_req(const VerifyArgs& a, int b) {
+    Req q;
+    if (a.row_off) { q.r0 = a.row_off[b]; q.r1 = a.row_off[b + 1]; }
+    else { q.r0 = (int64_t)b * (a.k_uniform + 1); q.r1 = q.r0 + a.k_uniform + 1; }
     const int n = a.hist_len[b];
-    if (n < 0 || n > a.hist_cap[b] || r1 <= r0) return 0;
-    int m = a.sel_len[b];
-    m = max(0, min(m, a.k_cap));
-    if ((int64_t)m > r1 - r0 - 1) m = (int)(r1 - r0 - 1);
-    return m + 1;
+    q.nr = 0;
+    if (n >= 0 && n <= a.hist_cap[b] && q.r1 > q.r0) {
+        int m = max(0, min(a.sel_len[b], a.k_cap));
+        if ((int64_t)m > q.r1 - q.r0 - 1) m = (int)(q.r1 - q.r0 - 1);
+        q.nr = m + 1;
+    }
+    return q;
 }
 
-// Commit of one request by one warp, after all its row partials are in scratch.
-__device__ void commit_request(const VerifyArgs& a, int b, int pref_b, int nr, int lane) {
-    int64_t r0;
-    (void)needed_rows(a, b, &r0);
-    const int64_t r1 = a.row_off ? a.row_off[b + 1] : r0 + a.k_uniform + 1;
-    const int m = nr - 1;
+// Commit of one request by one warp, after all its needed rows are folded into the row keys.
+__device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int lane) {
+    const Req q = load_req(a, b);
     const int kc = a.k_cap;
+    int32_t* z = a.committed + (int64_t)b * (kc + 1);
+    if (q.nr == 0) {
+        // skipped request: neutral outputs, nothing else touched
+        for (int j = lane; j <= kc; j += 32) z[j] = -1;
+        if (a.target_tok) for (int64_t r = q.r0 + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
+        if (lane == 0) { a.accepted[b] = 0; a.n_commit[b] = 0; a.status[b] = HVD_REQ_BAD_LEN; }
+        return;
+    }
+    const int m = q.nr - 1;
     const int32_t* d = a.sel_draft + (int64_t)b * kc;
     int acc = -1;
     int t_acc = 0;
-    // rows in rounds of 32: lane handles row i, finds its target token and compares with the draft
+    // rows in rounds of 32: lane handles row i, reads its target token, compares with the draft
     for (int base = 0; base <= m; base += 32) {
         const int i = base + lane;
         int t = 0;
         bool stop = true;
         if (i <= m) {
-            unsigned long long key = 0;
-            const unsigned long long* p = a.partial + (int64_t)(pref_b + i) * a.n_seg;
-            for (int s = 0; s < a.n_seg; ++s) {
-                const unsigned long long k = __ldcg(p + s);
-                key = k > key ? k : key;
-            }
+            const unsigned long long key = a.row_key[q.r0 + i];
+            a.row_key[q.r0 + i] = 0ull;  // scratch is zero at rest
             t = (int)(~(uint32_t)(key & 0xffffffffu));
-            t = (int)min((int64_t)max(t, 0), a.V - 1);  // stays inside the vocabulary whatever the data
-            if (a.target_tok) a.target_tok[r0 + i] = t;
+            t = (int)min((int64_t)max(t, 0), a.V - 1);  // inside the vocabulary whatever the data
+            if (a.target_tok) a.target_tok[q.r0 + i] = t;
             stop = (i >= m) || (d[i] != t);
         }
         const uint32_t stops = __ballot_sync(kFull, stop);
@@ -138,8 +196,7 @@ __device__ void commit_request(const VerifyArgs& a, int b, int pref_b, int nr, i
     }
     // acc <= m always (row m stops).  Rows beyond m were not read.
     if (a.target_tok)
-        for (int64_t r = r0 + nr + lane; r < r1; r += 32) a.target_tok[r] = -1;
-    int32_t* z = a.committed + (int64_t)b * (kc + 1);
+        for (int64_t r = q.r0 + q.nr + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
     const int n = a.hist_len[b];
     const int room = a.hist_cap[b] - n;
     const int w = min(acc + 1, room);
@@ -158,195 +215,213 @@ __device__ void commit_request(const VerifyArgs& a, int b, int pref_b, int nr, i
         st.sel_bits = (st.sel_bits << 1) | (a.select[b] ? 1u : 0u);
         st.acc_ring = (st.acc_ring << 8) | (unsigned long long)(acc & 0xff);
         a.state[b] = st;
-        a.req_cnt[b] = 0;  // scratch is zero at rest
     }
 }
 
+constexpr int kCommitWarps = 4;
+
+__global__ void __launch_bounds__(kCommitWarps * 32) verify_commit_kernel(const VerifyArgs a) {
+    const int b = blockIdx.x * kCommitWarps + (threadIdx.x >> 5);
+    if (b == 0 && (threadIdx.x & 31) < Q) a.next_unit[(threadIdx.x & 31) * kQueueStride] = 0u;  // zero at rest
+    if (b < a.B) commit_request(a, b, threadIdx.x & 31);
+}
+
+struct Smem {
+    long long* row0;  // [B] first logits row of each request
+    int* pref;        // [B+1] exclusive prefix of needed rows over requests
+    __device__ __forceinline__ Smem(unsigned char* base, int B) {
+        row0 = reinterpret_cast<long long*>(base);
+        pref = reinterpret_cast<int*>(base + (size_t)B * 8);
+    }
+};
+
+#ifdef HVD_TRACE
+__device__ __forceinline__ unsigned long long gtime() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define TR(...) __VA_ARGS__
+#else
+#define TR(...)
+#endif
+
 template <typename E>
-__global__ void __launch_bounds__(T) verify_commit_kernel(const VerifyArgs a) {
-    extern __shared__ int s_pref[];  // [B+1] exclusive prefix of needed rows
-    __shared__ uint32_t s_wmax[T / 32];
-    __shared__ uint32_t s_minidx;
-    __shared__ uint32_t s_next;
+__global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel(const VerifyArgs a) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    __shared__ int s_wsum[NW];
     __shared__ int s_carry;
+    const Smem sm(s_raw, a.B);
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    constexpr int EPV = Elem<E>::kPerVec;
+    constexpr int EPV = Tracker<E>::kPerVec;
     constexpr int ESZ = 16 / EPV;
+    TR(unsigned long long t_enter = gtime(); unsigned long long acc_wait = 0, acc_str = 0, acc_close = 0, n_b = 0;)
 
-    // ---- phase 0: which rows are needed (device data), prefix over requests -----------------
-    if (tid == 0) { s_carry = 0; s_pref[0] = 0; }
+    // Unit u belongs to queue u % Q.  The first unit of a warp is the one with its own number
+    // (queue warp % Q); the next one is requested now and its answer is looked at after the first
+    // unit has been streamed.
+    const uint32_t n_warps = gridDim.x * (uint32_t)NW;
+    uint32_t cur = blockIdx.x * (uint32_t)NW + (uint32_t)warp;
+    int queue = warp % Q;
+    int tries = 0;  // queues found dry so far
+    auto fetch = [&](int q) { return (n_warps / Q + atomicAdd(a.next_unit + q * kQueueStride, 1u)) * Q + (uint32_t)q; };
+    uint32_t nxt = 0;
+    if (lane == 0) nxt = fetch(queue);
+
+    // ---- phase 0: rows needed per request (device data), prefix over requests ----------------------
+    if (tid == 0) { s_carry = 0; sm.pref[0] = 0; }
     __syncthreads();
     for (int base = 0; base < a.B; base += T) {
         const int b = base + tid;
-        int64_t r0 = 0;
-        const int nr = (b < a.B) ? needed_rows(a, b, &r0) : 0;
-        if (b < a.B && nr == 0 && blockIdx.x == 0) {
-            // skipped request: neutral outputs, nothing else touched
-            const int64_t r1 = a.row_off ? a.row_off[b + 1] : r0 + a.k_uniform + 1;
-            a.accepted[b] = 0; a.n_commit[b] = 0; a.status[b] = HVD_REQ_BAD_LEN;
-            for (int j = 0; j <= a.k_cap; ++j) a.committed[(int64_t)b * (a.k_cap + 1) + j] = -1;
-            if (a.target_tok) for (int64_t r = r0; r < r1; ++r) a.target_tok[r] = -1;
+        int nr = 0;
+        if (b < a.B) {
+            const Req q = load_req(a, b);
+            nr = q.nr;
+            sm.row0[b] = q.r0;
         }
-        // inclusive scan of nr over the tile
-        int v = nr;
+        int v = nr;  // inclusive scan of nr over the tile
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const int o = __shfl_up_sync(kFull, v, off);
             if (lane >= off) v += o;
         }
-        __shared__ int s_wsum[T / 32];
         if (lane == 31) s_wsum[warp] = v;
         __syncthreads();
         int wbase = 0;
 #pragma unroll
-        for (int k = 0; k < T / 32; ++k) wbase += (k < warp) ? s_wsum[k] : 0;
+        for (int k = 0; k < NW; ++k) wbase += (k < warp) ? s_wsum[k] : 0;
         const int carry = s_carry;
-        if (b < a.B) s_pref[b + 1] = carry + wbase + v;
+        if (b < a.B) sm.pref[b + 1] = carry + wbase + v;
         __syncthreads();
         if (tid == T - 1) s_carry = carry + wbase + v;
         __syncthreads();
     }
-    const int total_rows = s_pref[a.B];
-    const uint32_t total_items = (uint32_t)total_rows * (uint32_t)a.n_seg;
 
-    if (tid == 0) s_next = atomicAdd(&a.ctrl->next_item, 1u);
-    __syncthreads();
-    uint32_t cur = s_next;
-
-    const int64_t row_bytes = a.V * ESZ;
+    const int nbr = a.n_batch_row;
+    const int64_t total = (int64_t)sm.pref[a.B] * nbr;  // batches of all needed rows
+    const uint32_t n_units = (uint32_t)((total + UB - 1) / UB);
     const char* base_ptr = static_cast<const char*>(a.logits);
+    TR(unsigned long long t_loop = gtime();)
 
-    while (cur < total_items) {
-        uint32_t nxt = 0;
-        if (tid == 0) nxt = atomicAdd(&a.ctrl->next_item, 1u);  // overlaps with this item's loads
-
-        // ---- decode the item -> (request b, row i, segment s) ------------------------------
-        const int r = (int)(cur / (uint32_t)a.n_seg);
-        const int s = (int)(cur - (uint32_t)r * (uint32_t)a.n_seg);
-        int lo = 0, hi = a.B;  // largest b with s_pref[b] <= r
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (s_pref[mid] <= r) lo = mid; else hi = mid;
+    // ---- phase 1: units of batches -------------------------------------------------------------------
+    while (cur < n_units) {
+        TR(unsigned long long tw0 = gtime();)
+        nxt = __shfl_sync(kFull, nxt, 0);
+        if (nxt >= n_units && tries == 0) {  // own queue is dry: one look at the neighbour queue
+            tries = 1;
+            queue = (queue + 1) % Q;
+            if (lane == 0) nxt = fetch(queue);
+            nxt = __shfl_sync(kFull, nxt, 0);
         }
-        const int b = lo;
-        const int i = r - s_pref[b];
-        const int64_t row0 = a.row_off ? a.row_off[b] : (int64_t)b * (a.k_uniform + 1);
-        const char* row = base_ptr + (row0 + i) * row_bytes;
+        uint32_t nn = 0;
+        if (lane == 0 && nxt < n_units) nn = fetch(queue);  // answer needed a unit from now
+        TR(acc_wait += gtime() - tw0;)
 
-        // 128-bit grid inside the row: `head` leading elements, then n_vec full vectors, then a tail
-        const int head_bytes = (int)((16 - (reinterpret_cast<uintptr_t>(row) & 15)) & 15);
-        const int head = (int)min((int64_t)(head_bytes / ESZ), a.V);
-        const int64_t n_vec = (a.V - head) / EPV;
-        const int tail = (int)(a.V - head - n_vec * EPV);
-        const uint4* vrow = reinterpret_cast<const uint4*>(row + (int64_t)head * ESZ);
-        const int64_t vbeg = (int64_t)s * kVerifyVecPerItem;
-        const int64_t nv = min((int64_t)kVerifyVecPerItem, n_vec - vbeg);  // may be <= 0
-
-        uint4 x[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int vi = u * T + tid;
-            if (vi < nv) x[u] = ld_stream(vrow + vbeg + vi);
-            else x[u] = make_uint4(Elem<E>::kFillWord, Elem<E>::kFillWord, Elem<E>::kFillWord, Elem<E>::kFillWord);
-        }
-        // ragged edges of the row (at most 2*(EPV-1) elements) ride along with segment 0
-        float edge = 0.0f;
-        int edge_idx = -1;
-        if (s == 0 && tid < head + tail) {
-            edge_idx = tid < head ? tid : (int)(head + n_vec * EPV + (tid - head));
-            edge = Elem<E>::scalar(row, edge_idx);
-        }
-
-        float tmax = Elem<E>::thread_max(x);
-        uint32_t tord = (tid < nv) ? ord32(tmax) : 0u;  // a thread without a vector holds nothing
-        if (edge_idx >= 0) tord = max(tord, ord32(edge));
-        const uint32_t word = __reduce_max_sync(kFull, tord);
-        if (lane == 0) s_wmax[warp] = word;
-        if (tid == 0) { s_minidx = 0xffffffffu; s_next = nxt; }
-        __syncthreads();  // A
-        uint32_t bord = s_wmax[0];
-#pragma unroll
-        for (int k = 1; k < T / 32; ++k) bord = max(bord, s_wmax[k]);
-        nxt = s_next;
-        if (tord == bord && bord != 0u) {
-            // this thread holds a maximum: find its lowest index (rare path)
-            uint32_t best = 0xffffffffu;
-            if (edge_idx >= 0 && ord32(edge) == bord) best = (uint32_t)edge_idx;
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int vi = u * T + tid;
-                if (vi < nv) {
-#pragma unroll
-                    for (int k = 0; k < EPV; ++k) {
-                        if (ord32(Elem<E>::get(x[u], k)) == bord) {
-                            const uint32_t idx = (uint32_t)(head + (vbeg + vi) * EPV + k);
-                            best = min(best, idx);
-                        }
-                    }
-                }
+        const int64_t c0 = (int64_t)cur * UB;
+        const int64_t c1 = min(c0 + UB, total);
+        int r = (int)(c0 / nbr);              // needed-row number of the batch
+        int gb = (int)(c0 - (int64_t)r * nbr);  // batch number inside that row
+        unsigned long long ukey = 0ull;       // best of the unit's batches in the current row
+        int64_t ugrow = -1;
+#pragma unroll 1
+        for (int64_t p = c0; p < c1; ++p, ++gb) {
+            TR(unsigned long long ts0 = gtime();)
+            if (gb >= nbr) { gb -= nbr; ++r; }
+            int lo = 0, hi = a.B;  // request of the row: largest b with pref[b] <= r
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (sm.pref[mid] <= r) lo = mid; else hi = mid;
             }
-            atomicMin(&s_minidx, best);
-        }
-        __syncthreads();  // B
+            const int64_t grow = sm.row0[lo] + (r - sm.pref[lo]);
+            if (grow != ugrow) {
+                if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + ugrow, ukey);
+                ukey = 0ull;
+                ugrow = grow;
+            }
+            // 128-bit grid inside the row: `head` leading elements, n_vec full vectors, a tail
+            const char* row = base_ptr + grow * a.V * ESZ;
+            const int head_bytes = (int)((16 - (reinterpret_cast<uintptr_t>(row) & 15)) & 15);
+            const int head = (int)min((int64_t)(head_bytes / ESZ), a.V);
+            const int n_vec = (int)((a.V - head) / EPV);
+            const int tail = (int)(a.V - head - (int64_t)n_vec * EPV);
+            const int left = n_vec - gb * kBatchVec;  // vectors of the row from this batch on
+            const uint4* ptr = reinterpret_cast<const uint4*>(row + (int64_t)head * ESZ) + (int64_t)gb * kBatchVec + lane;
 
-        // ---- warp 0: publish the partial, count the item, commit if the request is complete ----
-        if (warp == 0) {
-            const int nr = s_pref[b + 1] - s_pref[b];
-            uint32_t last = 0;
-            if (lane == 0) {
-                const uint32_t idx = s_minidx;
-                const unsigned long long key =
-                    (bord == 0u || idx == 0xffffffffu) ? 0ull : (((unsigned long long)bord << 32) | (uint32_t)(~idx));
-                a.partial[(int64_t)r * a.n_seg + s] = key;
-                __threadfence();
-                const uint32_t old = atomicAdd(a.req_cnt + b, 1u);
-                last = (old + 1 == (uint32_t)nr * (uint32_t)a.n_seg) ? 1u : 0u;
+            uint32_t lord = 0u, loff = 0xffffffffu;  // this lane's maximum and its element index in the row
+            if (left >= kBatchVec) {
+                uint4 x[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) x[u] = ld_stream(ptr + u * 32);
+                Tracker<E> t;
+                t.init(x[0]);
+#pragma unroll
+                for (int u = 1; u < U; ++u) t.fold(x[u], u);
+                t.best(lane, lord, loff);
+                loff += (uint32_t)(head + gb * kBatchVec * EPV);
+            } else if (lane < left) {  // ragged last batch of the row
+                Tracker<E> t;
+                t.init(ld_stream(ptr));
+#pragma unroll
+                for (int u = 1; u < U; ++u)
+                    if (u * 32 + lane < left) t.fold(ld_stream(ptr + u * 32), u);
+                t.best(lane, lord, loff);
+                loff += (uint32_t)(head + gb * kBatchVec * EPV);
             }
-            last = __shfl_sync(kFull, last, 0);
-            if (last) {
-                __threadfence();
-                commit_request(a, b, s_pref[b], nr, lane);
+            // the ragged edges of the row (at most 2*(EPV-1) elements) ride along with batch 0
+            if (gb == 0 && lane < head + tail) {
+                const int idx = lane < head ? lane : head + n_vec * EPV + (lane - head);
+                const uint32_t eord = ord32(Tracker<E>::scalar(row, idx));
+                if (eord > lord || (eord == lord && (uint32_t)idx < loff)) { lord = eord; loff = (uint32_t)idx; }
             }
+            const uint32_t word = __reduce_max_sync(kFull, lord);
+            const uint32_t widx = __reduce_min_sync(kFull, lord == word ? loff : 0xffffffffu);
+            if (word != 0u && widx != 0xffffffffu) {
+                const unsigned long long key = ((unsigned long long)word << 32) | (uint32_t)(~widx);
+                ukey = key > ukey ? key : ukey;
+            }
+            TR(acc_str += gtime() - ts0; ++n_b;)
         }
+        if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + ugrow, ukey);
         cur = nxt;
+        nxt = nn;
     }
-
-    // ---- the last CTA to leave resets the work counter for the next call -----------------------
-    if (tid == 0) {
-        const uint32_t old = atomicAdd(&a.ctrl->blocks_exited, 1u);
-        if (old + 1 == gridDim.x) {
-            a.ctrl->next_item = 0;
-            a.ctrl->blocks_exited = 0;
-        }
-    }
+    TR(if (a.trace && lane == 0) { unsigned long long* tr = a.trace + ((size_t)blockIdx.x * NW + warp) * 8; tr[0] = t_enter; tr[1] = t_loop; tr[2] = gtime(); tr[3] = acc_wait; tr[4] = acc_str; tr[5] = acc_close; tr[6] = 0; tr[7] = n_b; })
 }
 
 }  // namespace
 
-size_t verify_dyn_smem(int32_t B) { return (size_t)(B + 1) * sizeof(int); }
+size_t verify_dyn_smem(int32_t B) { return (size_t)B * 8 + (size_t)(B + 1) * 4; }
 
 int verify_occupancy(hvd_dtype dtype, size_t dyn_smem) {
     int n = 0;
     cudaError_t e;
     if (dtype == HVD_F32)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, verify_commit_kernel<float>, T, dyn_smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, verify_stream_kernel<float>, T, dyn_smem);
     else
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, verify_commit_kernel<__nv_bfloat16>, T, dyn_smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, verify_stream_kernel<__nv_bfloat16>, T, dyn_smem);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return 0; }
     return n;
 }
 
-hvd_status launch_verify(hvd_ctx* ctx, const VerifyArgs& a, hvd_dtype dtype, cudaStream_t stream) {
-    const size_t smem = verify_dyn_smem(a.B);
+hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream) {
     const int per_sm = ctx->vf_blocks_per_sm[dtype == HVD_F32 ? 0 : 1];
     const int grid = ctx->num_sms * (per_sm > 0 ? per_sm : 1);
+    const int64_t esz = dtype == HVD_F32 ? 4 : 2;
+    a.n_batch_row = (int32_t)((a.V * esz / 16 + kBatchVec - 1) / kBatchVec);
+    if (a.n_batch_row < 1) a.n_batch_row = 1;
+    // unit numbers are 32-bit
+    if (a.total_rows * (int64_t)a.n_batch_row / UB + 4 * (int64_t)grid * NW >= 0x7fffffffLL)
+        return fail(ctx, HVD_ERR_UNSUPPORTED, "hvd_verify_commit: too many batches");
+    const size_t smem = verify_dyn_smem(a.B);
     if (dtype == HVD_F32)
-        verify_commit_kernel<float><<<grid, T, smem, stream>>>(a);
+        verify_stream_kernel<float><<<grid, T, smem, stream>>>(a);
     else
-        verify_commit_kernel<__nv_bfloat16><<<grid, T, smem, stream>>>(a);
+        verify_stream_kernel<__nv_bfloat16><<<grid, T, smem, stream>>>(a);
+    HVD_CUDA_TRY(ctx, cudaGetLastError());
+    verify_commit_kernel<<<(a.B + kCommitWarps - 1) / kCommitWarps, kCommitWarps * 32, 0, stream>>>(a);
     HVD_CUDA_TRY(ctx, cudaGetLastError());
     return HVD_OK;
 }
