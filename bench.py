@@ -283,68 +283,69 @@ def main():
         hist_len_steps.copy_(hist_len_pristine)
         state_steps.copy_(state_pristine)
 
-    def step(slot, events=None):
+    def step(slot, events=None, with_verify=True):
         r = slot % R
         hl, st = hist_len_steps[slot], state_steps[slot]
         if events is not None:
             events[0].record()
         lookup(hists[r], hl)
-        if events is not None:
-            events[1].record()
         score_select(hl, st)
         if events is not None:
-            events[2].record()
-        verify(logits[r], hists[r], hl, st)
+            events[1].record()
+        if with_verify:
+            verify(logits[r], hists[r], hl, st)
         if events is not None:
-            events[3].record()
+            events[2].record()
 
     # ---- warm-up (eager), then the timed K steps --------------------------------------------------
     for s in range(W_steps):
         step(s)
     torch.cuda.synchronize()
-    use_events = not args.no_kernel_events
     mode = args.mode
-    kernel_events = None
-    graph = None
     stream = torch.cuda.Stream(device=dev)
+
+    def capture(events=None, with_verify=True):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            g.capture_begin()
+            for s in range(K_steps):
+                step(W_steps + s, events[s] if events else None, with_verify)
+            g.capture_end()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            g.replay()               # untimed: instantiation and upload costs
+        torch.cuda.synchronize()
+        restore()
+        return g
+
+    graph = None
     if mode == "graph":
         try:
-            if use_events:
-                kernel_events = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(4)]
-                                 for _ in range(K_steps)]
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.stream(stream):
-                graph.capture_begin()
-                for s in range(K_steps):
-                    step(W_steps + s, kernel_events[s] if kernel_events else None)
-                graph.capture_end()
-            torch.cuda.synchronize()
-            with torch.cuda.stream(stream):
-                graph.replay()               # untimed: instantiation and upload costs
-            torch.cuda.synchronize()
-            restore()
+            graph = capture()
         except Exception as e:  # pragma: no cover
             sys.stderr.write(f"bench.py: graph capture failed ({e!r}); timing plain stream launches\n")
-            mode, graph, kernel_events = "stream", None, None
+            mode, graph = "stream", None
             torch.cuda.synchronize()
             restore()
-    if mode == "stream" and use_events:
-        kernel_events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K_steps)]
 
+    def timed(run):
+        """Device time of run() on `stream`, bracketed by barrier + synchronize on both sides."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with torch.cuda.stream(stream):
+            e0.record()
+            run()
+            e1.record()
+        barrier()
+        return e0.elapsed_time(e1)
+
+    # ---- the timed region: K steps, nothing but the path's kernels between the two events -------------
     sampler = ClockSampler(local)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
     sampler.start()
-    with torch.cuda.stream(stream):
-        ev0.record()
-        if graph is not None:
-            graph.replay()
-        else:
-            for s in range(K_steps):
-                step(W_steps + s, kernel_events[s] if kernel_events else None)
-        ev1.record()
-    barrier()
-    elapsed_ms = ev0.elapsed_time(ev1)
+    if graph is not None:
+        elapsed_ms = timed(graph.replay)
+    else:
+        elapsed_ms = timed(lambda: [step(W_steps + s) for s in range(K_steps)])
     window = "timed region"
     # results of the timed steps (every step does the same work on identical copies)
     n_commit_h = n_commit.cpu().numpy()
@@ -364,14 +365,37 @@ def main():
     sampler.stop_flag.set()
     sampler.join(timeout=2)
 
+    # ---- per-kernel times: the same K steps again, (a) with event records around the verify call
+    # inside the graph (each record is a graph node of its own and costs a few microseconds of
+    # serialisation, so these are upper bounds), (b) without the verify call (difference to the
+    # timed region = what verify adds to a step) ------------------------------------------------------
     kt = None
-    if kernel_events:
+    if not args.no_kernel_events:
         try:
-            d = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in kernel_events])
-            kt = {"lookup_us": 1e3 * float(d[:, 0].mean()), "score_select_us": 1e3 * float(d[:, 1].mean()),
-                  "verify_commit_us": 1e3 * float(d[:, 2].mean()),
-                  "verify_commit_us_median": 1e3 * float(np.median(d[:, 2])),
-                  "lookup_us_median": 1e3 * float(np.median(d[:, 0]))}
+            restore()
+            ext = graph is not None
+            evs = [[torch.cuda.Event(enable_timing=True, external=ext) for _ in range(3)] for _ in range(K_steps)]
+            if graph is not None:
+                g_ev = capture(evs)
+                t_ev = timed(g_ev.replay)
+                restore()
+                g_nv = capture(None, with_verify=False)
+                restore()
+                t_nv = timed(g_nv.replay)
+            else:
+                t_ev = timed(lambda: [step(W_steps + s, evs[s]) for s in range(K_steps)])
+                restore()
+                t_nv = timed(lambda: [step(W_steps + s, None, False) for s in range(K_steps)])
+            restore()
+            d = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(2)] for e in evs])
+            kt = {"lookup_plus_score_select_us": 1e3 * float(d[:, 0].mean()),
+                  "verify_commit_us": 1e3 * float(d[:, 1].mean()),
+                  "verify_commit_us_median": 1e3 * float(np.median(d[:, 1])),
+                  "step_us_with_event_records": 1e3 * t_ev / K_steps,
+                  "step_us_without_verify": 1e3 * t_nv / K_steps,
+                  "verify_commit_us_by_difference": 1e3 * (elapsed_ms - t_nv) / K_steps,
+                  "note": "event-bracketed times include the serialisation the event records add; "
+                          "the headline region has no records in it"}
         except Exception as e:  # pragma: no cover
             sys.stderr.write(f"bench.py: per-kernel events unavailable ({e!r})\n")
 
@@ -383,19 +407,15 @@ def main():
     # ---- roofline of the dominant kernel (verify/commit): algorithmic bytes = needed rows x V x elt ----
     verify_bytes = int((sel_len_after.astype(np.int64) + 1).sum()) * w.V * w.elt
     lookup_bytes = int(rq.hist_len.astype(np.int64).sum()) * 4
-    roofline = {"bound": "hbm", "kernel": "verify_commit_kernel", "achieved": None, "peak": peak_gbs, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": "verify_stream_kernel (+ verify_commit_kernel)", "achieved": None, "peak": peak_gbs, "unit": "GB/s",
                 "frac": None, "traffic": NCU_VERIFY_TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": verify_bytes}
-    roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel", "achieved": None, "peak": peak_gbs, "unit": "GB/s",
-                       "frac": None, "traffic": None, "peak_kind": peak_kind,
-                       "algorithmic_bytes_per_launch": lookup_bytes}
     if kt:
         roofline["achieved"] = verify_bytes / (kt["verify_commit_us"] * 1e-6) / 1e9
         roofline["frac"] = roofline["achieved"] / peak_gbs
         roofline["frac_of_8000_nominal"] = roofline["achieved"] / 8000.0
-        roofline_lookup["achieved"] = lookup_bytes / (kt["lookup_us"] * 1e-6) / 1e9
-        roofline_lookup["frac"] = roofline_lookup["achieved"] / peak_gbs
-        roofline_lookup["frac_of_8000_nominal"] = roofline_lookup["achieved"] / 8000.0
+        roofline["achieved_by_difference"] = verify_bytes / (kt["verify_commit_us_by_difference"] * 1e-6) / 1e9
+        roofline["timing"] = "CUDA events recorded around the hvd_verify_commit call inside the graph"
 
     # ---- end to end through the host-buffer entry point --------------------------------------------
     e2e = None
@@ -469,14 +489,14 @@ def main():
                 "config": workload_config(w, world, {
                     "cold_cache": f"{R} rotating copies of histories+logits ({foot / 2**20:.0f} MiB each, "
                                   f"L2 is 126 MiB); inputs per step exceed L2",
-                    "launch": f"{mode}: {K_steps} steps x 3 kernels in one CUDA graph" if graph is not None
-                              else "stream: 3 kernel launches per step",
-                    "kernel_events_in_timed_region": bool(kernel_events), "tau": tau}),
+                    "launch": f"{mode}: {K_steps} steps x 4 kernels in one CUDA graph" if graph is not None
+                              else "stream: 4 kernel launches per step",
+                    "kernel_events_in_timed_region": False, "tau": tau}),
                 "tokens_per_s": world * K_steps * tokens_per_step / (elapsed_ms * 1e-3),
                 "tokens_per_step": tokens_per_step,
                 "mean_accepted": float(accepted_h.mean()), "cache_selected_frac": float(select_h.mean()),
-                "kernel_us": kt, "roofline": roofline, "roofline_lookup": roofline_lookup,
-                "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": 3 * K_steps,
+                "kernel_us": kt, "roofline": roofline, "lookup_algorithmic_bytes": lookup_bytes,
+                "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": 4 * K_steps,
                 "clocks": sampler.summary(window)}
         print(json.dumps(line), flush=True)
     ctx.close()

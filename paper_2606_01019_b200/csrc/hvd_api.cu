@@ -86,6 +86,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->vf_blocks_per_sm[1] = verify_occupancy(HVD_BF16, smem);
     if (c->vf_blocks_per_sm[0] < 1 || c->vf_blocks_per_sm[1] < 1) { release(c); return HVD_ERR_UNSUPPORTED; }
     c->has_predictor = false;
+    c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // measured: no gain on this path, off unless asked for
     c->host_ws = nullptr;
     c->host_ws_bytes = 0;
 #ifdef HVD_TRACE

@@ -64,6 +64,7 @@ struct hvd_ctx {
     int* dev_error;                  // device status word
     int vf_blocks_per_sm[2];         // per dtype
     // device staging of the host-buffer entry point (grown on demand)
+    bool use_pdl;  // programmatic dependent launch between the kernels of the path
     char* host_ws;
     size_t host_ws_bytes;
 #ifdef HVD_TRACE
@@ -90,6 +91,27 @@ inline hvd_status cuda_fail(hvd_ctx* ctx, cudaError_t e, const char* where) {
         cudaError_t e_ = (call);                                         \
         if (e_ != cudaSuccess) return hvd::cuda_fail((ctx), e_, #call);  \
     } while (0)
+
+// Programmatic dependent launch: every kernel of the path lets its successor in the stream be
+// scheduled early (pdl_trigger) and waits for its predecessor's memory (pdl_wait) before it reads
+// anything a predecessor wrote.  Both are no-ops for a launch without the attribute.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
 
 hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
                          const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,

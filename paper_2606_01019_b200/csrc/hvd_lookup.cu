@@ -71,6 +71,8 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
+    pdl_trigger();
+    pdl_wait();
 
     int n = a.hist_len[b];
     if (n < 0 || n > a.hist_cap[b] || n > a.n_max) n = 0;  // unusable length: empty history
@@ -241,13 +243,14 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
     const int64_t chunks = (span + chunk - 1) / chunk;
     if (chunks > ctx->lk_max_chunks) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max exceeds max_hist_len");
     dim3 grid((unsigned)chunks, (unsigned)B);
+    cudaError_t e;
     switch (iter) {
-        case 1: lookup_kernel<1><<<grid, kLookupThreads, 0, stream>>>(a); break;
-        case 2: lookup_kernel<2><<<grid, kLookupThreads, 0, stream>>>(a); break;
-        case 4: lookup_kernel<4><<<grid, kLookupThreads, 0, stream>>>(a); break;
-        default: lookup_kernel<8><<<grid, kLookupThreads, 0, stream>>>(a); break;
+        case 1: e = launch_kernel(ctx->use_pdl, lookup_kernel<1>, grid, kLookupThreads, 0, stream, a); break;
+        case 2: e = launch_kernel(ctx->use_pdl, lookup_kernel<2>, grid, kLookupThreads, 0, stream, a); break;
+        case 4: e = launch_kernel(ctx->use_pdl, lookup_kernel<4>, grid, kLookupThreads, 0, stream, a); break;
+        default: e = launch_kernel(ctx->use_pdl, lookup_kernel<8>, grid, kLookupThreads, 0, stream, a); break;
     }
-    HVD_CUDA_TRY(ctx, cudaGetLastError());
+    HVD_CUDA_TRY(ctx, e);
     return HVD_OK;
 }
 

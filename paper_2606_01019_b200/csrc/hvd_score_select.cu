@@ -43,6 +43,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) score_select_kernel(const
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int b = blockIdx.x * kWarpsPerBlock + warp;
+    pdl_trigger();
+    pdl_wait();
     if (b >= a.B) return;
 
     int n = a.hist_len[b];
@@ -132,8 +134,7 @@ hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
     a.W1 = ctx->d_W1; a.b1 = ctx->d_b1; a.W2 = ctx->d_W2; a.b2 = ctx->b2; a.tau = ctx->tau;
     a.hidden = ctx->cfg.hidden; a.k_cap = ctx->cfg.k_cap;
     const int blocks = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    score_select_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(a);
-    HVD_CUDA_TRY(ctx, cudaGetLastError());
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select_kernel, blocks, kWarpsPerBlock * 32, 0, stream, a));
     return HVD_OK;
 }
 

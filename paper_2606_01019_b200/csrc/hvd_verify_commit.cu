@@ -222,6 +222,8 @@ constexpr int kCommitWarps = 4;
 
 __global__ void __launch_bounds__(kCommitWarps * 32) verify_commit_kernel(const VerifyArgs a) {
     const int b = blockIdx.x * kCommitWarps + (threadIdx.x >> 5);
+    pdl_trigger();
+    pdl_wait();
     if (b == 0 && (threadIdx.x & 31) < Q) a.next_unit[(threadIdx.x & 31) * kQueueStride] = 0u;  // zero at rest
     if (b < a.B) commit_request(a, b, threadIdx.x & 31);
 }
@@ -259,6 +261,8 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
     constexpr int EPV = Tracker<E>::kPerVec;
     constexpr int ESZ = 16 / EPV;
     TR(unsigned long long t_enter = gtime(); unsigned long long acc_wait = 0, acc_str = 0, acc_close = 0, n_b = 0;)
+    pdl_trigger();
+    pdl_wait();
 
     // Unit u belongs to queue u % Q.  The first unit of a warp is the one with its own number
     // (queue warp % Q); the next one is requested now and its answer is looked at after the first
@@ -302,7 +306,10 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
 
     const int nbr = a.n_batch_row;
     const int64_t total = (int64_t)sm.pref[a.B] * nbr;  // batches of all needed rows
-    const uint32_t n_units = (uint32_t)((total + UB - 1) / UB);
+    // the first 7/8 of the batches go out in units of UB, the rest one by one: near the end a
+    // warp on a slow SM should not sit on more than it can finish quickly
+    const uint32_t n_big = (uint32_t)((total - total / 8) / UB);
+    const uint32_t n_units = n_big + (uint32_t)(total - (int64_t)n_big * UB);
     const char* base_ptr = static_cast<const char*>(a.logits);
     TR(unsigned long long t_loop = gtime();)
 
@@ -320,8 +327,8 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
         if (lane == 0 && nxt < n_units) nn = fetch(queue);  // answer needed a unit from now
         TR(acc_wait += gtime() - tw0;)
 
-        const int64_t c0 = (int64_t)cur * UB;
-        const int64_t c1 = min(c0 + UB, total);
+        const int64_t c0 = cur < n_big ? (int64_t)cur * UB : (int64_t)n_big * UB + (cur - n_big);
+        const int64_t c1 = cur < n_big ? c0 + UB : c0 + 1;
         int r = (int)(c0 / nbr);              // needed-row number of the batch
         int gb = (int)(c0 - (int64_t)r * nbr);  // batch number inside that row
         unsigned long long ukey = 0ull;       // best of the unit's batches in the current row
@@ -417,12 +424,11 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
         return fail(ctx, HVD_ERR_UNSUPPORTED, "hvd_verify_commit: too many batches");
     const size_t smem = verify_dyn_smem(a.B);
     if (dtype == HVD_F32)
-        verify_stream_kernel<float><<<grid, T, smem, stream>>>(a);
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_stream_kernel<float>, grid, T, smem, stream, a));
     else
-        verify_stream_kernel<__nv_bfloat16><<<grid, T, smem, stream>>>(a);
-    HVD_CUDA_TRY(ctx, cudaGetLastError());
-    verify_commit_kernel<<<(a.B + kCommitWarps - 1) / kCommitWarps, kCommitWarps * 32, 0, stream>>>(a);
-    HVD_CUDA_TRY(ctx, cudaGetLastError());
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_stream_kernel<__nv_bfloat16>, grid, T, smem, stream, a));
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+                                    kCommitWarps * 32, 0, stream, a));
     return HVD_OK;
 }
 
