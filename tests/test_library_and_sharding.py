@@ -82,7 +82,7 @@ tokens = sum_over_ranks(float(out.vf.n_commit.sum()))
 assert tokens == float(full.vf.n_commit.sum()), (tokens, full.vf.n_commit.sum())
 assert max_over_ranks(10.0 + rank) == 10.0 + world - 1
 dist.destroy_process_group()
-print("rank", rank, "ok", lo, hi)
+sys.stdout.write("rank %d ok %d %d\n" % (rank, lo, hi))
 """
 
 
