@@ -220,6 +220,38 @@ typedef struct {
 
 HVD_API hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args, void* stream);
 
+/*
+ * Greedy verification and commit without a context and without any allocation.  (The paper has
+ * no counterpart: this is a packaging variant of hvd_verify_commit.)
+ *
+ * For callers that cannot allocate device memory where the decoding step runs: an engine whose
+ * memory pool owns the whole device, a call made while a stream is being captured, a plugin that
+ * may only touch the tensors it is handed.  Arguments, layouts and results are those of
+ * hvd_verify_commit, with k_cap (row length of sel_draft, committed has k_cap+1) passed directly.
+ * The kernels' scratch memory is a static device array inside the library (about 129 KB, held by
+ * every GPU that loads the library until the process exits), so:
+ *   - B <= HVD_NOALLOC_MAX_BATCH and total_rows <= HVD_NOALLOC_MAX_ROWS; larger calls are
+ *     rejected with HVD_ERR_INVALID_ARG (hvd_noalloc_last_error() says which limit);
+ *   - all calls on a device share the array: two calls that overlap on the GPU (different
+ *     streams, or threads launching at once) race and give wrong results; serialise them;
+ *   - the array keeps the previous call's contents; each call first clears, on `stream`, the part
+ *     it will read;
+ *   - the first call on each device looks up the array's device address and the launch shape
+ *     (queries only); make that first call outside of any stream capture.
+ * It calls no cudaMalloc, cudaFree or allocating library routine.
+ */
+enum { HVD_NOALLOC_MAX_ROWS = 16384, HVD_NOALLOC_MAX_BATCH = 2048 };
+HVD_API hvd_status hvd_verify_commit_noalloc(int32_t B, int32_t k_cap, const void* logits, hvd_dtype dtype,
+                                             int64_t V, const int64_t* row_off, int32_t k_uniform,
+                                             int64_t total_rows, const int32_t* sel_draft,
+                                             const int32_t* sel_len, const int32_t* select, int32_t* hist,
+                                             const int64_t* hist_off, const int32_t* hist_cap,
+                                             int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                                             int32_t* committed, int32_t* n_commit, int32_t* target_tok,
+                                             int32_t* status, void* stream);
+/* text of the last error of hvd_verify_commit_noalloc on the calling thread ("" if none) */
+HVD_API const char* hvd_noalloc_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

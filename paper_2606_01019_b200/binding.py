@@ -50,6 +50,8 @@ _SIGNATURES = {
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
     "hvd_step_host": (_i32, [_vp, C.POINTER(HvdHostStepArgs), _vp]),
+    "hvd_verify_commit_noalloc": (_i32, [_i32, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
+    "hvd_noalloc_last_error": (C.c_char_p, []),
 }
 
 _lib = None
@@ -95,6 +97,25 @@ def _hptr(a):
 def _stream():
     import torch
     return torch.cuda.current_stream().cuda_stream
+
+
+NOALLOC_MAX_ROWS, NOALLOC_MAX_BATCH = 16384, 2048
+
+
+def hvd_verify_commit_noalloc(B, k_cap, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
+                              select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
+                              target_tok, status):
+    """Verification and commit for callers that cannot allocate: no context, scratch memory is a
+    static array inside the library (limits NOALLOC_MAX_ROWS / NOALLOC_MAX_BATCH).  Calls on one
+    device must not overlap.  Enqueues on the current CUDA stream."""
+    lib = load_library()
+    st = lib.hvd_verify_commit_noalloc(B, k_cap, _ptr(logits), dtype, V, _ptr(row_off), k_uniform, total_rows,
+                                       _ptr(sel_draft), _ptr(sel_len), _ptr(select), _ptr(hist), _ptr(hist_off),
+                                       _ptr(hist_cap), _ptr(hist_len), _ptr(state), _ptr(accepted),
+                                       _ptr(committed), _ptr(n_commit), _ptr(target_tok), _ptr(status), _stream())
+    if st != 0:
+        raise HvdError(f"hvd_verify_commit_noalloc: {lib.hvd_status_string(st).decode()}: "
+                       f"{lib.hvd_noalloc_last_error().decode()}")
 
 
 class Context:
