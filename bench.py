@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--unfused", action="store_true",
+                    help="call hvd_lookup and hvd_score_select separately instead of hvd_lookup_score_select")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="leave the per-kernel event records out of the timed graph")
     return ap.parse_args()
@@ -250,6 +252,11 @@ def main():
         ctx.hvd_score_select(B, hist_len, prompt_len, state, Kt, draft, draft_len, match_len, match_pos,
                              match_cnt, model_draft, model_len, None, score, select, sel_draft, sel_len)
 
+    def lookup_score_select(hist, hist_len, state):
+        ctx.hvd_lookup_score_select(B, hist, hist_off, hist_cap, hist_len, Kt, n_max, prompt_len, state,
+                                    model_draft, model_len, draft, draft_len, match_len, match_pos, match_cnt,
+                                    None, score, select, sel_draft, sel_len)
+
     dtype = H.F32 if w.dtype == "f32" else H.BF16
 
     def verify(logits, hist, hist_len, state):
@@ -288,8 +295,11 @@ def main():
         hl, st = hist_len_steps[slot], state_steps[slot]
         if events is not None:
             events[0].record()
-        lookup(hists[r], hl)
-        score_select(hl, st)
+        if args.unfused:
+            lookup(hists[r], hl)
+            score_select(hl, st)
+        else:
+            lookup_score_select(hists[r], hl, st)
         if events is not None:
             events[1].record()
         if with_verify:
@@ -489,14 +499,16 @@ def main():
                 "config": workload_config(w, world, {
                     "cold_cache": f"{R} rotating copies of histories+logits ({foot / 2**20:.0f} MiB each, "
                                   f"L2 is 126 MiB); inputs per step exceed L2",
-                    "launch": f"{mode}: {K_steps} steps x 4 kernels in one CUDA graph" if graph is not None
-                              else "stream: 4 kernel launches per step",
+                    "launch": f"{mode}: {K_steps} steps x {4 if args.unfused else 3} kernels in one CUDA graph"
+                              if graph is not None else f"stream: {4 if args.unfused else 3} kernel launches per step",
+                    "entry_points": "hvd_lookup + hvd_score_select + hvd_verify_commit" if args.unfused
+                                    else "hvd_lookup_score_select + hvd_verify_commit",
                     "kernel_events_in_timed_region": False, "tau": tau}),
                 "tokens_per_s": world * K_steps * tokens_per_step / (elapsed_ms * 1e-3),
                 "tokens_per_step": tokens_per_step,
                 "mean_accepted": float(accepted_h.mean()), "cache_selected_frac": float(select_h.mean()),
                 "kernel_us": kt, "roofline": roofline, "lookup_algorithmic_bytes": lookup_bytes,
-                "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": 4 * K_steps,
+                "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": (4 if args.unfused else 3) * K_steps,
                 "clocks": sampler.summary(window)}
         print(json.dumps(line), flush=True)
     ctx.close()

@@ -150,6 +150,20 @@ HVD_API hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist
                             void* stream);
 
 /*
+ * hvd_lookup and hvd_score_select in one launch (Alg. 1: draft, score and select are consecutive
+ * and per request): the thread block that finishes a request's history scan goes straight on to
+ * its features, score and selection.  Arguments and every output exactly as in the two separate
+ * calls; all lookup outputs are still written.
+ */
+HVD_API hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                                           const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
+                                           int32_t n_max, const int32_t* prompt_len, const hvd_req_state* state,
+                                           const int32_t* model_draft, const int32_t* model_len, int32_t* draft,
+                                           int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
+                                           int32_t* match_cnt, float* features, float* score, int32_t* select,
+                                           int32_t* sel_draft, int32_t* sel_len, void* stream);
+
+/*
  * Greedy verification and commit (Sec. 3.1 Verify; Sec. 3.4; Algorithm 1; the accepted length is
  * the label equation of Sec. 3.3).  Request b owns logits rows [r0, r1): r0 = row_off[b],
  * r1 = row_off[b+1], or r0 = b*(k_uniform+1), r1 = r0 + k_uniform + 1 when row_off is NULL.  Row r

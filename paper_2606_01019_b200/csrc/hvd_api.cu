@@ -3,7 +3,7 @@
 
 #include <new>
 
-#include "hvd_internal.cuh"
+#include "hvd_score.cuh"
 
 using namespace hvd;
 
@@ -150,7 +150,33 @@ hvd_status hvd_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_
     if (n_max < 0 || n_max > ctx->cfg.max_hist_len)
         return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max outside [0, max_hist_len]");
     return launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
-                         match_len, match_pos, match_cnt, static_cast<cudaStream_t>(stream));
+                         match_len, match_pos, match_cnt, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                                   const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
+                                   int32_t n_max, const int32_t* prompt_len, const hvd_req_state* state,
+                                   const int32_t* model_draft, const int32_t* model_len, int32_t* draft,
+                                   int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
+                                   int32_t* match_cnt, float* features, float* score, int32_t* select,
+                                   int32_t* sel_draft, int32_t* sel_len, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: B outside [1, max_batch]");
+    if (!ctx->has_predictor) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: call hvd_set_predictor first");
+    if (!hist || !hist_off || !hist_cap || !hist_len || !K || !prompt_len || !state || !draft || !draft_len ||
+        !match_len || !match_pos || !match_cnt || !score || !select || !sel_draft || !sel_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: NULL pointer");
+    if ((model_draft == nullptr) != (model_len == nullptr))
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: model_draft and model_len go together");
+    if (!aligned(hist, 16)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: hist must be 16-byte aligned");
+    if (!aligned(state, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: state must be 8-byte aligned");
+    if (n_max < 0 || n_max > ctx->cfg.max_hist_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: n_max outside [0, max_hist_len]");
+    const ScoreArgs sa = make_score_args(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len,
+                                         match_pos, match_cnt, model_draft, model_len, features, score,
+                                         select, sel_draft, sel_len);
+    return launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
+                         match_len, match_pos, match_cnt, &sa, static_cast<cudaStream_t>(stream));
 }
 
 hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,

@@ -113,10 +113,19 @@ inline cudaError_t launch_kernel(bool pdl, void (*kernel)(KArgs...), dim3 grid, 
 }
 #endif
 
+struct ScoreArgs;  // hvd_score.cuh
+
+// `fused` != NULL: the CTA that finishes a request also scores it and selects its draft
 hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
                          const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
                          int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
-                         int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream);
+                         int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream);
+
+ScoreArgs make_score_args(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
+                          const hvd_req_state* state, const int32_t* K, const int32_t* draft,
+                          const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
+                          const int32_t* match_cnt, const int32_t* model_draft, const int32_t* model_len,
+                          float* features, float* score, int32_t* select, int32_t* sel_draft, int32_t* sel_len);
 
 hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
                                const int32_t* prompt_len, const hvd_req_state* state, const int32_t* K,

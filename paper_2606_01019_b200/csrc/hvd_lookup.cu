@@ -5,8 +5,10 @@
 // extends the match backwards cooperatively (one compared token per lane, ballot + find-first-set
 // gives the match length).  Each CTA leaves one partial (best length, latest position, count) in
 // the context's scratch; the CTA that arrives last for a request combines the partials, applies the
-// minimum-length and draft-length rules and copies the draft.  No CTA waits for another.
-#include "hvd_internal.cuh"
+// minimum-length and draft-length rules and copies the draft -- and, in the fused form, goes
+// straight on to the payoff features, the predictor and the draft selection of that request
+// (one kernel and one global round trip less per decoding step).  No CTA waits for another.
+#include "hvd_score.cuh"
 
 namespace hvd {
 namespace {
@@ -64,8 +66,9 @@ __device__ __forceinline__ int4 ld_hist(const int4* p) {
     return v;
 }
 
-template <int ITER>
-__global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs a) {
+template <int ITER, bool FUSED>
+__global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
+    __shared__ float s_hid[FUSED ? HVD_MAX_HIDDEN : 1];
     const int b = blockIdx.y;
     const int chunk = blockIdx.x;
     const int tid = threadIdx.x;
@@ -74,7 +77,8 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
     pdl_trigger();
     pdl_wait();
 
-    int n = a.hist_len[b];
+    const int n_raw = a.hist_len[b];
+    int n = n_raw;
     if (n < 0 || n > a.hist_cap[b] || n > a.n_max) n = 0;  // unusable length: empty history
     const int32_t* __restrict__ slab = a.hist + a.hist_off[b];
     // 128-bit loads run on the 16-byte grid; `mis` tokens of the first vector lie before the slab
@@ -90,6 +94,7 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
             if (lane == 0) {
                 a.draft_len[b] = 0; a.match_len[b] = 0; a.match_pos[b] = -1; a.match_cnt[b] = 0;
             }
+            if (FUSED) score_select_request(sa, b, lane, s_hid, n_raw, 0, 0, -1, 0, -1, -1);
         }
         return;
     }
@@ -210,11 +215,14 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
         }
         d = min(min(K, lim), n - e);
     }
-    for (int j = lane; j < a.k_cap; j += 32)
-        a.draft[(int64_t)b * a.k_cap + j] = (j < d) ? slab[e + j] : -1;
+    const int tok0 = lane < d ? slab[e + lane] : -1;
+    const int tok1 = lane + 32 < d ? slab[e + lane + 32] : -1;
+    if (lane < a.k_cap) a.draft[(int64_t)b * a.k_cap + lane] = tok0;
+    if (lane + 32 < a.k_cap) a.draft[(int64_t)b * a.k_cap + lane + 32] = tok1;
     if (lane == 0) {
         a.draft_len[b] = d; a.match_len[b] = L; a.match_pos[b] = e; a.match_cnt[b] = cnt;
     }
+    if (FUSED) score_select_request(sa, b, lane, s_hid, n_raw, d, L, e, cnt, tok0, tok1);
 }
 
 }  // namespace
@@ -222,7 +230,7 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
 hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
                          const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
                          int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
-                         int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream) {
+                         int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream) {
     LookupArgs a;
     a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.K = K;
     a.n_max = n_max;
@@ -244,12 +252,17 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
     if (chunks > ctx->lk_max_chunks) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max exceeds max_hist_len");
     dim3 grid((unsigned)chunks, (unsigned)B);
     cudaError_t e;
+    const ScoreArgs sa = fused ? *fused : ScoreArgs();
+#define HVD_LAUNCH_LOOKUP(I)                                                                              \
+    (fused ? launch_kernel(ctx->use_pdl, lookup_kernel<I, true>, grid, kLookupThreads, 0, stream, a, sa)  \
+           : launch_kernel(ctx->use_pdl, lookup_kernel<I, false>, grid, kLookupThreads, 0, stream, a, sa))
     switch (iter) {
-        case 1: e = launch_kernel(ctx->use_pdl, lookup_kernel<1>, grid, kLookupThreads, 0, stream, a); break;
-        case 2: e = launch_kernel(ctx->use_pdl, lookup_kernel<2>, grid, kLookupThreads, 0, stream, a); break;
-        case 4: e = launch_kernel(ctx->use_pdl, lookup_kernel<4>, grid, kLookupThreads, 0, stream, a); break;
-        default: e = launch_kernel(ctx->use_pdl, lookup_kernel<8>, grid, kLookupThreads, 0, stream, a); break;
+        case 1: e = HVD_LAUNCH_LOOKUP(1); break;
+        case 2: e = HVD_LAUNCH_LOOKUP(2); break;
+        case 4: e = HVD_LAUNCH_LOOKUP(4); break;
+        default: e = HVD_LAUNCH_LOOKUP(8); break;
     }
+#undef HVD_LAUNCH_LOOKUP
     HVD_CUDA_TRY(ctx, e);
     return HVD_OK;
 }

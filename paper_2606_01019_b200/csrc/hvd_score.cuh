@@ -1,0 +1,109 @@
+// Payoff features, predictor and draft selection for ONE request, by one warp (Sec. 3.3, 3.4,
+// App. B feature groups).  Shared by the stand-alone kernel and by the lookup kernel's fused tail.
+#pragma once
+
+#include "hvd_internal.cuh"
+
+namespace hvd {
+
+struct ScoreArgs {
+    int32_t B;
+    const int32_t* hist_len;
+    const int32_t* prompt_len;
+    const hvd_req_state* state;
+    const int32_t* K;
+    const int32_t* draft;
+    const int32_t* draft_len;
+    const int32_t* match_len;
+    const int32_t* match_pos;
+    const int32_t* match_cnt;
+    const int32_t* model_draft;
+    const int32_t* model_len;
+    float* features;
+    float* score;
+    int32_t* select;
+    int32_t* sel_draft;
+    int32_t* sel_len;
+    const float* W1;
+    const float* b1;
+    const float* W2;
+    float b2, tau;
+    int32_t hidden, k_cap;
+};
+
+__device__ __forceinline__ int bit_width(uint32_t x) { return 32 - __clz((int)x); }
+
+// The work is a few hundred flops per request, far too small and too irregular for tensor cores:
+// lane j evaluates hidden unit j (and j+32, ...) with a left-to-right chain of fused multiply-adds,
+// lane 0 then accumulates the output layer in unit order, so the fp32 result does not depend on
+// the launch shape.  d, L, pos, cnt: the lookup results of the request; tok0 / tok1: cache draft
+// tokens lane and lane+32 (-1 beyond the draft); s_hid: shared memory, a.hidden floats, private to
+// the warp.
+__device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, int lane, float* s_hid, int n,
+                                                     int d, int L, int pos, int cnt, int tok0, int tok1) {
+    n = max(n, 0);
+    const int P = max(a.prompt_len[b], 0);
+    const hvd_req_state st = a.state[b];
+    const int kc = a.k_cap;
+    const int K = max(0, min(a.K[b], kc));
+    d = max(0, min(d, kc));
+    cnt = max(cnt, 0);
+
+    float phi[HVD_N_FEATURES];
+    phi[0] = (float)L;
+    phi[1] = (float)d;
+    phi[2] = (float)bit_width((uint32_t)cnt);
+    phi[3] = (pos < 0 || n == 0) ? 0.0f : __fdiv_rn((float)(n - pos), (float)n);
+    phi[4] = (float)bit_width((uint32_t)P);
+    phi[5] = (n == 0) ? 0.0f : __fdiv_rn((float)(n - P), (float)n);
+    phi[6] = __fdiv_rn((float)__popc(st.sel_bits & 0xFFu), 8.0f);
+    // sum of the eight bytes of the accepted-length ring
+    uint64_t r = st.acc_ring;
+    r = (r & 0x00FF00FF00FF00FFull) + ((r >> 8) & 0x00FF00FF00FF00FFull);
+    r = (r & 0x0000FFFF0000FFFFull) + ((r >> 16) & 0x0000FFFF0000FFFFull);
+    const int acc_sum = (int)((r & 0xFFFFFFFFull) + (r >> 32));
+    phi[7] = __fdiv_rn((float)acc_sum, 8.0f);
+
+    if (a.features && lane < HVD_N_FEATURES) {
+        float v = phi[0];
+#pragma unroll
+        for (int i = 1; i < HVD_N_FEATURES; ++i) v = (lane == i) ? phi[i] : v;
+        a.features[(int64_t)b * HVD_N_FEATURES + lane] = v;
+    }
+
+    for (int j = lane; j < a.hidden; j += 32) {
+        float acc = a.b1[j];
+        const float* w = a.W1 + (int64_t)j * HVD_N_FEATURES;
+#pragma unroll
+        for (int i = 0; i < HVD_N_FEATURES; ++i) acc = __fmaf_rn(w[i], phi[i], acc);
+        s_hid[j] = acc > 0.0f ? acc : 0.0f;
+    }
+    __syncwarp();
+    float y = a.b2;
+    if (lane == 0) {
+        for (int j = 0; j < a.hidden; ++j) y = __fmaf_rn(a.W2[j], s_hid[j], y);
+    }
+    y = __shfl_sync(0xffffffffu, y, 0);
+    const int sel = (d > 0 && y >= a.tau) ? 1 : 0;
+
+    int m = d;
+    if (!sel) {
+        m = 0;
+        tok0 = tok1 = -1;
+        if (a.model_draft && a.model_len) {
+            m = max(0, min(a.model_len[b], K));
+            const int32_t* src = a.model_draft + (int64_t)b * kc;
+            if (lane < m) tok0 = src[lane];
+            if (lane + 32 < m) tok1 = src[lane + 32];
+        }
+    }
+    if (lane < kc) a.sel_draft[(int64_t)b * kc + lane] = (lane < m) ? tok0 : -1;
+    if (lane + 32 < kc) a.sel_draft[(int64_t)b * kc + lane + 32] = (lane + 32 < m) ? tok1 : -1;
+    if (lane == 0) {
+        a.score[b] = y;
+        a.select[b] = sel;
+        a.sel_len[b] = m;
+    }
+}
+
+}  // namespace hvd

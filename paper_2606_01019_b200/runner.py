@@ -55,6 +55,13 @@ class DeviceBatch:
                                   self.model_draft, self.model_len, self.features, self.score,
                                   self.select, self.sel_draft, self.sel_len)
 
+    def lookup_score_select(self):
+        self.ctx.hvd_lookup_score_select(self.B, self.hist, self.hist_off, self.hist_cap, self.hist_len, self.K,
+                                         self.n_max, self.prompt_len, self.state, self.model_draft,
+                                         self.model_len, self.draft, self.draft_len, self.match_len,
+                                         self.match_pos, self.match_cnt, self.features, self.score,
+                                         self.select, self.sel_draft, self.sel_len)
+
     def verify_commit(self, logits, target_tok=True):
         self.ctx.hvd_verify_commit(self.B, logits, self.dtype, self.V, self.row_off, self.k_uniform,
                                    self.total_rows, self.sel_draft, self.sel_len, self.select, self.hist,
@@ -62,9 +69,12 @@ class DeviceBatch:
                                    self.accepted, self.committed, self.n_commit,
                                    self.target_tok if target_tok else None, self.status)
 
-    def step(self, logits, target_tok=True):
-        self.lookup()
-        self.score_select()
+    def step(self, logits, target_tok=True, fused=False):
+        if fused:
+            self.lookup_score_select()
+        else:
+            self.lookup()
+            self.score_select()
         self.verify_commit(logits, target_tok)
 
     def download(self) -> dict:

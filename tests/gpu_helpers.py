@@ -63,7 +63,7 @@ def compare_verify(g, vf, rq_after):
 
 
 def run_and_compare(inp, ctx=None, uniform_rows=False, logits=None, logits_np=None, rq=None, batch=None,
-                    nthreads=None):
+                    nthreads=None, fused=False):
     """One full step on the GPU and in the oracle from the same inputs; returns (gpu dict, StepOut)."""
     w = inp.w
     rq = inp.rq.copy() if rq is None else rq
@@ -76,7 +76,7 @@ def run_and_compare(inp, ctx=None, uniform_rows=False, logits=None, logits_np=No
     lg = inp.logits if logits is None else logits
     if lg.device.type != "cuda":
         lg = lg.cuda()
-    batch.step(lg)
+    batch.step(lg, fused=fused)
     g = batch.download()
     out = P.step(inp, rq, nthreads=nthreads or P.host_threads(), logits_np=logits_np)
     compare_lookup(g, out.lk)

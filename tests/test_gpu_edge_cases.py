@@ -39,7 +39,8 @@ def run(w, rq, **kw):
     return G.run_and_compare(inp, **kw), inp
 
 
-def test_tiny_histories():
+@pytest.mark.parametrize("fused", [False, True])
+def test_tiny_histories(fused):
     w = small()
     rng = np.random.default_rng(3)
     hists = []
@@ -47,7 +48,7 @@ def test_tiny_histories():
         hists.append(rng.integers(0, 3, n))                 # tiny vocabulary: matches everywhere
         hists.append(rng.integers(0, w.V, n))               # large vocabulary: rarely any match
     rq = hand_requests(w, hists, [8] * len(hists))
-    (g, out, _), _ = run(w, rq)
+    (g, out, _), _ = run(w, rq, fused=fused)
     assert (out.lk.match_len > 0).sum() > 10
 
 
@@ -103,6 +104,7 @@ def test_capacity_edges_and_bad_lengths():
     extra = [9, 5, 4, 3, 2, 1, 0, 9, 9, 9, 9, 0]
     hist_len = [500, 500, 500, 500, 500, 500, 500, -1, 510, 2**31 - 1, 500, 500]
     rq = hand_requests(w, hists, [8] * 12, cap_extra=extra, hist_len=hist_len)
+    run(w, rq.copy(), fused=True)
     (g, out, _), _ = run(w, rq)
     assert (out.vf.status == O.REQ_BAD_LEN).sum() == 3
     assert (out.vf.status == O.REQ_CAPACITY).sum() >= 1
@@ -116,6 +118,7 @@ def test_model_draft_clamp_and_out_of_vocab_tokens():
     md = rng.integers(0, w.V, (10, 16)).astype(np.int32)
     md[5, 3] = -1; md[6, 0] = w.V; md[2, 15] = 2**31 - 1
     rq = hand_requests(w, hists, K, model_len=[9, 8, 16, 5, 0, 16, 16, 1, 40, -3], model_draft=md)
+    run(w.scaled(calibrate_cache_frac=None), rq.copy(), fused=True)
     (g, out, _), _ = run(w.scaled(calibrate_cache_frac=None), rq)
     assert (out.sc.select == 0).all()
 

@@ -18,6 +18,14 @@ def test_c1_full():
     assert g["select"].sum() > 0
 
 
+@pytest.mark.parametrize("name,kw", [("C1", {}), ("C2", dict(B=24, n=9000, V=20011)), ("C4", dict(B=6, n=40000, V=5003)),
+                                     ("C5", dict(B=60, n=(2, 5000), V=32003))])
+def test_fused_lookup_score_select(name, kw):
+    """hvd_lookup_score_select gives what hvd_lookup followed by hvd_score_select gives."""
+    inp = P.prepare(W.CONFIGS[name].scaled(**kw), device="cuda")
+    G.run_and_compare(inp, fused=True)
+
+
 def test_c1_uniform_row_layout():
     inp = P.prepare(W.CONFIGS["C1"], device="cuda")
     G.run_and_compare(inp, uniform_rows=True)
@@ -28,7 +36,7 @@ def test_full_size_configs(name):
     """Every request, row and token of the full-size workloads, in the launch configuration the
     benchmark uses (same context limits, same entry points)."""
     inp = P.prepare(W.CONFIGS[name], device="cuda")
-    g, out, _ = G.run_and_compare(inp)
+    g, out, _ = G.run_and_compare(inp, fused=(name in ("C2", "C4")))      # the benchmark's launch configuration
     assert (g["accepted"] == inp.A)[inp.strict].all()
     sel = g["select"]
     assert 0 < sel.sum() < len(sel)                       # both draft sources in play
