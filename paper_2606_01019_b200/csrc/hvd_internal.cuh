@@ -36,8 +36,11 @@ constexpr int kVerifyUnroll = HVD_VERIFY_UNROLL;      // 128-bit loads in flight
 #define HVD_VERIFY_UNIT_BATCHES 2
 #endif
 constexpr int kVerifyUnitBatches = HVD_VERIFY_UNIT_BATCHES;  // 4 KB batches per unit drawn by a warp
+#ifndef HVD_VERIFY_ENDGAME_SHIFT
+#define HVD_VERIFY_ENDGAME_SHIFT 3
+#endif
 #ifndef HVD_VERIFY_QUEUES
-#define HVD_VERIFY_QUEUES 4
+#define HVD_VERIFY_QUEUES 8
 #endif
 constexpr int kVerifyQueues = HVD_VERIFY_QUEUES;  // unit counters
 

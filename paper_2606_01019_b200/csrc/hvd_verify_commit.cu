@@ -123,19 +123,32 @@ struct Tracker<__nv_bfloat16> {
             u[c] = (u[c] & ~m) | (tag & m);
         }
     }
+    __device__ static __forceinline__ uint32_t eq2(uint32_t a, uint32_t b) {  // 0xffff per equal half
+        uint32_t d;
+        asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+        return d;
+    }
+    __device__ static __forceinline__ uint32_t minu2(uint32_t a, uint32_t b) {
+        uint32_t d;
+        asm("min.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+        return d;
+    }
+    // all in packed form: the lane maximum, then the smallest (load, slot) among the slots equal to it
     __device__ __forceinline__ void best(int lane, uint32_t& ord, uint32_t& off) const {
-        ord = 0u; off = 0xffffffffu;
+        const uint32_t m = max2(max2(v[0], v[1]), max2(v[2], v[3]));
+        const float vmax = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
+        const uint32_t h = __float_as_uint(vmax) >> 16;
+        const uint32_t mm = h | (h << 16);
+        uint32_t cand = 0xffffffffu;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint32_t bits = h ? (v[c] & 0xffff0000u) : (v[c] << 16);
-                const uint32_t load = h ? (u[c] >> 16) : (u[c] & 0xffffu);
-                const uint32_t o = ord32(__uint_as_float(bits));
-                const uint32_t f = (load * 32u + (uint32_t)lane) * 8u + (uint32_t)(2 * c + h);
-                if (o > ord || (o == ord && f < off)) { ord = o; off = f; }
-            }
+            const uint32_t e = eq2(v[c], mm);
+            const uint32_t k = (u[c] << 3) | (uint32_t)(((2 * c + 1) << 16) | (2 * c));  // (load << 3 | slot) per half
+            cand = minu2(cand, (k & e) | ~e);
         }
+        const uint32_t b16 = min(cand & 0xffffu, cand >> 16);
+        ord = ord32(vmax);
+        off = ((b16 >> 3) * 32u + (uint32_t)lane) * 8u + (b16 & 7u);
     }
 };
 
@@ -159,9 +172,19 @@ __device__ __forceinline__ Req load_req(const VerifyArgs& a, int b) {
 }
 
 // Commit of one request by one warp, after all its needed rows are folded into the row keys.
+// Every load that does not depend on another is issued up front: the kernel is a short chain of
+// global round trips at the end of every decoding step.
 __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int lane) {
-    const Req q = load_req(a, b);
     const int kc = a.k_cap;
+    const int32_t* d = a.sel_draft + (int64_t)b * kc;
+    const int d0 = lane < kc ? d[lane] : -1;            // draft tokens lane, lane+32 (k_cap <= 64)
+    const int d1 = lane + 32 < kc ? d[lane + 32] : -1;
+    const int64_t hoff = a.hist_off[b];
+    const int sel = a.select[b];
+    hvd_req_state st = a.state[b];
+    const int n = a.hist_len[b];
+    const int cap = a.hist_cap[b];
+    const Req q = load_req(a, b);
     int32_t* z = a.committed + (int64_t)b * (kc + 1);
     if (q.nr == 0) {
         // skipped request: neutral outputs, nothing else touched
@@ -171,38 +194,46 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
         return;
     }
     const int m = q.nr - 1;
-    const int32_t* d = a.sel_draft + (int64_t)b * kc;
+    // rows lane, lane+32, lane+64 (at most 65 rows): target tokens from the row keys
+    unsigned long long key[3];
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const int i = lane + 32 * k;
+        key[k] = 0ull;
+        if (i <= m) {
+            key[k] = a.row_key[q.r0 + i];
+            a.row_key[q.r0 + i] = 0ull;  // scratch is zero at rest
+        }
+    }
     int acc = -1;
     int t_acc = 0;
-    // rows in rounds of 32: lane handles row i, reads its target token, compares with the draft
-    for (int base = 0; base <= m; base += 32) {
-        const int i = base + lane;
-        int t = 0;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const int i = lane + 32 * k;
+        int t = (int)(~(uint32_t)(key[k] & 0xffffffffu));
+        t = (int)min((int64_t)max(t, 0), a.V - 1);  // inside the vocabulary whatever the data
         bool stop = true;
         if (i <= m) {
-            const unsigned long long key = a.row_key[q.r0 + i];
-            a.row_key[q.r0 + i] = 0ull;  // scratch is zero at rest
-            t = (int)(~(uint32_t)(key & 0xffffffffu));
-            t = (int)min((int64_t)max(t, 0), a.V - 1);  // inside the vocabulary whatever the data
             if (a.target_tok) a.target_tok[q.r0 + i] = t;
-            stop = (i >= m) || (d[i] != t);
+            const int di = k == 0 ? d0 : (k == 1 ? d1 : -1);
+            stop = (i >= m) || (di != t);
         }
         const uint32_t stops = __ballot_sync(kFull, stop);
-        if (acc < 0 && stops != 0) {
+        if (acc < 0 && stops != 0 && 32 * k <= m) {
             const int j = __ffs(stops) - 1;
-            acc = base + j;
+            acc = 32 * k + j;
             t_acc = __shfl_sync(kFull, t, j);
         }
     }
     // acc <= m always (row m stops).  Rows beyond m were not read.
     if (a.target_tok)
         for (int64_t r = q.r0 + q.nr + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
-    const int n = a.hist_len[b];
-    const int room = a.hist_cap[b] - n;
+    const int room = cap - n;
     const int w = min(acc + 1, room);
-    int32_t* h = a.hist + a.hist_off[b];
+    int32_t* h = a.hist + hoff;
     for (int j = lane; j <= kc; j += 32) {
-        const int tok = (j < acc) ? d[j] : (j == acc ? t_acc : -1);
+        const int dj = j < 32 ? d0 : d1;
+        const int tok = (j < acc) ? dj : (j == acc ? t_acc : -1);
         z[j] = tok;
         if (j < w) h[n + j] = tok;
     }
@@ -211,8 +242,7 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
         a.n_commit[b] = w;
         a.accepted[b] = acc;
         a.status[b] = (w < acc + 1) ? HVD_REQ_CAPACITY : HVD_REQ_OK;
-        hvd_req_state st = a.state[b];
-        st.sel_bits = (st.sel_bits << 1) | (a.select[b] ? 1u : 0u);
+        st.sel_bits = (st.sel_bits << 1) | (sel ? 1u : 0u);
         st.acc_ring = (st.acc_ring << 8) | (unsigned long long)(acc & 0xff);
         a.state[b] = st;
     }
@@ -273,6 +303,7 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
     int tries = 0;  // queues found dry so far
     auto fetch = [&](int q) { return (n_warps / Q + atomicAdd(a.next_unit + q * kQueueStride, 1u)) * Q + (uint32_t)q; };
     uint32_t nxt = 0;
+    bool have_nxt = true;
     if (lane == 0) nxt = fetch(queue);
 
     // ---- phase 0: rows needed per request (device data), prefix over requests ----------------------
@@ -306,9 +337,9 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
 
     const int nbr = a.n_batch_row;
     const int64_t total = (int64_t)sm.pref[a.B] * nbr;  // batches of all needed rows
-    // the first 7/8 of the batches go out in units of UB, the rest one by one: near the end a
+    // all but the last 1/2^HVD_VERIFY_ENDGAME_SHIFT of the batches go out in units of UB, the rest one by one: near the end a
     // warp on a slow SM should not sit on more than it can finish quickly
-    const uint32_t n_big = (uint32_t)((total - total / 8) / UB);
+    const uint32_t n_big = (uint32_t)((total - (total >> HVD_VERIFY_ENDGAME_SHIFT)) / UB);
     const uint32_t n_units = n_big + (uint32_t)(total - (int64_t)n_big * UB);
     const char* base_ptr = static_cast<const char*>(a.logits);
     TR(unsigned long long t_loop = gtime();)
@@ -316,46 +347,57 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
     // ---- phase 1: units of batches -------------------------------------------------------------------
     while (cur < n_units) {
         TR(unsigned long long tw0 = gtime();)
-        nxt = __shfl_sync(kFull, nxt, 0);
-        if (nxt >= n_units && tries == 0) {  // own queue is dry: one look at the neighbour queue
-            tries = 1;
-            queue = (queue + 1) % Q;
-            if (lane == 0) nxt = fetch(queue);
-            nxt = __shfl_sync(kFull, nxt, 0);
-        }
+        // `nxt` was requested a unit ago.  In the end game (single-batch units) nothing is requested
+        // ahead: a warp on a slow SM must not sit on work that an idle warp could do.
         uint32_t nn = 0;
-        if (lane == 0 && nxt < n_units) nn = fetch(queue);  // answer needed a unit from now
+        bool have_nn = false;
+        if (have_nxt) {
+            nxt = __shfl_sync(kFull, nxt, 0);
+            if (nxt >= n_units && tries == 0) {  // own queue is dry: one look at the neighbour queue
+                tries = 1;
+                queue = (queue + 1) % Q;
+                if (lane == 0) nxt = fetch(queue);
+                nxt = __shfl_sync(kFull, nxt, 0);
+            }
+            if (nxt < n_big) { if (lane == 0) nn = fetch(queue); have_nn = true; }  // needed a unit from now
+            else if (nxt >= n_units) { nn = nxt; have_nn = true; }                  // nothing left, stays so
+        }
         TR(acc_wait += gtime() - tw0;)
 
         const int64_t c0 = cur < n_big ? (int64_t)cur * UB : (int64_t)n_big * UB + (cur - n_big);
         const int64_t c1 = cur < n_big ? c0 + UB : c0 + 1;
-        int r = (int)(c0 / nbr);              // needed-row number of the batch
+        int r = (int)(c0 / nbr);                // needed-row number of the batch
         int gb = (int)(c0 - (int64_t)r * nbr);  // batch number inside that row
-        unsigned long long ukey = 0ull;       // best of the unit's batches in the current row
-        int64_t ugrow = -1;
+        unsigned long long ukey = 0ull;         // best of the unit's batches in the current row
+        int64_t grow = -1;
+        // 128-bit grid inside the current row: `head` leading elements, n_vec full vectors, a tail
+        const char* row = nullptr;
+        const uint4* vrow = nullptr;
+        int head = 0, n_vec = 0, tail = 0;
+        int geom_r = -1;
 #pragma unroll 1
         for (int64_t p = c0; p < c1; ++p, ++gb) {
             TR(unsigned long long ts0 = gtime();)
             if (gb >= nbr) { gb -= nbr; ++r; }
-            int lo = 0, hi = a.B;  // request of the row: largest b with pref[b] <= r
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (sm.pref[mid] <= r) lo = mid; else hi = mid;
-            }
-            const int64_t grow = sm.row0[lo] + (r - sm.pref[lo]);
-            if (grow != ugrow) {
-                if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + ugrow, ukey);
+            if (r != geom_r) {
+                if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + grow, ukey);
                 ukey = 0ull;
-                ugrow = grow;
+                geom_r = r;
+                int lo = 0, hi = a.B;  // request of the row: largest b with pref[b] <= r
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (sm.pref[mid] <= r) lo = mid; else hi = mid;
+                }
+                grow = sm.row0[lo] + (r - sm.pref[lo]);
+                row = base_ptr + grow * a.V * ESZ;
+                const int head_bytes = (int)((16 - (reinterpret_cast<uintptr_t>(row) & 15)) & 15);
+                head = (int)min((int64_t)(head_bytes / ESZ), a.V);
+                n_vec = (int)((a.V - head) / EPV);
+                tail = (int)(a.V - head - (int64_t)n_vec * EPV);
+                vrow = reinterpret_cast<const uint4*>(row + (int64_t)head * ESZ);
             }
-            // 128-bit grid inside the row: `head` leading elements, n_vec full vectors, a tail
-            const char* row = base_ptr + grow * a.V * ESZ;
-            const int head_bytes = (int)((16 - (reinterpret_cast<uintptr_t>(row) & 15)) & 15);
-            const int head = (int)min((int64_t)(head_bytes / ESZ), a.V);
-            const int n_vec = (int)((a.V - head) / EPV);
-            const int tail = (int)(a.V - head - (int64_t)n_vec * EPV);
             const int left = n_vec - gb * kBatchVec;  // vectors of the row from this batch on
-            const uint4* ptr = reinterpret_cast<const uint4*>(row + (int64_t)head * ESZ) + (int64_t)gb * kBatchVec + lane;
+            const uint4* ptr = vrow + (int64_t)gb * kBatchVec + lane;
 
             uint32_t lord = 0u, loff = 0xffffffffu;  // this lane's maximum and its element index in the row
             if (left >= kBatchVec) {
@@ -391,9 +433,21 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
             }
             TR(acc_str += gtime() - ts0; ++n_b;)
         }
-        if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + ugrow, ukey);
-        cur = nxt;
+        if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + grow, ukey);
+        if (have_nxt) {
+            cur = nxt;
+        } else {  // end game: ask only now that this warp is free
+            if (lane == 0) cur = fetch(queue);
+            cur = __shfl_sync(kFull, cur, 0);
+            if (cur >= n_units && tries == 0) {
+                tries = 1;
+                queue = (queue + 1) % Q;
+                if (lane == 0) cur = fetch(queue);
+                cur = __shfl_sync(kFull, cur, 0);
+            }
+        }
         nxt = nn;
+        have_nxt = have_nn;
     }
     TR(if (a.trace && lane == 0) { unsigned long long* tr = a.trace + ((size_t)blockIdx.x * NW + warp) * 8; tr[0] = t_enter; tr[1] = t_loop; tr[2] = gtime(); tr[3] = acc_wait; tr[4] = acc_str; tr[5] = acc_close; tr[6] = 0; tr[7] = n_b; })
 }
