@@ -18,7 +18,7 @@ struct LookupPartial {
 
 constexpr int kLookupThreads = 256;
 constexpr int kLookupTokPerVec = 4;
-constexpr int kLookupMinChunk = kLookupThreads * kLookupTokPerVec;  // tokens, one 128-bit load per thread
+constexpr int kLookupMinChunk = kLookupThreads * kLookupTokPerVec;  // tokens: sizes the partial scratch
 
 // tunables of the verify kernel (overridable at compile time for experiments)
 #ifndef HVD_VERIFY_THREADS

@@ -1,7 +1,7 @@
 // Cache-draft lookup (Sec. 3.2): longest match of the history's own suffix inside the history.
 //
-// The history of a request is cut into chunks; one CTA scans one chunk with 128-bit loads, looking
-// for the last token of the history.  Every hit is a candidate end position; the warp that found it
+// One CTA scans a request's history (histories longer than 32 K tokens are cut into chunks, one
+// CTA each) with 128-bit loads, all issued up front, looking for the last token of the history.  Every hit is a candidate end position; the warp that found it
 // extends the match backwards cooperatively (one compared token per lane, ballot + find-first-set
 // gives the match length).  Each CTA leaves one partial (best length, latest position, count) in
 // the context's scratch; the CTA that arrives last for a request combines the partials, applies the
@@ -66,8 +66,8 @@ __device__ __forceinline__ int4 ld_hist(const int4* p) {
     return v;
 }
 
-template <int ITER, bool FUSED>
-__global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
+template <int THREADS, int ITER, bool FUSED>
+__global__ void __launch_bounds__(THREADS, 1) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
     __shared__ float s_hid[FUSED ? HVD_MAX_HIDDEN : 1];
     const int b = blockIdx.y;
     const int chunk = blockIdx.x;
@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
     const int32_t* __restrict__ slab = a.hist + a.hist_off[b];
     // 128-bit loads run on the 16-byte grid; `mis` tokens of the first vector lie before the slab
     const int mis = (int)((reinterpret_cast<uintptr_t>(slab) >> 2) & 3);
-    constexpr int CHUNK = kLookupMinChunk * ITER;  // tokens of the aligned grid per CTA
+    constexpr int CHUNK = THREADS * kLookupTokPerVec * ITER;  // tokens of the aligned grid per CTA
     // candidate positions p (index of the matched copy's last token) are 0 .. n-2
     const int g_end = (n >= 2) ? (n - 1 + mis) : 0;  // exclusive end on the aligned grid
     const int n_chunks = (g_end + CHUNK - 1) / CHUNK;
@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
     int4 x[ITER];
 #pragma unroll
     for (int i = 0; i < ITER; ++i) {
-        const int v = v0 + i * kLookupThreads + tid;
+        const int v = v0 + i * THREADS + tid;
         if (4 * v < g_end) x[i] = ld_hist(vbase + v);
         else x[i] = make_int4(0, 0, 0, 0);
     }
@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
 
 #pragma unroll
     for (int i = 0; i < ITER; ++i) {
-        const int p0 = 4 * (v0 + i * kLookupThreads + tid) - mis;  // position of x[i].x
+        const int p0 = 4 * (v0 + i * THREADS + tid) - mis;  // position of x[i].x
         uint32_t m = 0;
         m |= (x[i].x == q0 && p0 + 0 >= 0 && p0 + 0 <= n - 2) ? 1u : 0u;
         m |= (x[i].y == q0 && p0 + 1 >= 0 && p0 + 1 <= n - 2) ? 2u : 0u;
@@ -158,15 +158,15 @@ __global__ void __launch_bounds__(kLookupThreads) lookup_kernel(const LookupArgs
         }
     }
 
-    __shared__ unsigned long long s_key[kLookupThreads / 32];
-    __shared__ uint32_t s_cnt[kLookupThreads / 32];
+    __shared__ unsigned long long s_key[THREADS / 32];
+    __shared__ uint32_t s_cnt[THREADS / 32];
     if (lane == 0) { s_key[warp] = best.key; s_cnt[warp] = best.cnt; }
     __syncthreads();
     if (warp != 0) return;
 
     Best r;
-    r.key = lane < kLookupThreads / 32 ? s_key[lane] : 0ull;
-    r.cnt = lane < kLookupThreads / 32 ? s_cnt[lane] : 0u;
+    r.key = lane < THREADS / 32 ? s_key[lane] : 0ull;
+    r.cnt = lane < THREADS / 32 ? s_cnt[lane] : 0u;
     r = warp_combine(r);
 
     uint32_t last = 0;
@@ -242,25 +242,31 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
 
     // aligned-grid tokens to cover: n_max - 1 candidates plus up to 3 tokens of misalignment
     const int64_t span = (int64_t)(n_max > 1 ? n_max - 1 : 1) + 3;
-    // pick the loads per thread so that the grid is about two resident waves at most
-    const int64_t resident = (int64_t)ctx->num_sms * (2048 / kLookupThreads);
-    int iter = 1;
-    while (iter < 8 && ((span + (int64_t)kLookupMinChunk * iter - 1) / ((int64_t)kLookupMinChunk * iter)) * B > 2 * resident)
-        iter *= 2;
-    const int64_t chunk = (int64_t)kLookupMinChunk * iter;
+    // The kernel is a chain of dependent global round trips, and a request that fits one CTA skips
+    // two of them (no partials, no last-arrival counter): take the smallest CTA shape that covers
+    // the span, up to 1024 threads x 8 loads (32 K tokens, 128 KB in flight); longer histories are
+    // cut into chunks of that size.
+    struct Shape { int threads, iter; };
+    static const Shape shapes[] = {{256, 1}, {256, 2}, {256, 4}, {256, 8}, {256, 16}, {1024, 8}};
+    int pick = 5;
+    for (int k = 0; k < 6; ++k)
+        if ((int64_t)shapes[k].threads * kLookupTokPerVec * shapes[k].iter >= span) { pick = k; break; }
+    const int64_t chunk = (int64_t)shapes[pick].threads * kLookupTokPerVec * shapes[pick].iter;
     const int64_t chunks = (span + chunk - 1) / chunk;
     if (chunks > ctx->lk_max_chunks) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max exceeds max_hist_len");
     dim3 grid((unsigned)chunks, (unsigned)B);
     cudaError_t e;
     const ScoreArgs sa = fused ? *fused : ScoreArgs();
-#define HVD_LAUNCH_LOOKUP(I)                                                                              \
-    (fused ? launch_kernel(ctx->use_pdl, lookup_kernel<I, true>, grid, kLookupThreads, 0, stream, a, sa)  \
-           : launch_kernel(ctx->use_pdl, lookup_kernel<I, false>, grid, kLookupThreads, 0, stream, a, sa))
-    switch (iter) {
-        case 1: e = HVD_LAUNCH_LOOKUP(1); break;
-        case 2: e = HVD_LAUNCH_LOOKUP(2); break;
-        case 4: e = HVD_LAUNCH_LOOKUP(4); break;
-        default: e = HVD_LAUNCH_LOOKUP(8); break;
+#define HVD_LAUNCH_LOOKUP(TH, I)                                                                       \
+    (fused ? launch_kernel(ctx->use_pdl, lookup_kernel<TH, I, true>, grid, TH, 0, stream, a, sa)      \
+           : launch_kernel(ctx->use_pdl, lookup_kernel<TH, I, false>, grid, TH, 0, stream, a, sa))
+    switch (pick) {
+        case 0: e = HVD_LAUNCH_LOOKUP(256, 1); break;
+        case 1: e = HVD_LAUNCH_LOOKUP(256, 2); break;
+        case 2: e = HVD_LAUNCH_LOOKUP(256, 4); break;
+        case 3: e = HVD_LAUNCH_LOOKUP(256, 8); break;
+        case 4: e = HVD_LAUNCH_LOOKUP(256, 16); break;
+        default: e = HVD_LAUNCH_LOOKUP(1024, 8); break;
     }
 #undef HVD_LAUNCH_LOOKUP
     HVD_CUDA_TRY(ctx, e);

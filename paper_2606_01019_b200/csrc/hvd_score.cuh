@@ -42,10 +42,13 @@ __device__ __forceinline__ int bit_width(uint32_t x) { return 32 - __clz((int)x)
 __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, int lane, float* s_hid, int n,
                                                      int d, int L, int pos, int cnt, int tok0, int tok1) {
     n = max(n, 0);
-    const int P = max(a.prompt_len[b], 0);
-    const hvd_req_state st = a.state[b];
+    // read-only inputs go through the non-coherent path so that the compiler may issue them early
+    const int P = max(__ldg(a.prompt_len + b), 0);
+    hvd_req_state st;
+    st.sel_bits = __ldg(&a.state[b].sel_bits);
+    st.acc_ring = __ldg(reinterpret_cast<const unsigned long long*>(&a.state[b].acc_ring));
     const int kc = a.k_cap;
-    const int K = max(0, min(a.K[b], kc));
+    const int K = max(0, min(__ldg(a.K + b), kc));
     d = max(0, min(d, kc));
     cnt = max(cnt, 0);
 
@@ -72,8 +75,10 @@ __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, 
     }
 
     for (int j = lane; j < a.hidden; j += 32) {
-        float acc = a.b1[j];
-        const float* w = a.W1 + (int64_t)j * HVD_N_FEATURES;
+        float acc = __ldg(a.b1 + j);
+        const float4* w4 = reinterpret_cast<const float4*>(a.W1 + (int64_t)j * HVD_N_FEATURES);  // 32-byte rows
+        const float4 wa = __ldg(w4), wb = __ldg(w4 + 1);
+        const float w[HVD_N_FEATURES] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
         for (int i = 0; i < HVD_N_FEATURES; ++i) acc = __fmaf_rn(w[i], phi[i], acc);
         s_hid[j] = acc > 0.0f ? acc : 0.0f;
@@ -81,7 +86,7 @@ __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, 
     __syncwarp();
     float y = a.b2;
     if (lane == 0) {
-        for (int j = 0; j < a.hidden; ++j) y = __fmaf_rn(a.W2[j], s_hid[j], y);
+        for (int j = 0; j < a.hidden; ++j) y = __fmaf_rn(__ldg(a.W2 + j), s_hid[j], y);
     }
     y = __shfl_sync(0xffffffffu, y, 0);
     const int sel = (d > 0 && y >= a.tau) ? 1 : 0;
@@ -91,10 +96,10 @@ __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, 
         m = 0;
         tok0 = tok1 = -1;
         if (a.model_draft && a.model_len) {
-            m = max(0, min(a.model_len[b], K));
+            m = max(0, min(__ldg(a.model_len + b), K));
             const int32_t* src = a.model_draft + (int64_t)b * kc;
-            if (lane < m) tok0 = src[lane];
-            if (lane + 32 < m) tok1 = src[lane + 32];
+            if (lane < m) tok0 = __ldg(src + lane);
+            if (lane + 32 < m) tok1 = __ldg(src + lane + 32);
         }
     }
     if (lane < kc) a.sel_draft[(int64_t)b * kc + lane] = (lane < m) ? tok0 : -1;
