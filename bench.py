@@ -237,7 +237,7 @@ def main():
     state0 = torch.as_tensor(rq.state.view(np.int64).reshape(B, 2), device=dev)
     model_draft, model_len = up(rq.model_draft, np.int32), up(rq.model_len, np.int32)
     row_off = up(rq.row_off, np.int64)
-    n_max = int(rq.hist_cap.max())
+    n_max = int(rq.hist_len.max())   # every timed step starts from the pristine lengths
     i32 = lambda *s: torch.zeros(s, dtype=torch.int32, device=dev)
     draft, draft_len, match_len, match_pos, match_cnt = i32(B, kc), i32(B), i32(B), i32(B), i32(B)
     score = torch.zeros(B, dtype=torch.float32, device=dev)

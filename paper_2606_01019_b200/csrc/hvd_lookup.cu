@@ -67,7 +67,7 @@ __device__ __forceinline__ int4 ld_hist(const int4* p) {
 }
 
 template <int THREADS, int ITER, bool FUSED>
-__global__ void __launch_bounds__(THREADS, 1) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
+__global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 512 ? 2 : 4))) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
     __shared__ float s_hid[FUSED ? HVD_MAX_HIDDEN : 1];
     const int b = blockIdx.y;
     const int chunk = blockIdx.x;
@@ -244,13 +244,18 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
     const int64_t span = (int64_t)(n_max > 1 ? n_max - 1 : 1) + 3;
     // The kernel is a chain of dependent global round trips, and a request that fits one CTA skips
     // two of them (no partials, no last-arrival counter): take the smallest CTA shape that covers
-    // the span, up to 1024 threads x 8 loads (32 K tokens, 128 KB in flight); longer histories are
-    // cut into chunks of that size.
+    // the candidate positions, up to 32 K tokens (128 KB in flight); a misaligned slab may spill into
+    // a second chunk, which is launched but exits at once.  Longer histories are cut into chunks of
+    // 8 K tokens (256 threads x 8 loads, four CTAs per SM).
     struct Shape { int threads, iter; };
-    static const Shape shapes[] = {{256, 1}, {256, 2}, {256, 4}, {256, 8}, {256, 16}, {1024, 8}};
-    int pick = 5;
+    // single-CTA shapes by size class (wide CTAs with few loads per thread finish soonest), then
+    // the chunk shape for longer histories
+    static const Shape shapes[] = {{256, 1}, {256, 2}, {512, 2}, {1024, 2}, {1024, 4}, {1024, 8}, {512, 16}, {256, 8}};
+    int pick = 7;
     for (int k = 0; k < 6; ++k)
-        if ((int64_t)shapes[k].threads * kLookupTokPerVec * shapes[k].iter >= span) { pick = k; break; }
+        if ((int64_t)shapes[k].threads * kLookupTokPerVec * shapes[k].iter >= n_max - 1) { pick = k; break; }
+    // 32 K tokens: one 1024-thread CTA per SM; with more requests than SMs, two 512-thread CTAs per SM
+    if (pick == 5 && B > ctx->num_sms) pick = 6;
     const int64_t chunk = (int64_t)shapes[pick].threads * kLookupTokPerVec * shapes[pick].iter;
     const int64_t chunks = (span + chunk - 1) / chunk;
     if (chunks > ctx->lk_max_chunks) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max exceeds max_hist_len");
@@ -263,10 +268,12 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
     switch (pick) {
         case 0: e = HVD_LAUNCH_LOOKUP(256, 1); break;
         case 1: e = HVD_LAUNCH_LOOKUP(256, 2); break;
-        case 2: e = HVD_LAUNCH_LOOKUP(256, 4); break;
-        case 3: e = HVD_LAUNCH_LOOKUP(256, 8); break;
-        case 4: e = HVD_LAUNCH_LOOKUP(256, 16); break;
-        default: e = HVD_LAUNCH_LOOKUP(1024, 8); break;
+        case 2: e = HVD_LAUNCH_LOOKUP(512, 2); break;
+        case 3: e = HVD_LAUNCH_LOOKUP(1024, 2); break;
+        case 4: e = HVD_LAUNCH_LOOKUP(1024, 4); break;
+        case 5: e = HVD_LAUNCH_LOOKUP(1024, 8); break;
+        case 6: e = HVD_LAUNCH_LOOKUP(512, 16); break;
+        default: e = HVD_LAUNCH_LOOKUP(256, 8); break;
     }
 #undef HVD_LAUNCH_LOOKUP
     HVD_CUDA_TRY(ctx, e);

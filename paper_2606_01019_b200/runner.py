@@ -33,7 +33,11 @@ class DeviceBatch:
         self.total_rows = int(row_off[-1])
         self.k_uniform = int(row_off[1] - row_off[0]) - 1 if uniform_rows else 0
         self.row_off = None if uniform_rows else up(row_off, np.int64)
-        self.n_max = int(max(0, np.max(hist_cap))) if len(hist_cap) else 0
+        # host-side upper bound on hist_len: the longest valid history now, raised by every commit
+        self.cap_max = int(max(0, np.max(hist_cap))) if len(hist_cap) else 0
+        hl = np.asarray(hist_len, np.int64)
+        ok = (hl >= 0) & (hl <= np.asarray(hist_cap, np.int64))
+        self.n_max = int(hl[ok].max()) if ok.any() else 0
         B = self.B
         i32 = lambda *s: torch.full(s, -12345, dtype=torch.int32, device=self.dev)
         self.draft, self.draft_len = i32(B, kc), i32(B)
@@ -68,6 +72,7 @@ class DeviceBatch:
                                    self.hist_off, self.hist_cap, self.hist_len, self.state,
                                    self.accepted, self.committed, self.n_commit,
                                    self.target_tok if target_tok else None, self.status)
+        self.n_max = min(self.cap_max, self.n_max + self.ctx.k_cap + 1)
 
     def step(self, logits, target_tok=True, fused=False):
         if fused:
