@@ -153,7 +153,8 @@ def run_reference(args):
         rows = int(inp.rq.row_off[B_s])
         keep = slice(0, B_s)
         sub = P.Inputs(w, W.subset_requests(inp.rq, 0, B_s), inp.W1, inp.b1, inp.W2, inp.b2, inp.tau,
-                       inp.A[keep], inp.strict[keep], inp.logits[:rows], inp.logits_np[:rows])
+                       Wh=inp.Wh, bh=inp.bh, A=inp.A[keep], strict=inp.strict[keep], logits=inp.logits[:rows],
+                       logits_np=inp.logits_np[:rows])
     times, committed = [], 0
     for i in range(args.warmup + args.steps):
         rq = sub.rq.copy()
@@ -290,9 +291,12 @@ def main():
         hist_len_steps.copy_(hist_len_pristine)
         state_steps.copy_(state_pristine)
 
-    def step(slot, events=None, with_verify=True):
+    def step(slot, events=None, with_verify=True, lookup_only=False):
         r = slot % R
         hl, st = hist_len_steps[slot], state_steps[slot]
+        if lookup_only:
+            lookup(hists[r], hl)
+            return
         if events is not None:
             events[0].record()
         if args.unfused:
@@ -314,12 +318,12 @@ def main():
     mode = args.mode
     stream = torch.cuda.Stream(device=dev)
 
-    def capture(events=None, with_verify=True):
+    def capture(events=None, with_verify=True, lookup_only=False):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
             g.capture_begin()
             for s in range(K_steps):
-                step(W_steps + s, events[s] if events else None, with_verify)
+                step(W_steps + s, events[s] if events else None, with_verify, lookup_only)
             g.capture_end()
         torch.cuda.synchronize()
         with torch.cuda.stream(stream):
@@ -392,10 +396,13 @@ def main():
                 g_nv = capture(None, with_verify=False)
                 restore()
                 t_nv = timed(g_nv.replay)
+                g_lk = capture(None, lookup_only=True)
+                t_lk = timed(g_lk.replay)
             else:
                 t_ev = timed(lambda: [step(W_steps + s, evs[s]) for s in range(K_steps)])
                 restore()
                 t_nv = timed(lambda: [step(W_steps + s, None, False) for s in range(K_steps)])
+                t_lk = timed(lambda: [step(W_steps + s, None, False, True) for s in range(K_steps)])
             restore()
             d = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(2)] for e in evs])
             kt = {"lookup_plus_score_select_us": 1e3 * float(d[:, 0].mean()),
@@ -403,6 +410,7 @@ def main():
                   "verify_commit_us_median": 1e3 * float(np.median(d[:, 1])),
                   "step_us_with_event_records": 1e3 * t_ev / K_steps,
                   "step_us_without_verify": 1e3 * t_nv / K_steps,
+                  "lookup_only_us": 1e3 * t_lk / K_steps,
                   "verify_commit_us_by_difference": 1e3 * (elapsed_ms - t_nv) / K_steps,
                   "note": "event-bracketed times include the serialisation the event records add; "
                           "the headline region has no records in it"}
@@ -420,11 +428,16 @@ def main():
     roofline = {"bound": "hbm", "kernel": "verify_stream_kernel (+ verify_commit_kernel)", "achieved": None, "peak": peak_gbs, "unit": "GB/s",
                 "frac": None, "traffic": NCU_VERIFY_TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": verify_bytes}
+    roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel (hvd_lookup alone, back to back in one graph)",
+                       "achieved": None, "peak": peak_gbs, "unit": "GB/s", "frac": None, "traffic": None,
+                       "peak_kind": peak_kind, "algorithmic_bytes_per_launch": lookup_bytes}
     if kt:
         roofline["achieved"] = verify_bytes / (kt["verify_commit_us"] * 1e-6) / 1e9
         roofline["frac"] = roofline["achieved"] / peak_gbs
         roofline["frac_of_8000_nominal"] = roofline["achieved"] / 8000.0
         roofline["achieved_by_difference"] = verify_bytes / (kt["verify_commit_us_by_difference"] * 1e-6) / 1e9
+        roofline_lookup["achieved"] = lookup_bytes / (kt["lookup_only_us"] * 1e-6) / 1e9
+        roofline_lookup["frac"] = roofline_lookup["achieved"] / peak_gbs
         roofline["timing"] = "CUDA events recorded around the hvd_verify_commit call inside the graph"
 
     # ---- end to end through the host-buffer entry point --------------------------------------------
@@ -475,7 +488,7 @@ def main():
         from oracle import pipeline as P
         cores = P.host_threads()
         logits_np = W.logits_to_numpy(logits0)
-        inp = P.Inputs(w, rq, W1, b1, W2, b2, tau, A, np.ones(B, bool), None, logits_np)
+        inp = P.Inputs(w, rq, W1, b1, W2, b2, tau, A=A, strict=np.ones(B, bool), logits_np=logits_np)
         times, out = [], None
         t_begin = time.perf_counter()
         while len(times) < 5 or (time.perf_counter() - t_begin < 10.0 and len(times) < 200):
@@ -507,7 +520,8 @@ def main():
                 "tokens_per_s": world * K_steps * tokens_per_step / (elapsed_ms * 1e-3),
                 "tokens_per_step": tokens_per_step,
                 "mean_accepted": float(accepted_h.mean()), "cache_selected_frac": float(select_h.mean()),
-                "kernel_us": kt, "roofline": roofline, "lookup_algorithmic_bytes": lookup_bytes,
+                "kernel_us": kt, "roofline": roofline, "roofline_lookup": roofline_lookup,
+                "lookup_algorithmic_bytes": lookup_bytes,
                 "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": (4 if args.unfused else 3) * K_steps,
                 "clocks": sampler.summary(window)}
         print(json.dumps(line), flush=True)

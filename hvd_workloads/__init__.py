@@ -69,6 +69,7 @@ class Workload:
     b2: float
     calibrate_cache_frac: Optional[float] = None   # tau := score quantile so this fraction selects cache
     hidden: int = 32
+    hidden_layers: int = 1          # 2: the paper's predictor shape (two hidden layers)
     min_match: int = 2
     l_max: int = 64
     filler_run: Tuple[int, int] = (16, 256)
@@ -318,6 +319,17 @@ def make_predictor(w: Workload):
     b1 = rng.normal(0.0, 0.1, H).astype(np.float32)
     W2 = rng.normal(0.0, 0.1, H).astype(np.float32)
     return W1, b1, W2, float(np.float32(w.b2)), float(np.float32(w.tau))
+
+
+def make_second_layer(w: Workload):
+    """Wh [H,H], bh [H] ~ N(0, 0.1^2) fp32 of the second hidden layer (drawn after W1, b1, W2 from the
+    same stream, so the one-layer weights do not change)."""
+    rng = _rng(w.index, S_WEIGHTS)
+    H = w.hidden
+    rng.normal(0.0, 0.1, (H, 8)); rng.normal(0.0, 0.1, H); rng.normal(0.0, 0.1, H)
+    Wh = rng.normal(0.0, 0.1, (H, H)).astype(np.float32)
+    bh = rng.normal(0.0, 0.1, H).astype(np.float32)
+    return Wh, bh
 
 
 def calibrate_tau(scores: np.ndarray, eligible: np.ndarray, frac: float) -> float:

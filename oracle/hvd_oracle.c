@@ -201,12 +201,51 @@ double oracle_mlp_f64(const float* phi, int32_t F, int32_t H, const float* W1, c
     return y;
 }
 
+/* The same predictor with a second hidden ReLU layer (the paper's trained predictor has two hidden
+   layers of 256 units: App. B, table "Payoff predictor training configuration"):
+   h1 = relu(W1 phi + b1), h2 = relu(Wh h1 + bh), y = b2 + W2 . h2; same left-to-right fmaf chains. */
+float oracle_mlp2_f32(const float* phi, int32_t F, int32_t H, const float* W1 /*[H,F]*/, const float* b1,
+                      const float* Wh /*[H,H]*/, const float* bh, const float* W2, float b2) {
+    float h1[1024];
+    for (int32_t j = 0; j < H; ++j) {
+        float acc = b1[j];
+        for (int32_t i = 0; i < F; ++i) acc = fmaf(W1[(int64_t)j * F + i], phi[i], acc);
+        h1[j] = acc > 0.0f ? acc : 0.0f;
+    }
+    float y = b2;
+    for (int32_t j = 0; j < H; ++j) {
+        float acc = bh[j];
+        for (int32_t i = 0; i < H; ++i) acc = fmaf(Wh[(int64_t)j * H + i], h1[i], acc);
+        float hid = acc > 0.0f ? acc : 0.0f;
+        y = fmaf(W2[j], hid, y);
+    }
+    return y;
+}
+
+double oracle_mlp2_f64(const float* phi, int32_t F, int32_t H, const float* W1, const float* b1,
+                       const float* Wh, const float* bh, const float* W2, float b2) {
+    double h1[1024];
+    for (int32_t j = 0; j < H; ++j) {
+        double acc = (double)b1[j];
+        for (int32_t i = 0; i < F; ++i) acc += (double)W1[(int64_t)j * F + i] * (double)phi[i];
+        h1[j] = acc > 0.0 ? acc : 0.0;
+    }
+    double y = (double)b2;
+    for (int32_t j = 0; j < H; ++j) {
+        double acc = (double)bh[j];
+        for (int32_t i = 0; i < H; ++i) acc += (double)Wh[(int64_t)j * H + i] * h1[i];
+        y += (double)W2[j] * (acc > 0.0 ? acc : 0.0);
+    }
+    return y;
+}
+
 typedef struct {
     const int32_t *hist_len, *prompt_len; const oracle_req_state* state; const int32_t* K;
     const int32_t *draft, *draft_len, *match_len, *match_pos, *match_cnt;
     const int32_t *model_draft, *model_len; int32_t k_cap, H;
     const float *W1, *b1, *W2; float b2, tau;
     float *features, *score; double* score64; int32_t *select, *sel_draft, *sel_len;
+    const float *Wh, *bh; /* second hidden layer, NULL for the one-layer predictor */
 } score_args;
 
 static void score_req(int32_t b, void* p) {
@@ -222,9 +261,12 @@ static void score_req(int32_t b, void* p) {
     oracle_features_one(a->hist_len[b], a->prompt_len[b], a->state[b], d, a->match_len[b],
                         a->match_pos[b], a->match_cnt[b], phi);
     if (a->features) memcpy(a->features + (int64_t)b * ORACLE_N_FEATURES, phi, sizeof(phi));
-    float y = oracle_mlp_f32(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->W2, a->b2);
+    float y = a->Wh ? oracle_mlp2_f32(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->Wh, a->bh, a->W2, a->b2)
+                    : oracle_mlp_f32(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->W2, a->b2);
     a->score[b] = y;
-    if (a->score64) a->score64[b] = oracle_mlp_f64(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->W2, a->b2);
+    if (a->score64)
+        a->score64[b] = a->Wh ? oracle_mlp2_f64(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->Wh, a->bh, a->W2, a->b2)
+                              : oracle_mlp_f64(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->W2, a->b2);
     /* cache draft is verified iff it exists and its predicted payoff reaches the threshold */
     int32_t sel = (d > 0 && y >= a->tau) ? 1 : 0;
     a->select[b] = sel;
@@ -254,7 +296,21 @@ void oracle_score_select(int32_t B, const int32_t* hist_len, const int32_t* prom
                          int32_t* select, int32_t* sel_draft, int32_t* sel_len, int32_t nthreads) {
     score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
                     model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
-                    select, sel_draft, sel_len};
+                    select, sel_draft, sel_len, NULL, NULL};
+    for_each_request(B, nthreads, score_req, &a);
+}
+
+void oracle_score_select2(int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
+                          const oracle_req_state* state, const int32_t* K, const int32_t* draft,
+                          const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
+                          const int32_t* match_cnt, const int32_t* model_draft, const int32_t* model_len,
+                          int32_t k_cap, int32_t H, const float* W1, const float* b1, const float* Wh,
+                          const float* bh, const float* W2, float b2, float tau, float* features, float* score,
+                          double* score64, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
+                          int32_t nthreads) {
+    score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
+                    model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
+                    select, sel_draft, sel_len, Wh, bh};
     for_each_request(B, nthreads, score_req, &a);
 }
 

@@ -43,6 +43,8 @@ def lib():
         _lib.oracle_argmax_row.restype = C.c_int32
         _lib.oracle_mlp_f32.restype = C.c_float
         _lib.oracle_mlp_f64.restype = C.c_double
+        _lib.oracle_mlp2_f32.restype = C.c_float
+        _lib.oracle_mlp2_f64.restype = C.c_double
     return _lib
 
 
@@ -89,12 +91,16 @@ class ScoreOut:
 
 
 def score_select(hist_len, prompt_len, state, K, lk: LookupOut, model_draft, model_len, *, k_cap,
-                 W1, b1, W2, b2, tau, nthreads=1) -> ScoreOut:
+                 W1, b1, W2, b2, tau, nthreads=1, Wh=None, bh=None) -> ScoreOut:
+    """Wh [H,H], bh [H]: optional second hidden layer (between W1/b1 and the output weights W2/b2)."""
     B = len(hist_len)
     H = int(np.asarray(W2).shape[0])
     W1 = np.ascontiguousarray(W1, np.float32); b1 = np.ascontiguousarray(b1, np.float32)
     W2 = np.ascontiguousarray(W2, np.float32)
     assert W1.shape == (H, N_FEATURES)
+    if Wh is not None:
+        Wh = np.ascontiguousarray(Wh, np.float32); bh = np.ascontiguousarray(bh, np.float32)
+        assert Wh.shape == (H, H) and bh.shape == (H,) and H <= 1024
     state = np.ascontiguousarray(state, dtype=STATE_DTYPE)
     hist_len = _i32(hist_len); prompt_len = _i32(prompt_len); K = _i32(K)
     md = None if model_draft is None else _i32(model_draft)
@@ -102,12 +108,16 @@ def score_select(hist_len, prompt_len, state, K, lk: LookupOut, model_draft, mod
     out = ScoreOut(np.empty((B, N_FEATURES), np.float32), np.empty(B, np.float32),
                    np.empty(B, np.float64), np.empty(B, np.int32), np.empty((B, k_cap), np.int32),
                    np.empty(B, np.int32))
-    lib().oracle_score_select(C.c_int32(B), _p(hist_len), _p(prompt_len), _p(state), _p(K),
-                              _p(_i32(lk.draft)), _p(_i32(lk.draft_len)), _p(_i32(lk.match_len)),
-                              _p(_i32(lk.match_pos)), _p(_i32(lk.match_cnt)), _p(md), _p(ml),
-                              C.c_int32(k_cap), C.c_int32(H), _p(W1), _p(b1), _p(W2), C.c_float(b2),
-                              C.c_float(tau), _p(out.features), _p(out.score), _p(out.score64),
-                              _p(out.select), _p(out.sel_draft), _p(out.sel_len), C.c_int32(nthreads))
+    head = (C.c_int32(B), _p(hist_len), _p(prompt_len), _p(state), _p(K),
+            _p(_i32(lk.draft)), _p(_i32(lk.draft_len)), _p(_i32(lk.match_len)),
+            _p(_i32(lk.match_pos)), _p(_i32(lk.match_cnt)), _p(md), _p(ml),
+            C.c_int32(k_cap), C.c_int32(H), _p(W1), _p(b1))
+    tail = (_p(W2), C.c_float(b2), C.c_float(tau), _p(out.features), _p(out.score), _p(out.score64),
+            _p(out.select), _p(out.sel_draft), _p(out.sel_len), C.c_int32(nthreads))
+    if Wh is None:
+        lib().oracle_score_select(*head, *tail)
+    else:
+        lib().oracle_score_select2(*head, _p(Wh), _p(bh), *tail)
     return out
 
 
@@ -167,6 +177,18 @@ def mlp_f64(phi, W1, b1, W2, b2) -> float:
     b1 = np.ascontiguousarray(b1, np.float32); W2 = np.ascontiguousarray(W2, np.float32)
     return float(lib().oracle_mlp_f64(_p(phi), C.c_int32(phi.size), C.c_int32(W2.size), _p(W1), _p(b1),
                                       _p(W2), C.c_float(b2)))
+
+
+def mlp2_f32(phi, W1, b1, Wh, bh, W2, b2) -> float:
+    a = [np.ascontiguousarray(x, np.float32) for x in (phi, W1, b1, Wh, bh, W2)]
+    return float(lib().oracle_mlp2_f32(_p(a[0]), C.c_int32(a[0].size), C.c_int32(a[5].size), _p(a[1]), _p(a[2]),
+                                       _p(a[3]), _p(a[4]), _p(a[5]), C.c_float(b2)))
+
+
+def mlp2_f64(phi, W1, b1, Wh, bh, W2, b2) -> float:
+    a = [np.ascontiguousarray(x, np.float32) for x in (phi, W1, b1, Wh, bh, W2)]
+    return float(lib().oracle_mlp2_f64(_p(a[0]), C.c_int32(a[0].size), C.c_int32(a[5].size), _p(a[1]), _p(a[2]),
+                                       _p(a[3]), _p(a[4]), _p(a[5]), C.c_float(b2)))
 
 
 def features_one(n, prompt_len, sel_bits, acc_ring, draft_len, match_len, match_pos, match_cnt):

@@ -28,10 +28,12 @@ class Inputs:
     W2: np.ndarray
     b2: float
     tau: float
-    A: np.ndarray           # planted accepted lengths
-    strict: np.ndarray      # requests on which accepted == A must hold
-    logits: object          # torch tensor [rows, V] on the device it was drawn on
-    logits_np: np.ndarray   # host copy (float32, or uint16 bf16 bit patterns)
+    Wh: object = None       # second hidden layer [H,H] (None: one-layer predictor)
+    bh: object = None
+    A: np.ndarray = None    # planted accepted lengths
+    strict: np.ndarray = None      # requests on which accepted == A must hold
+    logits: object = None          # torch tensor [rows, V] on the device it was drawn on
+    logits_np: np.ndarray = None   # host copy (float32, or uint16 bf16 bit patterns)
 
 
 @dataclass
@@ -46,9 +48,9 @@ def lookup(w, rq, nthreads=1):
                     l_max=w.l_max, min_match=w.min_match, nthreads=nthreads)
 
 
-def score_select(w, rq, lk, W1, b1, W2, b2, tau, nthreads=1):
+def score_select(w, rq, lk, W1, b1, W2, b2, tau, nthreads=1, Wh=None, bh=None):
     return O.score_select(rq.hist_len, rq.prompt_len, rq.state, rq.K, lk, rq.model_draft, rq.model_len,
-                          k_cap=w.k_cap, W1=W1, b1=b1, W2=W2, b2=b2, tau=tau, nthreads=nthreads)
+                          k_cap=w.k_cap, W1=W1, b1=b1, W2=W2, b2=b2, tau=tau, nthreads=nthreads, Wh=Wh, bh=bh)
 
 
 def verify_commit(w, rq, sc, logits_np, nthreads=1):
@@ -63,21 +65,22 @@ def prepare(w: W.Workload, device="cpu", nthreads=None, salt: int = 0, rq: W.Req
     nthreads = nthreads or host_threads()
     rq = W.make_requests(w) if rq is None else rq
     W1, b1, W2, b2, tau = W.make_predictor(w)
+    Wh, bh = W.make_second_layer(w) if w.hidden_layers == 2 else (None, None)
     lk = lookup(w, rq, nthreads)
-    sc = score_select(w, rq, lk, W1, b1, W2, b2, tau, nthreads)
+    sc = score_select(w, rq, lk, W1, b1, W2, b2, tau, nthreads, Wh, bh)
     if w.calibrate_cache_frac is not None:
         tau = W.calibrate_tau(sc.score, lk.draft_len > 0, w.calibrate_cache_frac)
-        sc = score_select(w, rq, lk, W1, b1, W2, b2, tau, nthreads)
+        sc = score_select(w, rq, lk, W1, b1, W2, b2, tau, nthreads, Wh, bh)
     A = W.make_agreement(w, sc.sel_len)
     logits = W.make_logits(w, max(int(rq.row_off[-1]), 1), device=device, salt=salt)
     strict = W.plant_agreement(w, logits, rq.row_off, sc.sel_draft, sc.sel_len, A, salt=salt)
-    return Inputs(w, rq, W1, b1, W2, b2, tau, A, strict, logits, W.logits_to_numpy(logits))
+    return Inputs(w, rq, W1, b1, W2, b2, tau, Wh, bh, A, strict, logits, W.logits_to_numpy(logits))
 
 
 def step(inp: Inputs, rq: W.Requests, nthreads=1, logits_np=None) -> StepOut:
     """One decoding step on `rq` (updated in place: history, lengths, state)."""
     w = inp.w
     lk = lookup(w, rq, nthreads)
-    sc = score_select(w, rq, lk, inp.W1, inp.b1, inp.W2, inp.b2, inp.tau, nthreads)
+    sc = score_select(w, rq, lk, inp.W1, inp.b1, inp.W2, inp.b2, inp.tau, nthreads, inp.Wh, inp.bh)
     vf = verify_commit(w, rq, sc, inp.logits_np if logits_np is None else logits_np, nthreads)
     return StepOut(lk, sc, vf)

@@ -74,7 +74,7 @@ lo, hi = int(bounds[rank]), int(bounds[rank + 1])
 # each rank steps only its own requests (here with the CPU oracle standing in for the device)
 sub = W.subset_requests(inp.rq, lo, hi)
 rows = slice(int(inp.rq.row_off[lo]), int(inp.rq.row_off[hi]))
-part = P.Inputs(w, sub, inp.W1, inp.b1, inp.W2, inp.b2, inp.tau, inp.A[lo:hi], inp.strict[lo:hi], None, inp.logits_np[rows])
+part = P.Inputs(w, sub, inp.W1, inp.b1, inp.W2, inp.b2, inp.tau, A=inp.A[lo:hi], strict=inp.strict[lo:hi], logits_np=inp.logits_np[rows])
 out = P.step(part, sub.copy())
 full = P.step(inp, inp.rq.copy())
 assert (out.vf.accepted == full.vf.accepted[lo:hi]).all() and (out.vf.committed == full.vf.committed[lo:hi]).all()

@@ -123,3 +123,61 @@ def test_scores_on_workload_fp32_vs_fp64():
     assert ((sc.select == 1) == ((lk.draft_len > 0) & (sc.score >= np.float32(tau)))).all()
     assert (sc.sel_len[sc.select == 1] == lk.draft_len[sc.select == 1]).all()
     assert (sc.sel_len[sc.select == 0] == rq.model_len[sc.select == 0]).all()
+
+
+# ---- two hidden layers: the paper's predictor shape (App. B: 2 hidden layers, ReLU) -------------------
+def test_mlp2_closed_forms():
+    H, F = 16, 8
+    phi = np.arange(1, 9, dtype=np.float32) * f32(0.25)
+    Z1, z, ZH = np.zeros((H, F), np.float32), np.zeros(H, np.float32), np.zeros((H, H), np.float32)
+    assert O.mlp2_f32(phi, Z1, z, ZH, z, z, 3.5) == 3.5                       # all zero: y = output bias
+    # a single path phi_k -> h1[a] -> h2[c] -> y with unit weights: y = b + relu(relu(phi_k + b1) + bh)
+    for k, a, c in [(0, 0, 0), (5, 3, 11), (7, 15, 2)]:
+        W1 = Z1.copy(); W1[a, k] = 1.0
+        Wh = ZH.copy(); Wh[c, a] = 1.0                                            # row c reads h1[a]
+        W2 = z.copy(); W2[c] = 1.0
+        b1 = z.copy(); b1[a] = 0.5
+        bh = z.copy(); bh[c] = 0.125
+        assert O.mlp2_f32(phi, W1, b1, Wh, bh, W2, 1.0) == f32(1.0) + ((phi[k] + f32(0.5)) + f32(0.125))
+        if a != c:                                                                # a transposed Wh breaks the path:
+            Wt = ZH.copy(); Wt[a, c] = 1.0                                        # only relu(bh[c]) reaches the output
+            assert O.mlp2_f32(phi, W1, b1, Wt, bh, W2, 1.0) == f32(1.0) + f32(0.125)
+        bh[c] = -100.0                                                            # second ReLU cuts the path
+        assert O.mlp2_f32(phi, W1, b1, Wh, bh, W2, 1.0) == 1.0
+        bh[c] = 0.125; b1[a] = -100.0                                             # first ReLU cuts it: only bh is left
+        assert O.mlp2_f32(phi, W1, b1, Wh, bh, W2, 1.0) == f32(1.0) + f32(0.125)
+    # an identity second layer reduces the network to the one-layer predictor
+    W1 = np.random.default_rng(1).normal(0, 0.1, (H, F)).astype(np.float32)
+    b1 = np.random.default_rng(2).normal(0, 0.1, H).astype(np.float32)
+    W2 = np.random.default_rng(3).normal(0, 0.1, H).astype(np.float32)
+    assert O.mlp2_f32(phi, W1, b1, np.eye(H, dtype=np.float32), z, W2, 2.0) == O.mlp_f32(phi, W1, b1, W2, 2.0)
+
+
+def test_mlp2_against_fp64_and_torch():
+    rng = np.random.default_rng(12)
+    for H in (8, 64, 256):
+        W1 = rng.normal(0, 0.1, (H, 8)).astype(np.float32); b1 = rng.normal(0, 0.1, H).astype(np.float32)
+        Wh = rng.normal(0, 0.1, (H, H)).astype(np.float32); bh = rng.normal(0, 0.1, H).astype(np.float32)
+        W2 = rng.normal(0, 0.1, H).astype(np.float32)
+        for _ in range(20):
+            phi = np.abs(rng.normal(0, 10, 8)).astype(np.float32)
+            y32 = O.mlp2_f32(phi, W1, b1, Wh, bh, W2, 6.0)
+            y64 = O.mlp2_f64(phi, W1, b1, Wh, bh, W2, 6.0)
+            lin = torch.nn.functional.linear
+            d = lambda x: torch.from_numpy(x).double()
+            t = lin(torch.relu(lin(torch.relu(lin(d(phi), d(W1), d(b1))), d(Wh), d(bh))), d(W2)[None],
+                    torch.tensor([6.0]).double())
+            assert abs(y64 - float(t)) <= 1e-12 * max(1.0, abs(y64))
+            assert abs(y32 - y64) <= 2e-5 * max(1.0, abs(y64))
+
+
+def test_two_layer_scores_on_workload():
+    w = W.CONFIGS["C2"].scaled(B=32, n=2048, hidden=256, hidden_layers=2)
+    inp = P.prepare(w)
+    out = P.step(inp, inp.rq.copy())
+    sc = out.sc
+    assert inp.Wh.shape == (256, 256)
+    assert np.abs(sc.score - sc.score64).max() <= 2e-5 * np.abs(sc.score64).max()
+    assert 0 < sc.select.sum() < len(sc.select)
+    for b in range(4):
+        assert sc.score[b] == np.float32(O.mlp2_f32(sc.features[b], inp.W1, inp.b1, inp.Wh, inp.bh, inp.W2, inp.b2))
