@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--predictor", default="config", choices=["config", "2x256"],
+                    help="2x256: the paper's predictor shape (two hidden layers of 256 units) instead of the config's")
     ap.add_argument("--unfused", action="store_true",
                     help="call hvd_lookup and hvd_score_select separately instead of hvd_lookup_score_select")
     ap.add_argument("--no-kernel-events", action="store_true",
@@ -219,6 +221,8 @@ def main():
         torch.cuda.synchronize()
 
     w = W.CONFIGS[args.config]
+    if args.predictor == "2x256":
+        w = w.scaled(hidden=256, hidden_layers=2)
     K_steps, W_steps = args.steps, args.warmup
     n_slots = K_steps + W_steps
     peak_gbs, peak_kind = measured_peak()
@@ -230,7 +234,15 @@ def main():
     total_rows = int(rq.row_off[-1])
     ctx = H.Context(max_batch=B, k_cap=kc, max_hist_len=int(rq.hist_cap.max()), max_rows=total_rows,
                     max_vocab=w.V, l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
-    ctx.hvd_set_predictor(W1, b1, W2, b2, tau)
+    Wh, bh = W.make_second_layer(w) if w.hidden_layers == 2 else (None, None)
+
+    def set_predictor(t):
+        if Wh is not None:
+            ctx.hvd_set_predictor2(W1, b1, Wh, bh, W2, b2, t)
+        else:
+            ctx.hvd_set_predictor(W1, b1, W2, b2, t)
+
+    set_predictor(tau)
     up = lambda a, dt: torch.as_tensor(np.ascontiguousarray(a, dt), device=dev)
     hist0 = up(rq.hist, np.int32)
     hist_off, hist_cap, Kt = up(rq.hist_off, np.int64), up(rq.hist_cap, np.int32), up(rq.K, np.int32)
@@ -269,7 +281,7 @@ def main():
     if w.calibrate_cache_frac is not None:
         torch.cuda.synchronize()
         tau = W.calibrate_tau(score.cpu().numpy(), draft_len.cpu().numpy() > 0, w.calibrate_cache_frac)
-        ctx.hvd_set_predictor(W1, b1, W2, b2, tau)
+        set_predictor(tau)
         score_select(hist_len0, state0)
     torch.cuda.synchronize()
     sel_len_h = sel_len.cpu().numpy()
@@ -488,7 +500,7 @@ def main():
         from oracle import pipeline as P
         cores = P.host_threads()
         logits_np = W.logits_to_numpy(logits0)
-        inp = P.Inputs(w, rq, W1, b1, W2, b2, tau, A=A, strict=np.ones(B, bool), logits_np=logits_np)
+        inp = P.Inputs(w, rq, W1, b1, W2, b2, tau, Wh=Wh, bh=bh, A=A, strict=np.ones(B, bool), logits_np=logits_np)
         times, out = [], None
         t_begin = time.perf_counter()
         while len(times) < 5 or (time.perf_counter() - t_begin < 10.0 and len(times) < 200):
@@ -516,7 +528,8 @@ def main():
                               if graph is not None else f"stream: {4 if args.unfused else 3} kernel launches per step",
                     "entry_points": "hvd_lookup + hvd_score_select + hvd_verify_commit" if args.unfused
                                     else "hvd_lookup_score_select + hvd_verify_commit",
-                    "kernel_events_in_timed_region": False, "tau": tau}),
+                    "kernel_events_in_timed_region": False, "tau": tau,
+                    "predictor": f"8->{w.hidden}" + (f"->{w.hidden}" if w.hidden_layers == 2 else "") + "->1 fp32"}),
                 "tokens_per_s": world * K_steps * tokens_per_step / (elapsed_ms * 1e-3),
                 "tokens_per_step": tokens_per_step,
                 "mean_accepted": float(accepted_h.mean()), "cache_selected_frac": float(select_h.mean()),

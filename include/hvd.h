@@ -106,6 +106,15 @@ HVD_API hvd_status hvd_device_status(hvd_ctx* ctx, int32_t* code);
 HVD_API hvd_status hvd_set_predictor(hvd_ctx* ctx, const float* W1, const float* b1, const float* W2,
                              float b2, float tau, void* stream);
 
+/* The same predictor with two hidden ReLU layers, the shape the paper trains (App. B, table "Payoff
+   predictor training configuration": 2 hidden layers of 256 units):
+   h1 = relu(W1 phi + b1), h2 = relu(Wh h1 + bh), y = b2 + W2 . h2, same accumulation rule.
+   Wh [hidden, hidden] row-major (row j = inputs of unit j), bh [hidden]: HOST pointers, copied before
+   returning.  Afterwards hvd_score_select and hvd_lookup_score_select use this predictor (the
+   latter then runs as two kernels); hvd_set_predictor switches back to one layer. */
+HVD_API hvd_status hvd_set_predictor2(hvd_ctx* ctx, const float* W1, const float* b1, const float* Wh,
+                                      const float* bh, const float* W2, float b2, float tau, void* stream);
+
 /*
  * Cache-based drafting D_C (Sec. 3.2), with the request's own history as the cache.
  * For every request: among the positions e in [1, n-1], find the longest l <= l_max such that

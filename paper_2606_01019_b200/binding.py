@@ -46,6 +46,7 @@ _SIGNATURES = {
     "hvd_last_error": (C.c_char_p, [_vp]),
     "hvd_device_status": (_i32, [_vp, C.POINTER(_i32)]),
     "hvd_set_predictor": (_i32, [_vp, _vp, _vp, _vp, _f32, _f32, _vp]),
+    "hvd_set_predictor2": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _vp]),
     "hvd_lookup": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_score_select": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32] + [_vp] * 14 + [_vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
@@ -165,6 +166,17 @@ class Context:
             raise HvdError("hvd_set_predictor: weight shapes do not match the context")
         self._check(self._lib.hvd_set_predictor(self._h, W1.ctypes.data, b1.ctypes.data, W2.ctypes.data,
                                                 float(b2), float(tau), _stream()), "hvd_set_predictor")
+
+    def hvd_set_predictor2(self, W1, b1, Wh, bh, W2, b2, tau):
+        H = self.hidden
+        W1 = np.ascontiguousarray(W1, np.float32); b1 = np.ascontiguousarray(b1, np.float32)
+        Wh = np.ascontiguousarray(Wh, np.float32); bh = np.ascontiguousarray(bh, np.float32)
+        W2 = np.ascontiguousarray(W2, np.float32)
+        if W1.shape != (H, N_FEATURES) or b1.shape != (H,) or Wh.shape != (H, H) or bh.shape != (H,) or W2.shape != (H,):
+            raise HvdError("hvd_set_predictor2: weight shapes do not match the context")
+        self._check(self._lib.hvd_set_predictor2(self._h, W1.ctypes.data, b1.ctypes.data, Wh.ctypes.data,
+                                                 bh.ctypes.data, W2.ctypes.data, float(b2), float(tau), _stream()),
+                    "hvd_set_predictor2")
 
     def hvd_lookup(self, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len, match_len,
                    match_pos, match_cnt):

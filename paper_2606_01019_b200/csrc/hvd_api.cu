@@ -13,7 +13,7 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 void release(hvd_ctx* c) {
     if (!c) return;
-    cudaFree(c->d_W1); cudaFree(c->d_b1); cudaFree(c->d_W2);
+    cudaFree(c->d_W1); cudaFree(c->d_b1); cudaFree(c->d_W2); cudaFree(c->d_WhT); cudaFree(c->d_bh);
     cudaFree(c->lk_partial); cudaFree(c->lk_cnt);
     cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
@@ -73,6 +73,8 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->d_W1, H * HVD_N_FEATURES * sizeof(float)) == cudaSuccess;
     ok = ok && alloc_zero(&c->d_b1, H * sizeof(float)) == cudaSuccess;
     ok = ok && alloc_zero(&c->d_W2, H * sizeof(float)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->d_WhT, (size_t)HVD_MAX_HIDDEN * HVD_MAX_HIDDEN * sizeof(float)) == cudaSuccess;  // row stride 256
+    ok = ok && alloc_zero(&c->d_bh, H * sizeof(float)) == cudaSuccess;
     ok = ok && alloc_zero(&c->lk_partial, (size_t)cfg->max_batch * c->lk_max_chunks * sizeof(LookupPartial)) == cudaSuccess;
     ok = ok && alloc_zero(&c->lk_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_row_key, (size_t)cfg->max_rows * sizeof(unsigned long long)) == cudaSuccess;
@@ -86,6 +88,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->vf_blocks_per_sm[1] = verify_occupancy(HVD_BF16, smem);
     if (c->vf_blocks_per_sm[0] < 1 || c->vf_blocks_per_sm[1] < 1) { release(c); return HVD_ERR_UNSUPPORTED; }
     c->has_predictor = false;
+    c->two_layer = false;
     c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // measured: no gain on this path, off unless asked for
     c->host_ws = nullptr;
     c->host_ws_bytes = 0;
@@ -134,6 +137,30 @@ hvd_status hvd_set_predictor(hvd_ctx* ctx, const float* W1, const float* b1, con
     ctx->b2 = b2;
     ctx->tau = tau;
     ctx->has_predictor = true;
+    ctx->two_layer = false;
+    return HVD_OK;
+}
+
+hvd_status hvd_set_predictor2(hvd_ctx* ctx, const float* W1, const float* b1, const float* Wh, const float* bh,
+                              const float* W2, float b2, float tau, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (!Wh || !bh) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_predictor2: NULL weights");
+    const hvd_status r = hvd_set_predictor(ctx, W1, b1, W2, b2, tau, stream);
+    if (r != HVD_OK) return r;
+    const size_t H = (size_t)ctx->cfg.hidden;
+    // transposed copy with a fixed row stride (coalesced, 16-byte aligned rows on the device)
+    const size_t S = HVD_MAX_HIDDEN;
+    float* t = static_cast<float*>(calloc(S * S, sizeof(float)));
+    if (!t) return fail(ctx, HVD_ERR_ALLOC, "hvd_set_predictor2: out of host memory");
+    for (size_t j = 0; j < H; ++j)
+        for (size_t i = 0; i < H; ++i) t[i * S + j] = Wh[j * H + i];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(ctx->d_WhT, t, S * S * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_bh, bh, H * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    free(t);
+    if (e != cudaSuccess) { ctx->has_predictor = false; return cuda_fail(ctx, e, "hvd_set_predictor2"); }
+    ctx->two_layer = true;
     return HVD_OK;
 }
 
@@ -172,11 +199,20 @@ hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist,
     if (!aligned(state, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: state must be 8-byte aligned");
     if (n_max < 0 || n_max > ctx->cfg.max_hist_len)
         return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_score_select: n_max outside [0, max_hist_len]");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->two_layer) {
+        // the two-layer predictor needs a whole CTA per request: lookup, then its own kernel
+        const hvd_status r = launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
+                                           match_len, match_pos, match_cnt, nullptr, st);
+        if (r != HVD_OK) return r;
+        return launch_score_select(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
+                                   match_cnt, model_draft, model_len, features, score, select, sel_draft, sel_len, st);
+    }
     const ScoreArgs sa = make_score_args(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len,
                                          match_pos, match_cnt, model_draft, model_len, features, score,
                                          select, sel_draft, sel_len);
     return launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
-                         match_len, match_pos, match_cnt, &sa, static_cast<cudaStream_t>(stream));
+                         match_len, match_pos, match_cnt, &sa, st);
 }
 
 hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,

@@ -55,8 +55,11 @@ struct hvd_ctx {
     float* d_W1;
     float* d_b1;
     float* d_W2;
+    float* d_WhT;  // second hidden layer, transposed [hidden, hidden]
+    float* d_bh;
     float b2, tau;
     bool has_predictor;
+    bool two_layer;
     // lookup scratch
     hvd::LookupPartial* lk_partial;  // [max_batch, lk_max_chunks]
     uint32_t* lk_cnt;                // [max_batch], zero at rest

@@ -29,30 +29,23 @@ struct ScoreArgs {
     const float* W2;
     float b2, tau;
     int32_t hidden, k_cap;
+    const float* WhT;  // second hidden layer, transposed: WhT[i][j] = Wh[j][i]; NULL = one layer
+    const float* bh;
 };
 
 __device__ __forceinline__ int bit_width(uint32_t x) { return 32 - __clz((int)x); }
 
-// The work is a few hundred flops per request, far too small and too irregular for tensor cores:
-// lane j evaluates hidden unit j (and j+32, ...) with a left-to-right chain of fused multiply-adds,
-// lane 0 then accumulates the output layer in unit order, so the fp32 result does not depend on
-// the launch shape.  d, L, pos, cnt: the lookup results of the request; tok0 / tok1: cache draft
-// tokens lane and lane+32 (-1 beyond the draft); s_hid: shared memory, a.hidden floats, private to
-// the warp.
-__device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, int lane, float* s_hid, int n,
-                                                     int d, int L, int pos, int cnt, int tok0, int tok1) {
+// phi[8] of one request from its lookup results and decode state (every operation is an exact
+// integer->float conversion or one correctly rounded IEEE operation).
+__device__ __forceinline__ void payoff_features(const ScoreArgs& a, int b, int n, int d, int L, int pos, int cnt,
+                                                float (&phi)[HVD_N_FEATURES]) {
     n = max(n, 0);
     // read-only inputs go through the non-coherent path so that the compiler may issue them early
     const int P = max(__ldg(a.prompt_len + b), 0);
     hvd_req_state st;
     st.sel_bits = __ldg(&a.state[b].sel_bits);
     st.acc_ring = __ldg(reinterpret_cast<const unsigned long long*>(&a.state[b].acc_ring));
-    const int kc = a.k_cap;
-    const int K = max(0, min(__ldg(a.K + b), kc));
-    d = max(0, min(d, kc));
     cnt = max(cnt, 0);
-
-    float phi[HVD_N_FEATURES];
     phi[0] = (float)L;
     phi[1] = (float)d;
     phi[2] = (float)bit_width((uint32_t)cnt);
@@ -66,31 +59,25 @@ __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, 
     r = (r & 0x0000FFFF0000FFFFull) + ((r >> 16) & 0x0000FFFF0000FFFFull);
     const int acc_sum = (int)((r & 0xFFFFFFFFull) + (r >> 32));
     phi[7] = __fdiv_rn((float)acc_sum, 8.0f);
+}
 
-    if (a.features && lane < HVD_N_FEATURES) {
-        float v = phi[0];
+// hidden unit j of the first layer: relu(b1[j] + sum_i W1[j][i] phi[i]), left to right
+__device__ __forceinline__ float first_layer_unit(const ScoreArgs& a, int j, const float (&phi)[HVD_N_FEATURES]) {
+    float acc = __ldg(a.b1 + j);
+    const float4* w4 = reinterpret_cast<const float4*>(a.W1 + (int64_t)j * HVD_N_FEATURES);  // 32-byte rows
+    const float4 wa = __ldg(w4), wb = __ldg(w4 + 1);
+    const float w[HVD_N_FEATURES] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
-        for (int i = 1; i < HVD_N_FEATURES; ++i) v = (lane == i) ? phi[i] : v;
-        a.features[(int64_t)b * HVD_N_FEATURES + lane] = v;
-    }
+    for (int i = 0; i < HVD_N_FEATURES; ++i) acc = __fmaf_rn(w[i], phi[i], acc);
+    return acc > 0.0f ? acc : 0.0f;
+}
 
-    for (int j = lane; j < a.hidden; j += 32) {
-        float acc = __ldg(a.b1 + j);
-        const float4* w4 = reinterpret_cast<const float4*>(a.W1 + (int64_t)j * HVD_N_FEATURES);  // 32-byte rows
-        const float4 wa = __ldg(w4), wb = __ldg(w4 + 1);
-        const float w[HVD_N_FEATURES] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-        for (int i = 0; i < HVD_N_FEATURES; ++i) acc = __fmaf_rn(w[i], phi[i], acc);
-        s_hid[j] = acc > 0.0f ? acc : 0.0f;
-    }
-    __syncwarp();
-    float y = a.b2;
-    if (lane == 0) {
-        for (int j = 0; j < a.hidden; ++j) y = __fmaf_rn(__ldg(a.W2 + j), s_hid[j], y);
-    }
-    y = __shfl_sync(0xffffffffu, y, 0);
+// Selection rule and the selected draft, by one warp.  tok0 / tok1: cache draft tokens lane and
+// lane+32 (-1 beyond the draft).
+__device__ __forceinline__ void select_draft(const ScoreArgs& a, int b, int lane, float y, int d, int tok0, int tok1) {
+    const int kc = a.k_cap;
+    const int K = max(0, min(__ldg(a.K + b), kc));
     const int sel = (d > 0 && y >= a.tau) ? 1 : 0;
-
     int m = d;
     if (!sel) {
         m = 0;
@@ -109,6 +96,32 @@ __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, 
         a.select[b] = sel;
         a.sel_len[b] = m;
     }
+}
+
+// One-hidden-layer predictor for one request by one warp.  The work is a few hundred flops per
+// request, far too small and too irregular for tensor cores: lane j evaluates hidden unit j (and
+// j+32, ...) with a left-to-right chain of fused multiply-adds, lane 0 then accumulates the output
+// layer in unit order, so the fp32 result does not depend on the launch shape.  d, L, pos, cnt: the
+// lookup results of the request; s_hid: shared memory, a.hidden floats, private to the warp.
+__device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, int lane, float* s_hid, int n,
+                                                     int d, int L, int pos, int cnt, int tok0, int tok1) {
+    d = max(0, min(d, a.k_cap));
+    float phi[HVD_N_FEATURES];
+    payoff_features(a, b, n, d, L, pos, cnt, phi);
+    if (a.features && lane < HVD_N_FEATURES) {
+        float v = phi[0];
+#pragma unroll
+        for (int i = 1; i < HVD_N_FEATURES; ++i) v = (lane == i) ? phi[i] : v;
+        a.features[(int64_t)b * HVD_N_FEATURES + lane] = v;
+    }
+    for (int j = lane; j < a.hidden; j += 32) s_hid[j] = first_layer_unit(a, j, phi);
+    __syncwarp();
+    float y = a.b2;
+    if (lane == 0) {
+        for (int j = 0; j < a.hidden; ++j) y = __fmaf_rn(__ldg(a.W2 + j), s_hid[j], y);
+    }
+    y = __shfl_sync(0xffffffffu, y, 0);
+    select_draft(a, b, lane, y, d, tok0, tok1);
 }
 
 }  // namespace hvd

@@ -18,6 +18,13 @@ def make_ctx(w, rq, **over):
     return H.Context(**kw)
 
 
+def set_predictor(ctx, inp):
+    if inp.Wh is not None:
+        ctx.hvd_set_predictor2(inp.W1, inp.b1, inp.Wh, inp.bh, inp.W2, inp.b2, inp.tau)
+    else:
+        ctx.hvd_set_predictor(inp.W1, inp.b1, inp.W2, inp.b2, inp.tau)
+
+
 def make_batch(ctx, w, rq, uniform_rows=False):
     from paper_2606_01019_b200.runner import DeviceBatch
     return DeviceBatch(ctx, hist=rq.hist, hist_off=rq.hist_off, hist_cap=rq.hist_cap, hist_len=rq.hist_len,
@@ -71,7 +78,7 @@ def run_and_compare(inp, ctx=None, uniform_rows=False, logits=None, logits_np=No
     if batch is None:
         if own:
             ctx = make_ctx(w, rq)
-        ctx.hvd_set_predictor(inp.W1, inp.b1, inp.W2, inp.b2, inp.tau)
+        set_predictor(ctx, inp)
         batch = make_batch(ctx, w, rq, uniform_rows)
     lg = inp.logits if logits is None else logits
     if lg.device.type != "cuda":

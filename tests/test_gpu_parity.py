@@ -26,6 +26,29 @@ def test_fused_lookup_score_select(name, kw):
     G.run_and_compare(inp, fused=True)
 
 
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("name,kw", [("C2", dict(B=40, n=6000, V=20011, hidden=256, hidden_layers=2)),
+                                     ("C1", dict(hidden=64, hidden_layers=2)),
+                                     ("C5", dict(B=33, n=(8, 3000), V=32003, hidden=200, hidden_layers=2))])
+def test_two_hidden_layer_predictor(name, kw, fused):
+    """The paper's predictor shape (two hidden ReLU layers): scores within 1e-5, same selections."""
+    inp = P.prepare(W.CONFIGS[name].scaled(**kw), device="cuda")
+    g, out, _ = G.run_and_compare(inp, fused=fused)
+    assert 0 < out.sc.select.sum() < len(out.sc.select)
+
+
+def test_switching_between_one_and_two_layers_on_one_context():
+    w2 = W.CONFIGS["C1"].scaled(hidden=32, hidden_layers=2)
+    w1 = W.CONFIGS["C1"]
+    inp2, inp1 = P.prepare(w2, device="cuda"), P.prepare(w1, device="cuda")
+    ctx = G.make_ctx(w1, inp1.rq)
+    for inp in (inp2, inp1, inp2):
+        G.set_predictor(ctx, inp)
+        batch = G.make_batch(ctx, inp.w, inp.rq.copy())
+        G.run_and_compare(inp, ctx=ctx, batch=batch, rq=inp.rq.copy())
+    ctx.close()
+
+
 def test_c1_uniform_row_layout():
     inp = P.prepare(W.CONFIGS["C1"], device="cuda")
     G.run_and_compare(inp, uniform_rows=True)
