@@ -139,6 +139,38 @@ void oracle_lookup(int32_t B, const int32_t* hist, const int64_t* hist_off, cons
 }
 
 /* ------------------------------------------------------------------ */
+/* Payoff labels by trace replay (Sec. 3.3 "training labels"; App. B   */
+/* "Payoff Label Construction"): every position t of a recorded trace  */
+/* is a decoding state with prefix x[0..t); its cache draft comes from */
+/* the lookup above on that prefix; the label is the number of draft   */
+/* tokens that agree with the trace's own continuation x[t..).         */
+/* Outputs are indexed by t-1, t = 1..n.                               */
+/* ------------------------------------------------------------------ */
+typedef struct {
+    const int32_t* x; int32_t n, K, k_cap, l_max, min_match; float spec_factor, spec_offset;
+    int32_t *label, *draft_len, *match_len, *match_pos, *match_cnt;
+} replay_args;
+
+static void replay_state(int32_t j, void* p) {
+    replay_args* a = (replay_args*)p;
+    const int32_t t = j + 1;
+    int32_t draft[64];
+    oracle_lookup_one(a->x, t, a->K, a->k_cap, a->l_max, a->min_match, a->spec_factor, a->spec_offset, draft,
+                      a->draft_len + j, a->match_len + j, a->match_pos + j, a->match_cnt + j);
+    int32_t y = 0;
+    while (y < a->draft_len[j] && t + y < a->n && draft[y] == a->x[t + y]) ++y;
+    a->label[j] = y;
+}
+
+void oracle_replay_labels(const int32_t* x, int32_t n, int32_t K, int32_t k_cap, int32_t l_max, int32_t min_match,
+                          float spec_factor, float spec_offset, int32_t* label, int32_t* draft_len,
+                          int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, int32_t nthreads) {
+    replay_args a = {x, n, K, k_cap, l_max, min_match, spec_factor, spec_offset, label, draft_len, match_len,
+                     match_pos, match_cnt};
+    for_each_request(n, nthreads, replay_state, &a);
+}
+
+/* ------------------------------------------------------------------ */
 /* Step 2: payoff features (Sec. 3.3; App. B feature-group table).     */
 /* Every operation is an exact integer->float conversion or a single   */
 /* correctly rounded IEEE operation.                                   */

@@ -81,6 +81,29 @@ def lookup(hist, hist_off, hist_cap, hist_len, K, *, k_cap, l_max=64, min_match=
 
 
 @dataclass
+class ReplayOut:
+    label: np.ndarray
+    draft_len: np.ndarray
+    match_len: np.ndarray
+    match_pos: np.ndarray
+    match_cnt: np.ndarray
+
+
+def replay_labels(trace, K, *, k_cap=None, l_max=64, min_match=2, spec_factor=1.0, spec_offset=0.0,
+                  nthreads=1) -> ReplayOut:
+    """Labels y_t for every prefix length t = 1..n of one trace (arrays indexed by t-1)."""
+    x = _i32(trace)
+    n = len(x)
+    k_cap = k_cap or max(K, 1)
+    out = ReplayOut(*(np.empty(n, np.int32) for _ in range(5)))
+    lib().oracle_replay_labels(_p(x), C.c_int32(n), C.c_int32(K), C.c_int32(k_cap), C.c_int32(l_max),
+                               C.c_int32(min_match), C.c_float(spec_factor), C.c_float(spec_offset),
+                               _p(out.label), _p(out.draft_len), _p(out.match_len), _p(out.match_pos),
+                               _p(out.match_cnt), C.c_int32(nthreads))
+    return out
+
+
+@dataclass
 class ScoreOut:
     features: np.ndarray
     score: np.ndarray
