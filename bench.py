@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--predictor", default="config", choices=["config", "2x256"],
                     help="2x256: the paper's predictor shape (two hidden layers of 256 units) instead of the config's")
+    ap.add_argument("--replay", action="store_true",
+                    help="second workload: payoff labels by trace replay (hvd_replay_labels) on one history of the config")
     ap.add_argument("--unfused", action="store_true",
                     help="call hvd_lookup and hvd_score_select separately instead of hvd_lookup_score_select")
     ap.add_argument("--no-kernel-events", action="store_true",
@@ -182,6 +184,53 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------------------------
+# second workload: trace-replay labels (training-data path)
+# ----------------------------------------------------------------------------------------------
+def run_replay(args):
+    import torch
+    import hvd_workloads as W
+    import paper_2606_01019_b200 as H
+    torch.cuda.set_device(0)
+    w = W.CONFIGS[args.config]
+    rq = W.make_requests(w.scaled(B=min(w.B, 4)))
+    x = np.ascontiguousarray(rq.history(0), np.int32)
+    n, K = len(x), int(rq.K[0])
+    ctx = H.Context(max_batch=4096, k_cap=w.k_cap, max_hist_len=n, max_rows=1, max_vocab=1, l_max=w.l_max,
+                    min_match=w.min_match)
+    xd = torch.as_tensor(x, device="cuda")
+    outs = [torch.zeros(n, dtype=torch.int32, device="cuda") for _ in range(5)]
+    for _ in range(max(3, args.warmup)):
+        ctx.hvd_replay_labels(xd, n, K, *outs)
+    torch.cuda.synchronize()
+    reps = max(1, min(args.steps, 50))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        ctx.hvd_replay_labels(xd, n, K, *outs)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    label = outs[0].cpu().numpy()
+    from oracle import hvd_oracle as O
+    from oracle import pipeline as P
+    cores = P.host_threads()
+    t0 = time.perf_counter()
+    ref = O.replay_labels(x, K, k_cap=w.k_cap, l_max=w.l_max, min_match=w.min_match, nthreads=cores)
+    cpu_s = time.perf_counter() - t0
+    line = {"metric": "trace-replay labelled positions/s", "value": n / (ms * 1e-3), "unit": "positions/s",
+            "n_gpus": 1, "steps": reps, "ms_per_trace": ms, "higher_is_better": True, "dtype": "int32",
+            "data": "synthetic", "config": {"workload": f"replay of one {w.name} history: {n} positions, K {K}",
+                                            "launches_per_trace": 3 * ((n + 4095) // 4096)},
+            "prefix_tokens_scanned_per_trace": int(n) * (int(n) + 1) // 2,
+            "scan_rate_gtokens_per_s": int(n) * (int(n) + 1) / 2 / (ms * 1e-3) / 1e9,
+            "mean_label": float(label.mean()), "labels_ge_6_frac": float((label >= 6).mean()),
+            "cpu_baseline": {"value": n / cpu_s, "unit": "positions/s", "cores": cores, "kind": "oracle",
+                             "sample": "the same whole trace, once", "agrees_with_gpu": bool((ref.label == label).all())}}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def workload_config(w, n_gpus, extra=None):
     cfg = {"workload": f"{w.name}: batch {w.B}, histories {w.n} tokens, vocab {w.V}, K {w.K}, {w.dtype} logits",
            "requests_per_gpu": w.B, "parallelism": f"requests sharded over {n_gpus} GPU(s), no collective"}
@@ -197,6 +246,9 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.replay:
+        run_replay(args)
         return
 
     import torch

@@ -173,6 +173,20 @@ HVD_API hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_
                                            int32_t* sel_draft, int32_t* sel_len, void* stream);
 
 /*
+ * Payoff labels by trace replay (Sec. 3.3, "We derive training labels ..."; App. B "Payoff Label
+ * Construction").  Every position t = 1..n of a recorded trace x[0..n) is a decoding state with prefix
+ * x[0..t): its cache draft is the hvd_lookup result on that prefix (same rules, K for every state),
+ * and its label is y_t = max{ l <= draft_len : draft[0..l) == x[t .. t+l) }, the number of draft tokens
+ * the trace's own continuation confirms.  Outputs (int32 [n], index t-1): label, draft_len, match_len,
+ * match_pos, match_cnt.  trace: DEVICE, 16-byte aligned; n (HOST value) <= max_hist_len; states are
+ * processed in slices of max_batch.  These are the regression targets of the payoff predictor; the
+ * recent-history features depend on the decoding loop and are not produced here.
+ */
+HVD_API hvd_status hvd_replay_labels(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label,
+                                     int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
+                                     int32_t* match_cnt, void* stream);
+
+/*
  * Greedy verification and commit (Sec. 3.1 Verify; Sec. 3.4; Algorithm 1; the accepted length is
  * the label equation of Sec. 3.3).  Request b owns logits rows [r0, r1): r0 = row_off[b],
  * r1 = row_off[b+1], or r0 = b*(k_uniform+1), r1 = r0 + k_uniform + 1 when row_off is NULL.  Row r

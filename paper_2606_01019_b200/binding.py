@@ -49,6 +49,7 @@ _SIGNATURES = {
     "hvd_set_predictor2": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _vp]),
     "hvd_lookup": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_score_select": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32] + [_vp] * 14 + [_vp]),
+    "hvd_replay_labels": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
     "hvd_step_host": (_i32, [_vp, C.POINTER(HvdHostStepArgs), _vp]),
@@ -193,6 +194,11 @@ class Context:
             _ptr(prompt_len), _ptr(state), _ptr(model_draft), _ptr(model_len), _ptr(draft), _ptr(draft_len),
             _ptr(match_len), _ptr(match_pos), _ptr(match_cnt), _ptr(features), _ptr(score), _ptr(select),
             _ptr(sel_draft), _ptr(sel_len), _stream()), "hvd_lookup_score_select")
+
+    def hvd_replay_labels(self, trace, n, K, label, draft_len, match_len, match_pos, match_cnt):
+        self._check(self._lib.hvd_replay_labels(self._h, _ptr(trace), n, K, _ptr(label), _ptr(draft_len),
+                                                _ptr(match_len), _ptr(match_pos), _ptr(match_cnt), _stream()),
+                    "hvd_replay_labels")
 
     def hvd_score_select(self, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
                          match_cnt, model_draft, model_len, features, score, select, sel_draft, sel_len):

@@ -15,6 +15,7 @@ void release(hvd_ctx* c) {
     if (!c) return;
     cudaFree(c->d_W1); cudaFree(c->d_b1); cudaFree(c->d_W2); cudaFree(c->d_WhT); cudaFree(c->d_bh);
     cudaFree(c->lk_partial); cudaFree(c->lk_cnt);
+    cudaFree(c->rp_off); cudaFree(c->rp_cap); cudaFree(c->rp_len); cudaFree(c->rp_K); cudaFree(c->rp_draft);
     cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
     delete c;
@@ -77,6 +78,12 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->d_bh, H * sizeof(float)) == cudaSuccess;
     ok = ok && alloc_zero(&c->lk_partial, (size_t)cfg->max_batch * c->lk_max_chunks * sizeof(LookupPartial)) == cudaSuccess;
     ok = ok && alloc_zero(&c->lk_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
+    const size_t MB = (size_t)cfg->max_batch;
+    ok = ok && alloc_zero(&c->rp_off, MB * sizeof(int64_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->rp_cap, MB * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->rp_len, MB * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->rp_K, MB * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->rp_draft, MB * (size_t)cfg->k_cap * sizeof(int32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_row_key, (size_t)cfg->max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_next_unit, (size_t)kVerifyQueues * 32 * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->dev_error, sizeof(int)) == cudaSuccess;
@@ -178,6 +185,19 @@ hvd_status hvd_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_
         return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max outside [0, max_hist_len]");
     return launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
                          match_len, match_pos, match_cnt, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_replay_labels(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label,
+                             int32_t* draft_len, int32_t* match_len, int32_t* match_pos, int32_t* match_cnt,
+                             void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (!trace || !label || !draft_len || !match_len || !match_pos || !match_cnt)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_replay_labels: NULL pointer");
+    if (n < 1 || n > ctx->cfg.max_hist_len) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_replay_labels: n outside [1, max_hist_len]");
+    if (K < 0 || K > ctx->cfg.k_cap) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_replay_labels: K outside [0, k_cap]");
+    if (!aligned(trace, 16)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_replay_labels: trace must be 16-byte aligned");
+    return launch_replay(ctx, trace, n, K, label, draft_len, match_len, match_pos, match_cnt,
+                         static_cast<cudaStream_t>(stream));
 }
 
 hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,

@@ -70,6 +70,9 @@ struct hvd_ctx {
     int* dev_error;                  // device status word
     int vf_blocks_per_sm[2];         // per dtype
     // device staging of the host-buffer entry point (grown on demand)
+    // trace replay: the virtual batch of one slice of states, and its drafts
+    int64_t* rp_off;
+    int32_t *rp_cap, *rp_len, *rp_K, *rp_draft;
     bool use_pdl;  // programmatic dependent launch between the kernels of the path
     char* host_ws;
     size_t host_ws_bytes;
@@ -140,6 +143,9 @@ hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
                                const int32_t* model_draft, const int32_t* model_len, float* features,
                                float* score, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
                                cudaStream_t stream);
+
+hvd_status launch_replay(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label, int32_t* draft_len,
+                         int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream);
 
 struct VerifyArgs {
     int32_t B;

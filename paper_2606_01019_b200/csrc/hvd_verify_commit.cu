@@ -458,7 +458,12 @@ size_t verify_dyn_smem(int32_t B) { return (size_t)B * 8 + (size_t)(B + 1) * 4; 
 
 int verify_occupancy(hvd_dtype dtype, size_t dyn_smem) {
     int n = 0;
-    cudaError_t e;
+    cudaError_t e = cudaSuccess;
+    if (dyn_smem > 48 * 1024) {  // large batches: the per-request tables need the opt-in shared memory size
+        e = dtype == HVD_F32 ? cudaFuncSetAttribute(verify_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem)
+                             : cudaFuncSetAttribute(verify_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    }
     if (dtype == HVD_F32)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, verify_stream_kernel<float>, T, dyn_smem);
     else

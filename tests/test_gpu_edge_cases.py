@@ -186,6 +186,15 @@ def test_batch_of_one_and_full_context_batch():
     run(w, rq)
 
 
+def test_batch_beyond_the_default_shared_memory_size():
+    """5000 requests: the verify kernel's per-request tables exceed 48 KB of shared memory."""
+    w = small(V=11, k_cap=2)
+    rng = np.random.default_rng(13)
+    hists = [rng.integers(0, 3, int(n)) for n in rng.integers(0, 40, 5000)]
+    rq = hand_requests(w, hists, rng.integers(0, 3, 5000))
+    run(w, rq)
+
+
 def test_two_calls_with_different_shapes_share_a_context():
     """A context sized for the larger call serves a smaller one afterwards (scratch at rest)."""
     w = small()
