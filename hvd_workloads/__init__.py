@@ -23,7 +23,7 @@ import numpy as np
 
 BASE_SEED = 260601019 * 10**4
 # stream ids
-S_TEMPLATES, S_HIST, S_TAIL, S_STATE, S_WEIGHTS, S_MODEL, S_AGREE, S_LOGITS, S_PLANT = range(9)
+S_TEMPLATES, S_HIST, S_TAIL, S_STATE, S_WEIGHTS, S_MODEL, S_AGREE, S_LOGITS, S_PLANT, S_TREE = range(10)
 
 GUARD_WORDS = 64          # canary words either side of every history slab
 GUARD_VALUE = -1515870811  # 0xA5A5A5A5 as int32
@@ -426,3 +426,59 @@ def logits_to_numpy(logits) -> np.ndarray:
     if t.dtype == torch.bfloat16:
         return t.view(torch.int16).numpy().view(np.uint16)
     return t.numpy()
+
+
+def make_tree_drafts(w: Workload, K: np.ndarray, max_nodes: int = 32, max_depth: int = 8, top_k: int = 4):
+    """Model-drafter token trees in the shape the paper's drafter uses (App. A: 32 draft tokens, depth 8,
+    top-k 4): per request up to min(max_nodes, K_b) nodes; node i hangs under a uniformly drawn earlier
+    node (or under the prefix, parent -1) that is shallower than max_depth and has fewer than top_k
+    children; sibling tokens are distinct.  Returns (tokens [B,k_cap], parent [B,k_cap], n_nodes [B])."""
+    rng = _rng(w.index, S_TREE)
+    B = len(K)
+    tok = np.full((B, w.k_cap), -1, np.int32)
+    par = np.full((B, w.k_cap), -2, np.int32)
+    cnt = np.zeros(B, np.int32)
+    for b in range(B):
+        m = int(min(max_nodes, K[b], w.k_cap))
+        depth, kids = {-1: 0}, {-1: []}
+        for i in range(m):
+            open_nodes = [p for p in depth if depth[p] < max_depth and len(kids[p]) < top_k]
+            p = open_nodes[int(rng.integers(0, len(open_nodes)))]
+            t = int(rng.integers(0, w.V))
+            while t in [int(tok[b, c]) for c in kids[p]] and w.V > top_k:
+                t = int(rng.integers(0, w.V))
+            tok[b, i], par[b, i] = t, p
+            kids[p].append(i); kids[i] = []; depth[i] = depth[p] + 1
+        cnt[b] = m
+    return tok, par, cnt
+
+
+def plant_tree_agreement(w: Workload, logits, row_off: np.ndarray, tok: np.ndarray, par: np.ndarray,
+                         n_nodes: np.ndarray, A: np.ndarray, salt: int = 0) -> np.ndarray:
+    """Plants PLANT_VALUE so that greedy verification walks a random root path of (up to) A_b nodes and
+    then stops: row(cur) gets its maximum at the chosen child's token; the row of the last node gets it
+    at a token none of its children carries.  Returns the planted path lengths."""
+    import torch
+    rng = _rng(w.index, S_PLANT, 7919 + salt)
+    rows, cols = [], []
+    depth = np.zeros(len(n_nodes), np.int32)
+    for b in range(len(n_nodes)):
+        m, r0 = int(n_nodes[b]), int(row_off[b])
+        cur, a = -1, 0
+        while a < int(A[b]):
+            kids = [c for c in range(m) if par[b, c] == cur]
+            if not kids:
+                break
+            c = kids[int(rng.integers(0, len(kids)))]
+            rows.append(r0 + cur + 1); cols.append(int(tok[b, c]))
+            cur, a = c, a + 1
+        kid_toks = {int(tok[b, c]) for c in range(m) if par[b, c] == cur}
+        t = int(rng.integers(0, w.V))
+        while t in kid_toks and w.V > len(kid_toks):
+            t = int(rng.integers(0, w.V))
+        rows.append(r0 + cur + 1); cols.append(t)
+        depth[b] = a
+    ri = torch.as_tensor(np.asarray(rows, np.int64), device=logits.device)
+    ci = torch.as_tensor(np.asarray(cols, np.int64), device=logits.device)
+    logits[ri, ci] = PLANT_VALUE
+    return depth

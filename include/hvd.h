@@ -216,6 +216,28 @@ HVD_API hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits
                              int32_t* status, void* stream);
 
 /*
+ * Greedy verification of a token TREE and commit.  The paper's model drafter (EAGLE3) proposes a
+ * tree (App. A "Drafting configuration": 32 draft tokens, depth 8, top-k 4); the verification rule is
+ * unchanged (Sec. 3.1, Sec. 3.4).  Node i of request b has token sel_draft[b, i] and parent
+ * parent[b, i] in {-1, 0..i-1} (-1: the node follows the prefix directly; any other value makes the
+ * node unreachable); sel_len[b] = number of nodes.  Row r0 of the request's logits is the target's
+ * output after the prefix, row r0+i+1 its output after node i.  The walk starts at the prefix: the
+ * target's token at the current node is the argmax of that node's row; the first child (lowest
+ * index) that carries this token is accepted and the walk goes on there; otherwise it stops.
+ * accepted[b] = number of accepted nodes, committed[b] = their tokens followed by the target's token
+ * at the last node.  Everything else (rows, ties, append, capacity, state, target_tok, status) is as
+ * in hvd_verify_commit, which is the special case parent[b, i] = i-1.
+ */
+HVD_API hvd_status hvd_verify_commit_tree(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                                          const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                                          const int32_t* sel_draft, const int32_t* sel_len,
+                                          const int32_t* parent /*[B, k_cap]*/, const int32_t* select,
+                                          int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                                          int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                                          int32_t* committed, int32_t* n_commit, int32_t* target_tok,
+                                          int32_t* status, void* stream);
+
+/*
  * The same decoding cycle with HOST buffers: one call copies the step's inputs to the device,
  * runs hvd_lookup, hvd_score_select and hvd_verify_commit there, copies the results back, waits
  * for the stream, and appends the committed tokens to the host histories.  Every pointer in the

@@ -444,3 +444,90 @@ void oracle_verify_commit(int32_t B, const void* logits, int32_t dtype, int64_t 
                      status};
     for_each_request(B, nthreads, verify_req, &a);
 }
+
+/* ------------------------------------------------------------------ */
+/* Verification of a token TREE (the model drafter of the paper,       */
+/* EAGLE3, proposes a tree: App. A "Drafting configuration": 32 draft  */
+/* tokens, depth 8, top-k 4).  Node i has token d[i] and parent        */
+/* par[i] in {-1, 0..i-1} (-1: it follows the prefix directly).  Row 0 */
+/* of the request's logits is the target's output after the prefix,    */
+/* row i+1 its output after node i.  Greedy verification (Sec. 3.1,    */
+/* Sec. 3.4) walks down from the prefix: the target's token at the     */
+/* current node is the argmax of that node's row; if a child carries   */
+/* that token (the first such child) it is accepted and the walk goes  */
+/* on there, else the walk stops and the target's token is committed   */
+/* as the last token.  A chain (par[i] = i-1) gives exactly            */
+/* oracle_verify_commit.                                               */
+/* ------------------------------------------------------------------ */
+typedef struct {
+    verify_args v;
+    const int32_t* parent;
+} verify_tree_args;
+
+static void verify_tree_req(int32_t b, void* p) {
+    verify_tree_args* ta = (verify_tree_args*)p;
+    verify_args* a = &ta->v;
+    int32_t kc = a->k_cap;
+    int64_t r0 = a->row_off ? a->row_off[b] : (int64_t)b * (a->k_uniform + 1);
+    int64_t r1 = a->row_off ? a->row_off[b + 1] : r0 + (a->k_uniform + 1);
+    int64_t rows = r1 - r0;
+    size_t elt = a->dtype == ORACLE_BF16 ? 2 : 4;
+    int32_t* z = a->committed + (int64_t)b * (kc + 1);
+    for (int32_t j = 0; j <= kc; ++j) z[j] = -1;
+    if (a->target_tok)
+        for (int64_t i = 0; i < rows; ++i) a->target_tok[r0 + i] = -1;
+    int32_t n = a->hist_len[b];
+    if (n < 0 || n > a->hist_cap[b] || rows <= 0) {
+        a->status[b] = ORACLE_REQ_BAD_LEN; a->accepted[b] = 0; a->n_commit[b] = 0;
+        return;
+    }
+    int32_t m = a->sel_len[b];
+    if (m < 0) m = 0;
+    if (m > kc) m = kc;
+    if (m > rows - 1) m = (int32_t)(rows - 1);
+    int32_t t[65 + 1];
+    for (int32_t i = 0; i <= m; ++i) {
+        const char* row = (const char*)a->logits + (size_t)(r0 + i) * (size_t)a->V * elt;
+        t[i] = oracle_argmax_row(row, a->dtype, a->V);
+        if (a->target_tok) a->target_tok[r0 + i] = t[i];
+    }
+    const int32_t* d = a->sel_draft + (int64_t)b * kc;
+    const int32_t* par = ta->parent + (int64_t)b * kc;
+    int32_t acc = 0, cur = -1;
+    for (;;) {
+        int32_t want = t[cur + 1]; /* the target's token after the current node */
+        int32_t next = -1;
+        for (int32_t c = cur + 1; c < m; ++c)
+            if (par[c] == cur && d[c] == want) { next = c; break; }
+        if (next < 0) { z[acc] = want; break; }
+        z[acc++] = d[next];
+        cur = next;
+    }
+    int32_t room = a->hist_cap[b] - n;
+    int32_t w = acc + 1;
+    int32_t st = ORACLE_REQ_OK;
+    if (w > room) { w = room; st = ORACLE_REQ_CAPACITY; }
+    int32_t* h = a->hist + a->hist_off[b];
+    for (int32_t j = 0; j < w; ++j) h[n + j] = z[j];
+    a->hist_len[b] = n + w;
+    a->n_commit[b] = w;
+    a->accepted[b] = acc;
+    a->status[b] = st;
+    oracle_req_state s = a->state[b];
+    s.sel_bits = (s.sel_bits << 1) | (uint32_t)(a->select[b] ? 1 : 0);
+    s.acc_ring = (s.acc_ring << 8) | (uint64_t)(uint8_t)acc;
+    a->state[b] = s;
+}
+
+void oracle_verify_commit_tree(int32_t B, const void* logits, int32_t dtype, int64_t V,
+                               const int64_t* row_off, int32_t k_uniform, const int32_t* sel_draft,
+                               const int32_t* sel_len, const int32_t* parent, const int32_t* select,
+                               int32_t k_cap, int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                               int32_t* hist_len, oracle_req_state* state, int32_t* accepted,
+                               int32_t* committed, int32_t* n_commit, int32_t* target_tok, int32_t* status,
+                               int32_t nthreads) {
+    verify_tree_args ta = {{logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, select, k_cap, hist,
+                            hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, target_tok,
+                            status}, parent};
+    for_each_request(B, nthreads, verify_tree_req, &ta);
+}

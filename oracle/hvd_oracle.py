@@ -154,8 +154,9 @@ class VerifyOut:
 
 
 def verify_commit(logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, select, *, k_cap, hist,
-                  hist_off, hist_cap, hist_len, state, nthreads=1) -> VerifyOut:
-    """`hist`, `hist_len` and `state` are updated IN PLACE (they must be writable, contiguous
+                  hist_off, hist_cap, hist_len, state, nthreads=1, parent=None) -> VerifyOut:
+    """`parent` (int32 [B, k_cap]) makes the draft a token tree.
+    `hist`, `hist_len` and `state` are updated IN PLACE (they must be writable, contiguous
     int32 / int32 / STATE_DTYPE arrays).  `logits` is a contiguous float32 array (dtype F32) or a
     uint16 array of bfloat16 bit patterns (dtype BF16), rows of V."""
     B = len(hist_len)
@@ -174,12 +175,15 @@ def verify_commit(logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, sele
     assert logits.size >= total_rows * V
     out = VerifyOut(np.empty(B, np.int32), np.empty((B, k_cap + 1), np.int32), np.empty(B, np.int32),
                     np.empty(total_rows, np.int32), np.empty(B, np.int32))
-    lib().oracle_verify_commit(C.c_int32(B), _p(logits), C.c_int32(dtype), C.c_int64(V), _p(row_off),
-                               C.c_int32(k_uniform), _p(_i32(sel_draft)), _p(_i32(sel_len)),
-                               _p(_i32(select)), C.c_int32(k_cap), _p(hist), _p(hist_off),
-                               _p(hist_cap), _p(hist_len), _p(state), _p(out.accepted),
-                               _p(out.committed), _p(out.n_commit), _p(out.target_tok),
-                               _p(out.status), C.c_int32(nthreads))
+    tail = (_p(_i32(select)), C.c_int32(k_cap), _p(hist), _p(hist_off), _p(hist_cap), _p(hist_len), _p(state),
+            _p(out.accepted), _p(out.committed), _p(out.n_commit), _p(out.target_tok), _p(out.status),
+            C.c_int32(nthreads))
+    head = (C.c_int32(B), _p(logits), C.c_int32(dtype), C.c_int64(V), _p(row_off), C.c_int32(k_uniform),
+            _p(_i32(sel_draft)), _p(_i32(sel_len)))
+    if parent is None:
+        lib().oracle_verify_commit(*head, *tail)
+    else:       # the draft is a token tree: parent[b, i] in {-1, 0..i-1}
+        lib().oracle_verify_commit_tree(*head, _p(_i32(parent)), *tail)
     return out
 
 

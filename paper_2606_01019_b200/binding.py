@@ -52,6 +52,7 @@ _SIGNATURES = {
     "hvd_replay_labels": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
+    "hvd_verify_commit_tree": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 14 + [_vp]),
     "hvd_step_host": (_i32, [_vp, C.POINTER(HvdHostStepArgs), _vp]),
     "hvd_verify_commit_noalloc": (_i32, [_i32, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
     "hvd_noalloc_last_error": (C.c_char_p, []),
@@ -219,6 +220,15 @@ class Context:
                                                 _ptr(committed), _ptr(n_commit), _ptr(target_tok),
                                                 _ptr(status), _stream()),
                     "hvd_verify_commit")
+
+    def hvd_verify_commit_tree(self, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
+                               parent, select, hist, hist_off, hist_cap, hist_len, state, accepted, committed,
+                               n_commit, target_tok, status):
+        self._check(self._lib.hvd_verify_commit_tree(
+            self._h, B, _ptr(logits), dtype, V, _ptr(row_off), k_uniform, total_rows, _ptr(sel_draft),
+            _ptr(sel_len), _ptr(parent), _ptr(select), _ptr(hist), _ptr(hist_off), _ptr(hist_cap),
+            _ptr(hist_len), _ptr(state), _ptr(accepted), _ptr(committed), _ptr(n_commit), _ptr(target_tok),
+            _ptr(status), _stream()), "hvd_verify_commit_tree")
 
     def hvd_step_host(self, *, B, n_max, hist, hist_off, hist_cap, hist_len, K, prompt_len, state,
                       model_draft, model_len, logits, dtype, V, row_off, k_uniform, total_rows, score,

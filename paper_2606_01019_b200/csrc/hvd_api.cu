@@ -256,9 +256,9 @@ hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
                                sel_draft, sel_len, static_cast<cudaStream_t>(stream));
 }
 
-hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
                              const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
-                             const int32_t* sel_draft, const int32_t* sel_len, const int32_t* select,
+                             const int32_t* sel_draft, const int32_t* sel_len, const int32_t* parent, const int32_t* select,
                              int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
                              int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
                              int32_t* committed, int32_t* n_commit, int32_t* target_tok,
@@ -284,7 +284,7 @@ hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dt
 
     VerifyArgs a;
     a.B = B; a.logits = logits; a.V = V; a.row_off = row_off; a.k_uniform = k_uniform;
-    a.sel_draft = sel_draft; a.sel_len = sel_len; a.select = select;
+    a.sel_draft = sel_draft; a.sel_len = sel_len; a.parent = parent; a.select = select;
     a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.state = state;
     a.accepted = accepted; a.committed = committed; a.n_commit = n_commit; a.target_tok = target_tok;
     a.status = status; a.k_cap = ctx->cfg.k_cap;
@@ -295,6 +295,32 @@ hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dt
     a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error;
     a.row_key = ctx->vf_row_key; a.total_rows = total_rows;
     return launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                             const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                             const int32_t* sel_draft, const int32_t* sel_len, const int32_t* select,
+                             int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                             int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                             int32_t* committed, int32_t* n_commit, int32_t* target_tok,
+                             int32_t* status, void* stream) {
+    return verify_commit_impl(ctx, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len, nullptr,
+                              select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
+                              target_tok, status, stream);
+}
+
+hvd_status hvd_verify_commit_tree(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                                  const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                                  const int32_t* sel_draft, const int32_t* sel_len, const int32_t* parent,
+                                  const int32_t* select, int32_t* hist, const int64_t* hist_off,
+                                  const int32_t* hist_cap, int32_t* hist_len, hvd_req_state* state,
+                                  int32_t* accepted, int32_t* committed, int32_t* n_commit, int32_t* target_tok,
+                                  int32_t* status, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (!parent) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_tree: NULL parent");
+    return verify_commit_impl(ctx, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len, parent,
+                              select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
+                              target_tok, status, stream);
 }
 
 }  // extern "C"

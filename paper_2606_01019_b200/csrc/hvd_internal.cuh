@@ -155,6 +155,7 @@ struct VerifyArgs {
     int32_t k_uniform;
     const int32_t* sel_draft;
     const int32_t* sel_len;
+    const int32_t* parent;  // NULL: the draft is a chain; else parent[b, i] of tree node i
     const int32_t* select;
     int32_t* hist;
     const int64_t* hist_off;

@@ -129,7 +129,7 @@ hvd_status hvd_verify_commit_noalloc(int32_t B, int32_t k_cap, const void* logit
 
     VerifyArgs a;
     a.B = B; a.logits = logits; a.V = V; a.row_off = row_off; a.k_uniform = k_uniform;
-    a.sel_draft = sel_draft; a.sel_len = sel_len; a.select = select;
+    a.sel_draft = sel_draft; a.sel_len = sel_len; a.parent = nullptr; a.select = select;
     a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.state = state;
     a.accepted = accepted; a.committed = committed; a.n_commit = n_commit; a.target_tok = target_tok;
     a.status = status; a.k_cap = k_cap;

@@ -248,6 +248,89 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
     }
 }
 
+// Commit of one request whose draft is a token TREE (node i: token sel_draft[i], parent[i] in
+// {-1, 0..i-1}; logits row 0 follows the prefix, row i+1 follows node i), by one warp.  The walk
+// starts at the prefix; at each node the target's token is the argmax of that node's row; the first
+// child that carries it is accepted, else the walk stops and that token is the last one committed.
+__device__ __forceinline__ void commit_tree_request(const VerifyArgs& a, int b, int lane) {
+    const int kc = a.k_cap;
+    const int32_t* d = a.sel_draft + (int64_t)b * kc;
+    const int32_t* par = a.parent + (int64_t)b * kc;
+    int dt[2], pr[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {  // nodes lane, lane+32 (k_cap <= 64)
+        const int node = lane + 32 * k;
+        dt[k] = node < kc ? d[node] : -1;
+        pr[k] = node < kc ? par[node] : -2;
+    }
+    const int64_t hoff = a.hist_off[b];
+    const int sel = a.select[b];
+    hvd_req_state st = a.state[b];
+    const int n = a.hist_len[b];
+    const int cap = a.hist_cap[b];
+    const Req q = load_req(a, b);
+    int32_t* z = a.committed + (int64_t)b * (kc + 1);
+    if (q.nr == 0) {
+        for (int j = lane; j <= kc; j += 32) z[j] = -1;
+        if (a.target_tok) for (int64_t r = q.r0 + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
+        if (lane == 0) { a.accepted[b] = 0; a.n_commit[b] = 0; a.status[b] = HVD_REQ_BAD_LEN; }
+        return;
+    }
+    const int m = q.nr - 1;
+    int tok[3];  // target tokens of rows lane, lane+32, lane+64
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const int i = lane + 32 * k;
+        tok[k] = 0;
+        if (i <= m) {
+            const unsigned long long key = a.row_key[q.r0 + i];
+            a.row_key[q.r0 + i] = 0ull;  // scratch is zero at rest
+            const int t = (int)(~(uint32_t)(key & 0xffffffffu));
+            tok[k] = (int)min((int64_t)max(t, 0), a.V - 1);
+            if (a.target_tok) a.target_tok[q.r0 + i] = tok[k];
+        }
+    }
+    if (a.target_tok)
+        for (int64_t r = q.r0 + q.nr + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
+    int zr[3] = {-1, -1, -1};  // committed tokens lane, lane+32, lane+64
+    int acc = 0, cur = -1;
+    for (;;) {
+        const int row = cur + 1;
+        const int t0 = __shfl_sync(kFull, tok[0], row & 31);
+        const int t1 = __shfl_sync(kFull, tok[1], row & 31);
+        const int t2 = __shfl_sync(kFull, tok[2], row & 31);
+        const int want = row < 32 ? t0 : (row < 64 ? t1 : t2);  // the target's token after the current node
+        if ((acc & 31) == lane) zr[acc >> 5] = want;             // accepted tokens equal the target's tokens
+        const bool ok0 = lane < m && lane > cur && pr[0] == cur && dt[0] == want;
+        const bool ok1 = lane + 32 < m && lane + 32 > cur && pr[1] == cur && dt[1] == want;
+        const uint32_t b0 = __ballot_sync(kFull, ok0), b1 = __ballot_sync(kFull, ok1);
+        if ((b0 | b1) == 0u) break;
+        cur = b0 ? __ffs(b0) - 1 : 32 + __ffs(b1) - 1;
+        ++acc;
+    }
+    const int room = cap - n;
+    const int w = min(acc + 1, room);
+    int32_t* h = a.hist + hoff;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const int j = lane + 32 * k;
+        if (j <= kc) {
+            const int tk = j <= acc ? zr[k] : -1;
+            z[j] = tk;
+            if (j < w) h[n + j] = tk;
+        }
+    }
+    if (lane == 0) {
+        a.hist_len[b] = n + w;
+        a.n_commit[b] = w;
+        a.accepted[b] = acc;
+        a.status[b] = (w < acc + 1) ? HVD_REQ_CAPACITY : HVD_REQ_OK;
+        st.sel_bits = (st.sel_bits << 1) | (sel ? 1u : 0u);
+        st.acc_ring = (st.acc_ring << 8) | (unsigned long long)(acc & 0xff);
+        a.state[b] = st;
+    }
+}
+
 constexpr int kCommitWarps = 4;
 
 __global__ void __launch_bounds__(kCommitWarps * 32) verify_commit_kernel(const VerifyArgs a) {
@@ -255,7 +338,10 @@ __global__ void __launch_bounds__(kCommitWarps * 32) verify_commit_kernel(const 
     pdl_trigger();
     pdl_wait();
     if (b == 0 && (threadIdx.x & 31) < Q) a.next_unit[(threadIdx.x & 31) * kQueueStride] = 0u;  // zero at rest
-    if (b < a.B) commit_request(a, b, threadIdx.x & 31);
+    if (b < a.B) {
+        if (a.parent) commit_tree_request(a, b, threadIdx.x & 31);
+        else commit_request(a, b, threadIdx.x & 31);
+    }
 }
 
 struct Smem {

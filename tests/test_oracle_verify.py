@@ -167,3 +167,79 @@ def test_multi_step_loop_keeps_appending():
         assert (out.vf.status == O.REQ_OK).all()
     assert (rq.hist_len == inp.rq.hist_len + total).all() and (total >= 4).all()
     assert (rq.hist[rq.guard_mask] == W.GUARD_VALUE).all()
+
+
+# ---- token-tree drafts (the paper's model drafter proposes trees: App. A drafting configuration) --------
+def run_tree(draft, parent, targets, V=50, k_cap=None, n0=5, cap_extra=12):
+    m = len(draft)
+    k_cap = k_cap or max(m, 1)
+    rows = len(targets)
+    logits = np.random.default_rng(1).normal(0, 1, (rows, V)).astype(np.float32)
+    for i, t in enumerate(targets):
+        logits[i, t] = 20.0
+    hist = np.full(n0 + cap_extra, -7, np.int32); hist[:n0] = np.arange(n0) + 40
+    hist_len = np.array([n0], np.int32)
+    state = np.zeros(1, O.STATE_DTYPE)
+    sd = np.full((1, k_cap), -1, np.int32); sd[0, :m] = draft
+    par = np.full((1, k_cap), -9, np.int32); par[0, :m] = parent
+    out = O.verify_commit(logits, O.F32, V, np.array([0, rows], np.int64), 0, sd, [m], [0], k_cap=k_cap, hist=hist,
+                          hist_off=[0], hist_cap=[n0 + cap_extra], hist_len=hist_len, state=state, parent=par)
+    return out, hist, hist_len
+
+
+def test_tree_hand_worked():
+    #            prefix
+    #          /        \
+    #      n0:5          n1:6
+    #     /    \           \
+    #  n2:7    n3:8        n4:9
+    #            \
+    #            n5:3
+    draft, parent = [5, 6, 7, 8, 9, 3], [-1, -1, 0, 0, 1, 3]
+    # rows: 0 after the prefix, i+1 after node i.  Target says 5, then (after n0) 8, then (after n3) 3,
+    # then (after n5) 4: path n0 n3 n5 accepted, bonus 4.
+    targets = [5, 8, 1, 1, 3, 1, 4]
+    out, hist, hl = run_tree(draft, parent, targets)
+    assert out.accepted[0] == 3 and list(out.committed[0, :4]) == [5, 8, 3, 4] and hl[0] == 9
+    assert list(hist[5:9]) == [5, 8, 3, 4]
+    # the target prefers 6 at the root and then something no child of n1 carries: one accepted, bonus 2
+    out, *_ = run_tree(draft, parent, [6, 1, 2, 1, 1, 1, 1])
+    assert out.accepted[0] == 1 and list(out.committed[0, :2]) == [6, 2]
+    # the target's first token is nobody's: nothing accepted
+    out, *_ = run_tree(draft, parent, [4, 8, 9, 1, 3, 1, 1])
+    assert out.accepted[0] == 0 and out.committed[0, 0] == 4
+    # siblings with the same token: the first one is taken (and its subtree decides what follows)
+    out, *_ = run_tree([5, 5, 7, 8], [-1, -1, 0, 1], [5, 8, 7, 1, 1])
+    assert out.accepted[0] == 1 and list(out.committed[0, :2]) == [5, 8]
+
+
+def test_tree_chain_equals_linear_verification():
+    rng = np.random.default_rng(31)
+    for _ in range(50):
+        m = int(rng.integers(0, 9))
+        draft = list(rng.integers(0, 6, m))
+        targets = list(rng.integers(0, 6, m + 1))
+        a, h1, l1, _ = run_verify(draft, targets, V=50, k_cap=8)
+        b, h2, l2 = run_tree(draft, list(range(-1, m - 1)), targets, V=50, k_cap=8)
+        assert a.accepted[0] == b.accepted[0] and (a.committed == b.committed).all() and l1[0] == l2[0]
+
+
+def test_tree_against_path_enumeration():
+    """Brute force: among all root paths, the accepted one is the path whose every token equals the
+    target's token at its parent and that cannot be extended; children are tried in index order."""
+    rng = np.random.default_rng(32)
+    for _ in range(300):
+        m = int(rng.integers(1, 12))
+        parent = [int(rng.integers(-1, i)) for i in range(m)]
+        draft = [int(x) for x in rng.integers(0, 4, m)]
+        targets = [int(x) for x in rng.integers(0, 4, m + 1)]
+        cur, path = -1, []
+        while True:
+            kids = [c for c in range(m) if parent[c] == cur and draft[c] == targets[cur + 1]]
+            if not kids:
+                break
+            cur = kids[0]
+            path.append(draft[cur])
+        out, *_ = run_tree(draft, parent, targets, V=10, k_cap=12)
+        assert out.accepted[0] == len(path)
+        assert list(out.committed[0, :len(path) + 1]) == path + [targets[cur + 1]]
