@@ -96,6 +96,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     if (c->vf_blocks_per_sm[0] < 1 || c->vf_blocks_per_sm[1] < 1) { release(c); return HVD_ERR_UNSUPPORTED; }
     c->has_predictor = false;
     c->two_layer = false;
+    c->score2_ready = false;
     c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // measured: no gain on this path, off unless asked for
     c->host_ws = nullptr;
     c->host_ws_bytes = 0;

@@ -60,6 +60,7 @@ struct hvd_ctx {
     float b2, tau;
     bool has_predictor;
     bool two_layer;
+    bool score2_ready;  // the two-layer kernel's shared-memory size has been opted in on this device
     // lookup scratch
     hvd::LookupPartial* lk_partial;  // [max_batch, lk_max_chunks]
     uint32_t* lk_cnt;                // [max_batch], zero at rest

@@ -180,11 +180,10 @@ hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
                                         match_pos, match_cnt, model_draft, model_len, features, score, select,
                                         sel_draft, sel_len);
     if (a.WhT) {
-        static bool smem_opted_in = false;  // a per-function attribute, set once
-        if (!smem_opted_in) {
+        if (!ctx->score2_ready) {  // per device: the kernel needs the opt-in shared memory size
             HVD_CUDA_TRY(ctx, cudaFuncSetAttribute(score_select2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    (int)kScore2Smem));
-            smem_opted_in = true;
+            ctx->score2_ready = true;
         }
         HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select2_kernel, (B + kReqPerCta - 1) / kReqPerCta,
                                         kScore2Threads, kScore2Smem, stream, a));

@@ -226,6 +226,7 @@ def test_host_side_argument_errors():
     with pytest.raises(H.HvdError, match="n_max"):
         ctx.hvd_lookup(3, b.hist, b.hist_off, b.hist_cap, b.hist_len, b.K, 10**6, b.draft, b.draft_len,
                        b.match_len, b.match_pos, b.match_cnt)
+    assert ctx.hvd_device_status() == 0
     with pytest.raises(H.HvdError):
         H.Context(max_batch=0, k_cap=8, max_hist_len=10, max_rows=10, max_vocab=10)
     with pytest.raises(H.HvdError):
