@@ -139,6 +139,111 @@ void oracle_lookup(int32_t B, const int32_t* hist, const int64_t* hist_off, cons
 }
 
 /* ------------------------------------------------------------------ */
+/* Frequency-weighted continuation and the suffix score (the cache     */
+/* drafter of the paper follows SuffixDecoding, Sec. 3.2; its limits   */
+/* are in App. A "Drafting configuration": speculative factor/offset,  */
+/* minimum token probability 0.1; the Frequency-Based Hybrid baseline  */
+/* of Sec. 4.2 thresholds "the frequency-derived cache score").        */
+/* All occurrences of the longest matched suffix are merged: the walk  */
+/* starts with the set of their end positions; at each step the next   */
+/* token carried by most of the occurrences still alive is taken (ties:*/
+/* the token whose latest alive occurrence is latest), with            */
+/* probability count / alive; the walk stops when that probability is  */
+/* below min_prob or the draft limit is reached; the score is the sum  */
+/* of the probabilities.  With more than max_occ occurrences only the  */
+/* latest one is followed (probability 1 per token).                   */
+/* ------------------------------------------------------------------ */
+void oracle_lookup_freq_one(const int32_t* h, int32_t n, int32_t K, int32_t k_cap, int32_t l_max,
+                            int32_t min_match, float spec_factor, float spec_offset, float min_prob,
+                            int32_t max_occ, int32_t* draft /*[k_cap]*/, int32_t* draft_len, float* score,
+                            int32_t* match_len, int32_t* match_pos, int32_t* match_cnt) {
+    int32_t plain[64];
+    int32_t plain_len;
+    oracle_lookup_one(h, n, K, k_cap, l_max, min_match, spec_factor, spec_offset, plain, &plain_len, match_len,
+                      match_pos, match_cnt);
+    for (int32_t j = 0; j < k_cap; ++j) draft[j] = -1;
+    *draft_len = 0;
+    *score = 0.0f;
+    const int32_t L = *match_len;
+    if (L == 0) return;
+    if (K < 0) K = 0;
+    if (K > k_cap) K = k_cap;
+    int32_t limit = K;
+    if (spec_factor > 0.0f) {
+        float lim = spec_factor * (float)L;
+        lim = lim + spec_offset;
+        int32_t cap = (int32_t)floorf(lim);
+        if (cap < 0) cap = 0;
+        if (cap < limit) limit = cap;
+    }
+    if (*match_cnt > max_occ) { /* too many to merge: follow the latest occurrence only */
+        for (int32_t j = 0; j < plain_len; ++j) { draft[j] = plain[j]; *score = *score + 1.0f; }
+        *draft_len = plain_len;
+        return;
+    }
+    /* the occurrences: every e whose (capped) match length equals L */
+    int32_t* alive = (int32_t*)malloc(sizeof(int32_t) * (size_t)(*match_cnt > 0 ? *match_cnt : 1));
+    int32_t na = 0;
+    for (int32_t e = 1; e <= n - 1; ++e) {
+        int32_t l = 0;
+        while (l < l_max && l < e && h[e - 1 - l] == h[n - 1 - l]) ++l;
+        if (l == L) alive[na++] = e;
+    }
+    int32_t d = 0;
+    float sc = 0.0f;
+    while (d < limit) {
+        /* best next token among the alive occurrences */
+        int32_t best_tok = -1, best_cnt = 0, best_last = -1;
+        for (int32_t i = 0; i < na; ++i) {
+            if (alive[i] + d >= n) continue;
+            const int32_t x = h[alive[i] + d];
+            int32_t c = 0, last = -1;
+            for (int32_t j = 0; j < na; ++j)
+                if (alive[j] + d < n && h[alive[j] + d] == x) { ++c; if (alive[j] > last) last = alive[j]; }
+            if (c > best_cnt || (c == best_cnt && last > best_last)) { best_cnt = c; best_tok = x; best_last = last; }
+        }
+        if (best_cnt == 0) break;
+        const float prob = (float)best_cnt / (float)na;
+        if (prob < min_prob) break;
+        draft[d] = best_tok;
+        sc = sc + prob;
+        int32_t nb = 0;
+        for (int32_t i = 0; i < na; ++i)
+            if (alive[i] + d < n && h[alive[i] + d] == best_tok) alive[nb++] = alive[i];
+        na = nb;
+        ++d;
+    }
+    free(alive);
+    *draft_len = d;
+    *score = sc;
+}
+
+typedef struct {
+    lookup_args l; float min_prob; int32_t max_occ; float* score;
+} lookup_freq_args;
+
+static void lookup_freq_req(int32_t b, void* p) {
+    lookup_freq_args* fa = (lookup_freq_args*)p;
+    lookup_args* a = &fa->l;
+    int32_t n = a->hist_len[b];
+    if (n < 0 || n > a->hist_cap[b]) n = 0;
+    oracle_lookup_freq_one(a->hist + a->hist_off[b], n, a->K[b], a->k_cap, a->l_max, a->min_match, a->spec_factor,
+                           a->spec_offset, fa->min_prob, fa->max_occ, a->draft + (int64_t)b * a->k_cap,
+                           a->draft_len + b, fa->score + b, a->match_len + b, a->match_pos + b, a->match_cnt + b);
+}
+
+void oracle_lookup_freq(int32_t B, const int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                        const int32_t* hist_len, const int32_t* K, int32_t k_cap, int32_t l_max,
+                        int32_t min_match, float spec_factor, float spec_offset, float min_prob, int32_t max_occ,
+                        int32_t* draft, int32_t* draft_len, float* score, int32_t* match_len,
+                        int32_t* match_pos, int32_t* match_cnt, int32_t nthreads) {
+    lookup_freq_args fa = {{hist, hist_off, hist_cap, hist_len, K, k_cap, l_max, min_match, spec_factor,
+                            spec_offset, draft, draft_len, match_len, match_pos, match_cnt}, min_prob, max_occ,
+                           score};
+    for_each_request(B, nthreads, lookup_freq_req, &fa);
+}
+
+/* ------------------------------------------------------------------ */
 /* Payoff labels by trace replay (Sec. 3.3 "training labels"; App. B   */
 /* "Payoff Label Construction"): every position t of a recorded trace  */
 /* is a decoding state with prefix x[0..t); its cache draft comes from */
