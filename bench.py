@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--predictor", default="config", choices=["config", "2x256"],
                     help="2x256: the paper's predictor shape (two hidden layers of 256 units) instead of the config's")
+    ap.add_argument("--freq", action="store_true",
+                    help="variant of the lookup step: frequency-weighted draft and score (hvd_lookup_freq) on the config's requests")
     ap.add_argument("--replay", action="store_true",
                     help="second workload: payoff labels by trace replay (hvd_replay_labels) on one history of the config")
     ap.add_argument("--unfused", action="store_true",
@@ -231,6 +233,72 @@ def run_replay(args):
     ctx.close()
 
 
+# ----------------------------------------------------------------------------------------------
+# variant of the lookup step: frequency-weighted draft and suffix score
+# ----------------------------------------------------------------------------------------------
+def run_freq(args):
+    import torch
+    import hvd_workloads as W
+    import paper_2606_01019_b200 as H
+    torch.cuda.set_device(0)
+    w = W.CONFIGS[args.config]
+    rq = W.make_requests(w)
+    B, n_max = rq.B, int(rq.hist_len.max())
+    dev = lambda a: torch.as_tensor(np.ascontiguousarray(a), device="cuda")
+    hist, off, cap, ln, K = dev(rq.hist), dev(rq.hist_off), dev(rq.hist_cap), dev(rq.hist_len), dev(rq.K)
+    i32 = lambda *shape: torch.zeros(shape, dtype=torch.int32, device="cuda")
+    draft, dlen, mlen, mpos, mcnt = i32(B, w.k_cap), i32(B), i32(B), i32(B), i32(B)
+    score = torch.zeros(B, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    from oracle import hvd_oracle as O
+    from oracle import pipeline as P
+    cores = P.host_threads()
+    reps = max(3, min(args.steps, 50))
+    cases = []
+    for l_max in (w.l_max, 2):   # the configured maximum match length, and a short one (many occurrences per request)
+        ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=1, max_vocab=1,
+                        l_max=l_max, min_match=min(w.min_match, l_max), spec_factor=8.0)
+        calls = {"hvd_lookup": lambda: ctx.hvd_lookup(B, hist, off, cap, ln, K, n_max, draft, dlen, mlen, mpos, mcnt),
+                 "hvd_lookup_freq": lambda: ctx.hvd_lookup_freq(B, hist, off, cap, ln, K, n_max, 0.1, H.FREQ_MAX_OCC, 0.0,
+                                                                None, None, draft, dlen, score, mlen, mpos, mcnt)}
+        us = {}
+        for name, call in calls.items():
+            for _ in range(max(3, args.warmup)):
+                call()
+            evs = []
+            for _ in range(reps):   # all enqueued ahead: the fills hide the host's launch latency
+                flush.fill_(1)      # L2 flush between timed calls
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); call(); e1.record()
+                evs.append((e0, e1))
+            torch.cuda.synchronize()
+            us[name] = sum(a.elapsed_time(b) for a, b in evs) / reps * 1e3
+        t0 = time.perf_counter()
+        ref = O.lookup_freq(rq.hist, rq.hist_off, rq.hist_cap, rq.hist_len, rq.K, k_cap=w.k_cap, l_max=l_max,
+                            min_match=min(w.min_match, l_max), spec_factor=8.0, min_prob=0.1, max_occ=H.FREQ_MAX_OCC,
+                            nthreads=cores)
+        cpu_s = time.perf_counter() - t0
+        agrees = bool((ref.draft == draft.cpu().numpy()).all() and
+                      (ref.score.view(np.uint32) == score.cpu().numpy().view(np.uint32)).all())
+        cases.append({"l_max": l_max, "us_lookup": us["hvd_lookup"], "us_lookup_freq": us["hvd_lookup_freq"],
+                      "mean_occurrences": float(ref.match_cnt.mean()), "max_occurrences": int(ref.match_cnt.max()),
+                      "merged_requests": int(((ref.match_cnt > 0) & (ref.match_cnt <= H.FREQ_MAX_OCC)).sum()),
+                      "mean_draft_len": float(ref.draft_len.mean()), "mean_score": float(ref.score.mean()),
+                      "oracle_ms": cpu_s * 1e3, "agrees_with_oracle": agrees})
+        ctx.close()
+    hist_bytes = int(rq.hist_len.sum()) * 4
+    c0 = cases[0]
+    line = {"metric": "frequency-weighted lookups/s", "value": B / (c0["us_lookup_freq"] * 1e-6), "unit": "requests/s",
+            "n_gpus": 1, "steps": reps, "higher_is_better": True, "dtype": "int32 (fp32 score)", "data": "synthetic",
+            "config": {"workload": f"{w.name}: batch {B}, histories {w.n} tokens; 3 launches per call, "
+                                   "L2 flushed between calls", "history_bytes": hist_bytes},
+            "history_scan_gbs": 2 * hist_bytes / (c0["us_lookup_freq"] * 1e-6) / 1e9,
+            "cases": cases,
+            "cpu_baseline": {"value": B / (c0["oracle_ms"] * 1e-3), "unit": "requests/s", "cores": cores, "kind": "oracle",
+                             "sample": "the same batch, once"}}
+    print(json.dumps(line), flush=True)
+
+
 def workload_config(w, n_gpus, extra=None):
     cfg = {"workload": f"{w.name}: batch {w.B}, histories {w.n} tokens, vocab {w.V}, K {w.K}, {w.dtype} logits",
            "requests_per_gpu": w.B, "parallelism": f"requests sharded over {n_gpus} GPU(s), no collective"}
@@ -246,6 +314,9 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.freq:
+        run_freq(args)
         return
     if args.replay:
         run_replay(args)

@@ -173,6 +173,36 @@ HVD_API hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_
                                            int32_t* sel_draft, int32_t* sel_len, void* stream);
 
 /*
+ * Frequency-weighted cache draft, suffix score and the score-threshold selection (Sec. 4.1
+ * "Frequency-Based Hybrid Decoding": same cache-first structure, the decision taken on the
+ * frequency-derived cache score; App. A drafting table: speculation limits and the minimum token
+ * probability).  Steps, per request:
+ *   1. hvd_lookup's search: longest match length L, its latest occurrence, the number c of
+ *      occurrences (match_len / match_pos / match_cnt exactly as hvd_lookup writes them).
+ *   2. limit = min(K, floor(spec_factor * L + spec_offset)) as in hvd_lookup.  If c <= max_occ all c
+ *      occurrences are merged: starting with all of them alive, step s takes the token that most
+ *      alive occurrences continue with at offset s (ties: the token whose latest such occurrence is
+ *      later; occurrences that run into the end of the history have no token), p = count / alive in
+ *      fp32 (one IEEE division); the walk stops when p < min_prob, at `limit` tokens, or when no alive
+ *      occurrence has a token left; otherwise the token joins the draft, p is added to the score
+ *      (fp32, in step order) and only the occurrences that continue with it stay alive.
+ *      If c > max_occ the draft is hvd_lookup's (latest occurrence only) and score = draft_len.
+ *   3. optional (select, sel_draft, sel_len all non-NULL): select = (draft_len > 0 && score >= threshold);
+ *      sel_draft / sel_len as in hvd_score_select (the model draft, or an empty draft, otherwise).
+ * draft int32 [B, k_cap] (-1 beyond draft_len), draft_len int32 [B], score float [B]: DEVICE outputs.
+ * min_prob, max_occ (1 .. HVD_FREQ_MAX_OCC), threshold: HOST values.  Everything else as in hvd_lookup.
+ * Uses context scratch: one call at a time per context.
+ */
+enum { HVD_FREQ_MAX_OCC = 128 };
+HVD_API hvd_status hvd_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                                   const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
+                                   int32_t n_max, float min_prob, int32_t max_occ, float threshold,
+                                   const int32_t* model_draft, const int32_t* model_len, int32_t* draft,
+                                   int32_t* draft_len, float* score, int32_t* match_len, int32_t* match_pos,
+                                   int32_t* match_cnt, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
+                                   void* stream);
+
+/*
  * Payoff labels by trace replay (Sec. 3.3, "We derive training labels ..."; App. B "Payoff Label
  * Construction").  Every position t = 1..n of a recorded trace x[0..n) is a decoding state with prefix
  * x[0..t): its cache draft is the hvd_lookup result on that prefix (same rules, K for every state),

@@ -19,7 +19,10 @@
  *   - most-recent-occurrence tie-break among equally long matches,
  *   - the exact formulas of the eight payoff features (the paper names only
  *     feature groups, App. B table "Payoff predictor feature groups"),
- *   - the layout of the recent-history summary h.
+ *   - the layout of the recent-history summary h,
+ *   - the frequency-weighted continuation and its score (the paper names the
+ *     baseline's "frequency-derived cache score" without defining it; pinned
+ *     to an independent restatement and hand-worked cases only).
  */
 #include <math.h>
 #include <pthread.h>
@@ -241,6 +244,27 @@ void oracle_lookup_freq(int32_t B, const int32_t* hist, const int64_t* hist_off,
                             spec_offset, draft, draft_len, match_len, match_pos, match_cnt}, min_prob, max_occ,
                            score};
     for_each_request(B, nthreads, lookup_freq_req, &fa);
+}
+
+/* Selection of the frequency-based hybrid rule (Sec. 4.1): verify the cache draft when it is not
+   empty and its frequency score reaches the threshold, the model draft otherwise. */
+void oracle_freq_select(int32_t B, int32_t k_cap, const int32_t* draft, const int32_t* draft_len,
+                        const float* score, float threshold, const int32_t* model_draft /*may be NULL*/,
+                        const int32_t* model_len, int32_t* select, int32_t* sel_draft, int32_t* sel_len) {
+    for (int32_t b = 0; b < B; ++b) {
+        const int32_t s = (draft_len[b] > 0 && score[b] >= threshold) ? 1 : 0;
+        const int32_t* src = NULL;
+        int32_t m = 0;
+        if (s) { src = draft + (int64_t)b * k_cap; m = draft_len[b]; }
+        else if (model_draft) {
+            src = model_draft + (int64_t)b * k_cap; m = model_len[b];
+            if (m < 0) m = 0;
+            if (m > k_cap) m = k_cap;
+        }
+        select[b] = s;
+        sel_len[b] = m;
+        for (int32_t j = 0; j < k_cap; ++j) sel_draft[(int64_t)b * k_cap + j] = j < m ? src[j] : -1;
+    }
 }
 
 /* ------------------------------------------------------------------ */

@@ -101,6 +101,18 @@ def lookup_freq(hist, hist_off, hist_cap, hist_len, K, *, k_cap, l_max=64, min_m
     return out
 
 
+def freq_select(out: FreqOut, threshold, model_draft=None, model_len=None):
+    """The frequency-based hybrid rule on lookup_freq's result: (select, sel_draft, sel_len)."""
+    B, k_cap = out.draft.shape
+    select = np.empty(B, np.int32); sel_len = np.empty(B, np.int32); sel_draft = np.empty((B, k_cap), np.int32)
+    md = None if model_draft is None else _i32(model_draft)
+    ml = None if model_len is None else _i32(model_len)
+    lib().oracle_freq_select(C.c_int32(B), C.c_int32(k_cap), _p(out.draft), _p(out.draft_len), _p(out.score),
+                             C.c_float(threshold), None if md is None else _p(md), None if ml is None else _p(ml),
+                             _p(select), _p(sel_draft), _p(sel_len))
+    return select, sel_draft, sel_len
+
+
 @dataclass
 class ReplayOut:
     label: np.ndarray

@@ -49,6 +49,7 @@ _SIGNATURES = {
     "hvd_set_predictor2": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _vp]),
     "hvd_lookup": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_score_select": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32] + [_vp] * 14 + [_vp]),
+    "hvd_lookup_freq": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _f32, _i32, _f32] + [_vp] * 11 + [_vp]),
     "hvd_replay_labels": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
@@ -104,6 +105,7 @@ def _stream():
 
 
 NOALLOC_MAX_ROWS, NOALLOC_MAX_BATCH = 16384, 2048
+FREQ_MAX_OCC = 128   # HVD_FREQ_MAX_OCC
 
 
 def hvd_verify_commit_noalloc(B, k_cap, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
@@ -195,6 +197,15 @@ class Context:
             _ptr(prompt_len), _ptr(state), _ptr(model_draft), _ptr(model_len), _ptr(draft), _ptr(draft_len),
             _ptr(match_len), _ptr(match_pos), _ptr(match_cnt), _ptr(features), _ptr(score), _ptr(select),
             _ptr(sel_draft), _ptr(sel_len), _stream()), "hvd_lookup_score_select")
+
+    def hvd_lookup_freq(self, B, hist, hist_off, hist_cap, hist_len, K, n_max, min_prob, max_occ, threshold,
+                        model_draft, model_len, draft, draft_len, score, match_len, match_pos, match_cnt,
+                        select=None, sel_draft=None, sel_len=None):
+        self._check(self._lib.hvd_lookup_freq(
+            self._h, B, _ptr(hist), _ptr(hist_off), _ptr(hist_cap), _ptr(hist_len), _ptr(K), n_max, min_prob,
+            max_occ, threshold, _ptr(model_draft), _ptr(model_len), _ptr(draft), _ptr(draft_len), _ptr(score),
+            _ptr(match_len), _ptr(match_pos), _ptr(match_cnt), _ptr(select), _ptr(sel_draft), _ptr(sel_len),
+            _stream()), "hvd_lookup_freq")
 
     def hvd_replay_labels(self, trace, n, K, label, draft_len, match_len, match_pos, match_cnt):
         self._check(self._lib.hvd_replay_labels(self._h, _ptr(trace), n, K, _ptr(label), _ptr(draft_len),

@@ -15,6 +15,7 @@ void release(hvd_ctx* c) {
     if (!c) return;
     cudaFree(c->d_W1); cudaFree(c->d_b1); cudaFree(c->d_W2); cudaFree(c->d_WhT); cudaFree(c->d_bh);
     cudaFree(c->lk_partial); cudaFree(c->lk_cnt);
+    cudaFree(c->fq_occ); cudaFree(c->fq_cnt);
     cudaFree(c->rp_off); cudaFree(c->rp_cap); cudaFree(c->rp_len); cudaFree(c->rp_K); cudaFree(c->rp_draft);
     cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
@@ -78,6 +79,8 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->d_bh, H * sizeof(float)) == cudaSuccess;
     ok = ok && alloc_zero(&c->lk_partial, (size_t)cfg->max_batch * c->lk_max_chunks * sizeof(LookupPartial)) == cudaSuccess;
     ok = ok && alloc_zero(&c->lk_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->fq_occ, (size_t)cfg->max_batch * HVD_FREQ_MAX_OCC * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->fq_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
     const size_t MB = (size_t)cfg->max_batch;
     ok = ok && alloc_zero(&c->rp_off, MB * sizeof(int64_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->rp_cap, MB * sizeof(int32_t)) == cudaSuccess;
@@ -186,6 +189,33 @@ hvd_status hvd_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_
         return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max outside [0, max_hist_len]");
     return launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
                          match_len, match_pos, match_cnt, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                           const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K, int32_t n_max,
+                           float min_prob, int32_t max_occ, float threshold, const int32_t* model_draft,
+                           const int32_t* model_len, int32_t* draft, int32_t* draft_len, float* score,
+                           int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, int32_t* select,
+                           int32_t* sel_draft, int32_t* sel_len, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_freq: B outside [1, max_batch]");
+    if (!hist || !hist_off || !hist_cap || !hist_len || !K || !draft || !draft_len || !score || !match_len ||
+        !match_pos || !match_cnt)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_freq: NULL pointer");
+    const int n_sel = (select != nullptr) + (sel_draft != nullptr) + (sel_len != nullptr);
+    if (n_sel != 0 && n_sel != 3)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_freq: select, sel_draft and sel_len go together");
+    if ((model_draft == nullptr) != (model_len == nullptr))
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_freq: model_draft and model_len go together");
+    if (!aligned(hist, 16)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_freq: hist must be 16-byte aligned");
+    if (n_max < 0 || n_max > ctx->cfg.max_hist_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_freq: n_max outside [0, max_hist_len]");
+    if (max_occ < 1 || max_occ > HVD_FREQ_MAX_OCC)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_freq: max_occ outside [1, HVD_FREQ_MAX_OCC]");
+    if (!(min_prob >= 0.0f)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_freq: min_prob must be >= 0");
+    return launch_lookup_freq(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, min_prob, max_occ, threshold,
+                              model_draft, model_len, draft, draft_len, score, match_len, match_pos, match_cnt,
+                              select, sel_draft, sel_len, static_cast<cudaStream_t>(stream));
 }
 
 hvd_status hvd_replay_labels(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label,

@@ -65,6 +65,9 @@ struct hvd_ctx {
     hvd::LookupPartial* lk_partial;  // [max_batch, lk_max_chunks]
     uint32_t* lk_cnt;                // [max_batch], zero at rest
     int lk_max_chunks;
+    // occurrence lists of the frequency-weighted draft
+    int32_t* fq_occ;    // [max_batch, HVD_FREQ_MAX_OCC]
+    uint32_t* fq_cnt;   // [max_batch], zero at rest
     // verify scratch
     unsigned long long* vf_row_key;  // [max_rows], zero at rest
     uint32_t* vf_next_unit;          // zero at rest
@@ -147,6 +150,13 @@ hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
 
 hvd_status launch_replay(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label, int32_t* draft_len,
                          int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream);
+
+hvd_status launch_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                              const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K, int32_t n_max,
+                              float min_prob, int32_t max_occ, float threshold, const int32_t* model_draft,
+                              const int32_t* model_len, int32_t* draft, int32_t* draft_len, float* score,
+                              int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, int32_t* select,
+                              int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream);
 
 struct VerifyArgs {
     int32_t B;

@@ -101,3 +101,19 @@ def test_minimum_probability_cut():
     assert d == [109, 209] and sc == f32(f32(0.1) + f32(1.0))
     d, sc, _ = run_one(fan(12), 4, max_occ=8)    # more occurrences than are merged: the latest one alone
     assert d == [111, 211] and sc == 2.0
+
+
+def test_freq_select_hand_cases():
+    """Rule of the frequency-based hybrid baseline: cache draft iff non-empty and score >= threshold."""
+    out = O.FreqOut(np.array([[5, 6, -1], [7, -1, -1], [-1, -1, -1], [8, 9, 4]], np.int32),
+                    np.array([2, 1, 0, 3], np.int32), None, None, None,
+                    np.array([1.5, 0.99, 0.0, 1.0], np.float32))
+    md = np.array([[1, 2, 3], [1, 2, 3], [1, 2, 3], [1, 2, 3]], np.int32)
+    ml = np.array([3, 2, 5, -1], np.int32)
+    sel, sd, sl = O.freq_select(out, 1.0, md, ml)
+    assert list(sel) == [1, 0, 0, 1]
+    assert list(sl) == [2, 2, 3, 3]
+    assert sd.tolist() == [[5, 6, -1], [1, 2, -1], [1, 2, 3], [8, 9, 4]]
+    sel, sd, sl = O.freq_select(out, 0.0)               # no model draft: empty selection when not chosen
+    assert list(sel) == [1, 1, 0, 1] and list(sl) == [2, 1, 0, 3]
+    assert sd[2].tolist() == [-1, -1, -1]
