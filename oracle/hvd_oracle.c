@@ -20,6 +20,8 @@
  *   - the exact formulas of the eight payoff features (the paper names only
  *     feature groups, App. B table "Payoff predictor feature groups"),
  *   - the layout of the recent-history summary h,
+ *   - how warm-up traces and the own history share the cache (history before
+ *     corpus at equal match length; separators between traces),
  *   - the frequency-weighted continuation and its score (the paper names the
  *     baseline's "frequency-derived cache score" without defining it; pinned
  *     to an independent restatement and hand-worked cases only).
@@ -139,6 +141,94 @@ void oracle_lookup(int32_t B, const int32_t* hist, const int64_t* hist_off, cons
     lookup_args a = {hist, hist_off, hist_cap, hist_len, K, k_cap, l_max, min_match, spec_factor,
                      spec_offset, draft, draft_len, match_len, match_pos, match_cnt};
     for_each_request(B, nthreads, lookup_req, &a);
+}
+
+/* ------------------------------------------------------------------ */
+/* Step 1 with a shared warm-up corpus (Algorithm 1, "Initialize C from */
+/* cache-warmup traces and the input prompt"; App. C: warm-up prompts  */
+/* of the same dataset initialise the suffix cache).  The cache of a   */
+/* request is then [corpus, own history]: the corpus is one token      */
+/* array shared by all requests; a negative entry separates two        */
+/* traces, is never part of a match and ends a draft.  Candidates:     */
+/*   history e in [1, n-1] as in oracle_lookup_one;                    */
+/*   corpus  e in [1, m-1] with corpus[e] >= 0 (a continuation token    */
+/*   exists), match length l <= min(l_max, e, n).                       */
+/* The longest match wins; among equally long ones the history comes   */
+/* before the corpus, and within a source the latest position.         */
+/* match_src = 0 (history) or 1 (corpus); match_pos is the position in  */
+/* that source; match_cnt counts both sources.                         */
+/* ------------------------------------------------------------------ */
+void oracle_lookup_corpus_one(const int32_t* h, int32_t n, const int32_t* corpus, int32_t m, int32_t K,
+                              int32_t k_cap, int32_t l_max, int32_t min_match, float spec_factor,
+                              float spec_offset, int32_t* draft /*[k_cap]*/, int32_t* draft_len,
+                              int32_t* match_len, int32_t* match_pos, int32_t* match_src, int32_t* match_cnt) {
+    int32_t best_L = 0, best_e = -1, best_src = 0, cnt = 0;
+    if (K < 0) K = 0;
+    if (K > k_cap) K = k_cap;
+    /* corpus first, history second: with ">=" on ties the later candidate of this order wins */
+    for (int32_t e = 1; e <= m - 1; ++e) {
+        if (corpus[e] < 0) continue;
+        int32_t l = 0;
+        while (l < l_max && l < e && l < n && corpus[e - 1 - l] >= 0 && corpus[e - 1 - l] == h[n - 1 - l]) ++l;
+        if (l == 0) continue;
+        if (l > best_L) { best_L = l; best_e = e; best_src = 1; cnt = 1; }
+        else if (l == best_L) { best_e = e; best_src = 1; ++cnt; }
+    }
+    for (int32_t e = 1; e <= n - 1; ++e) {
+        int32_t l = 0;
+        while (l < l_max && l < e && h[e - 1 - l] == h[n - 1 - l]) ++l;
+        if (l == 0) continue;
+        if (l > best_L) { best_L = l; best_e = e; best_src = 0; cnt = 1; }
+        else if (l == best_L) { best_e = e; best_src = 0; ++cnt; }
+    }
+    for (int32_t j = 0; j < k_cap; ++j) draft[j] = -1;
+    if (best_L < min_match || best_L == 0) {
+        *match_len = 0; *match_pos = -1; *match_src = 0; *match_cnt = 0; *draft_len = 0;
+        return;
+    }
+    int32_t d = K;
+    if (spec_factor > 0.0f) {
+        float prod = spec_factor * (float)best_L;
+        float lim = prod + spec_offset;
+        int32_t cap = (int32_t)floorf(lim);
+        if (cap < 0) cap = 0;
+        if (cap < d) d = cap;
+    }
+    if (best_src == 0) {
+        if (n - best_e < d) d = n - best_e;
+        for (int32_t j = 0; j < d; ++j) draft[j] = h[best_e + j];
+    } else {
+        if (m - best_e < d) d = m - best_e;
+        int32_t j = 0;
+        while (j < d && corpus[best_e + j] >= 0) { draft[j] = corpus[best_e + j]; ++j; } /* a separator ends the draft */
+        d = j;
+    }
+    *match_len = best_L; *match_pos = best_e; *match_src = best_src; *match_cnt = cnt; *draft_len = d;
+}
+
+typedef struct {
+    lookup_args l; const int32_t* corpus; int32_t m; int32_t* match_src;
+} lookup_corpus_args;
+
+static void lookup_corpus_req(int32_t b, void* p) {
+    lookup_corpus_args* ca = (lookup_corpus_args*)p;
+    lookup_args* a = &ca->l;
+    int32_t n = a->hist_len[b];
+    if (n < 0 || n > a->hist_cap[b]) n = 0;
+    oracle_lookup_corpus_one(a->hist + a->hist_off[b], n, ca->corpus, ca->m, a->K[b], a->k_cap, a->l_max,
+                             a->min_match, a->spec_factor, a->spec_offset, a->draft + (int64_t)b * a->k_cap,
+                             a->draft_len + b, a->match_len + b, a->match_pos + b, ca->match_src + b,
+                             a->match_cnt + b);
+}
+
+void oracle_lookup_corpus(int32_t B, const int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                          const int32_t* hist_len, const int32_t* K, const int32_t* corpus, int32_t m,
+                          int32_t k_cap, int32_t l_max, int32_t min_match, float spec_factor, float spec_offset,
+                          int32_t* draft, int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
+                          int32_t* match_src, int32_t* match_cnt, int32_t nthreads) {
+    lookup_corpus_args ca = {{hist, hist_off, hist_cap, hist_len, K, k_cap, l_max, min_match, spec_factor,
+                              spec_offset, draft, draft_len, match_len, match_pos, match_cnt}, corpus, m, match_src};
+    for_each_request(B, nthreads, lookup_corpus_req, &ca);
 }
 
 /* ------------------------------------------------------------------ */

@@ -81,6 +81,27 @@ def lookup(hist, hist_off, hist_cap, hist_len, K, *, k_cap, l_max=64, min_match=
 
 
 @dataclass
+class CorpusOut(LookupOut):
+    match_src: np.ndarray = None
+
+
+def lookup_corpus(hist, hist_off, hist_cap, hist_len, K, corpus, *, k_cap, l_max=64, min_match=2, spec_factor=1.0,
+                  spec_offset=0.0, nthreads=1) -> CorpusOut:
+    """Cache draft from [shared warm-up corpus, own history]; negative corpus entries separate traces."""
+    B = len(hist_len)
+    hist = _i32(hist); hist_len = _i32(hist_len); hist_cap = _i32(hist_cap); K = _i32(K); corpus = _i32(corpus)
+    hist_off = np.ascontiguousarray(hist_off, dtype=np.int64)
+    out = CorpusOut(np.empty((B, k_cap), np.int32), np.empty(B, np.int32), np.empty(B, np.int32),
+                    np.empty(B, np.int32), np.empty(B, np.int32), np.empty(B, np.int32))
+    lib().oracle_lookup_corpus(C.c_int32(B), _p(hist), _p(hist_off), _p(hist_cap), _p(hist_len), _p(K), _p(corpus),
+                               C.c_int32(len(corpus)), C.c_int32(k_cap), C.c_int32(l_max), C.c_int32(min_match),
+                               C.c_float(spec_factor), C.c_float(spec_offset), _p(out.draft), _p(out.draft_len),
+                               _p(out.match_len), _p(out.match_pos), _p(out.match_src), _p(out.match_cnt),
+                               C.c_int32(nthreads))
+    return out
+
+
+@dataclass
 class FreqOut(LookupOut):
     score: np.ndarray = None
 
