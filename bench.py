@@ -52,6 +52,8 @@ def parse_args():
                     help="2x256: the paper's predictor shape (two hidden layers of 256 units) instead of the config's")
     ap.add_argument("--freq", action="store_true",
                     help="variant of the lookup step: frequency-weighted draft and score (hvd_lookup_freq) on the config's requests")
+    ap.add_argument("--corpus", action="store_true",
+                    help="variant of the lookup step: shared warm-up corpus scanned with the history (hvd_lookup_corpus)")
     ap.add_argument("--replay", action="store_true",
                     help="second workload: payoff labels by trace replay (hvd_replay_labels) on one history of the config")
     ap.add_argument("--unfused", action="store_true",
@@ -299,6 +301,76 @@ def run_freq(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------------------------
+# variant of the lookup step: shared warm-up corpus
+# ----------------------------------------------------------------------------------------------
+def run_corpus(args):
+    import torch
+    import hvd_workloads as W
+    import paper_2606_01019_b200 as H
+    torch.cuda.set_device(0)
+    w = W.CONFIGS[args.config]
+    rq = W.make_requests(w)
+    B, n_max = rq.B, int(rq.hist_len.max())
+    dev = lambda a: torch.as_tensor(np.ascontiguousarray(a), device="cuda")
+    hist, off, cap, ln, K = dev(rq.hist), dev(rq.hist_off), dev(rq.hist_cap), dev(rq.hist_len), dev(rq.K)
+    i32 = lambda *shape: torch.zeros(shape, dtype=torch.int32, device="cuda")
+    draft, dlen, mlen, mpos, msrc, mcnt = i32(B, w.k_cap), i32(B), i32(B), i32(B), i32(B), i32(B)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    from oracle import hvd_oracle as O
+    from oracle import pipeline as P
+    cores = P.host_threads()
+    reps = max(3, min(args.steps, 50))
+    ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=1, max_vocab=1,
+                    l_max=w.l_max, min_match=w.min_match)
+
+    def timed(call, cold):
+        for _ in range(max(3, args.warmup)):
+            call()
+        evs = []
+        for _ in range(reps):   # all enqueued ahead: the fills hide the host's launch latency
+            if cold:
+                flush.fill_(1)  # L2 flush between timed calls
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); call(); e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in evs) / reps * 1e3
+
+    plain = lambda: ctx.hvd_lookup(B, hist, off, cap, ln, K, n_max, draft, dlen, mlen, mpos, mcnt)
+    both = lambda: ctx.hvd_lookup_corpus(B, hist, off, cap, ln, K, n_max, draft, dlen, mlen, mpos, msrc, mcnt)
+    us_plain = timed(plain, True)
+    cases = []
+    for n_traces in (16, 64, 256):
+        corpus = W.make_corpus(w, n_traces=n_traces)
+        cd = dev(corpus)
+        ctx.hvd_set_corpus(cd)
+        us_cold, us_warm = timed(both, True), timed(both, False)
+        t0 = time.perf_counter()
+        ref = O.lookup_corpus(rq.hist, rq.hist_off, rq.hist_cap, rq.hist_len, rq.K, corpus, k_cap=w.k_cap,
+                              l_max=w.l_max, min_match=w.min_match, nthreads=cores)
+        cpu_s = time.perf_counter() - t0
+        agrees = all(bool((getattr(ref, k) == t.cpu().numpy()).all()) for k, t in
+                     (("draft", draft), ("draft_len", dlen), ("match_len", mlen), ("match_pos", mpos),
+                      ("match_src", msrc), ("match_cnt", mcnt)))
+        m = len(corpus)
+        cases.append({"corpus_tokens": m, "us_lookup_corpus_cold": us_cold, "us_lookup_corpus_corpus_in_l2": us_warm,
+                      "token_compares_per_s": float(B) * m / (us_warm * 1e-6),
+                      "requests_matched_in_corpus": int(ref.match_src.sum()), "oracle_ms": cpu_s * 1e3,
+                      "agrees_with_oracle": agrees})
+    c = cases[1]
+    line = {"metric": "lookups over corpus and history per second", "value": B / (c["us_lookup_corpus_cold"] * 1e-6),
+            "unit": "requests/s", "n_gpus": 1, "steps": reps, "higher_is_better": True, "dtype": "int32",
+            "data": "synthetic",
+            "config": {"workload": f"{w.name}: batch {B}, histories {w.n} tokens, warm-up corpus of {c['corpus_tokens']} "
+                                   "tokens (64 traces); 2 launches per call, L2 flushed between calls"},
+            "us_lookup_history_only": us_plain, "cases": cases,
+            "cpu_baseline": {"value": B / (c["oracle_ms"] * 1e-3), "unit": "requests/s", "cores": cores, "kind": "oracle",
+                             "sample": "the same batch and corpus, once"}}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def workload_config(w, n_gpus, extra=None):
     cfg = {"workload": f"{w.name}: batch {w.B}, histories {w.n} tokens, vocab {w.V}, K {w.K}, {w.dtype} logits",
            "requests_per_gpu": w.B, "parallelism": f"requests sharded over {n_gpus} GPU(s), no collective"}
@@ -317,6 +389,9 @@ def main():
         return
     if args.freq:
         run_freq(args)
+        return
+    if args.corpus:
+        run_corpus(args)
         return
     if args.replay:
         run_replay(args)

@@ -23,7 +23,7 @@ import numpy as np
 
 BASE_SEED = 260601019 * 10**4
 # stream ids
-S_TEMPLATES, S_HIST, S_TAIL, S_STATE, S_WEIGHTS, S_MODEL, S_AGREE, S_LOGITS, S_PLANT, S_TREE = range(10)
+S_TEMPLATES, S_HIST, S_TAIL, S_STATE, S_WEIGHTS, S_MODEL, S_AGREE, S_LOGITS, S_PLANT, S_TREE, S_CORPUS = range(11)
 
 GUARD_WORDS = 64          # canary words either side of every history slab
 GUARD_VALUE = -1515870811  # 0xA5A5A5A5 as int32
@@ -264,6 +264,24 @@ def make_requests(w: Workload) -> Requests:
     for b in range(B):
         model_draft[b, :int(K_all[b])] = r_model.integers(0, w.V, int(K_all[b]))
     return pack_requests(hists, K_all, cap, prompt_len, state, model_draft, K_all.astype(np.int32))
+
+
+def make_corpus(w: Workload, n_traces: int = 16, trace_len: IntOrRange = (1024, 8192), rep: float = 0.6,
+                separator: int = -1) -> np.ndarray:
+    """Shared warm-up corpus: `n_traces` recorded traces drawn from the workload's own template family
+    (so that requests of the workload find some of their suffixes in it), joined by a negative
+    separator.  Stands in for the warm-up prompts of the paper's datasets."""
+    templates = make_templates(w)
+    tprobs = _template_probs(w)
+    rng = _rng(w.index, S_CORPUS)
+    parts = []
+    for t in range(n_traces):
+        n = int(_draw_int(rng, trace_len, log=True))
+        h, _ = _one_history(w, rng, templates, tprobs, n, rep)
+        if t:
+            parts.append(np.array([separator], np.int32))
+        parts.append(h)
+    return np.concatenate(parts).astype(np.int32) if parts else np.zeros(0, np.int32)
 
 
 def pack_requests(hists, K, cap, prompt_len, state, model_draft, model_len, hist_len=None,

@@ -173,6 +173,31 @@ HVD_API hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_
                                            int32_t* sel_draft, int32_t* sel_len, void* stream);
 
 /*
+ * Shared warm-up corpus (Algorithm 1: the suffix cache is initialised from cache-warmup traces and
+ * the prompt; App. C: warm-up prompts of the same dataset).  hvd_set_corpus registers one token
+ * array shared by all requests: corpus int32 [m], DEVICE, 16-byte aligned, owned by the caller and
+ * kept alive and unchanged while registered; a negative entry separates two traces (it is never
+ * part of a match and ends a draft); m (HOST value) in [0, 2^31 - 2]; corpus = NULL or m = 0
+ * unregisters.  Takes effect for later hvd_lookup_corpus calls on any stream.
+ *
+ * hvd_lookup_corpus is hvd_lookup over [corpus, own history].  Candidates are the history positions
+ * of hvd_lookup and the corpus positions e in [1, m-1] whose token corpus[e] is not a separator,
+ * with match length l <= min(l_max, e, n) and no separator inside the match.  The longest match
+ * wins; at equal length the history comes before the corpus, and within a source the latest
+ * position.  match_src int32 [B] (DEVICE output): 0 = history (or no match), 1 = corpus; match_pos
+ * is the position in that source; match_cnt counts both sources; a corpus draft is
+ * corpus[e .. e + d), d = min(K, floor(spec_factor * L + spec_offset), m - e), cut before the first
+ * separator.  Everything else as in hvd_lookup.  For the payoff features of a corpus match pass
+ * match_pos = 0 to hvd_score_select (the corpus is older than every history token).
+ * Uses context scratch: one call at a time per context.
+ */
+HVD_API hvd_status hvd_set_corpus(hvd_ctx* ctx, const int32_t* corpus, int64_t m);
+HVD_API hvd_status hvd_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                                     const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
+                                     int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
+                                     int32_t* match_pos, int32_t* match_src, int32_t* match_cnt, void* stream);
+
+/*
  * Frequency-weighted cache draft, suffix score and the score-threshold selection (Sec. 4.1
  * "Frequency-Based Hybrid Decoding": same cache-first structure, the decision taken on the
  * frequency-derived cache score; App. A drafting table: speculation limits and the minimum token

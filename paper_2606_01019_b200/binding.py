@@ -49,6 +49,8 @@ _SIGNATURES = {
     "hvd_set_predictor2": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _vp]),
     "hvd_lookup": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_score_select": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32] + [_vp] * 14 + [_vp]),
+    "hvd_set_corpus": (_i32, [_vp, _vp, _i64]),
+    "hvd_lookup_corpus": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_freq": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _f32, _i32, _f32] + [_vp] * 11 + [_vp]),
     "hvd_replay_labels": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
@@ -197,6 +199,20 @@ class Context:
             _ptr(prompt_len), _ptr(state), _ptr(model_draft), _ptr(model_len), _ptr(draft), _ptr(draft_len),
             _ptr(match_len), _ptr(match_pos), _ptr(match_cnt), _ptr(features), _ptr(score), _ptr(select),
             _ptr(sel_draft), _ptr(sel_len), _stream()), "hvd_lookup_score_select")
+
+    def hvd_set_corpus(self, corpus, m=None):
+        """Registers a device int32 tensor as the shared warm-up corpus (None unregisters); the context
+        keeps a reference so that the tensor stays alive while registered."""
+        self._corpus = corpus
+        n = 0 if corpus is None else (int(corpus.numel()) if m is None else int(m))
+        self._check(self._lib.hvd_set_corpus(self._h, _ptr(corpus), n), "hvd_set_corpus")
+
+    def hvd_lookup_corpus(self, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len, match_len,
+                          match_pos, match_src, match_cnt):
+        self._check(self._lib.hvd_lookup_corpus(self._h, B, _ptr(hist), _ptr(hist_off), _ptr(hist_cap),
+                                                _ptr(hist_len), _ptr(K), n_max, _ptr(draft), _ptr(draft_len),
+                                                _ptr(match_len), _ptr(match_pos), _ptr(match_src),
+                                                _ptr(match_cnt), _stream()), "hvd_lookup_corpus")
 
     def hvd_lookup_freq(self, B, hist, hist_off, hist_cap, hist_len, K, n_max, min_prob, max_occ, threshold,
                         model_draft, model_len, draft, draft_len, score, match_len, match_pos, match_cnt,

@@ -16,6 +16,7 @@ void release(hvd_ctx* c) {
     cudaFree(c->d_W1); cudaFree(c->d_b1); cudaFree(c->d_W2); cudaFree(c->d_WhT); cudaFree(c->d_bh);
     cudaFree(c->lk_partial); cudaFree(c->lk_cnt);
     cudaFree(c->fq_occ); cudaFree(c->fq_cnt);
+    cudaFree(c->cp_key); cudaFree(c->cp_cnt); cudaFree(c->cp_arrived);
     cudaFree(c->rp_off); cudaFree(c->rp_cap); cudaFree(c->rp_len); cudaFree(c->rp_K); cudaFree(c->rp_draft);
     cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
@@ -81,6 +82,9 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->lk_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->fq_occ, (size_t)cfg->max_batch * HVD_FREQ_MAX_OCC * sizeof(int32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->fq_cnt, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->cp_key, (size_t)cfg->max_batch * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->cp_cnt, (size_t)cfg->max_batch * (HVD_MAX_L + 1) * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->cp_arrived, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
     const size_t MB = (size_t)cfg->max_batch;
     ok = ok && alloc_zero(&c->rp_off, MB * sizeof(int64_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->rp_cap, MB * sizeof(int32_t)) == cudaSuccess;
@@ -189,6 +193,31 @@ hvd_status hvd_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_
         return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max outside [0, max_hist_len]");
     return launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
                          match_len, match_pos, match_cnt, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_set_corpus(hvd_ctx* ctx, const int32_t* corpus, int64_t m) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (corpus == nullptr || m == 0) { ctx->corpus = nullptr; ctx->corpus_len = 0; return HVD_OK; }
+    if (m < 0 || m > 2147483646LL) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_corpus: m outside [0, 2^31 - 2]");
+    if (!aligned(corpus, 16)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_corpus: corpus must be 16-byte aligned");
+    ctx->corpus = corpus; ctx->corpus_len = (int32_t)m;
+    return HVD_OK;
+}
+
+hvd_status hvd_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                             const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K, int32_t n_max,
+                             int32_t* draft, int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
+                             int32_t* match_src, int32_t* match_cnt, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_corpus: B outside [1, max_batch]");
+    if (!hist || !hist_off || !hist_cap || !hist_len || !K || !draft || !draft_len || !match_len || !match_pos ||
+        !match_src || !match_cnt)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_corpus: NULL pointer");
+    if (!aligned(hist, 16)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_corpus: hist must be 16-byte aligned");
+    if (n_max < 0 || n_max > ctx->cfg.max_hist_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup_corpus: n_max outside [0, max_hist_len]");
+    return launch_lookup_corpus(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len, match_len,
+                                match_pos, match_src, match_cnt, static_cast<cudaStream_t>(stream));
 }
 
 hvd_status hvd_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,

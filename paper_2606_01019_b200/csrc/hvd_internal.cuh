@@ -68,6 +68,12 @@ struct hvd_ctx {
     // occurrence lists of the frequency-weighted draft
     int32_t* fq_occ;    // [max_batch, HVD_FREQ_MAX_OCC]
     uint32_t* fq_cnt;   // [max_batch], zero at rest
+    // shared warm-up corpus (caller-owned) and the scratch its scan meets in, zero at rest
+    const int32_t* corpus;
+    int32_t corpus_len;
+    unsigned long long* cp_key;  // [max_batch]
+    uint32_t* cp_cnt;            // [max_batch, HVD_MAX_L + 1]
+    uint32_t* cp_arrived;        // [max_batch]
     // verify scratch
     unsigned long long* vf_row_key;  // [max_rows], zero at rest
     uint32_t* vf_next_unit;          // zero at rest
@@ -157,6 +163,11 @@ hvd_status launch_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist, cons
                               const int32_t* model_len, int32_t* draft, int32_t* draft_len, float* score,
                               int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, int32_t* select,
                               int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream);
+
+hvd_status launch_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
+                                const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K, int32_t n_max,
+                                int32_t* draft, int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
+                                int32_t* match_src, int32_t* match_cnt, cudaStream_t stream);
 
 struct VerifyArgs {
     int32_t B;
