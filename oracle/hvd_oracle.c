@@ -20,6 +20,8 @@
  *   - the exact formulas of the eight payoff features (the paper names only
  *     feature groups, App. B table "Payoff predictor feature groups"),
  *   - the layout of the recent-history summary h,
+ *   - the draft-structure features (shares of the draft's tokens per token
+ *     class; the paper lists the classes, not the formula),
  *   - how warm-up traces and the own history share the cache (history before
  *     corpus at equal match length; separators between traces),
  *   - the frequency-weighted continuation and its score (the paper names the
@@ -422,6 +424,30 @@ void oracle_features_one(int32_t n, int32_t prompt_len, oracle_req_state st, int
     phi[7] = (float)acc_sum / 8.0f;
 }
 
+/* Extended feature vector (App. B feature-group table, all four groups): the eight features above,
+   then the draft-structure group -- for each of five token classes (bit 0 whitespace, 1 punctuation,
+   2 line break, 3 bracket, 4 delimiter-like; one byte of class bits per vocabulary entry, supplied
+   by the caller from its tokenizer) the share of the cache draft's tokens that carry the class, one
+   IEEE division count / draft_len (0 for an empty draft; tokens outside [0, V) carry no class) --
+   and last the cache-match group's suffix score (the frequency score of oracle_lookup_freq; 0 when
+   the caller has none). */
+enum { ORACLE_N_FEATURES_EXT = 14, ORACLE_N_TOKEN_CLASSES = 5 };
+
+void oracle_features_ext_one(int32_t n, int32_t prompt_len, oracle_req_state st, int32_t draft_len,
+                             int32_t match_len, int32_t match_pos, int32_t match_cnt, const int32_t* draft,
+                             const uint8_t* cls, int32_t cls_V, float suffix_score, float* phi /*[14]*/) {
+    oracle_features_one(n, prompt_len, st, draft_len, match_len, match_pos, match_cnt, phi);
+    for (int k = 0; k < ORACLE_N_TOKEN_CLASSES; ++k) {
+        int32_t c = 0;
+        for (int32_t j = 0; j < draft_len; ++j) {
+            const int32_t t = draft[j];
+            if (t >= 0 && t < cls_V && ((cls[t] >> k) & 1u)) ++c;
+        }
+        phi[ORACLE_N_FEATURES + k] = draft_len > 0 ? (float)c / (float)draft_len : 0.0f;
+    }
+    phi[ORACLE_N_FEATURES + ORACLE_N_TOKEN_CLASSES] = suffix_score;
+}
+
 /* ------------------------------------------------------------------ */
 /* Step 3: payoff score y = g_theta(phi) and the rule y >= tau          */
 /* (Sec. 3.3 predictor; Sec. 3.4 selection equation; Algorithm 1).     */
@@ -497,11 +523,12 @@ typedef struct {
     const float *W1, *b1, *W2; float b2, tau;
     float *features, *score; double* score64; int32_t *select, *sel_draft, *sel_len;
     const float *Wh, *bh; /* second hidden layer, NULL for the one-layer predictor */
+    const uint8_t* cls; int32_t cls_V; const float* suffix; /* cls != NULL: the extended feature vector */
 } score_args;
 
 static void score_req(int32_t b, void* p) {
     score_args* a = (score_args*)p;
-    float phi[ORACLE_N_FEATURES];
+    float phi[ORACLE_N_FEATURES_EXT];
     int32_t kc = a->k_cap;
     int32_t K = a->K[b];
     if (K < 0) K = 0;
@@ -509,15 +536,23 @@ static void score_req(int32_t b, void* p) {
     int32_t d = a->draft_len[b];
     if (d < 0) d = 0;
     if (d > kc) d = kc;
-    oracle_features_one(a->hist_len[b], a->prompt_len[b], a->state[b], d, a->match_len[b],
-                        a->match_pos[b], a->match_cnt[b], phi);
-    if (a->features) memcpy(a->features + (int64_t)b * ORACLE_N_FEATURES, phi, sizeof(phi));
-    float y = a->Wh ? oracle_mlp2_f32(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->Wh, a->bh, a->W2, a->b2)
-                    : oracle_mlp_f32(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->W2, a->b2);
+    int32_t F = ORACLE_N_FEATURES;
+    if (a->cls) {
+        F = ORACLE_N_FEATURES_EXT;
+        oracle_features_ext_one(a->hist_len[b], a->prompt_len[b], a->state[b], d, a->match_len[b], a->match_pos[b],
+                                a->match_cnt[b], a->draft + (int64_t)b * kc, a->cls, a->cls_V,
+                                a->suffix ? a->suffix[b] : 0.0f, phi);
+    } else {
+        oracle_features_one(a->hist_len[b], a->prompt_len[b], a->state[b], d, a->match_len[b],
+                            a->match_pos[b], a->match_cnt[b], phi);
+    }
+    if (a->features) memcpy(a->features + (int64_t)b * F, phi, sizeof(float) * (size_t)F);
+    float y = a->Wh ? oracle_mlp2_f32(phi, F, a->H, a->W1, a->b1, a->Wh, a->bh, a->W2, a->b2)
+                    : oracle_mlp_f32(phi, F, a->H, a->W1, a->b1, a->W2, a->b2);
     a->score[b] = y;
     if (a->score64)
-        a->score64[b] = a->Wh ? oracle_mlp2_f64(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->Wh, a->bh, a->W2, a->b2)
-                              : oracle_mlp_f64(phi, ORACLE_N_FEATURES, a->H, a->W1, a->b1, a->W2, a->b2);
+        a->score64[b] = a->Wh ? oracle_mlp2_f64(phi, F, a->H, a->W1, a->b1, a->Wh, a->bh, a->W2, a->b2)
+                              : oracle_mlp_f64(phi, F, a->H, a->W1, a->b1, a->W2, a->b2);
     /* cache draft is verified iff it exists and its predicted payoff reaches the threshold */
     int32_t sel = (d > 0 && y >= a->tau) ? 1 : 0;
     a->select[b] = sel;
@@ -547,7 +582,7 @@ void oracle_score_select(int32_t B, const int32_t* hist_len, const int32_t* prom
                          int32_t* select, int32_t* sel_draft, int32_t* sel_len, int32_t nthreads) {
     score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
                     model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
-                    select, sel_draft, sel_len, NULL, NULL};
+                    select, sel_draft, sel_len, NULL, NULL, NULL, 0, NULL};
     for_each_request(B, nthreads, score_req, &a);
 }
 
@@ -561,7 +596,23 @@ void oracle_score_select2(int32_t B, const int32_t* hist_len, const int32_t* pro
                           int32_t nthreads) {
     score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
                     model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
-                    select, sel_draft, sel_len, Wh, bh};
+                    select, sel_draft, sel_len, Wh, bh, NULL, 0, NULL};
+    for_each_request(B, nthreads, score_req, &a);
+}
+
+/* The same step on the extended feature vector: W1 is [H, 14]; Wh / bh NULL for one hidden layer;
+   features [B, 14]; suffix (float [B]) may be NULL. */
+void oracle_score_select_ext(int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
+                             const oracle_req_state* state, const int32_t* K, const int32_t* draft,
+                             const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
+                             const int32_t* match_cnt, const float* suffix, const uint8_t* cls, int32_t cls_V,
+                             const int32_t* model_draft, const int32_t* model_len, int32_t k_cap, int32_t H,
+                             const float* W1, const float* b1, const float* Wh, const float* bh, const float* W2,
+                             float b2, float tau, float* features, float* score, double* score64,
+                             int32_t* select, int32_t* sel_draft, int32_t* sel_len, int32_t nthreads) {
+    score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
+                    model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
+                    select, sel_draft, sel_len, Wh, bh, cls, cls_V, suffix};
     for_each_request(B, nthreads, score_req, &a);
 }
 

@@ -198,6 +198,51 @@ def score_select(hist_len, prompt_len, state, K, lk: LookupOut, model_draft, mod
     return out
 
 
+N_FEATURES_EXT = 14
+N_TOKEN_CLASSES = 5
+
+
+def score_select_ext(hist_len, prompt_len, state, K, lk: LookupOut, suffix, cls, model_draft, model_len, *, k_cap,
+                     W1, b1, W2, b2, tau, nthreads=1, Wh=None, bh=None) -> ScoreOut:
+    """score_select on the extended feature vector: cls uint8 [V] token-class bits, suffix float [B] or None,
+    W1 [H, 14]."""
+    B = len(hist_len)
+    H = int(np.asarray(W2).shape[0])
+    W1 = np.ascontiguousarray(W1, np.float32); b1 = np.ascontiguousarray(b1, np.float32)
+    W2 = np.ascontiguousarray(W2, np.float32)
+    assert W1.shape == (H, N_FEATURES_EXT)
+    if Wh is not None:
+        Wh = np.ascontiguousarray(Wh, np.float32); bh = np.ascontiguousarray(bh, np.float32)
+        assert Wh.shape == (H, H) and bh.shape == (H,)
+    cls = np.ascontiguousarray(cls, np.uint8)
+    sfx = None if suffix is None else np.ascontiguousarray(suffix, np.float32)
+    state = np.ascontiguousarray(state, dtype=STATE_DTYPE)
+    hist_len = _i32(hist_len); prompt_len = _i32(prompt_len); K = _i32(K)
+    md = None if model_draft is None else _i32(model_draft)
+    ml = None if model_len is None else _i32(model_len)
+    out = ScoreOut(np.empty((B, N_FEATURES_EXT), np.float32), np.empty(B, np.float32), np.empty(B, np.float64),
+                   np.empty(B, np.int32), np.empty((B, k_cap), np.int32), np.empty(B, np.int32))
+    lib().oracle_score_select_ext(
+        C.c_int32(B), _p(hist_len), _p(prompt_len), _p(state), _p(K), _p(_i32(lk.draft)), _p(_i32(lk.draft_len)),
+        _p(_i32(lk.match_len)), _p(_i32(lk.match_pos)), _p(_i32(lk.match_cnt)), _p(sfx), _p(cls),
+        C.c_int32(len(cls)), _p(md), _p(ml), C.c_int32(k_cap), C.c_int32(H), _p(W1), _p(b1), _p(Wh), _p(bh), _p(W2),
+        C.c_float(b2), C.c_float(tau), _p(out.features), _p(out.score), _p(out.score64), _p(out.select),
+        _p(out.sel_draft), _p(out.sel_len), C.c_int32(nthreads))
+    return out
+
+
+def features_ext_one(n, prompt_len, sel_bits, acc_ring, draft, match_len, match_pos, match_cnt, cls, suffix_score=0.0):
+    class St(C.Structure):
+        _fields_ = [("sel_bits", C.c_uint32), ("pad", C.c_uint32), ("acc_ring", C.c_uint64)]
+    phi = np.empty(N_FEATURES_EXT, np.float32)
+    draft = _i32(draft); cls = np.ascontiguousarray(cls, np.uint8)
+    lib().oracle_features_ext_one(C.c_int32(n), C.c_int32(prompt_len), St(sel_bits, 0, acc_ring),
+                                  C.c_int32(len(draft)), C.c_int32(match_len), C.c_int32(match_pos),
+                                  C.c_int32(match_cnt), _p(draft), _p(cls), C.c_int32(len(cls)),
+                                  C.c_float(suffix_score), _p(phi))
+    return phi
+
+
 @dataclass
 class VerifyOut:
     accepted: np.ndarray
