@@ -74,6 +74,7 @@ typedef struct {
 } hvd_req_state;
 
 enum { HVD_N_FEATURES = 8, HVD_MAX_K = 64, HVD_MAX_L = 64, HVD_MAX_HIDDEN = 256 };
+enum { HVD_N_TOKEN_CLASSES = 5, HVD_N_FEATURES_EXT = 14 };
 
 typedef struct {
     int32_t max_batch;    /* largest B of any call, 1..8192 */
@@ -157,6 +158,34 @@ HVD_API hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist
                             const int32_t* model_draft, const int32_t* model_len, float* features,
                             float* score, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
                             void* stream);
+
+/*
+ * The same step on the extended feature vector (App. B feature-group table, all four groups):
+ * features 0..7 as in hvd_score_select; 8..12 the draft-structure group, for each of
+ * HVD_N_TOKEN_CLASSES token classes (bit 0 whitespace, 1 punctuation, 2 line break, 3 bracket,
+ * 4 delimiter-like) the share of the cache draft's tokens that carry the class, count / draft_len as
+ * one IEEE division (0 for an empty draft; tokens outside [0, V) carry no class); 13 the suffix
+ * score of the cache match (suffix_score float [B], DEVICE, e.g. hvd_lookup_freq's score; NULL: 0).
+ *
+ * hvd_set_token_classes registers the class bits: cls uint8 [V], DEVICE, owned by the caller and kept
+ * alive while registered (NULL or V = 0 unregisters).  hvd_set_predictor_ext stores a predictor that
+ * takes the 14 features: W1 [hidden, 14] row-major, b1 [hidden], optional second layer Wh [hidden,
+ * hidden] / bh [hidden] (both NULL: one hidden layer), W2 [hidden], HOST pointers, copied before the
+ * call returns; it replaces the predictor of hvd_set_predictor / hvd_set_predictor2 and vice versa
+ * (hvd_score_select then fails until its own predictor is set again).  Evaluation order as in
+ * hvd_score_select, over 14 inputs.  features float [B, 14] or NULL.  Everything else as in
+ * hvd_score_select.
+ */
+HVD_API hvd_status hvd_set_token_classes(hvd_ctx* ctx, const uint8_t* cls, int64_t V);
+HVD_API hvd_status hvd_set_predictor_ext(hvd_ctx* ctx, const float* W1, const float* b1, const float* Wh,
+                                         const float* bh, const float* W2, float b2, float tau, void* stream);
+HVD_API hvd_status hvd_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
+                                        const hvd_req_state* state, const int32_t* K, const int32_t* draft,
+                                        const int32_t* draft_len, const int32_t* match_len,
+                                        const int32_t* match_pos, const int32_t* match_cnt,
+                                        const float* suffix_score, const int32_t* model_draft,
+                                        const int32_t* model_len, float* features, float* score, int32_t* select,
+                                        int32_t* sel_draft, int32_t* sel_len, void* stream);
 
 /*
  * hvd_lookup and hvd_score_select in one launch (Alg. 1: draft, score and select are consecutive

@@ -49,6 +49,9 @@ _SIGNATURES = {
     "hvd_set_predictor2": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _vp]),
     "hvd_lookup": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_score_select": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32] + [_vp] * 14 + [_vp]),
+    "hvd_set_token_classes": (_i32, [_vp, _vp, _i64]),
+    "hvd_set_predictor_ext": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _vp]),
+    "hvd_score_select_ext": (_i32, [_vp, _i32] + [_vp] * 17 + [_vp]),
     "hvd_set_corpus": (_i32, [_vp, _vp, _i64]),
     "hvd_lookup_corpus": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_freq": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _f32, _i32, _f32] + [_vp] * 11 + [_vp]),
@@ -108,6 +111,7 @@ def _stream():
 
 NOALLOC_MAX_ROWS, NOALLOC_MAX_BATCH = 16384, 2048
 FREQ_MAX_OCC = 128   # HVD_FREQ_MAX_OCC
+N_FEATURES_EXT, N_TOKEN_CLASSES = 14, 5
 
 
 def hvd_verify_commit_noalloc(B, k_cap, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
@@ -183,6 +187,38 @@ class Context:
         self._check(self._lib.hvd_set_predictor2(self._h, W1.ctypes.data, b1.ctypes.data, Wh.ctypes.data,
                                                  bh.ctypes.data, W2.ctypes.data, float(b2), float(tau), _stream()),
                     "hvd_set_predictor2")
+
+    def hvd_set_token_classes(self, cls):
+        """Registers a device uint8 tensor of class bits per vocabulary entry (None unregisters); the
+        context keeps a reference so that the tensor stays alive while registered."""
+        self._cls = cls
+        self._check(self._lib.hvd_set_token_classes(self._h, _ptr(cls), 0 if cls is None else int(cls.numel())),
+                    "hvd_set_token_classes")
+
+    def hvd_set_predictor_ext(self, W1, b1, W2, b2, tau, Wh=None, bh=None):
+        H = self.hidden
+        W1 = np.ascontiguousarray(W1, np.float32); b1 = np.ascontiguousarray(b1, np.float32)
+        W2 = np.ascontiguousarray(W2, np.float32)
+        if W1.shape != (H, N_FEATURES_EXT) or b1.shape != (H,) or W2.shape != (H,):
+            raise HvdError("hvd_set_predictor_ext: weight shapes do not match the context")
+        if Wh is not None:
+            Wh = np.ascontiguousarray(Wh, np.float32); bh = np.ascontiguousarray(bh, np.float32)
+            if Wh.shape != (H, H) or bh.shape != (H,):
+                raise HvdError("hvd_set_predictor_ext: second-layer shapes do not match the context")
+        self._check(self._lib.hvd_set_predictor_ext(self._h, W1.ctypes.data, b1.ctypes.data,
+                                                    None if Wh is None else Wh.ctypes.data,
+                                                    None if Wh is None else bh.ctypes.data, W2.ctypes.data,
+                                                    float(b2), float(tau), _stream()), "hvd_set_predictor_ext")
+
+    def hvd_score_select_ext(self, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
+                             match_cnt, suffix_score, model_draft, model_len, features, score, select, sel_draft,
+                             sel_len):
+        self._check(self._lib.hvd_score_select_ext(self._h, B, _ptr(hist_len), _ptr(prompt_len), _ptr(state),
+                                                   _ptr(K), _ptr(draft), _ptr(draft_len), _ptr(match_len),
+                                                   _ptr(match_pos), _ptr(match_cnt), _ptr(suffix_score),
+                                                   _ptr(model_draft), _ptr(model_len), _ptr(features), _ptr(score),
+                                                   _ptr(select), _ptr(sel_draft), _ptr(sel_len), _stream()),
+                    "hvd_score_select_ext")
 
     def hvd_lookup(self, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len, match_len,
                    match_pos, match_cnt):

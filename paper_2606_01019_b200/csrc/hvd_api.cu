@@ -73,7 +73,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
 
     const size_t H = (size_t)cfg->hidden;
     bool ok = true;
-    ok = ok && alloc_zero(&c->d_W1, H * HVD_N_FEATURES * sizeof(float)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->d_W1, H * 16 * sizeof(float)) == cudaSuccess;  // row stride 8, or 16 for the extended vector
     ok = ok && alloc_zero(&c->d_b1, H * sizeof(float)) == cudaSuccess;
     ok = ok && alloc_zero(&c->d_W2, H * sizeof(float)) == cudaSuccess;
     ok = ok && alloc_zero(&c->d_WhT, (size_t)HVD_MAX_HIDDEN * HVD_MAX_HIDDEN * sizeof(float)) == cudaSuccess;  // row stride 256
@@ -102,6 +102,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->vf_blocks_per_sm[1] = verify_occupancy(HVD_BF16, smem);
     if (c->vf_blocks_per_sm[0] < 1 || c->vf_blocks_per_sm[1] < 1) { release(c); return HVD_ERR_UNSUPPORTED; }
     c->has_predictor = false;
+    c->has_predictor_ext = false;
     c->two_layer = false;
     c->score2_ready = false;
     c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // measured: no gain on this path, off unless asked for
@@ -152,7 +153,25 @@ hvd_status hvd_set_predictor(hvd_ctx* ctx, const float* W1, const float* b1, con
     ctx->b2 = b2;
     ctx->tau = tau;
     ctx->has_predictor = true;
+    ctx->has_predictor_ext = false;
     ctx->two_layer = false;
+    return HVD_OK;
+}
+
+// second hidden layer: transposed copy with a fixed row stride (coalesced, 16-byte aligned rows on the device)
+static hvd_status store_second_layer(hvd_ctx* ctx, const float* Wh, const float* bh, cudaStream_t st, const char* who) {
+    const size_t H = (size_t)ctx->cfg.hidden;
+    const size_t S = HVD_MAX_HIDDEN;
+    float* t = static_cast<float*>(calloc(S * S, sizeof(float)));
+    if (!t) return fail(ctx, HVD_ERR_ALLOC, "out of host memory");
+    for (size_t j = 0; j < H; ++j)
+        for (size_t i = 0; i < H; ++i) t[i * S + j] = Wh[j * H + i];
+    cudaError_t e = cudaMemcpyAsync(ctx->d_WhT, t, S * S * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_bh, bh, H * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    free(t);
+    if (e != cudaSuccess) { ctx->has_predictor = false; ctx->has_predictor_ext = false; return cuda_fail(ctx, e, who); }
+    ctx->two_layer = true;
     return HVD_OK;
 }
 
@@ -162,20 +181,41 @@ hvd_status hvd_set_predictor2(hvd_ctx* ctx, const float* W1, const float* b1, co
     if (!Wh || !bh) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_predictor2: NULL weights");
     const hvd_status r = hvd_set_predictor(ctx, W1, b1, W2, b2, tau, stream);
     if (r != HVD_OK) return r;
-    const size_t H = (size_t)ctx->cfg.hidden;
-    // transposed copy with a fixed row stride (coalesced, 16-byte aligned rows on the device)
-    const size_t S = HVD_MAX_HIDDEN;
-    float* t = static_cast<float*>(calloc(S * S, sizeof(float)));
-    if (!t) return fail(ctx, HVD_ERR_ALLOC, "hvd_set_predictor2: out of host memory");
-    for (size_t j = 0; j < H; ++j)
-        for (size_t i = 0; i < H; ++i) t[i * S + j] = Wh[j * H + i];
+    return store_second_layer(ctx, Wh, bh, static_cast<cudaStream_t>(stream), "hvd_set_predictor2");
+}
+
+hvd_status hvd_set_token_classes(hvd_ctx* ctx, const uint8_t* cls, int64_t V) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (cls == nullptr || V == 0) { ctx->cls = nullptr; ctx->cls_V = 0; return HVD_OK; }
+    if (V < 0 || V > 0x7fffffffLL) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_token_classes: V outside [0, 2^31 - 1]");
+    ctx->cls = cls; ctx->cls_V = (int32_t)V;
+    return HVD_OK;
+}
+
+hvd_status hvd_set_predictor_ext(hvd_ctx* ctx, const float* W1, const float* b1, const float* Wh, const float* bh,
+                                 const float* W2, float b2, float tau, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (!W1 || !b1 || !W2) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_predictor_ext: NULL weights");
+    if ((Wh == nullptr) != (bh == nullptr)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_predictor_ext: Wh and bh go together");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemcpyAsync(ctx->d_WhT, t, S * S * sizeof(float), cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_bh, bh, H * sizeof(float), cudaMemcpyHostToDevice, st);
+    const size_t H = (size_t)ctx->cfg.hidden;
+    float* t = static_cast<float*>(calloc(H * 16, sizeof(float)));  // rows padded to 16 floats
+    if (!t) return fail(ctx, HVD_ERR_ALLOC, "hvd_set_predictor_ext: out of host memory");
+    for (size_t j = 0; j < H; ++j)
+        for (size_t i = 0; i < HVD_N_FEATURES_EXT; ++i) t[j * 16 + i] = W1[j * HVD_N_FEATURES_EXT + i];
+    cudaError_t e = cudaMemcpyAsync(ctx->d_W1, t, H * 16 * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_b1, b1, H * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_W2, W2, H * sizeof(float), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     free(t);
-    if (e != cudaSuccess) { ctx->has_predictor = false; return cuda_fail(ctx, e, "hvd_set_predictor2"); }
-    ctx->two_layer = true;
+    ctx->has_predictor = false;
+    ctx->has_predictor_ext = false;
+    ctx->two_layer = false;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "hvd_set_predictor_ext");
+    ctx->b2 = b2;
+    ctx->tau = tau;
+    ctx->has_predictor_ext = true;
+    if (Wh) return store_second_layer(ctx, Wh, bh, st, "hvd_set_predictor_ext");
     return HVD_OK;
 }
 
@@ -314,6 +354,27 @@ hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
     return launch_score_select(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len,
                                match_pos, match_cnt, model_draft, model_len, features, score, select,
                                sel_draft, sel_len, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
+                                const hvd_req_state* state, const int32_t* K, const int32_t* draft,
+                                const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
+                                const int32_t* match_cnt, const float* suffix_score, const int32_t* model_draft,
+                                const int32_t* model_len, float* features, float* score, int32_t* select,
+                                int32_t* sel_draft, int32_t* sel_len, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: B outside [1, max_batch]");
+    if (!ctx->has_predictor_ext) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: call hvd_set_predictor_ext first");
+    if (!ctx->cls) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: call hvd_set_token_classes first");
+    if (!hist_len || !prompt_len || !state || !K || !draft || !draft_len || !match_len || !match_pos ||
+        !match_cnt || !score || !select || !sel_draft || !sel_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: NULL pointer");
+    if ((model_draft == nullptr) != (model_len == nullptr))
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: model_draft and model_len go together");
+    if (!aligned(state, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: state must be 8-byte aligned");
+    return launch_score_select_ext(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
+                                   match_cnt, suffix_score, model_draft, model_len, features, score, select, sel_draft,
+                                   sel_len, static_cast<cudaStream_t>(stream));
 }
 
 static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,

@@ -58,9 +58,13 @@ struct hvd_ctx {
     float* d_WhT;  // second hidden layer, transposed [hidden, hidden]
     float* d_bh;
     float b2, tau;
-    bool has_predictor;
+    bool has_predictor;      // a predictor on the 8 base features is stored
+    bool has_predictor_ext;  // a predictor on the extended feature vector is stored (same buffers)
     bool two_layer;
     bool score2_ready;  // the two-layer kernel's shared-memory size has been opted in on this device
+    bool score2x_ready; // the same for its extended-feature instance
+    const uint8_t* cls; // token-class bits per vocabulary entry (caller-owned), NULL = none
+    int32_t cls_V;
     // lookup scratch
     hvd::LookupPartial* lk_partial;  // [max_batch, lk_max_chunks]
     uint32_t* lk_cnt;                // [max_batch], zero at rest
@@ -153,6 +157,13 @@ hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
                                const int32_t* model_draft, const int32_t* model_len, float* features,
                                float* score, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
                                cudaStream_t stream);
+
+hvd_status launch_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
+                                   const hvd_req_state* state, const int32_t* K, const int32_t* draft,
+                                   const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
+                                   const int32_t* match_cnt, const float* suffix, const int32_t* model_draft,
+                                   const int32_t* model_len, float* features, float* score, int32_t* select,
+                                   int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream);
 
 hvd_status launch_replay(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label, int32_t* draft_len,
                          int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream);

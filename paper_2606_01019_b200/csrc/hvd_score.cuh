@@ -31,14 +31,23 @@ struct ScoreArgs {
     int32_t hidden, k_cap;
     const float* WhT;  // second hidden layer, transposed: WhT[i][j] = Wh[j][i]; NULL = one layer
     const float* bh;
+    // extended feature vector only: token-class bits per vocabulary entry, optional suffix scores
+    const uint8_t* cls;
+    int32_t cls_V;
+    const float* suffix;
 };
+
+constexpr int kW1StrideExt = 16;  // row stride of the first layer's weights for the extended vector
+template <bool EXT>
+struct NFeat { static constexpr int value = EXT ? HVD_N_FEATURES_EXT : HVD_N_FEATURES; };
 
 __device__ __forceinline__ int bit_width(uint32_t x) { return 32 - __clz((int)x); }
 
 // phi[8] of one request from its lookup results and decode state (every operation is an exact
 // integer->float conversion or one correctly rounded IEEE operation).
+template <int N>
 __device__ __forceinline__ void payoff_features(const ScoreArgs& a, int b, int n, int d, int L, int pos, int cnt,
-                                                float (&phi)[HVD_N_FEATURES]) {
+                                                float (&phi)[N]) {
     n = max(n, 0);
     // read-only inputs go through the non-coherent path so that the compiler may issue them early
     const int P = max(__ldg(a.prompt_len + b), 0);
@@ -62,14 +71,36 @@ __device__ __forceinline__ void payoff_features(const ScoreArgs& a, int b, int n
 }
 
 // hidden unit j of the first layer: relu(b1[j] + sum_i W1[j][i] phi[i]), left to right
-__device__ __forceinline__ float first_layer_unit(const ScoreArgs& a, int j, const float (&phi)[HVD_N_FEATURES]) {
+template <int N>
+__device__ __forceinline__ float first_layer_unit(const ScoreArgs& a, int j, const float (&phi)[N]) {
     float acc = __ldg(a.b1 + j);
-    const float4* w4 = reinterpret_cast<const float4*>(a.W1 + (int64_t)j * HVD_N_FEATURES);  // 32-byte rows
-    const float4 wa = __ldg(w4), wb = __ldg(w4 + 1);
-    const float w[HVD_N_FEATURES] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+    constexpr int STRIDE = (N == HVD_N_FEATURES) ? HVD_N_FEATURES : kW1StrideExt;  // 32- or 64-byte rows
+    const float4* w4 = reinterpret_cast<const float4*>(a.W1 + (int64_t)j * STRIDE);
+    float w[STRIDE];
 #pragma unroll
-    for (int i = 0; i < HVD_N_FEATURES; ++i) acc = __fmaf_rn(w[i], phi[i], acc);
+    for (int q = 0; q < STRIDE / 4; ++q) {
+        const float4 v = __ldg(w4 + q);
+        w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) acc = __fmaf_rn(w[i], phi[i], acc);
     return acc > 0.0f ? acc : 0.0f;
+}
+
+// Draft-structure group and suffix score of the extended vector (App. B feature groups), by one
+// converged warp: the share of the draft's tokens in each of five token classes (one IEEE division
+// count / d), then the caller's suffix score.  tok0 / tok1: draft tokens lane and lane + 32.
+__device__ __forceinline__ void structure_features(const ScoreArgs& a, int b, int lane, int d, int tok0, int tok1,
+                                                   float (&phi)[HVD_N_FEATURES_EXT]) {
+    uint32_t c0 = 0, c1 = 0;
+    if (lane < d && tok0 >= 0 && tok0 < a.cls_V) c0 = __ldg(a.cls + tok0);
+    if (lane + 32 < d && tok1 >= 0 && tok1 < a.cls_V) c1 = __ldg(a.cls + tok1);
+#pragma unroll
+    for (int k = 0; k < HVD_N_TOKEN_CLASSES; ++k) {
+        const int cnt = __popc(__ballot_sync(0xffffffffu, (c0 >> k) & 1u)) + __popc(__ballot_sync(0xffffffffu, (c1 >> k) & 1u));
+        phi[HVD_N_FEATURES + k] = d > 0 ? __fdiv_rn((float)cnt, (float)d) : 0.0f;
+    }
+    phi[HVD_N_FEATURES + HVD_N_TOKEN_CLASSES] = a.suffix ? __ldg(a.suffix + b) : 0.0f;
 }
 
 // Selection rule and the selected draft, by one warp.  tok0 / tok1: cache draft tokens lane and
@@ -103,16 +134,19 @@ __device__ __forceinline__ void select_draft(const ScoreArgs& a, int b, int lane
 // j+32, ...) with a left-to-right chain of fused multiply-adds, lane 0 then accumulates the output
 // layer in unit order, so the fp32 result does not depend on the launch shape.  d, L, pos, cnt: the
 // lookup results of the request; s_hid: shared memory, a.hidden floats, private to the warp.
+template <bool EXT = false>
 __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, int lane, float* s_hid, int n,
                                                      int d, int L, int pos, int cnt, int tok0, int tok1) {
+    constexpr int N = NFeat<EXT>::value;
     d = max(0, min(d, a.k_cap));
-    float phi[HVD_N_FEATURES];
+    float phi[N];
     payoff_features(a, b, n, d, L, pos, cnt, phi);
-    if (a.features && lane < HVD_N_FEATURES) {
+    if constexpr (EXT) structure_features(a, b, lane, d, tok0, tok1, phi);
+    if (a.features && lane < N) {
         float v = phi[0];
 #pragma unroll
-        for (int i = 1; i < HVD_N_FEATURES; ++i) v = (lane == i) ? phi[i] : v;
-        a.features[(int64_t)b * HVD_N_FEATURES + lane] = v;
+        for (int i = 1; i < N; ++i) v = (lane == i) ? phi[i] : v;
+        a.features[(int64_t)b * N + lane] = v;
     }
     for (int j = lane; j < a.hidden; j += 32) s_hid[j] = first_layer_unit(a, j, phi);
     __syncwarp();

@@ -8,6 +8,7 @@ namespace {
 
 constexpr int kWarpsPerBlock = 4;
 
+template <bool EXT>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) score_select_kernel(const ScoreArgs a) {
     __shared__ float s_hid[kWarpsPerBlock][HVD_MAX_HIDDEN];
     const int lane = threadIdx.x & 31;
@@ -21,8 +22,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) score_select_kernel(const
     const int32_t* src = a.draft + (int64_t)b * kc;
     const int tok0 = lane < d ? src[lane] : -1;
     const int tok1 = lane + 32 < d ? src[lane + 32] : -1;
-    score_select_request(a, b, lane, s_hid[warp], a.hist_len[b], d, a.match_len[b], a.match_pos[b],
-                         a.match_cnt[b], tok0, tok1);
+    score_select_request<EXT>(a, b, lane, s_hid[warp], a.hist_len[b], d, a.match_len[b], a.match_pos[b],
+                              a.match_cnt[b], tok0, tok1);
 }
 
 // Two hidden layers (the paper's predictor shape, 2 x 256).  One CTA scores kReqPerCta (4) requests:
@@ -52,9 +53,11 @@ __device__ __forceinline__ void copy_tile_async(float* dst, const float* src, in
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
+template <bool EXT>
 __global__ void __launch_bounds__(kScore2Threads) score_select2_kernel(const ScoreArgs a) {
+    constexpr int N = NFeat<EXT>::value;
     extern __shared__ __align__(16) float s_tiles[];  // [2][kTileRows][HVD_MAX_HIDDEN]
-    __shared__ float s_phi[kReqPerCta][HVD_N_FEATURES];
+    __shared__ float s_phi[kReqPerCta][N];
     __shared__ __align__(16) float s_h1[HVD_MAX_HIDDEN][kReqPerCta];  // [input unit][request]
     __shared__ float s_h2[kReqPerCta][kHidPad];
     __shared__ float s_w2[HVD_MAX_HIDDEN];
@@ -78,14 +81,18 @@ __global__ void __launch_bounds__(kScore2Threads) score_select2_kernel(const Sco
     if (warp < nreq) {
         const int b = b0 + warp;
         const int d = max(0, min(a.draft_len[b], kc));
-        float phi[HVD_N_FEATURES];
+        float phi[N];
         payoff_features(a, b, a.hist_len[b], d, a.match_len[b], a.match_pos[b], a.match_cnt[b], phi);
-        if (lane < HVD_N_FEATURES) {
+        if constexpr (EXT) {
+            const int32_t* src = a.draft + (int64_t)b * kc;
+            structure_features(a, b, lane, d, lane < d ? src[lane] : -1, lane + 32 < d ? src[lane + 32] : -1, phi);
+        }
+        if (lane < N) {
             float v = phi[0];
 #pragma unroll
-            for (int i = 1; i < HVD_N_FEATURES; ++i) v = (lane == i) ? phi[i] : v;
+            for (int i = 1; i < N; ++i) v = (lane == i) ? phi[i] : v;
             s_phi[warp][lane] = v;
-            if (a.features) a.features[(int64_t)b * HVD_N_FEATURES + lane] = v;
+            if (a.features) a.features[(int64_t)b * N + lane] = v;
         }
         if (lane == 0) s_d[warp] = d;
     }
@@ -99,9 +106,9 @@ __global__ void __launch_bounds__(kScore2Threads) score_select2_kernel(const Sco
             acc[r] = bias;
             h1[r] = 0.0f;
             if (r < nreq) {
-                float phi[HVD_N_FEATURES];
+                float phi[N];
 #pragma unroll
-                for (int i = 0; i < HVD_N_FEATURES; ++i) phi[i] = s_phi[r][i];
+                for (int i = 0; i < N; ++i) phi[i] = s_phi[r][i];
                 h1[r] = first_layer_unit(a, tid, phi);
             }
         }
@@ -166,7 +173,26 @@ ScoreArgs make_score_args(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, cons
     a.W1 = ctx->d_W1; a.b1 = ctx->d_b1; a.W2 = ctx->d_W2; a.b2 = ctx->b2; a.tau = ctx->tau;
     a.hidden = ctx->cfg.hidden; a.k_cap = ctx->cfg.k_cap;
     a.WhT = ctx->two_layer ? ctx->d_WhT : nullptr; a.bh = ctx->d_bh;
+    a.cls = nullptr; a.cls_V = 0; a.suffix = nullptr;
     return a;
+}
+
+template <bool EXT>
+static hvd_status launch_score_kernels(hvd_ctx* ctx, const ScoreArgs& a, int32_t B, cudaStream_t stream) {
+    if (a.WhT) {
+        bool& ready = EXT ? ctx->score2x_ready : ctx->score2_ready;
+        if (!ready) {  // per device: the kernel needs the opt-in shared memory size
+            HVD_CUDA_TRY(ctx, cudaFuncSetAttribute(score_select2_kernel<EXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)kScore2Smem));
+            ready = true;
+        }
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select2_kernel<EXT>, (B + kReqPerCta - 1) / kReqPerCta,
+                                        kScore2Threads, kScore2Smem, stream, a));
+        return HVD_OK;
+    }
+    const int blocks = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select_kernel<EXT>, blocks, kWarpsPerBlock * 32, 0, stream, a));
+    return HVD_OK;
 }
 
 hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
@@ -179,19 +205,19 @@ hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
     const ScoreArgs a = make_score_args(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len,
                                         match_pos, match_cnt, model_draft, model_len, features, score, select,
                                         sel_draft, sel_len);
-    if (a.WhT) {
-        if (!ctx->score2_ready) {  // per device: the kernel needs the opt-in shared memory size
-            HVD_CUDA_TRY(ctx, cudaFuncSetAttribute(score_select2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)kScore2Smem));
-            ctx->score2_ready = true;
-        }
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select2_kernel, (B + kReqPerCta - 1) / kReqPerCta,
-                                        kScore2Threads, kScore2Smem, stream, a));
-        return HVD_OK;
-    }
-    const int blocks = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select_kernel, blocks, kWarpsPerBlock * 32, 0, stream, a));
-    return HVD_OK;
+    return launch_score_kernels<false>(ctx, a, B, stream);
+}
+
+hvd_status launch_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
+                                   const hvd_req_state* state, const int32_t* K, const int32_t* draft,
+                                   const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
+                                   const int32_t* match_cnt, const float* suffix, const int32_t* model_draft,
+                                   const int32_t* model_len, float* features, float* score, int32_t* select,
+                                   int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream) {
+    ScoreArgs a = make_score_args(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
+                                  match_cnt, model_draft, model_len, features, score, select, sel_draft, sel_len);
+    a.cls = ctx->cls; a.cls_V = ctx->cls_V; a.suffix = suffix;
+    return launch_score_kernels<true>(ctx, a, B, stream);
 }
 
 }  // namespace hvd
