@@ -166,6 +166,8 @@ HVD_API hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist
  * 4 delimiter-like) the share of the cache draft's tokens that carry the class, count / draft_len as
  * one IEEE division (0 for an empty draft; tokens outside [0, V) carry no class); 13 the suffix
  * score of the cache match (suffix_score float [B], DEVICE, e.g. hvd_lookup_freq's score; NULL: 0).
+ * match_src (int32 [B], DEVICE, hvd_lookup_corpus's output; may be NULL): where it is 1 the match lies
+ * in the shared corpus and feature 3 (recency) is taken at position 0, i.e. older than the history.
  *
  * hvd_set_token_classes registers the class bits: cls uint8 [V], DEVICE, owned by the caller and kept
  * alive while registered (NULL or V = 0 unregisters).  hvd_set_predictor_ext stores a predictor that
@@ -183,9 +185,10 @@ HVD_API hvd_status hvd_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* 
                                         const hvd_req_state* state, const int32_t* K, const int32_t* draft,
                                         const int32_t* draft_len, const int32_t* match_len,
                                         const int32_t* match_pos, const int32_t* match_cnt,
-                                        const float* suffix_score, const int32_t* model_draft,
-                                        const int32_t* model_len, float* features, float* score, int32_t* select,
-                                        int32_t* sel_draft, int32_t* sel_len, void* stream);
+                                        const int32_t* match_src, const float* suffix_score,
+                                        const int32_t* model_draft, const int32_t* model_len, float* features,
+                                        float* score, int32_t* select, int32_t* sel_draft, int32_t* sel_len,
+                                        void* stream);
 
 /*
  * hvd_lookup and hvd_score_select in one launch (Alg. 1: draft, score and select are consecutive
@@ -216,8 +219,8 @@ HVD_API hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_
  * position.  match_src int32 [B] (DEVICE output): 0 = history (or no match), 1 = corpus; match_pos
  * is the position in that source; match_cnt counts both sources; a corpus draft is
  * corpus[e .. e + d), d = min(K, floor(spec_factor * L + spec_offset), m - e), cut before the first
- * separator.  Everything else as in hvd_lookup.  For the payoff features of a corpus match pass
- * match_pos = 0 to hvd_score_select (the corpus is older than every history token).
+ * separator.  Everything else as in hvd_lookup.  hvd_score_select_ext takes match_src for the payoff
+ * features of corpus matches.
  * Uses context scratch: one call at a time per context.
  */
 HVD_API hvd_status hvd_set_corpus(hvd_ctx* ctx, const int32_t* corpus, int64_t m);

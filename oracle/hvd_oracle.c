@@ -524,6 +524,7 @@ typedef struct {
     float *features, *score; double* score64; int32_t *select, *sel_draft, *sel_len;
     const float *Wh, *bh; /* second hidden layer, NULL for the one-layer predictor */
     const uint8_t* cls; int32_t cls_V; const float* suffix; /* cls != NULL: the extended feature vector */
+    const int32_t* match_src; /* extended only, may be NULL: 1 = the match lies in the shared corpus */
 } score_args;
 
 static void score_req(int32_t b, void* p) {
@@ -539,7 +540,9 @@ static void score_req(int32_t b, void* p) {
     int32_t F = ORACLE_N_FEATURES;
     if (a->cls) {
         F = ORACLE_N_FEATURES_EXT;
-        oracle_features_ext_one(a->hist_len[b], a->prompt_len[b], a->state[b], d, a->match_len[b], a->match_pos[b],
+        /* a match in the shared corpus is older than every history token: position 0 for the recency feature */
+        const int32_t pos = (a->match_src && a->match_src[b] == 1) ? 0 : a->match_pos[b];
+        oracle_features_ext_one(a->hist_len[b], a->prompt_len[b], a->state[b], d, a->match_len[b], pos,
                                 a->match_cnt[b], a->draft + (int64_t)b * kc, a->cls, a->cls_V,
                                 a->suffix ? a->suffix[b] : 0.0f, phi);
     } else {
@@ -582,7 +585,7 @@ void oracle_score_select(int32_t B, const int32_t* hist_len, const int32_t* prom
                          int32_t* select, int32_t* sel_draft, int32_t* sel_len, int32_t nthreads) {
     score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
                     model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
-                    select, sel_draft, sel_len, NULL, NULL, NULL, 0, NULL};
+                    select, sel_draft, sel_len, NULL, NULL, NULL, 0, NULL, NULL};
     for_each_request(B, nthreads, score_req, &a);
 }
 
@@ -596,23 +599,23 @@ void oracle_score_select2(int32_t B, const int32_t* hist_len, const int32_t* pro
                           int32_t nthreads) {
     score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
                     model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
-                    select, sel_draft, sel_len, Wh, bh, NULL, 0, NULL};
+                    select, sel_draft, sel_len, Wh, bh, NULL, 0, NULL, NULL};
     for_each_request(B, nthreads, score_req, &a);
 }
 
 /* The same step on the extended feature vector: W1 is [H, 14]; Wh / bh NULL for one hidden layer;
-   features [B, 14]; suffix (float [B]) may be NULL. */
+   features [B, 14]; suffix (float [B]) and match_src (int32 [B], from oracle_lookup_corpus) may be NULL. */
 void oracle_score_select_ext(int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
                              const oracle_req_state* state, const int32_t* K, const int32_t* draft,
                              const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
-                             const int32_t* match_cnt, const float* suffix, const uint8_t* cls, int32_t cls_V,
-                             const int32_t* model_draft, const int32_t* model_len, int32_t k_cap, int32_t H,
+                             const int32_t* match_cnt, const int32_t* match_src, const float* suffix,
+                             const uint8_t* cls, int32_t cls_V, const int32_t* model_draft, const int32_t* model_len, int32_t k_cap, int32_t H,
                              const float* W1, const float* b1, const float* Wh, const float* bh, const float* W2,
                              float b2, float tau, float* features, float* score, double* score64,
                              int32_t* select, int32_t* sel_draft, int32_t* sel_len, int32_t nthreads) {
     score_args a = {hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos, match_cnt,
                     model_draft, model_len, k_cap, H, W1, b1, W2, b2, tau, features, score, score64,
-                    select, sel_draft, sel_len, Wh, bh, cls, cls_V, suffix};
+                    select, sel_draft, sel_len, Wh, bh, cls, cls_V, suffix, match_src};
     for_each_request(B, nthreads, score_req, &a);
 }
 

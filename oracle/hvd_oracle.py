@@ -203,7 +203,7 @@ N_TOKEN_CLASSES = 5
 
 
 def score_select_ext(hist_len, prompt_len, state, K, lk: LookupOut, suffix, cls, model_draft, model_len, *, k_cap,
-                     W1, b1, W2, b2, tau, nthreads=1, Wh=None, bh=None) -> ScoreOut:
+                     W1, b1, W2, b2, tau, nthreads=1, Wh=None, bh=None, match_src=None) -> ScoreOut:
     """score_select on the extended feature vector: cls uint8 [V] token-class bits, suffix float [B] or None,
     W1 [H, 14]."""
     B = len(hist_len)
@@ -224,7 +224,8 @@ def score_select_ext(hist_len, prompt_len, state, K, lk: LookupOut, suffix, cls,
                    np.empty(B, np.int32), np.empty((B, k_cap), np.int32), np.empty(B, np.int32))
     lib().oracle_score_select_ext(
         C.c_int32(B), _p(hist_len), _p(prompt_len), _p(state), _p(K), _p(_i32(lk.draft)), _p(_i32(lk.draft_len)),
-        _p(_i32(lk.match_len)), _p(_i32(lk.match_pos)), _p(_i32(lk.match_cnt)), _p(sfx), _p(cls),
+        _p(_i32(lk.match_len)), _p(_i32(lk.match_pos)), _p(_i32(lk.match_cnt)),
+        None if match_src is None else _p(_i32(match_src)), _p(sfx), _p(cls),
         C.c_int32(len(cls)), _p(md), _p(ml), C.c_int32(k_cap), C.c_int32(H), _p(W1), _p(b1), _p(Wh), _p(bh), _p(W2),
         C.c_float(b2), C.c_float(tau), _p(out.features), _p(out.score), _p(out.score64), _p(out.select),
         _p(out.sel_draft), _p(out.sel_len), C.c_int32(nthreads))

@@ -51,7 +51,7 @@ _SIGNATURES = {
     "hvd_lookup_score_select": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32] + [_vp] * 14 + [_vp]),
     "hvd_set_token_classes": (_i32, [_vp, _vp, _i64]),
     "hvd_set_predictor_ext": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _vp]),
-    "hvd_score_select_ext": (_i32, [_vp, _i32] + [_vp] * 17 + [_vp]),
+    "hvd_score_select_ext": (_i32, [_vp, _i32] + [_vp] * 18 + [_vp]),
     "hvd_set_corpus": (_i32, [_vp, _vp, _i64]),
     "hvd_lookup_corpus": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_freq": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _f32, _i32, _f32] + [_vp] * 11 + [_vp]),
@@ -212,10 +212,10 @@ class Context:
 
     def hvd_score_select_ext(self, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
                              match_cnt, suffix_score, model_draft, model_len, features, score, select, sel_draft,
-                             sel_len):
+                             sel_len, match_src=None):
         self._check(self._lib.hvd_score_select_ext(self._h, B, _ptr(hist_len), _ptr(prompt_len), _ptr(state),
                                                    _ptr(K), _ptr(draft), _ptr(draft_len), _ptr(match_len),
-                                                   _ptr(match_pos), _ptr(match_cnt), _ptr(suffix_score),
+                                                   _ptr(match_pos), _ptr(match_cnt), _ptr(match_src), _ptr(suffix_score),
                                                    _ptr(model_draft), _ptr(model_len), _ptr(features), _ptr(score),
                                                    _ptr(select), _ptr(sel_draft), _ptr(sel_len), _stream()),
                     "hvd_score_select_ext")

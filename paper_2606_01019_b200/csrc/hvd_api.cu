@@ -359,9 +359,9 @@ hvd_status hvd_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
 hvd_status hvd_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
                                 const hvd_req_state* state, const int32_t* K, const int32_t* draft,
                                 const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
-                                const int32_t* match_cnt, const float* suffix_score, const int32_t* model_draft,
-                                const int32_t* model_len, float* features, float* score, int32_t* select,
-                                int32_t* sel_draft, int32_t* sel_len, void* stream) {
+                                const int32_t* match_cnt, const int32_t* match_src, const float* suffix_score,
+                                const int32_t* model_draft, const int32_t* model_len, float* features, float* score,
+                                int32_t* select, int32_t* sel_draft, int32_t* sel_len, void* stream) {
     if (!ctx) return HVD_ERR_INVALID_ARG;
     if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: B outside [1, max_batch]");
     if (!ctx->has_predictor_ext) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: call hvd_set_predictor_ext first");
@@ -373,8 +373,8 @@ hvd_status hvd_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_len
         return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: model_draft and model_len go together");
     if (!aligned(state, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_score_select_ext: state must be 8-byte aligned");
     return launch_score_select_ext(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
-                                   match_cnt, suffix_score, model_draft, model_len, features, score, select, sel_draft,
-                                   sel_len, static_cast<cudaStream_t>(stream));
+                                   match_cnt, match_src, suffix_score, model_draft, model_len, features, score, select,
+                                   sel_draft, sel_len, static_cast<cudaStream_t>(stream));
 }
 
 static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,

@@ -161,9 +161,9 @@ hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
 hvd_status launch_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
                                    const hvd_req_state* state, const int32_t* K, const int32_t* draft,
                                    const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
-                                   const int32_t* match_cnt, const float* suffix, const int32_t* model_draft,
-                                   const int32_t* model_len, float* features, float* score, int32_t* select,
-                                   int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream);
+                                   const int32_t* match_cnt, const int32_t* match_src, const float* suffix,
+                                   const int32_t* model_draft, const int32_t* model_len, float* features, float* score,
+                                   int32_t* select, int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream);
 
 hvd_status launch_replay(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label, int32_t* draft_len,
                          int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream);

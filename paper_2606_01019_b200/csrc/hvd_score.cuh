@@ -35,6 +35,7 @@ struct ScoreArgs {
     const uint8_t* cls;
     int32_t cls_V;
     const float* suffix;
+    const int32_t* match_src;  // may be NULL; 1 = the match lies in the shared corpus (recency position 0)
 };
 
 constexpr int kW1StrideExt = 16;  // row stride of the first layer's weights for the extended vector

@@ -22,8 +22,9 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) score_select_kernel(const
     const int32_t* src = a.draft + (int64_t)b * kc;
     const int tok0 = lane < d ? src[lane] : -1;
     const int tok1 = lane + 32 < d ? src[lane + 32] : -1;
-    score_select_request<EXT>(a, b, lane, s_hid[warp], a.hist_len[b], d, a.match_len[b], a.match_pos[b],
-                              a.match_cnt[b], tok0, tok1);
+    int pos = a.match_pos[b];
+    if (EXT && a.match_src && a.match_src[b] == 1) pos = 0;
+    score_select_request<EXT>(a, b, lane, s_hid[warp], a.hist_len[b], d, a.match_len[b], pos, a.match_cnt[b], tok0, tok1);
 }
 
 // Two hidden layers (the paper's predictor shape, 2 x 256).  One CTA scores kReqPerCta (4) requests:
@@ -82,7 +83,9 @@ __global__ void __launch_bounds__(kScore2Threads) score_select2_kernel(const Sco
         const int b = b0 + warp;
         const int d = max(0, min(a.draft_len[b], kc));
         float phi[N];
-        payoff_features(a, b, a.hist_len[b], d, a.match_len[b], a.match_pos[b], a.match_cnt[b], phi);
+        int pos = a.match_pos[b];
+        if (EXT && a.match_src && a.match_src[b] == 1) pos = 0;
+        payoff_features(a, b, a.hist_len[b], d, a.match_len[b], pos, a.match_cnt[b], phi);
         if constexpr (EXT) {
             const int32_t* src = a.draft + (int64_t)b * kc;
             structure_features(a, b, lane, d, lane < d ? src[lane] : -1, lane + 32 < d ? src[lane + 32] : -1, phi);
@@ -173,7 +176,7 @@ ScoreArgs make_score_args(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, cons
     a.W1 = ctx->d_W1; a.b1 = ctx->d_b1; a.W2 = ctx->d_W2; a.b2 = ctx->b2; a.tau = ctx->tau;
     a.hidden = ctx->cfg.hidden; a.k_cap = ctx->cfg.k_cap;
     a.WhT = ctx->two_layer ? ctx->d_WhT : nullptr; a.bh = ctx->d_bh;
-    a.cls = nullptr; a.cls_V = 0; a.suffix = nullptr;
+    a.cls = nullptr; a.cls_V = 0; a.suffix = nullptr; a.match_src = nullptr;
     return a;
 }
 
@@ -211,12 +214,12 @@ hvd_status launch_score_select(hvd_ctx* ctx, int32_t B, const int32_t* hist_len,
 hvd_status launch_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
                                    const hvd_req_state* state, const int32_t* K, const int32_t* draft,
                                    const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,
-                                   const int32_t* match_cnt, const float* suffix, const int32_t* model_draft,
-                                   const int32_t* model_len, float* features, float* score, int32_t* select,
-                                   int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream) {
+                                   const int32_t* match_cnt, const int32_t* match_src, const float* suffix,
+                                   const int32_t* model_draft, const int32_t* model_len, float* features, float* score,
+                                   int32_t* select, int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream) {
     ScoreArgs a = make_score_args(ctx, B, hist_len, prompt_len, state, K, draft, draft_len, match_len, match_pos,
                                   match_cnt, model_draft, model_len, features, score, select, sel_draft, sel_len);
-    a.cls = ctx->cls; a.cls_V = ctx->cls_V; a.suffix = suffix;
+    a.cls = ctx->cls; a.cls_V = ctx->cls_V; a.suffix = suffix; a.match_src = match_src;
     return launch_score_kernels<true>(ctx, a, B, stream);
 }
 

@@ -43,6 +43,10 @@ class DeviceBatch:
         self.draft, self.draft_len = i32(B, kc), i32(B)
         self.match_len, self.match_pos, self.match_cnt = i32(B), i32(B), i32(B)
         self.features = torch.full((B, 8), float("nan"), dtype=torch.float32, device=self.dev)
+        # outputs of the variants: frequency score, source of a corpus match, the extended feature vector
+        self.freq_score = torch.full((B,), float("nan"), dtype=torch.float32, device=self.dev)
+        self.match_src = i32(B)
+        self.features_ext = torch.full((B, 14), float("nan"), dtype=torch.float32, device=self.dev)
         self.score = torch.full((B,), float("nan"), dtype=torch.float32, device=self.dev)
         self.select, self.sel_draft, self.sel_len = i32(B), i32(B, kc), i32(B)
         self.accepted, self.committed, self.n_commit = i32(B), i32(B, kc + 1), i32(B)
@@ -66,6 +70,26 @@ class DeviceBatch:
                                          self.match_pos, self.match_cnt, self.features, self.score,
                                          self.select, self.sel_draft, self.sel_len)
 
+    def lookup_freq(self, min_prob=0.1, max_occ=128, threshold=None):
+        """Frequency-weighted draft and score; with a threshold also the score-threshold selection."""
+        sel = (self.select, self.sel_draft, self.sel_len) if threshold is not None else (None, None, None)
+        self.ctx.hvd_lookup_freq(self.B, self.hist, self.hist_off, self.hist_cap, self.hist_len, self.K, self.n_max,
+                                 float(min_prob), int(max_occ), float(threshold or 0.0), self.model_draft,
+                                 self.model_len, self.draft, self.draft_len, self.freq_score, self.match_len,
+                                 self.match_pos, self.match_cnt, *sel)
+
+    def lookup_corpus(self):
+        self.ctx.hvd_lookup_corpus(self.B, self.hist, self.hist_off, self.hist_cap, self.hist_len, self.K, self.n_max,
+                                   self.draft, self.draft_len, self.match_len, self.match_pos, self.match_src,
+                                   self.match_cnt)
+
+    def score_select_ext(self, suffix=False, src=False):
+        self.ctx.hvd_score_select_ext(self.B, self.hist_len, self.prompt_len, self.state, self.K, self.draft,
+                                      self.draft_len, self.match_len, self.match_pos, self.match_cnt,
+                                      self.freq_score if suffix else None, self.model_draft, self.model_len,
+                                      self.features_ext, self.score, self.select, self.sel_draft, self.sel_len,
+                                      match_src=self.match_src if src else None)
+
     def verify_commit(self, logits, target_tok=True):
         self.ctx.hvd_verify_commit(self.B, logits, self.dtype, self.V, self.row_off, self.k_uniform,
                                    self.total_rows, self.sel_draft, self.sel_len, self.select, self.hist,
@@ -86,7 +110,7 @@ class DeviceBatch:
         """Host copies of every output and in/out array (synchronises)."""
         names = ["draft", "draft_len", "match_len", "match_pos", "match_cnt", "features", "score",
                  "select", "sel_draft", "sel_len", "accepted", "committed", "n_commit", "target_tok",
-                 "status", "hist", "hist_len"]
+                 "status", "hist", "hist_len", "freq_score", "match_src", "features_ext"]
         out = {k: getattr(self, k).cpu().numpy() for k in names}
         out["target_tok"] = out["target_tok"][:self.total_rows]
         out["state"] = self.state.cpu().numpy().reshape(-1).view(STATE_DTYPE)

@@ -106,3 +106,17 @@ def test_single_feature_probes():
     none = O.score_select_ext(*args, None, cls, None, None, k_cap=w.k_cap, W1=np.zeros((1, 14), f32), b1=[0.0], W2=[1.0],
                               b2=0.0, tau=0.5)
     assert (none.features[:, 13] == 0).all()
+
+
+def test_corpus_matches_take_position_zero():
+    w, rq, lk, cls, sfx = _inputs()
+    args = (rq.hist_len, rq.prompt_len, rq.state, rq.K, lk)
+    kw = dict(k_cap=w.k_cap, W1=np.zeros((1, 14), f32), b1=[0.0], W2=[1.0], b2=0.0, tau=0.5)
+    src = (np.arange(rq.B) % 2).astype(np.int32)
+    a = O.score_select_ext(*args, sfx, cls, None, None, **kw)
+    b = O.score_select_ext(*args, sfx, cls, None, None, match_src=src, **kw)
+    has = lk.match_len > 0
+    assert (b.features[(src == 1) & has, 3] == 1.0).all()            # (n - 0) / n
+    assert (b.features[src == 0] == a.features[src == 0]).all()
+    cols = [i for i in range(14) if i != 3]
+    assert (b.features[:, cols] == a.features[:, cols]).all()
