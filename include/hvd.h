@@ -210,7 +210,10 @@ HVD_API hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_
  * array shared by all requests: corpus int32 [m], DEVICE, 16-byte aligned, owned by the caller and
  * kept alive and unchanged while registered; a negative entry separates two traces (it is never
  * part of a match and ends a draft); m (HOST value) in [0, 2^31 - 2]; corpus = NULL or m = 0
- * unregisters.  Takes effect for later hvd_lookup_corpus calls on any stream.
+ * unregisters.  Registration builds an index of the corpus (device memory of about 12 bytes per
+ * token, kernels on the default stream) and returns when it is ready: a set-up call, not for the
+ * decoding loop and not under stream capture.  Takes effect for later hvd_lookup_corpus calls on any
+ * stream.  The index is keyed on the last min(min_match, 2) tokens of a match.
  *
  * hvd_lookup_corpus is hvd_lookup over [corpus, own history].  Candidates are the history positions
  * of hvd_lookup and the corpus positions e in [1, m-1] whose token corpus[e] is not a separator,

@@ -17,6 +17,7 @@ void release(hvd_ctx* c) {
     cudaFree(c->lk_partial); cudaFree(c->lk_cnt);
     cudaFree(c->fq_occ); cudaFree(c->fq_cnt);
     cudaFree(c->cp_key); cudaFree(c->cp_cnt); cudaFree(c->cp_arrived);
+    cudaFree(c->cp_start); cudaFree(c->cp_pos);
     cudaFree(c->rp_off); cudaFree(c->rp_cap); cudaFree(c->rp_len); cudaFree(c->rp_K); cudaFree(c->rp_draft);
     cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
@@ -237,11 +238,10 @@ hvd_status hvd_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_
 
 hvd_status hvd_set_corpus(hvd_ctx* ctx, const int32_t* corpus, int64_t m) {
     if (!ctx) return HVD_ERR_INVALID_ARG;
-    if (corpus == nullptr || m == 0) { ctx->corpus = nullptr; ctx->corpus_len = 0; return HVD_OK; }
+    if (corpus == nullptr || m == 0) { release_corpus_index(ctx); return HVD_OK; }
     if (m < 0 || m > 2147483646LL) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_corpus: m outside [0, 2^31 - 2]");
     if (!aligned(corpus, 16)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_set_corpus: corpus must be 16-byte aligned");
-    ctx->corpus = corpus; ctx->corpus_len = (int32_t)m;
-    return HVD_OK;
+    return build_corpus_index(ctx, corpus, m);
 }
 
 hvd_status hvd_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,

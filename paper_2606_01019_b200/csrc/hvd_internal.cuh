@@ -75,6 +75,10 @@ struct hvd_ctx {
     // shared warm-up corpus (caller-owned) and the scratch its scan meets in, zero at rest
     const int32_t* corpus;
     int32_t corpus_len;
+    uint32_t* cp_start;  // index of the corpus: bucket boundaries [buckets + 1] ...
+    int32_t* cp_pos;     // ... and the indexed positions, bucket by bucket
+    uint32_t cp_mask;    // buckets - 1
+    int cp_g;            // tokens in a key (min(min_match, 2))
     unsigned long long* cp_key;  // [max_batch]
     uint32_t* cp_cnt;            // [max_batch, HVD_MAX_L + 1]
     uint32_t* cp_arrived;        // [max_batch]
@@ -179,6 +183,9 @@ hvd_status launch_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, co
                                 const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K, int32_t n_max,
                                 int32_t* draft, int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
                                 int32_t* match_src, int32_t* match_cnt, cudaStream_t stream);
+
+hvd_status build_corpus_index(hvd_ctx* ctx, const int32_t* corpus, int64_t m);
+void release_corpus_index(hvd_ctx* ctx);
 
 struct VerifyArgs {
     int32_t B;

@@ -132,6 +132,29 @@ def test_workload_requests_and_warm_up_traces(name, B, n):
     run.close()
 
 
+@pytest.mark.parametrize("min_match,l_max", [(2, 64), (1, 64), (2, 1), (3, 5)])
+def test_long_buckets(min_match, l_max):
+    """Keys that occur thousands of times (runs of one token, a two-token cycle): every CTA of a request
+    gets candidates, counts run into the thousands, and the longest lengths saturate at l_max."""
+    rng = np.random.default_rng(31)
+    corpus = np.concatenate([np.full(9000, 5, np.int32), [-1], np.tile(np.array([7, 8], np.int32), 4000), [-1],
+                             rng.integers(0, 3, 6000).astype(np.int32), np.full(70, 5, np.int32), [9]])
+    hs = [[5] * 10, [5] * 100, [1, 5], [7, 8] * 40, [8, 7, 8], [3, 7, 8, 7], list(rng.integers(0, 3, 50)), [9, 5, 5, 5],
+          [5] * 3 + [6] + [5] * 3]
+    flat, off, cap, ln = pack(hs)
+    K = np.full(len(hs), 8, np.int32)
+    cfg = dict(min_match=min_match, l_max=l_max, spec_factor=2.0)
+    run = CorpusRunner(len(hs), 8, 128, **cfg)
+    run.set_corpus(corpus)
+    want = O.lookup_corpus(flat, off, cap, ln, K, corpus, k_cap=8, nthreads=8, **cfg)
+    check(run(flat, off, cap, ln, K), want)
+    if l_max >= min_match:
+        assert want.match_cnt.max() > 3000
+    else:
+        assert (want.match_len == 0).all()
+    run.close()
+
+
 def test_degenerate_requests_and_bad_arguments():
     import torch
     import paper_2606_01019_b200 as H
