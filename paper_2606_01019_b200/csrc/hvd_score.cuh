@@ -71,21 +71,39 @@ __device__ __forceinline__ void payoff_features(const ScoreArgs& a, int b, int n
     phi[7] = __fdiv_rn((float)acc_sum, 8.0f);
 }
 
-// hidden unit j of the first layer: relu(b1[j] + sum_i W1[j][i] phi[i]), left to right
+// hidden unit j of the first layer: relu(b1[j] + sum_i W1[j][i] phi[i]), left to right.  The weights
+// can be fetched ahead of the features (load_first_layer) and applied later (apply_first_layer).
+template <int N>
+struct FirstLayerRow {
+    static constexpr int STRIDE = (N == HVD_N_FEATURES) ? HVD_N_FEATURES : kW1StrideExt;  // 32- or 64-byte rows
+    float w[STRIDE];
+    float bias;
+};
+
+template <int N>
+__device__ __forceinline__ FirstLayerRow<N> load_first_layer(const ScoreArgs& a, int j) {
+    FirstLayerRow<N> row;
+    row.bias = __ldg(a.b1 + j);
+    const float4* w4 = reinterpret_cast<const float4*>(a.W1 + (int64_t)j * FirstLayerRow<N>::STRIDE);
+#pragma unroll
+    for (int q = 0; q < FirstLayerRow<N>::STRIDE / 4; ++q) {
+        const float4 v = __ldg(w4 + q);
+        row.w[4 * q] = v.x; row.w[4 * q + 1] = v.y; row.w[4 * q + 2] = v.z; row.w[4 * q + 3] = v.w;
+    }
+    return row;
+}
+
+template <int N>
+__device__ __forceinline__ float apply_first_layer(const FirstLayerRow<N>& row, const float (&phi)[N]) {
+    float acc = row.bias;
+#pragma unroll
+    for (int i = 0; i < N; ++i) acc = __fmaf_rn(row.w[i], phi[i], acc);
+    return acc > 0.0f ? acc : 0.0f;
+}
+
 template <int N>
 __device__ __forceinline__ float first_layer_unit(const ScoreArgs& a, int j, const float (&phi)[N]) {
-    float acc = __ldg(a.b1 + j);
-    constexpr int STRIDE = (N == HVD_N_FEATURES) ? HVD_N_FEATURES : kW1StrideExt;  // 32- or 64-byte rows
-    const float4* w4 = reinterpret_cast<const float4*>(a.W1 + (int64_t)j * STRIDE);
-    float w[STRIDE];
-#pragma unroll
-    for (int q = 0; q < STRIDE / 4; ++q) {
-        const float4 v = __ldg(w4 + q);
-        w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
-    }
-#pragma unroll
-    for (int i = 0; i < N; ++i) acc = __fmaf_rn(w[i], phi[i], acc);
-    return acc > 0.0f ? acc : 0.0f;
+    return apply_first_layer(load_first_layer<N>(a, j), phi);
 }
 
 // Draft-structure group and suffix score of the extended vector (App. B feature groups), by one
@@ -105,22 +123,33 @@ __device__ __forceinline__ void structure_features(const ScoreArgs& a, int b, in
 }
 
 // Selection rule and the selected draft, by one warp.  tok0 / tok1: cache draft tokens lane and
-// lane+32 (-1 beyond the draft).
-__device__ __forceinline__ void select_draft(const ScoreArgs& a, int b, int lane, float y, int d, int tok0, int tok1) {
+// lane+32 (-1 beyond the draft).  The model draft's length and tokens can be fetched ahead of the
+// score (load_model_draft).
+struct ModelDraft {
+    int m;       // usable length of the model draft (0 without one)
+    int t0, t1;  // its tokens lane and lane + 32 (-1 beyond m)
+};
+
+__device__ __forceinline__ ModelDraft load_model_draft(const ScoreArgs& a, int b, int lane) {
+    ModelDraft md;
+    md.m = 0; md.t0 = -1; md.t1 = -1;
+    if (a.model_draft && a.model_len) {
+        const int kc = a.k_cap;
+        const int K = max(0, min(__ldg(a.K + b), kc));
+        md.m = max(0, min(__ldg(a.model_len + b), K));
+        const int32_t* src = a.model_draft + (int64_t)b * kc;
+        if (lane < md.m) md.t0 = __ldg(src + lane);
+        if (lane + 32 < md.m) md.t1 = __ldg(src + lane + 32);
+    }
+    return md;
+}
+
+__device__ __forceinline__ void select_draft(const ScoreArgs& a, int b, int lane, float y, int d, int tok0, int tok1,
+                                             const ModelDraft& md) {
     const int kc = a.k_cap;
-    const int K = max(0, min(__ldg(a.K + b), kc));
     const int sel = (d > 0 && y >= a.tau) ? 1 : 0;
     int m = d;
-    if (!sel) {
-        m = 0;
-        tok0 = tok1 = -1;
-        if (a.model_draft && a.model_len) {
-            m = max(0, min(__ldg(a.model_len + b), K));
-            const int32_t* src = a.model_draft + (int64_t)b * kc;
-            if (lane < m) tok0 = __ldg(src + lane);
-            if (lane + 32 < m) tok1 = __ldg(src + lane + 32);
-        }
-    }
+    if (!sel) { m = md.m; tok0 = md.t0; tok1 = md.t1; }
     if (lane < kc) a.sel_draft[(int64_t)b * kc + lane] = (lane < m) ? tok0 : -1;
     if (lane + 32 < kc) a.sel_draft[(int64_t)b * kc + lane + 32] = (lane + 32 < m) ? tok1 : -1;
     if (lane == 0) {
@@ -128,6 +157,14 @@ __device__ __forceinline__ void select_draft(const ScoreArgs& a, int b, int lane
         a.select[b] = sel;
         a.sel_len[b] = m;
     }
+}
+
+__device__ __forceinline__ void select_draft(const ScoreArgs& a, int b, int lane, float y, int d, int tok0, int tok1) {
+    const int sel = (d > 0 && y >= a.tau) ? 1 : 0;
+    ModelDraft md;
+    md.m = 0; md.t0 = -1; md.t1 = -1;
+    if (!sel) md = load_model_draft(a, b, lane);  // only fetched when it is the one verified
+    select_draft(a, b, lane, y, d, tok0, tok1, md);
 }
 
 // One-hidden-layer predictor for one request by one warp.  The work is a few hundred flops per

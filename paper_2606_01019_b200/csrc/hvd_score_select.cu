@@ -1,7 +1,11 @@
 // Payoff features, predictor and draft selection (Sec. 3.3, Sec. 3.4, App. B feature groups).
 //
 // Stand-alone kernel: one warp per request (the per-request arithmetic is in hvd_score.cuh).
+#include <cooperative_groups.h>
+
 #include "hvd_score.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace hvd {
 namespace {
@@ -27,58 +31,77 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) score_select_kernel(const
     score_select_request<EXT>(a, b, lane, s_hid[warp], a.hist_len[b], d, a.match_len[b], pos, a.match_cnt[b], tok0, tok1);
 }
 
-// Two hidden layers (the paper's predictor shape, 2 x 256).  One CTA scores kReqPerCta (4) requests:
-// the second layer's 256 KB of weights are the traffic that matters, and every request a CTA
-// handles reuses the tile it has staged.  Thread j evaluates unit j of each layer, for each of the
-// CTA's requests, with the same left-to-right fused multiply-add chains as the one-layer kernel
-// (64 K multiply-adds per request: still far from a tensor-core shape at batch sizes of tens to
-// hundreds, and a sequential order keeps the result independent of the launch).  The second
-// layer's weights are stored transposed with a row stride of HVD_MAX_HIDDEN (WhT[i][j] = Wh[j][i])
-// and are staged through shared memory with asynchronous 16-byte copies, two tiles of kTileRows
-// rows in flight, so that the chains never wait for a global load.
+// Two hidden layers (the paper's predictor shape, 2 x 256).  A thread-block cluster of four CTAs
+// scores four requests: CTA `rank` owns 64 of the second layer's 256 output units, so it stages only
+// its 64 KB column slab of the weights (stored transposed with a row stride of HVD_MAX_HIDDEN:
+// WhT[i][j] = Wh[j][i]) with asynchronous 16-byte copies issued before anything else; thread
+// (request r, unit jj) runs one left-to-right chain of fused multiply-adds over the 256 inputs --
+// the same order as the one-layer kernel and as a plain loop, so the fp32 result does not depend on
+// the launch (64 K multiply-adds per request: far from a tensor-core shape at batch sizes of tens to
+// hundreds).  The first layer is cheap and every CTA evaluates it for itself; the second layer's
+// activations go to CTA 0 of the cluster through distributed shared memory, and after the cluster
+// barrier CTA 0 runs the output layer (one sequential chain per request) and the selection.
 constexpr int kScore2Threads = HVD_MAX_HIDDEN;
-constexpr int kReqPerCta = 4;  // requests per CTA: one float4 of first-layer activations per input unit
-constexpr int kTileRows = 64;
-constexpr int kTileFloats = kTileRows * HVD_MAX_HIDDEN;
+constexpr int kClusterSize = 4;
+constexpr int kReqPerCluster = 4;  // one float4 of first-layer activations per input unit
+constexpr int kColsPerCta = HVD_MAX_HIDDEN / kClusterSize;
 constexpr int kHidPad = HVD_MAX_HIDDEN + 1;  // row stride of the second-layer activations
-constexpr size_t kScore2Smem = 2 * (size_t)kTileFloats * sizeof(float);  // 128 KB
-
-__device__ __forceinline__ void copy_tile_async(float* dst, const float* src, int tid) {
-    // kTileFloats floats = 4096 x 16 bytes, 16 per thread
-    const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(dst);
-#pragma unroll
-    for (int k = 0; k < kTileFloats / 4 / kScore2Threads; ++k) {
-        const int v = k * kScore2Threads + tid;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d0 + v * 16), "l"(src + v * 4) : "memory");
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-}
+constexpr size_t kScore2Smem = (size_t)HVD_MAX_HIDDEN * kColsPerCta * sizeof(float);  // 64 KB slab
+static_assert(kScore2Threads == kReqPerCluster * kColsPerCta, "one thread per (request, unit) pair");
 
 template <bool EXT>
-__global__ void __launch_bounds__(kScore2Threads) score_select2_kernel(const ScoreArgs a) {
+__global__ void __cluster_dims__(kClusterSize, 1, 1) __launch_bounds__(kScore2Threads)
+score_select2_kernel(const ScoreArgs a) {
     constexpr int N = NFeat<EXT>::value;
-    extern __shared__ __align__(16) float s_tiles[];  // [2][kTileRows][HVD_MAX_HIDDEN]
-    __shared__ float s_phi[kReqPerCta][N];
-    __shared__ __align__(16) float s_h1[HVD_MAX_HIDDEN][kReqPerCta];  // [input unit][request]
-    __shared__ float s_h2[kReqPerCta][kHidPad];
+    extern __shared__ __align__(16) float s_w[];  // [HVD_MAX_HIDDEN inputs][kColsPerCta units]
+    __shared__ float s_phi[kReqPerCluster][N];
+    __shared__ __align__(16) float s_h1[HVD_MAX_HIDDEN][kReqPerCluster];  // [input unit][request]
+    __shared__ float s_h2[kReqPerCluster][kHidPad];                        // filled by the whole cluster in CTA 0
     __shared__ float s_w2[HVD_MAX_HIDDEN];
-    __shared__ float s_y[kReqPerCta];
-    __shared__ int s_d[kReqPerCta];
+    __shared__ float s_y[kReqPerCluster];
+    __shared__ int s_d[kReqPerCluster];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    const int b0 = blockIdx.x * kReqPerCta;
-    const int nreq = min(kReqPerCta, a.B - b0);
+    const int b0 = (int)(blockIdx.x / kClusterSize) * kReqPerCluster;
+    const int nreq = min(kReqPerCluster, a.B - b0);
     const int kc = a.k_cap;
     const int H = a.hidden;
-    const int n_tiles = (H + kTileRows - 1) / kTileRows;
-    // the weights do not depend on the previous kernel: their first tiles are requested at once
-    copy_tile_async(s_tiles, a.WhT, tid);
-    if (n_tiles > 1) copy_tile_async(s_tiles + kTileFloats, a.WhT + kTileFloats, tid);
+    // the weights do not depend on the previous kernel: this CTA's slab is requested at once
+    {
+        const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(s_w);
+        const float* src = a.WhT + rank * kColsPerCta;
+#pragma unroll
+        for (int k = 0; k < HVD_MAX_HIDDEN * kColsPerCta / 4 / kScore2Threads; ++k) {
+            const int v = k * kScore2Threads + tid;       // 16-byte vector: row v / 16, vector v % 16 of the row
+            const int row = v / (kColsPerCta / 4), c4 = v % (kColsPerCta / 4);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d0 + v * 16),
+                         "l"(src + (size_t)row * HVD_MAX_HIDDEN + c4 * 4) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
     if (tid < H) s_w2[tid] = __ldg(a.W2 + tid);
+    // so are this thread's first-layer weights and its second-layer bias
+    FirstLayerRow<N> row1;
+    if (tid < H) row1 = load_first_layer<N>(a, tid);
+    const int my_j = rank * kColsPerCta + tid % kColsPerCta;
+    const float my_bh = (my_j < H) ? __ldg(a.bh + my_j) : 0.0f;
     pdl_trigger();
     pdl_wait();
-    // features: warp r for request b0 + r
+    // CTA 0 selects at the end: its warps fetch the drafts they will choose between now
+    ModelDraft md;
+    int ctok0 = -1, ctok1 = -1;
+    if (rank == 0 && warp < nreq) {
+        const int b = b0 + warp;
+        md = load_model_draft(a, b, lane);
+        const int d = max(0, min(a.draft_len[b], kc));
+        const int32_t* src = a.draft + (int64_t)b * kc;
+        ctok0 = lane < d ? src[lane] : -1;
+        ctok1 = lane + 32 < d ? src[lane + 32] : -1;
+    }
+    // features: warp r for request b0 + r (every CTA of the cluster needs them; CTA 0 writes them out)
     if (warp < nreq) {
         const int b = b0 + warp;
         const int d = max(0, min(a.draft_len[b], kc));
@@ -95,54 +118,43 @@ __global__ void __launch_bounds__(kScore2Threads) score_select2_kernel(const Sco
 #pragma unroll
             for (int i = 1; i < N; ++i) v = (lane == i) ? phi[i] : v;
             s_phi[warp][lane] = v;
-            if (a.features) a.features[(int64_t)b * N + lane] = v;
+            if (a.features && rank == 0) a.features[(int64_t)b * N + lane] = v;
         }
         if (lane == 0) s_d[warp] = d;
     }
     __syncthreads();
-    float acc[kReqPerCta];
-    if (tid < H) {
-        const float bias = __ldg(a.bh + tid);
-        float h1[kReqPerCta];
+    {   // first layer: thread j evaluates unit j for the four requests
+        float h1[kReqPerCluster] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (tid < H) {
 #pragma unroll
-        for (int r = 0; r < kReqPerCta; ++r) {
-            acc[r] = bias;
-            h1[r] = 0.0f;
-            if (r < nreq) {
-                float phi[N];
+            for (int r = 0; r < kReqPerCluster; ++r) {
+                if (r < nreq) {
+                    float phi[N];
 #pragma unroll
-                for (int i = 0; i < N; ++i) phi[i] = s_phi[r][i];
-                h1[r] = first_layer_unit(a, tid, phi);
+                    for (int i = 0; i < N; ++i) phi[i] = s_phi[r][i];
+                    h1[r] = apply_first_layer(row1, phi);
+                }
             }
         }
         *reinterpret_cast<float4*>(s_h1[tid]) = make_float4(h1[0], h1[1], h1[2], h1[3]);
-    } else {
-        *reinterpret_cast<float4*>(s_h1[tid]) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
     }
-    for (int t = 0; t < n_tiles; ++t) {
-        if (t + 1 < n_tiles) asm volatile("cp.async.wait_group 1;" ::: "memory");
-        else asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncthreads();  // tile t has landed for every thread (and, for t = 0, s_h1 is complete)
-        const float* w = s_tiles + (t & 1) * kTileFloats + tid;
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();  // the slab and s_h1 are complete
+    {   // second layer: thread (r, jj) -> unit j = rank * 64 + jj of request r
+        const int r = tid / kColsPerCta, jj = tid % kColsPerCta;
+        const int j = rank * kColsPerCta + jj;
+        float acc = my_bh;
         // rows beyond H hold zero weights and zero activations: adding their products changes nothing,
-        // and a fixed trip count lets all the shared-memory loads of a tile be issued ahead of the chains
-        if (tid < H) {
+        // and a fixed trip count lets the shared-memory loads be issued ahead of the chain
+        const float* w = s_w + jj;
 #pragma unroll 16
-            for (int i = 0; i < kTileRows; ++i) {
-                const float wv = w[i * HVD_MAX_HIDDEN];
-                const float4 h = *reinterpret_cast<const float4*>(s_h1[t * kTileRows + i]);  // broadcast
-                acc[0] = __fmaf_rn(wv, h.x, acc[0]); acc[1] = __fmaf_rn(wv, h.y, acc[1]);
-                acc[2] = __fmaf_rn(wv, h.z, acc[2]); acc[3] = __fmaf_rn(wv, h.w, acc[3]);
-            }
-        }
-        __syncthreads();  // everyone is done with this buffer
-        if (t + 2 < n_tiles) copy_tile_async(s_tiles + (t & 1) * kTileFloats, a.WhT + (size_t)(t + 2) * kTileFloats, tid);
+        for (int i = 0; i < HVD_MAX_HIDDEN; ++i) acc = __fmaf_rn(w[i * kColsPerCta], s_h1[i][r], acc);
+        const float h2 = (j < H && r < nreq && acc > 0.0f) ? acc : 0.0f;
+        float* dst = cluster.map_shared_rank(&s_h2[0][0], 0);  // CTA 0's copy
+        dst[r * kHidPad + j] = h2;
     }
-    if (tid < H) {
-#pragma unroll
-        for (int r = 0; r < kReqPerCta; ++r) s_h2[r][tid] = acc[r] > 0.0f ? acc[r] : 0.0f;
-    }
-    __syncthreads();
+    cluster.sync();  // all four slabs of activations have arrived in CTA 0
+    if (rank != 0) return;
     if (tid < nreq) {  // output layer: one sequential chain per request, operands from shared memory
         float y = a.b2;
 #pragma unroll 8
@@ -151,12 +163,7 @@ __global__ void __launch_bounds__(kScore2Threads) score_select2_kernel(const Sco
     }
     __syncthreads();
     if (warp < nreq) {
-        const int b = b0 + warp;
-        const int d = s_d[warp];
-        const int32_t* src = a.draft + (int64_t)b * kc;
-        const int tok0 = lane < d ? src[lane] : -1;
-        const int tok1 = lane + 32 < d ? src[lane + 32] : -1;
-        select_draft(a, b, lane, s_y[warp], d, tok0, tok1);
+        select_draft(a, b0 + warp, lane, s_y[warp], s_d[warp], ctok0, ctok1, md);
     }
 }
 
@@ -189,7 +196,8 @@ static hvd_status launch_score_kernels(hvd_ctx* ctx, const ScoreArgs& a, int32_t
                                                    (int)kScore2Smem));
             ready = true;
         }
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select2_kernel<EXT>, (B + kReqPerCta - 1) / kReqPerCta,
+        const int clusters = (B + kReqPerCluster - 1) / kReqPerCluster;
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select2_kernel<EXT>, clusters * kClusterSize,
                                         kScore2Threads, kScore2Smem, stream, a));
         return HVD_OK;
     }
