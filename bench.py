@@ -501,11 +501,14 @@ def main():
         hist_len_steps.copy_(hist_len_pristine)
         state_steps.copy_(state_pristine)
 
-    def step(slot, events=None, with_verify=True, lookup_only=False):
+    def step(slot, events=None, with_verify=True, lookup_only=False, verify_only=False):
         r = slot % R
         hl, st = hist_len_steps[slot], state_steps[slot]
         if lookup_only:
             lookup(hists[r], hl)
+            return
+        if verify_only:   # the selection of the last lookup is still in place: every step starts from the same state
+            verify(logits[r], hists[r], hl, st)
             return
         if events is not None:
             events[0].record()
@@ -528,12 +531,12 @@ def main():
     mode = args.mode
     stream = torch.cuda.Stream(device=dev)
 
-    def capture(events=None, with_verify=True, lookup_only=False):
+    def capture(events=None, with_verify=True, lookup_only=False, verify_only=False):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
             g.capture_begin()
             for s in range(K_steps):
-                step(W_steps + s, events[s] if events else None, with_verify, lookup_only)
+                step(W_steps + s, events[s] if events else None, with_verify, lookup_only, verify_only)
             g.capture_end()
         torch.cuda.synchronize()
         with torch.cuda.stream(stream):
@@ -608,11 +611,17 @@ def main():
                 t_nv = timed(g_nv.replay)
                 g_lk = capture(None, lookup_only=True)
                 t_lk = timed(g_lk.replay)
+                restore()
+                g_vo = capture(None, verify_only=True)
+                restore()
+                t_vo = timed(g_vo.replay)
             else:
                 t_ev = timed(lambda: [step(W_steps + s, evs[s]) for s in range(K_steps)])
                 restore()
                 t_nv = timed(lambda: [step(W_steps + s, None, False) for s in range(K_steps)])
                 t_lk = timed(lambda: [step(W_steps + s, None, False, True) for s in range(K_steps)])
+                restore()
+                t_vo = timed(lambda: [step(W_steps + s, None, True, False, True) for s in range(K_steps)])
             restore()
             d = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(2)] for e in evs])
             kt = {"lookup_plus_score_select_us": 1e3 * float(d[:, 0].mean()),
@@ -622,6 +631,7 @@ def main():
                   "step_us_without_verify": 1e3 * t_nv / K_steps,
                   "lookup_only_us": 1e3 * t_lk / K_steps,
                   "verify_commit_us_by_difference": 1e3 * (elapsed_ms - t_nv) / K_steps,
+                  "verify_commit_us_back_to_back": 1e3 * t_vo / K_steps,
                   "note": "event-bracketed times include the serialisation the event records add; "
                           "the headline region has no records in it"}
         except Exception as e:  # pragma: no cover
@@ -642,13 +652,15 @@ def main():
                        "achieved": None, "peak": peak_gbs, "unit": "GB/s", "frac": None, "traffic": None,
                        "peak_kind": peak_kind, "algorithmic_bytes_per_launch": lookup_bytes}
     if kt:
-        roofline["achieved"] = verify_bytes / (kt["verify_commit_us"] * 1e-6) / 1e9
+        roofline["achieved"] = verify_bytes / (kt["verify_commit_us_back_to_back"] * 1e-6) / 1e9
         roofline["frac"] = roofline["achieved"] / peak_gbs
         roofline["frac_of_8000_nominal"] = roofline["achieved"] / 8000.0
         roofline["achieved_by_difference"] = verify_bytes / (kt["verify_commit_us_by_difference"] * 1e-6) / 1e9
+        roofline["achieved_with_event_records_in_graph"] = verify_bytes / (kt["verify_commit_us"] * 1e-6) / 1e9
         roofline_lookup["achieved"] = lookup_bytes / (kt["lookup_only_us"] * 1e-6) / 1e9
         roofline_lookup["frac"] = roofline_lookup["achieved"] / peak_gbs
-        roofline["timing"] = "CUDA events recorded around the hvd_verify_commit call inside the graph"
+        roofline["timing"] = ("CUDA events around a graph of the same K hvd_verify_commit launches back to back "
+                              "(both kernels of the call, launch gaps included), on rotating inputs larger than L2")
 
     # ---- end to end through the host-buffer entry point --------------------------------------------
     e2e = None
