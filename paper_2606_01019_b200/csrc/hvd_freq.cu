@@ -25,7 +25,8 @@ constexpr int kCollectThreads = 256;
 constexpr int kCollectIter = 4;
 constexpr int kCollectChunk = kCollectThreads * kLookupTokPerVec * kCollectIter;  // tokens per CTA
 constexpr int kWalkThreads = HVD_FREQ_MAX_OCC;                                    // one thread per occurrence
-constexpr int kSlots = HVD_FREQ_MAX_OCC / 32;                                     // occurrences per lane of the walking warp
+constexpr int kSlots = HVD_FREQ_MAX_OCC / 32;
+constexpr int kBatchMaxAlive = 6;   // agreement runs are looked for while at most this many occurrences are alive                                     // occurrences per lane of the walking warp
 
 struct FreqArgs {
     const int32_t* hist;
@@ -135,8 +136,8 @@ using TokTile = int32_t[HVD_FREQ_MAX_OCC + 1];
 // The walk over SLOTS * 32 listed occurrences by one warp; lane l owns occurrences l, l + 32, ...
 template <int SLOTS>
 __device__ __forceinline__ void walk_merged(const FreqArgs& a, const int32_t* __restrict__ slab, int n, int limit,
-                                            int lane, const TokTile* s_tok, const int32_t* s_e, int& d, float& sc,
-                                            int& tok0, int& tok1) {
+                                            int lane, const TokTile* s_tok, const int32_t* s_e, int32_t* s_alive,
+                                            int& d, float& sc, int& tok0, int& tok1) {
     int e[SLOTS], len[SLOTS];
     bool alive[SLOTS];
     int na = 0;
@@ -147,7 +148,49 @@ __device__ __forceinline__ void walk_merged(const FreqArgs& a, const int32_t* __
         len[j] = alive[j] ? min(limit, n - e[j]) : 0;
         na += __popc(__ballot_sync(0xffffffffu, alive[j]));
     }
+    bool listed = false;  // s_alive holds the indices of the alive occurrences
     while (d < limit) {
+        if (na >= 2 && na <= kBatchMaxAlive && 1.0f >= a.min_prob) {
+            // Steps on which every alive occurrence continues with the same token have probability 1 and
+            // keep the set as it is: all of them are taken at once.  Lane l looks at draft positions l, l + 32.
+            if (!listed) {
+                int base = 0;
+#pragma unroll
+                for (int j = 0; j < SLOTS; ++j) {
+                    const uint32_t mask = __ballot_sync(0xffffffffu, alive[j]);
+                    if (alive[j]) s_alive[base + __popc(mask & ((1u << lane) - 1u))] = lane + 32 * j;
+                    base += __popc(mask);
+                }
+                __syncwarp();
+                listed = true;
+            }
+            bool ok[2];
+            int t[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int q = lane + 32 * h;
+                ok[h] = q >= d && q < limit;
+                t[h] = -1;
+                if (ok[h]) {
+                    t[h] = s_tok[q][s_alive[0]];
+                    for (int k = 0; k < na; ++k) {
+                        const int i = s_alive[k];
+                        ok[h] = ok[h] && (s_e[i] + q < n) && (s_tok[q][i] == t[h]);
+                    }
+                }
+            }
+            const unsigned long long agree = ((unsigned long long)__ballot_sync(0xffffffffu, ok[1]) << 32) |
+                                             __ballot_sync(0xffffffffu, ok[0]);
+            const unsigned long long miss = ~(agree >> d);  // bit r: position d + r does not agree (or is past the limit)
+            const int run = miss ? __ffsll((long long)miss) - 1 : 64;
+            if (run > 0) {
+                if (lane >= d && lane < d + run) tok0 = t[0];
+                if (lane + 32 >= d && lane + 32 < d + run) tok1 = t[1];
+                for (int k = 0; k < run; ++k) sc = __fadd_rn(sc, 1.0f);  // the same additions, one by one
+                d += run;
+                continue;
+            }
+        }
         if (na == 1) {
             // one occurrence left: each further token has probability 1 until it or the limit ends
             int me = -1;
@@ -199,6 +242,7 @@ __device__ __forceinline__ void walk_merged(const FreqArgs& a, const int32_t* __
         sc = __fadd_rn(sc, prob);
 #pragma unroll
         for (int j = 0; j < SLOTS; ++j) alive[j] = alive[j] && d < len[j] && t[j] == best_tok;
+        listed = listed && best_cnt == na;  // the list stays valid only if nobody dropped out
         na = best_cnt;
         ++d;
     }
@@ -207,6 +251,7 @@ __device__ __forceinline__ void walk_merged(const FreqArgs& a, const int32_t* __
 __global__ void __launch_bounds__(kWalkThreads) freq_walk_kernel(const FreqArgs a) {
     __shared__ int32_t s_tok[HVD_MAX_K][HVD_FREQ_MAX_OCC + 1];  // [step][occurrence]; odd stride: no bank conflicts
     __shared__ int32_t s_e[HVD_FREQ_MAX_OCC];
+    __shared__ int32_t s_alive[HVD_FREQ_MAX_OCC];
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -248,8 +293,8 @@ __global__ void __launch_bounds__(kWalkThreads) freq_walk_kernel(const FreqArgs 
     float sc = 0.0f;
     int tok0 = -1, tok1 = -1;  // draft tokens lane and lane + 32
     if (merged) {
-        if (c <= 32) walk_merged<1>(a, slab, n, limit, lane, s_tok, s_e, d, sc, tok0, tok1);
-        else walk_merged<kSlots>(a, slab, n, limit, lane, s_tok, s_e, d, sc, tok0, tok1);
+        if (c <= 32) walk_merged<1>(a, slab, n, limit, lane, s_tok, s_e, s_alive, d, sc, tok0, tok1);
+        else walk_merged<kSlots>(a, slab, n, limit, lane, s_tok, s_e, s_alive, d, sc, tok0, tok1);
     } else if (L > 0) {
         // one occurrence: every token has probability 1 (nothing passes a minimum above 1);
         // too many occurrences: the latest one, every token taken as certain
