@@ -268,8 +268,9 @@ HVD_API hvd_status hvd_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist,
  * x[0..t): its cache draft is the hvd_lookup result on that prefix (same rules, K for every state),
  * and its label is y_t = max{ l <= draft_len : draft[0..l) == x[t .. t+l) }, the number of draft tokens
  * the trace's own continuation confirms.  Outputs (int32 [n], index t-1): label, draft_len, match_len,
- * match_pos, match_cnt.  trace: DEVICE, 16-byte aligned; n (HOST value) <= max_hist_len; states are
- * processed in slices of max_batch.  These are the regression targets of the payoff predictor; the
+ * match_pos, match_cnt.  trace: DEVICE, 16-byte aligned; n (HOST value) <= max_hist_len.  The first
+ * call, and any call with a longer trace than before, allocates per-state scratch (268 bytes per
+ * position) after waiting for the stream: not for use under stream capture.  These are the regression targets of the payoff predictor; the
  * recent-history features depend on the decoding loop and are not produced here.
  */
 HVD_API hvd_status hvd_replay_labels(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label,

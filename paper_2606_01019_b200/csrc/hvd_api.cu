@@ -18,7 +18,7 @@ void release(hvd_ctx* c) {
     cudaFree(c->fq_occ); cudaFree(c->fq_cnt);
     cudaFree(c->cp_key); cudaFree(c->cp_cnt); cudaFree(c->cp_arrived);
     cudaFree(c->cp_start); cudaFree(c->cp_pos);
-    cudaFree(c->rp_off); cudaFree(c->rp_cap); cudaFree(c->rp_len); cudaFree(c->rp_K); cudaFree(c->rp_draft);
+    cudaFree(c->rp_key); cudaFree(c->rp_cnt);
     cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
     delete c;
@@ -86,12 +86,6 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->cp_key, (size_t)cfg->max_batch * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && alloc_zero(&c->cp_cnt, (size_t)cfg->max_batch * (HVD_MAX_L + 1) * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->cp_arrived, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
-    const size_t MB = (size_t)cfg->max_batch;
-    ok = ok && alloc_zero(&c->rp_off, MB * sizeof(int64_t)) == cudaSuccess;
-    ok = ok && alloc_zero(&c->rp_cap, MB * sizeof(int32_t)) == cudaSuccess;
-    ok = ok && alloc_zero(&c->rp_len, MB * sizeof(int32_t)) == cudaSuccess;
-    ok = ok && alloc_zero(&c->rp_K, MB * sizeof(int32_t)) == cudaSuccess;
-    ok = ok && alloc_zero(&c->rp_draft, MB * (size_t)cfg->k_cap * sizeof(int32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_row_key, (size_t)cfg->max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_next_unit, (size_t)kVerifyQueues * 32 * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->dev_error, sizeof(int)) == cudaSuccess;

@@ -72,7 +72,8 @@ struct hvd_ctx {
     // occurrence lists of the frequency-weighted draft
     int32_t* fq_occ;    // [max_batch, HVD_FREQ_MAX_OCC]
     uint32_t* fq_cnt;   // [max_batch], zero at rest
-    // shared warm-up corpus (caller-owned) and the scratch its scan meets in, zero at rest
+    // shared warm-up corpus (caller-owned); cp_key / cp_cnt / cp_arrived: scratch in which the CTAs of a corpus
+    // probe, or the diagonals of a trace replay, meet per request or state; zero at rest
     const int32_t* corpus;
     int32_t corpus_len;
     uint32_t* cp_start;  // index of the corpus: bucket boundaries [buckets + 1] ...
@@ -82,15 +83,16 @@ struct hvd_ctx {
     unsigned long long* cp_key;  // [max_batch]
     uint32_t* cp_cnt;            // [max_batch, HVD_MAX_L + 1]
     uint32_t* cp_arrived;        // [max_batch]
+    // trace replay: per-state maximum and counts for a whole trace, grown on demand, zero at rest
+    unsigned long long* rp_key;  // [rp_states]
+    uint32_t* rp_cnt;            // [rp_states, HVD_MAX_L + 1]
+    int64_t rp_states;
     // verify scratch
     unsigned long long* vf_row_key;  // [max_rows], zero at rest
     uint32_t* vf_next_unit;          // zero at rest
     int* dev_error;                  // device status word
     int vf_blocks_per_sm[2];         // per dtype
     // device staging of the host-buffer entry point (grown on demand)
-    // trace replay: the virtual batch of one slice of states, and its drafts
-    int64_t* rp_off;
-    int32_t *rp_cap, *rp_len, *rp_K, *rp_draft;
     bool use_pdl;  // programmatic dependent launch between the kernels of the path
     char* host_ws;
     size_t host_ws_bytes;
