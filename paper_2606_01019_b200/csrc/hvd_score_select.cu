@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) score_select_kernel(const
 }
 
 // Two hidden layers (the paper's predictor shape, 2 x 256).  A thread-block cluster of four CTAs
-// scores four requests: CTA `rank` owns 64 of the second layer's 256 output units, so it stages only
+// scores four requests (eight or sixteen for larger batches): CTA `rank` owns 64 of the second layer's 256 output units, so it stages only
 // its 64 KB column slab of the weights (stored transposed with a row stride of HVD_MAX_HIDDEN:
 // WhT[i][j] = Wh[j][i]) with asynchronous 16-byte copies issued before anything else; thread
 // (request r, unit jj) runs one left-to-right chain of fused multiply-adds over the 256 inputs --
@@ -43,30 +43,35 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) score_select_kernel(const
 // barrier CTA 0 runs the output layer (one sequential chain per request) and the selection.
 constexpr int kScore2Threads = HVD_MAX_HIDDEN;
 constexpr int kClusterSize = 4;
-constexpr int kReqPerCluster = 4;  // one float4 of first-layer activations per input unit
+constexpr int kReqPerGroup = 4;  // requests that share a pass over the slab: thread (request, unit)
 constexpr int kColsPerCta = HVD_MAX_HIDDEN / kClusterSize;
 constexpr int kHidPad = HVD_MAX_HIDDEN + 1;  // row stride of the second-layer activations
 constexpr size_t kScore2Smem = (size_t)HVD_MAX_HIDDEN * kColsPerCta * sizeof(float);  // 64 KB slab
-static_assert(kScore2Threads == kReqPerCluster * kColsPerCta, "one thread per (request, unit) pair");
+static_assert(kScore2Threads == kReqPerGroup * kColsPerCta, "one thread per (request, unit) pair");
 
-template <bool EXT>
+// G: groups of four requests per cluster (1, 2 or 4).  Larger batches take more requests per cluster so
+// that a slab staged once serves more chains and the grid stays within one wave.
+template <bool EXT, int G>
 __global__ void __cluster_dims__(kClusterSize, 1, 1) __launch_bounds__(kScore2Threads)
 score_select2_kernel(const ScoreArgs a) {
     constexpr int N = NFeat<EXT>::value;
+    constexpr int REQ = kReqPerGroup * G;                  // requests per cluster
+    constexpr int RW = (REQ + kScore2Threads / 32 - 1) / (kScore2Threads / 32);  // requests per warp
     extern __shared__ __align__(16) float s_w[];  // [HVD_MAX_HIDDEN inputs][kColsPerCta units]
-    __shared__ float s_phi[kReqPerCluster][N];
-    __shared__ __align__(16) float s_h1[HVD_MAX_HIDDEN][kReqPerCluster];  // [input unit][request]
-    __shared__ float s_h2[kReqPerCluster][kHidPad];                        // filled by the whole cluster in CTA 0
+    __shared__ float s_phi[REQ][N];
+    __shared__ __align__(16) float s_h1[HVD_MAX_HIDDEN][REQ];  // [input unit][request]
+    __shared__ float s_h2[REQ][kHidPad];                        // filled by the whole cluster in CTA 0
     __shared__ float s_w2[HVD_MAX_HIDDEN];
-    __shared__ float s_y[kReqPerCluster];
-    __shared__ int s_d[kReqPerCluster];
+    __shared__ float s_y[REQ];
+    __shared__ int s_d[REQ];
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    const int b0 = (int)(blockIdx.x / kClusterSize) * kReqPerCluster;
-    const int nreq = min(kReqPerCluster, a.B - b0);
+    constexpr int NWARP = kScore2Threads / 32;
+    const int b0 = (int)(blockIdx.x / kClusterSize) * REQ;
+    const int nreq = min(REQ, a.B - b0);
     const int kc = a.k_cap;
     const int H = a.hidden;
     // the weights do not depend on the previous kernel: this CTA's slab is requested at once
@@ -91,19 +96,25 @@ score_select2_kernel(const ScoreArgs a) {
     pdl_trigger();
     pdl_wait();
     // CTA 0 selects at the end: its warps fetch the drafts they will choose between now
-    ModelDraft md;
-    int ctok0 = -1, ctok1 = -1;
-    if (rank == 0 && warp < nreq) {
-        const int b = b0 + warp;
-        md = load_model_draft(a, b, lane);
-        const int d = max(0, min(a.draft_len[b], kc));
-        const int32_t* src = a.draft + (int64_t)b * kc;
-        ctok0 = lane < d ? src[lane] : -1;
-        ctok1 = lane + 32 < d ? src[lane + 32] : -1;
+    ModelDraft md[RW];
+    int ctok0[RW], ctok1[RW];
+#pragma unroll
+    for (int k = 0; k < RW; ++k) {
+        const int r = warp + k * NWARP;
+        ctok0[k] = -1; ctok1[k] = -1;
+        md[k].m = 0; md[k].t0 = -1; md[k].t1 = -1;
+        if (rank == 0 && r < nreq) {
+            const int b = b0 + r;
+            md[k] = load_model_draft(a, b, lane);
+            const int d = max(0, min(a.draft_len[b], kc));
+            const int32_t* src = a.draft + (int64_t)b * kc;
+            ctok0[k] = lane < d ? src[lane] : -1;
+            ctok1[k] = lane + 32 < d ? src[lane + 32] : -1;
+        }
     }
-    // features: warp r for request b0 + r (every CTA of the cluster needs them; CTA 0 writes them out)
-    if (warp < nreq) {
-        const int b = b0 + warp;
+    // features: one warp per request (every CTA of the cluster needs them; CTA 0 writes them out)
+    for (int r = warp; r < nreq; r += NWARP) {
+        const int b = b0 + r;
         const int d = max(0, min(a.draft_len[b], kc));
         float phi[N];
         int pos = a.match_pos[b];
@@ -117,41 +128,48 @@ score_select2_kernel(const ScoreArgs a) {
             float v = phi[0];
 #pragma unroll
             for (int i = 1; i < N; ++i) v = (lane == i) ? phi[i] : v;
-            s_phi[warp][lane] = v;
+            s_phi[r][lane] = v;
             if (a.features && rank == 0) a.features[(int64_t)b * N + lane] = v;
         }
-        if (lane == 0) s_d[warp] = d;
+        if (lane == 0) s_d[r] = d;
     }
     __syncthreads();
-    {   // first layer: thread j evaluates unit j for the four requests
-        float h1[kReqPerCluster] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (tid < H) {
+    {   // first layer: thread j evaluates unit j for every request of the cluster
 #pragma unroll
-            for (int r = 0; r < kReqPerCluster; ++r) {
-                if (r < nreq) {
-                    float phi[N];
+        for (int r = 0; r < REQ; ++r) {
+            float h1 = 0.0f;
+            if (tid < H && r < nreq) {
+                float phi[N];
 #pragma unroll
-                    for (int i = 0; i < N; ++i) phi[i] = s_phi[r][i];
-                    h1[r] = apply_first_layer(row1, phi);
-                }
+                for (int i = 0; i < N; ++i) phi[i] = s_phi[r][i];
+                h1 = apply_first_layer(row1, phi);
             }
+            s_h1[tid][r] = h1;
         }
-        *reinterpret_cast<float4*>(s_h1[tid]) = make_float4(h1[0], h1[1], h1[2], h1[3]);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();  // the slab and s_h1 are complete
-    {   // second layer: thread (r, jj) -> unit j = rank * 64 + jj of request r
-        const int r = tid / kColsPerCta, jj = tid % kColsPerCta;
+    {   // second layer: thread (r4, jj) -> unit j = rank * 64 + jj of requests r4, r4 + 4, ...
+        const int r4 = tid / kColsPerCta, jj = tid % kColsPerCta;
         const int j = rank * kColsPerCta + jj;
-        float acc = my_bh;
+        float acc[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) acc[g] = my_bh;
         // rows beyond H hold zero weights and zero activations: adding their products changes nothing,
-        // and a fixed trip count lets the shared-memory loads be issued ahead of the chain
+        // and a fixed trip count lets the shared-memory loads be issued ahead of the chains
         const float* w = s_w + jj;
-#pragma unroll 16
-        for (int i = 0; i < HVD_MAX_HIDDEN; ++i) acc = __fmaf_rn(w[i * kColsPerCta], s_h1[i][r], acc);
-        const float h2 = (j < H && r < nreq && acc > 0.0f) ? acc : 0.0f;
+#pragma unroll 8
+        for (int i = 0; i < HVD_MAX_HIDDEN; ++i) {
+            const float wv = w[i * kColsPerCta];
+#pragma unroll
+            for (int g = 0; g < G; ++g) acc[g] = __fmaf_rn(wv, s_h1[i][r4 + kReqPerGroup * g], acc[g]);
+        }
         float* dst = cluster.map_shared_rank(&s_h2[0][0], 0);  // CTA 0's copy
-        dst[r * kHidPad + j] = h2;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const int r = r4 + kReqPerGroup * g;
+            dst[r * kHidPad + j] = (j < H && r < nreq && acc[g] > 0.0f) ? acc[g] : 0.0f;
+        }
     }
     cluster.sync();  // all four slabs of activations have arrived in CTA 0
     if (rank != 0) return;
@@ -162,8 +180,10 @@ score_select2_kernel(const ScoreArgs a) {
         s_y[tid] = y;
     }
     __syncthreads();
-    if (warp < nreq) {
-        select_draft(a, b0 + warp, lane, s_y[warp], s_d[warp], ctok0, ctok1, md);
+#pragma unroll
+    for (int k = 0; k < RW; ++k) {
+        const int r = warp + k * NWARP;
+        if (r < nreq) select_draft(a, b0 + r, lane, s_y[r], s_d[r], ctok0[k], ctok1[k], md[k]);
     }
 }
 
@@ -191,14 +211,21 @@ template <bool EXT>
 static hvd_status launch_score_kernels(hvd_ctx* ctx, const ScoreArgs& a, int32_t B, cudaStream_t stream) {
     if (a.WhT) {
         bool& ready = EXT ? ctx->score2x_ready : ctx->score2_ready;
-        if (!ready) {  // per device: the kernel needs the opt-in shared memory size
-            HVD_CUDA_TRY(ctx, cudaFuncSetAttribute(score_select2_kernel<EXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)kScore2Smem));
+        if (!ready) {  // per device: the kernels need the opt-in shared memory size
+            HVD_CUDA_TRY(ctx, cudaFuncSetAttribute(score_select2_kernel<EXT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScore2Smem));
+            HVD_CUDA_TRY(ctx, cudaFuncSetAttribute(score_select2_kernel<EXT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScore2Smem));
+            HVD_CUDA_TRY(ctx, cudaFuncSetAttribute(score_select2_kernel<EXT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScore2Smem));
             ready = true;
         }
-        const int clusters = (B + kReqPerCluster - 1) / kReqPerCluster;
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, score_select2_kernel<EXT>, clusters * kClusterSize,
-                                        kScore2Threads, kScore2Smem, stream, a));
+        // requests per cluster: 4, 8 or 16, the fewest that keep the grid within one CTA per SM
+        const int G = B <= ctx->num_sms ? 1 : (B <= 2 * ctx->num_sms ? 2 : 4);
+        const int clusters = (B + kReqPerGroup * G - 1) / (kReqPerGroup * G);
+        const dim3 grid((unsigned)(clusters * kClusterSize));
+        cudaError_t e;
+        if (G == 1) e = launch_kernel(ctx->use_pdl, score_select2_kernel<EXT, 1>, grid, kScore2Threads, kScore2Smem, stream, a);
+        else if (G == 2) e = launch_kernel(ctx->use_pdl, score_select2_kernel<EXT, 2>, grid, kScore2Threads, kScore2Smem, stream, a);
+        else e = launch_kernel(ctx->use_pdl, score_select2_kernel<EXT, 4>, grid, kScore2Threads, kScore2Smem, stream, a);
+        HVD_CUDA_TRY(ctx, e);
         return HVD_OK;
     }
     const int blocks = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
