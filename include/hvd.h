@@ -212,8 +212,10 @@ HVD_API hvd_status hvd_lookup_score_select(hvd_ctx* ctx, int32_t B, const int32_
  * part of a match and ends a draft); m (HOST value) in [0, 2^31 - 2]; corpus = NULL or m = 0
  * unregisters.  Registration builds an index of the corpus (device memory of about 12 bytes per
  * token, kernels on the default stream) and returns when it is ready: a set-up call, not for the
- * decoding loop and not under stream capture.  Takes effect for later hvd_lookup_corpus calls on any
- * stream.  The index is keyed on the last min(min_match, 2) tokens of a match.
+ * decoding loop and not under stream capture; no hvd_lookup_corpus call of this context may be in
+ * flight.  Takes effect for later hvd_lookup_corpus calls on any stream.  The index is keyed on the
+ * last min(min_match, 2) tokens of a match.  Errors: HVD_ERR_INVALID_ARG (alignment, m),
+ * HVD_ERR_CUDA (allocation or build failed: no corpus is registered afterwards).
  *
  * hvd_lookup_corpus is hvd_lookup over [corpus, own history].  Candidates are the history positions
  * of hvd_lookup and the corpus positions e in [1, m-1] whose token corpus[e] is not a separator,
@@ -270,8 +272,9 @@ HVD_API hvd_status hvd_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist,
  * the trace's own continuation confirms.  Outputs (int32 [n], index t-1): label, draft_len, match_len,
  * match_pos, match_cnt.  trace: DEVICE, 16-byte aligned; n (HOST value) <= max_hist_len.  The first
  * call, and any call with a longer trace than before, allocates per-state scratch (268 bytes per
- * position) after waiting for the stream: not for use under stream capture.  These are the regression targets of the payoff predictor; the
- * recent-history features depend on the decoding loop and are not produced here.
+ * position) after waiting for the stream: not for use under stream capture.  These are the
+ * regression targets of the payoff predictor; the recent-history features depend on the decoding
+ * loop and are not produced here.  Uses context scratch: one call at a time per context.
  */
 HVD_API hvd_status hvd_replay_labels(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label,
                                      int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
