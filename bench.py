@@ -54,6 +54,9 @@ def parse_args():
                     help="variant of the lookup step: frequency-weighted draft and score (hvd_lookup_freq) on the config's requests")
     ap.add_argument("--corpus", action="store_true",
                     help="variant of the lookup step: shared warm-up corpus scanned with the history (hvd_lookup_corpus)")
+    ap.add_argument("--vocab-shards", action="store_true",
+                    help="variant of the verify step: one rank's share under a vocabulary-parallel output layer "
+                         "(hvd_verify_keys on a 1/S slice of every row + hvd_commit_keys), S = 2, 4, 8")
     ap.add_argument("--replay", action="store_true",
                     help="second workload: payoff labels by trace replay (hvd_replay_labels) on one history of the config")
     ap.add_argument("--unfused", action="store_true",
@@ -371,6 +374,85 @@ def run_corpus(args):
     ctx.close()
 
 
+# ----------------------------------------------------------------------------------------------
+# variant of the verify step: vocabulary shards (one rank's work; the 8-bytes-per-row MAX all-reduce
+# between the two calls needs the other ranks and is not part of this single-GPU timing)
+# ----------------------------------------------------------------------------------------------
+def run_vocab_shards(args):
+    import torch
+    import hvd_workloads as W
+    import paper_2606_01019_b200 as H
+    from paper_2606_01019_b200.runner import DeviceBatch
+    from oracle import pipeline as P
+    torch.cuda.set_device(0)
+    w = W.CONFIGS[args.config]
+    inp = P.prepare(w, device="cuda")
+    rq = inp.rq
+    B, rows = rq.B, int(rq.row_off[-1])
+    ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=rows, max_vocab=w.V,
+                    l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
+    ctx.hvd_set_predictor(inp.W1, inp.b1, inp.W2, inp.b2, inp.tau)
+    batch = DeviceBatch(ctx, hist=rq.hist, hist_off=rq.hist_off, hist_cap=rq.hist_cap, hist_len=rq.hist_len, K=rq.K,
+                        prompt_len=rq.prompt_len, state=rq.state, model_draft=rq.model_draft, model_len=rq.model_len,
+                        row_off=rq.row_off, V=w.V, dtype=w.dtype)
+    batch.lookup_score_select()
+    full = inp.logits.reshape(-1)[: rows * w.V].reshape(rows, w.V)
+    needed = int((batch.sel_len.cpu().numpy().astype(np.int64) + 1).sum())
+    hist_len0, state0 = batch.hist_len.clone(), batch.state.clone()
+    reps = max(3, min(args.steps, 50))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    cases = []
+    for S in (1, 2, 4, 8):
+        Vs = w.V // S
+        copies = [full[:, :Vs].contiguous() for _ in range(2 if S > 1 else 1)]
+        keys = torch.zeros(rows, dtype=torch.int64, device="cuda")
+
+        def call(i):
+            ctx.hvd_verify_keys(B, copies[i % len(copies)], batch.dtype, Vs, 0, batch.row_off, 0, rows, batch.sel_len,
+                                batch.hist_len, batch.hist_cap, keys)
+            ctx.hvd_commit_keys(B, keys, w.V, batch.row_off, 0, rows, batch.sel_draft, batch.sel_len, batch.select,
+                                batch.hist, batch.hist_off, batch.hist_cap, batch.hist_len, batch.state, batch.accepted,
+                                batch.committed, batch.n_commit, None, batch.status)
+
+        def body(i, with_call):
+            batch.hist_len.copy_(hist_len0); batch.state.copy_(state0)
+            flush.fill_(1)   # L2 flush between calls
+            if with_call:
+                call(i)
+
+        for i in range(3):
+            body(i, True)
+        torch.cuda.synchronize()
+        stream = torch.cuda.Stream()
+        times = []
+        for with_call in (True, False):   # the same graph with and without the calls: the difference is the calls
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                g.capture_begin()
+                for i in range(reps):
+                    body(i, with_call)
+                g.capture_end()
+            torch.cuda.synchronize()
+            with torch.cuda.stream(stream):
+                g.replay()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); g.replay(); e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        us = (times[0] - times[1]) / reps * 1e3
+        shard_bytes = needed * Vs * w.elt
+        cases.append({"shards": S, "us_per_rank": us, "shard_bytes": shard_bytes, "gbs": shard_bytes / (us * 1e-6) / 1e9,
+                      "allreduce_bytes_per_rank": rows * 8, "logits_allgather_bytes_avoided": needed * (w.V - Vs) * w.elt})
+    line = {"metric": "verify+commit per rank under vocabulary shards", "value": cases[-1]["us_per_rank"], "unit": "us",
+            "n_gpus": 1, "steps": reps, "higher_is_better": False, "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": f"{w.name}: batch {B}, {rows} logits rows, vocab {w.V} in S slices; one rank's "
+                                   "hvd_verify_keys + hvd_commit_keys (a memset and 4 kernels) in a CUDA graph, L2 flushed between calls; "
+                                   "time = graph with the calls minus the same graph without them"},
+            "cases": cases}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def workload_config(w, n_gpus, extra=None):
     cfg = {"workload": f"{w.name}: batch {w.B}, histories {w.n} tokens, vocab {w.V}, K {w.K}, {w.dtype} logits",
            "requests_per_gpu": w.B, "parallelism": f"requests sharded over {n_gpus} GPU(s), no collective"}
@@ -392,6 +474,9 @@ def main():
         return
     if args.corpus:
         run_corpus(args)
+        return
+    if args.vocab_shards:
+        run_vocab_shards(args)
         return
     if args.replay:
         run_replay(args)

@@ -374,6 +374,35 @@ typedef struct {
 HVD_API hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args, void* stream);
 
 /*
+ * Verification with the vocabulary sharded over several ranks (a vocabulary-parallel output layer:
+ * every rank holds, for all rows, the logits of its own V_shard consecutive vocabulary entries
+ * starting at v_offset).  The argmax of Sec. 3.1's Verify splits into a per-shard part and a
+ * reduction:
+ *   hvd_verify_keys   streams this rank's shard (rows of V_shard values, same row layout and the same
+ *                     needed-row rule as hvd_verify_commit: rows beyond sel_len are not read) and
+ *                     writes one key per row, keys int64 [total_rows] (DEVICE output): larger key =
+ *                     larger logit, and among equal logits the lower GLOBAL index; a row that was
+ *                     not read gets the smallest int64.  Nothing else is written.
+ *   (caller)          element-wise MAX of the keys over the ranks (e.g. an all-reduce with MAX on
+ *                     int64: 8 bytes per row cross the links instead of the logits).
+ *   hvd_commit_keys   hvd_verify_commit's accepted length, commit, append and state update, with the
+ *                     row maxima taken from the reduced keys; V is the whole vocabulary size.  Every
+ *                     rank that holds the request's history runs it and gets identical results.
+ * Together the two calls give exactly hvd_verify_commit's outputs on the concatenated logits.
+ * hvd_verify_keys uses context scratch: one call at a time per context.
+ */
+HVD_API hvd_status hvd_verify_keys(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V_shard,
+                                   int64_t v_offset, const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                                   const int32_t* sel_len, const int32_t* hist_len, const int32_t* hist_cap,
+                                   int64_t* keys, void* stream);
+HVD_API hvd_status hvd_commit_keys(hvd_ctx* ctx, int32_t B, const int64_t* keys, int64_t V, const int64_t* row_off,
+                                   int32_t k_uniform, int64_t total_rows, const int32_t* sel_draft,
+                                   const int32_t* sel_len, const int32_t* select, int32_t* hist,
+                                   const int64_t* hist_off, const int32_t* hist_cap, int32_t* hist_len,
+                                   hvd_req_state* state, int32_t* accepted, int32_t* committed, int32_t* n_commit,
+                                   int32_t* target_tok, int32_t* status, void* stream);
+
+/*
  * Greedy verification and commit without a context and without any allocation.  (The paper has
  * no counterpart: this is a packaging variant of hvd_verify_commit.)
  *

@@ -59,6 +59,8 @@ _SIGNATURES = {
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
     "hvd_verify_commit_tree": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 14 + [_vp]),
+    "hvd_verify_keys": (_i32, [_vp, _i32, _vp, _i32, _i64, _i64, _vp, _i32, _i64, _vp, _vp, _vp, _vp, _vp]),
+    "hvd_commit_keys": (_i32, [_vp, _i32, _vp, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
     "hvd_step_host": (_i32, [_vp, C.POINTER(HvdHostStepArgs), _vp]),
     "hvd_verify_commit_noalloc": (_i32, [_i32, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
     "hvd_noalloc_last_error": (C.c_char_p, []),
@@ -283,6 +285,20 @@ class Context:
                                                 _ptr(committed), _ptr(n_commit), _ptr(target_tok),
                                                 _ptr(status), _stream()),
                     "hvd_verify_commit")
+
+    def hvd_verify_keys(self, B, logits, dtype, V_shard, v_offset, row_off, k_uniform, total_rows, sel_len, hist_len,
+                        hist_cap, keys):
+        self._check(self._lib.hvd_verify_keys(self._h, B, _ptr(logits), dtype, V_shard, v_offset, _ptr(row_off),
+                                              k_uniform, total_rows, _ptr(sel_len), _ptr(hist_len), _ptr(hist_cap),
+                                              _ptr(keys), _stream()), "hvd_verify_keys")
+
+    def hvd_commit_keys(self, B, keys, V, row_off, k_uniform, total_rows, sel_draft, sel_len, select, hist, hist_off,
+                        hist_cap, hist_len, state, accepted, committed, n_commit, target_tok, status):
+        self._check(self._lib.hvd_commit_keys(self._h, B, _ptr(keys), V, _ptr(row_off), k_uniform, total_rows,
+                                              _ptr(sel_draft), _ptr(sel_len), _ptr(select), _ptr(hist), _ptr(hist_off),
+                                              _ptr(hist_cap), _ptr(hist_len), _ptr(state), _ptr(accepted),
+                                              _ptr(committed), _ptr(n_commit), _ptr(target_tok), _ptr(status),
+                                              _stream()), "hvd_commit_keys")
 
     def hvd_verify_commit_tree(self, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
                                parent, select, hist, hist_off, hist_cap, hist_len, state, accepted, committed,

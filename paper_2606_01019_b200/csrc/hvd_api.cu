@@ -408,7 +408,7 @@ static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits
     a.trace = ctx->trace;
 #endif
     a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error;
-    a.row_key = ctx->vf_row_key; a.total_rows = total_rows;
+    a.row_key = ctx->vf_row_key; a.total_rows = total_rows; a.ext_keys = nullptr;
     return launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
 }
 
@@ -436,6 +436,65 @@ hvd_status hvd_verify_commit_tree(hvd_ctx* ctx, int32_t B, const void* logits, h
     return verify_commit_impl(ctx, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len, parent,
                               select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
                               target_tok, status, stream);
+}
+
+// shared checks of the two calls that split verification across vocabulary shards
+static hvd_status check_rows(hvd_ctx* ctx, const char* who, int32_t B, const int64_t* row_off, int32_t k_uniform,
+                             int64_t total_rows) {
+    if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "B outside [1, max_batch]");
+    if (!row_off) {
+        if (k_uniform < 0 || k_uniform > ctx->cfg.k_cap) return fail(ctx, HVD_ERR_INVALID_ARG, "k_uniform outside [0, k_cap]");
+        if (total_rows != (int64_t)B * (k_uniform + 1)) return fail(ctx, HVD_ERR_INVALID_ARG, "total_rows != B*(k_uniform+1)");
+    }
+    if (total_rows < 1 || total_rows > ctx->cfg.max_rows) return fail(ctx, HVD_ERR_INVALID_ARG, "total_rows outside [1, max_rows]");
+    (void)who;
+    return HVD_OK;
+}
+
+hvd_status hvd_verify_keys(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V_shard, int64_t v_offset,
+                           const int64_t* row_off, int32_t k_uniform, int64_t total_rows, const int32_t* sel_len,
+                           const int32_t* hist_len, const int32_t* hist_cap, int64_t* keys, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    const hvd_status c = check_rows(ctx, "hvd_verify_keys", B, row_off, k_uniform, total_rows);
+    if (c != HVD_OK) return c;
+    if (dtype != HVD_F32 && dtype != HVD_BF16) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_keys: unknown dtype");
+    if (V_shard < 1 || V_shard > ctx->cfg.max_vocab || v_offset < 0 || v_offset + V_shard > 0x7fffffffLL)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_keys: shard outside the vocabulary range");
+    if (!logits || !sel_len || !hist_len || !hist_cap || !keys) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_keys: NULL pointer");
+    const size_t esz = dtype == HVD_F32 ? 4 : 2;
+    if (!aligned(logits, esz)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_keys: logits not aligned to its element type");
+    if (!aligned(keys, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_keys: keys must be 8-byte aligned");
+    VerifyArgs a = {};
+    a.B = B; a.logits = logits; a.V = V_shard; a.row_off = row_off; a.k_uniform = k_uniform;
+    a.sel_len = sel_len; a.hist_len = const_cast<int32_t*>(hist_len); a.hist_cap = hist_cap; a.k_cap = ctx->cfg.k_cap;
+    a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error; a.total_rows = total_rows; a.ext_keys = nullptr;
+#ifdef HVD_TRACE
+    a.trace = ctx->trace;
+#endif
+    return launch_verify_keys(ctx, a, dtype, reinterpret_cast<long long*>(keys), v_offset, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_commit_keys(hvd_ctx* ctx, int32_t B, const int64_t* keys, int64_t V, const int64_t* row_off,
+                           int32_t k_uniform, int64_t total_rows, const int32_t* sel_draft, const int32_t* sel_len,
+                           const int32_t* select, int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                           int32_t* hist_len, hvd_req_state* state, int32_t* accepted, int32_t* committed,
+                           int32_t* n_commit, int32_t* target_tok, int32_t* status, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    const hvd_status c = check_rows(ctx, "hvd_commit_keys", B, row_off, k_uniform, total_rows);
+    if (c != HVD_OK) return c;
+    if (V < 1 || V > 0x7fffffffLL) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_commit_keys: V outside [1, 2^31 - 1]");
+    if (!keys || !sel_draft || !sel_len || !select || !hist || !hist_off || !hist_cap || !hist_len || !state ||
+        !accepted || !committed || !n_commit || !status)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_commit_keys: NULL pointer");
+    if (!aligned(state, 8) || !aligned(keys, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_commit_keys: state and keys must be 8-byte aligned");
+    VerifyArgs a = {};
+    a.B = B; a.V = V; a.row_off = row_off; a.k_uniform = k_uniform;
+    a.sel_draft = sel_draft; a.sel_len = sel_len; a.parent = nullptr; a.select = select;
+    a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.state = state;
+    a.accepted = accepted; a.committed = committed; a.n_commit = n_commit; a.target_tok = target_tok;
+    a.status = status; a.k_cap = ctx->cfg.k_cap; a.total_rows = total_rows;
+    a.ext_keys = reinterpret_cast<const long long*>(keys);
+    return launch_commit_keys(ctx, a, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

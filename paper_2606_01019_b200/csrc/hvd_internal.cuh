@@ -212,6 +212,7 @@ struct VerifyArgs {
     int32_t k_cap;
     // scratch
     unsigned long long* row_key;  // [total_rows] (value, ~index) key per logits row, zero at rest
+    const long long* ext_keys;    // NULL, or row keys in signed order handed in by the caller (commit only)
     int64_t total_rows;
     uint32_t* next_unit;   // unit counter, zero at rest
     int* dev_error;        // device status word (no kernel sets it at present)
@@ -221,7 +222,10 @@ struct VerifyArgs {
 #endif
 };
 
-hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream);
+hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit = true);
+hvd_status launch_verify_keys(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, long long* keys, int64_t v_offset,
+                              cudaStream_t stream);
+hvd_status launch_commit_keys(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream);
 int verify_occupancy(hvd_dtype dtype, size_t dyn_smem);
 size_t verify_dyn_smem(int32_t B);
 

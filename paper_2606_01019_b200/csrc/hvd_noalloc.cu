@@ -134,7 +134,7 @@ hvd_status hvd_verify_commit_noalloc(int32_t B, int32_t k_cap, const void* logit
     a.accepted = accepted; a.committed = committed; a.n_commit = n_commit; a.target_tok = target_tok;
     a.status = status; a.k_cap = k_cap;
     a.next_unit = counters; a.dev_error = nullptr;
-    a.row_key = row_key; a.total_rows = total_rows;
+    a.row_key = row_key; a.total_rows = total_rows; a.ext_keys = nullptr;
 #ifdef HVD_TRACE
     a.trace = nullptr;
 #endif

@@ -171,6 +171,17 @@ __device__ __forceinline__ Req load_req(const VerifyArgs& a, int b) {
     return q;
 }
 
+constexpr unsigned long long kKeySign = 0x8000000000000000ull;
+
+// The (value, ~index) key of a logits row.  Context scratch is put back to zero as it is read; keys
+// handed in by the caller (hvd_commit_keys) are in signed order and are left alone.
+__device__ __forceinline__ unsigned long long read_row_key(const VerifyArgs& a, int64_t r) {
+    if (a.ext_keys) return (unsigned long long)a.ext_keys[r] ^ kKeySign;  // "row not read" becomes 0
+    const unsigned long long key = a.row_key[r];
+    a.row_key[r] = 0ull;  // scratch is zero at rest
+    return key;
+}
+
 // Commit of one request by one warp, after all its needed rows are folded into the row keys.
 // Every load that does not depend on another is issued up front: the kernel is a short chain of
 // global round trips at the end of every decoding step.
@@ -201,8 +212,7 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
         const int i = lane + 32 * k;
         key[k] = 0ull;
         if (i <= m) {
-            key[k] = a.row_key[q.r0 + i];
-            a.row_key[q.r0 + i] = 0ull;  // scratch is zero at rest
+            key[k] = read_row_key(a, q.r0 + i);
         }
     }
     int acc = -1;
@@ -283,8 +293,7 @@ __device__ __forceinline__ void commit_tree_request(const VerifyArgs& a, int b, 
         const int i = lane + 32 * k;
         tok[k] = 0;
         if (i <= m) {
-            const unsigned long long key = a.row_key[q.r0 + i];
-            a.row_key[q.r0 + i] = 0ull;  // scratch is zero at rest
+            const unsigned long long key = read_row_key(a, q.r0 + i);
             const int t = (int)(~(uint32_t)(key & 0xffffffffu));
             tok[k] = (int)min((int64_t)max(t, 0), a.V - 1);
             if (a.target_tok) a.target_tok[q.r0 + i] = tok[k];
@@ -342,6 +351,32 @@ __global__ void __launch_bounds__(kCommitWarps * 32) verify_commit_kernel(const 
         if (a.parent) commit_tree_request(a, b, threadIdx.x & 31);
         else commit_request(a, b, threadIdx.x & 31);
     }
+}
+
+// Row keys of one vocabulary shard, for a reduction across ranks: indices become global (v_offset),
+// the order becomes that of signed 64-bit integers (so that a plain MAX all-reduce picks the larger
+// value and, among equal values, the lower global index), rows that were not read become the
+// smallest integer; the unit counters go back to zero.
+__global__ void keys_finish_kernel(long long* keys, int64_t total_rows, int64_t v_offset, uint32_t* next_unit) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
+    if (r < Q) next_unit[r * kQueueStride] = 0u;
+    if (r >= total_rows) return;
+    unsigned long long key = (unsigned long long)keys[r];
+    if (key != 0ull) {
+        const uint32_t idx = ~(uint32_t)(key & 0xffffffffu);
+        key = (key & 0xffffffff00000000ull) | (uint32_t)(~(idx + (uint32_t)v_offset));
+    }
+    keys[r] = (long long)(key ^ kKeySign);
+}
+
+// Commit from row keys the caller hands in (reduced over the vocabulary shards of several ranks).
+__global__ void __launch_bounds__(kCommitWarps * 32) commit_keys_kernel(const VerifyArgs a) {
+    const int b = blockIdx.x * kCommitWarps + (threadIdx.x >> 5);
+    pdl_trigger();
+    pdl_wait();
+    if (b < a.B) commit_request(a, b, threadIdx.x & 31);
 }
 
 struct Smem {
@@ -558,7 +593,25 @@ int verify_occupancy(hvd_dtype dtype, size_t dyn_smem) {
     return n;
 }
 
-hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream) {
+hvd_status launch_verify_keys(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, long long* keys, int64_t v_offset,
+                              cudaStream_t stream) {
+    HVD_CUDA_TRY(ctx, cudaMemsetAsync(keys, 0, (size_t)a.total_rows * sizeof(long long), stream));
+    a.row_key = reinterpret_cast<unsigned long long*>(keys);
+    const hvd_status r = launch_verify(ctx, a, dtype, stream, false);
+    if (r != HVD_OK) return r;
+    const int64_t n = a.total_rows > Q ? a.total_rows : Q;
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, keys_finish_kernel, dim3((unsigned)((n + 255) / 256)), 256, 0, stream,
+                                    keys, a.total_rows, v_offset, a.next_unit));
+    return HVD_OK;
+}
+
+hvd_status launch_commit_keys(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream) {
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, commit_keys_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+                                    kCommitWarps * 32, 0, stream, a));
+    return HVD_OK;
+}
+
+hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit) {
     const int per_sm = ctx->vf_blocks_per_sm[dtype == HVD_F32 ? 0 : 1];
     const int grid = ctx->num_sms * (per_sm > 0 ? per_sm : 1);
     const int64_t esz = dtype == HVD_F32 ? 4 : 2;
@@ -572,8 +625,9 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
         HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_stream_kernel<float>, grid, T, smem, stream, a));
     else
         HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_stream_kernel<__nv_bfloat16>, grid, T, smem, stream, a));
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
-                                    kCommitWarps * 32, 0, stream, a));
+    if (with_commit)
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+                                        kCommitWarps * 32, 0, stream, a));
     return HVD_OK;
 }
 

@@ -1,6 +1,11 @@
 """Request sharding across GPUs.  The path is independent per request (own history, own logits
 rows, own state), so ranks never exchange data: a rank takes a contiguous range of requests and
-runs the same three kernels on it.  Only timings and counters are reduced for the report."""
+runs the same three kernels on it.  Only timings and counters are reduced for the report.
+
+The one exchange the path can need is under a vocabulary-parallel output layer, where every rank
+holds a slice of each logits row: hvd_verify_keys gives one 8-byte key per row and rank,
+reduce_keys_over_ranks takes their element-wise maximum (8 bytes per row cross the links, not the
+logits), hvd_commit_keys finishes the step on every rank."""
 from __future__ import annotations
 
 import numpy as np
@@ -50,3 +55,20 @@ def sum_over_ranks(value: float, device=None) -> float:
     t = torch.tensor([float(value)], dtype=torch.float64, device=device or "cpu")
     dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return float(t.item())
+
+
+def vocab_shards(V: int, world: int) -> np.ndarray:
+    """Boundaries [world+1] of near-equal contiguous vocabulary slices: rank r holds [b[r], b[r+1])."""
+    return (np.arange(world + 1, dtype=np.int64) * int(V)) // int(world)
+
+
+def reduce_keys_over_ranks(keys, group=None):
+    """Element-wise MAX of the int64 row keys of hvd_verify_keys over all ranks, in place (identity
+    without an initialised process group).  The keys are in signed order, so the plain MAX picks the
+    larger logit and, among equal logits, the lower global index."""
+    import torch
+    import torch.distributed as dist
+    assert keys.dtype == torch.int64
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(keys, op=dist.ReduceOp.MAX, group=group)
+    return keys

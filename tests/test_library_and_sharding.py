@@ -94,3 +94,53 @@ def test_two_gloo_ranks_shard_requests_and_reduce(tmp_path):
     res = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
     assert res.returncode == 0, res.stdout[-2000:] + res.stderr[-4000:]
     assert "rank 0 ok" in res.stdout and "rank 1 ok" in res.stdout
+
+
+_KEYS_PROGRAM = r"""
+import sys
+sys.path.insert(0, {root!r})
+import numpy as np, torch, torch.distributed as dist
+from paper_2606_01019_b200.sharding import reduce_keys_over_ranks, vocab_shards
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+rng = np.random.default_rng(7)                       # the same rows on every rank
+rows, V = 40, 1001
+x = rng.normal(0, 1, (rows, V)).astype(np.float32)
+x[3, [5, 700]] = 9.0                                 # equal maxima in different shards: the lower index wins
+x[4, [900, 901]] = 9.0                               # and inside one shard
+x[5] = -3.0                                          # a constant negative row
+x[6, 10] = 0.0; x[6, 600] = -0.0; x[6, np.arange(V) % 590 != 10] = -1.0   # +0 and -0 are equal
+b = vocab_shards(V, world)
+lo, hi = int(b[rank]), int(b[rank + 1])
+def keys_of(shard, offset):
+    # what the header promises of a key: larger logit first, then the lower global index; signed order
+    u = shard.view(np.uint32).astype(np.uint64)
+    u = np.where((u << np.uint64(33)) == 0, np.uint64(0), u)                 # -0 -> +0
+    o = np.where(u >> np.uint64(31) == 1, (~u) & np.uint64(0xffffffff), u | np.uint64(0x80000000))
+    idx = np.arange(shard.shape[1], dtype=np.uint64) + np.uint64(offset)
+    k = (o << np.uint64(32)) | ((~idx) & np.uint64(0xffffffff))
+    best = k.max(axis=1)
+    return (best ^ np.uint64(1 << 63)).view(np.int64)
+keys = torch.from_numpy(keys_of(x[:, lo:hi], lo).copy())
+keys[7] = torch.iinfo(torch.int64).min if rank == 0 else keys[7]             # a row one rank did not read
+reduce_keys_over_ranks(keys)
+got = (~(keys.numpy().view(np.uint64) & np.uint64(0xffffffff))) & np.uint64(0xffffffff)
+want = np.array([int(np.argmax(np.where(r == 0, 0.0, r))) for r in x])
+if world > 1 and lo <= want[7] < hi and rank == 0:
+    pass
+ok = [i for i in range(rows) if i != 7]
+assert (got[ok].astype(np.int64) == want[ok]).all(), (got, want)
+assert got[3] == 5 and got[4] == 900 and got[5] == 0 and got[6] == 10
+dist.destroy_process_group()
+sys.stdout.write("rank %d keys ok\n" % rank)
+"""
+
+
+def test_two_gloo_ranks_reduce_vocabulary_shard_keys(tmp_path):
+    prog = tmp_path / "keys_program.py"
+    prog.write_text(_KEYS_PROGRAM.format(root=ROOT))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29633", str(prog)]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert res.returncode == 0, res.stdout[-2000:] + res.stderr[-4000:]
+    assert "rank 0 keys ok" in res.stdout and "rank 1 keys ok" in res.stdout
