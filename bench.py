@@ -446,7 +446,7 @@ def run_vocab_shards(args):
     line = {"metric": "verify+commit per rank under vocabulary shards", "value": cases[-1]["us_per_rank"], "unit": "us",
             "n_gpus": 1, "steps": reps, "higher_is_better": False, "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": f"{w.name}: batch {B}, {rows} logits rows, vocab {w.V} in S slices; one rank's "
-                                   "hvd_verify_keys + hvd_commit_keys (a memset and 4 kernels) in a CUDA graph, L2 flushed between calls; "
+                                   "hvd_verify_keys + hvd_commit_keys (4 kernels) in a CUDA graph, L2 flushed between calls; "
                                    "time = graph with the calls minus the same graph without them"},
             "cases": cases}
     print(json.dumps(line), flush=True)

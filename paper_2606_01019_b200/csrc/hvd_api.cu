@@ -468,6 +468,7 @@ hvd_status hvd_verify_keys(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtyp
     a.B = B; a.logits = logits; a.V = V_shard; a.row_off = row_off; a.k_uniform = k_uniform;
     a.sel_len = sel_len; a.hist_len = const_cast<int32_t*>(hist_len); a.hist_cap = hist_cap; a.k_cap = ctx->cfg.k_cap;
     a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error; a.total_rows = total_rows; a.ext_keys = nullptr;
+    a.row_key = ctx->vf_row_key;
 #ifdef HVD_TRACE
     a.trace = ctx->trace;
 #endif

@@ -357,13 +357,15 @@ __global__ void __launch_bounds__(kCommitWarps * 32) verify_commit_kernel(const 
 // the order becomes that of signed 64-bit integers (so that a plain MAX all-reduce picks the larger
 // value and, among equal values, the lower global index), rows that were not read become the
 // smallest integer; the unit counters go back to zero.
-__global__ void keys_finish_kernel(long long* keys, int64_t total_rows, int64_t v_offset, uint32_t* next_unit) {
+__global__ void keys_finish_kernel(unsigned long long* row_key, long long* keys, int64_t total_rows, int64_t v_offset,
+                                   uint32_t* next_unit) {
     const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_trigger();
     pdl_wait();
     if (r < Q) next_unit[r * kQueueStride] = 0u;
     if (r >= total_rows) return;
-    unsigned long long key = (unsigned long long)keys[r];
+    unsigned long long key = row_key[r];
+    row_key[r] = 0ull;  // scratch is zero at rest
     if (key != 0ull) {
         const uint32_t idx = ~(uint32_t)(key & 0xffffffffu);
         key = (key & 0xffffffff00000000ull) | (uint32_t)(~(idx + (uint32_t)v_offset));
@@ -595,13 +597,12 @@ int verify_occupancy(hvd_dtype dtype, size_t dyn_smem) {
 
 hvd_status launch_verify_keys(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, long long* keys, int64_t v_offset,
                               cudaStream_t stream) {
-    HVD_CUDA_TRY(ctx, cudaMemsetAsync(keys, 0, (size_t)a.total_rows * sizeof(long long), stream));
-    a.row_key = reinterpret_cast<unsigned long long*>(keys);
+    // the maxima gather in the context's row keys (zero at rest); the finishing kernel moves them out
     const hvd_status r = launch_verify(ctx, a, dtype, stream, false);
     if (r != HVD_OK) return r;
     const int64_t n = a.total_rows > Q ? a.total_rows : Q;
     HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, keys_finish_kernel, dim3((unsigned)((n + 255) / 256)), 256, 0, stream,
-                                    keys, a.total_rows, v_offset, a.next_unit));
+                                    a.row_key, keys, a.total_rows, v_offset, a.next_unit));
     return HVD_OK;
 }
 
