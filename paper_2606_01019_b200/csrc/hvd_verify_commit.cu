@@ -161,10 +161,13 @@ __device__ __forceinline__ Req load_req(const VerifyArgs& a, int b) {
     Req q;
     if (a.row_off) { q.r0 = a.row_off[b]; q.r1 = a.row_off[b + 1]; }
     else { q.r0 = (int64_t)b * (a.k_uniform + 1); q.r1 = q.r0 + a.k_uniform + 1; }
+    // every input is fetched before any is looked at: one round trip, not a chain of three
     const int n = a.hist_len[b];
+    const int cap = a.hist_cap[b];
+    const int sl = a.sel_len[b];
     q.nr = 0;
-    if (n >= 0 && n <= a.hist_cap[b] && q.r1 > q.r0) {
-        int m = max(0, min(a.sel_len[b], a.k_cap));
+    if (n >= 0 && n <= cap && q.r1 > q.r0) {
+        int m = max(0, min(sl, a.k_cap));
         if ((int64_t)m > q.r1 - q.r0 - 1) m = (int)(q.r1 - q.r0 - 1);
         q.nr = m + 1;
     }
