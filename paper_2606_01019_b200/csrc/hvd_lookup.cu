@@ -77,10 +77,15 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
     pdl_trigger();
     pdl_wait();
 
+    // the request's scalars are fetched together, before any of them is looked at: the kernel is a chain
+    // of dependent round trips and this keeps them to one
     const int n_raw = a.hist_len[b];
+    const int cap_b = a.hist_cap[b];
+    const int64_t off_b = a.hist_off[b];
+    const int K_b = a.K[b];
     int n = n_raw;
-    if (n < 0 || n > a.hist_cap[b] || n > a.n_max) n = 0;  // unusable length: empty history
-    const int32_t* __restrict__ slab = a.hist + a.hist_off[b];
+    if (n < 0 || n > cap_b || n > a.n_max) n = 0;  // unusable length: empty history
+    const int32_t* __restrict__ slab = a.hist + off_b;
     // 128-bit loads run on the 16-byte grid; `mis` tokens of the first vector lie before the slab
     const int mis = (int)((reinterpret_cast<uintptr_t>(slab) >> 2) & 3);
     constexpr int CHUNK = THREADS * kLookupTokPerVec * ITER;  // tokens of the aligned grid per CTA
@@ -205,8 +210,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
     if (L < a.min_match || L == 0) {
         L = 0; e = -1; cnt = 0;
     } else {
-        int K = a.K[b];
-        K = max(0, min(K, a.k_cap));
+        const int K = max(0, min(K_b, a.k_cap));
         int lim = K;
         if (a.spec_factor > 0.0f) {
             // two separately rounded operations, as written: multiply, then add
@@ -217,12 +221,17 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
     }
     const int tok0 = lane < d ? slab[e + lane] : -1;
     const int tok1 = lane + 32 < d ? slab[e + lane + 32] : -1;
+    if (FUSED) {
+        // everything the scoring reads is requested before the lookup's own results are stored (a store
+        // would hold back the loads behind it): draft tokens, decode state and model draft in one round trip
+        const ModelDraft md = load_model_draft(sa, b, lane);
+        score_select_request(sa, b, lane, s_hid, n_raw, d, L, e, cnt, tok0, tok1, &md);
+    }
     if (lane < a.k_cap) a.draft[(int64_t)b * a.k_cap + lane] = tok0;
     if (lane + 32 < a.k_cap) a.draft[(int64_t)b * a.k_cap + lane + 32] = tok1;
     if (lane == 0) {
         a.draft_len[b] = d; a.match_len[b] = L; a.match_pos[b] = e; a.match_cnt[b] = cnt;
     }
-    if (FUSED) score_select_request(sa, b, lane, s_hid, n_raw, d, L, e, cnt, tok0, tok1);
 }
 
 }  // namespace

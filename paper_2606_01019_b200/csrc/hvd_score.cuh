@@ -174,7 +174,8 @@ __device__ __forceinline__ void select_draft(const ScoreArgs& a, int b, int lane
 // lookup results of the request; s_hid: shared memory, a.hidden floats, private to the warp.
 template <bool EXT = false>
 __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, int lane, float* s_hid, int n,
-                                                     int d, int L, int pos, int cnt, int tok0, int tok1) {
+                                                     int d, int L, int pos, int cnt, int tok0, int tok1,
+                                                     const ModelDraft* fetched = nullptr) {
     constexpr int N = NFeat<EXT>::value;
     d = max(0, min(d, a.k_cap));
     float phi[N];
@@ -193,7 +194,8 @@ __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, 
         for (int j = 0; j < a.hidden; ++j) y = __fmaf_rn(__ldg(a.W2 + j), s_hid[j], y);
     }
     y = __shfl_sync(0xffffffffu, y, 0);
-    select_draft(a, b, lane, y, d, tok0, tok1);
+    if (fetched) select_draft(a, b, lane, y, d, tok0, tok1, *fetched);  // the model draft was fetched ahead
+    else select_draft(a, b, lane, y, d, tok0, tok1);
 }
 
 }  // namespace hvd
