@@ -48,11 +48,20 @@ __device__ __forceinline__ uint32_t ord32(float f) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+// The logits are read once and are larger than the L2: they bypass the L1 and are marked to leave the
+// L2 first, so that what the other kernels of a step reuse (histories, per-request arrays, predictor
+// weights) is still there when the stream has passed.
+__device__ __forceinline__ unsigned long long stream_policy() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p, unsigned long long pol) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
+                 : "l"(p), "l"(pol));
     return v;
 }
 
@@ -468,6 +477,7 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
     const uint32_t n_big = (uint32_t)((total - (total >> HVD_VERIFY_ENDGAME_SHIFT)) / UB);
     const uint32_t n_units = n_big + (uint32_t)(total - (int64_t)n_big * UB);
     const char* base_ptr = static_cast<const char*>(a.logits);
+    const unsigned long long pol = stream_policy();
     TR(unsigned long long t_loop = gtime();)
 
     // ---- phase 1: units of batches -------------------------------------------------------------------
@@ -529,7 +539,7 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
             if (left >= kBatchVec) {
                 uint4 x[U];
 #pragma unroll
-                for (int u = 0; u < U; ++u) x[u] = ld_stream(ptr + u * 32);
+                for (int u = 0; u < U; ++u) x[u] = ld_stream(ptr + u * 32, pol);
                 Tracker<E> t;
                 t.init(x[0]);
 #pragma unroll
@@ -538,10 +548,10 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
                 loff += (uint32_t)(head + gb * kBatchVec * EPV);
             } else if (lane < left) {  // ragged last batch of the row
                 Tracker<E> t;
-                t.init(ld_stream(ptr));
+                t.init(ld_stream(ptr, pol));
 #pragma unroll
                 for (int u = 1; u < U; ++u)
-                    if (u * 32 + lane < left) t.fold(ld_stream(ptr + u * 32), u);
+                    if (u * 32 + lane < left) t.fold(ld_stream(ptr + u * 32, pol), u);
                 t.best(lane, lord, loff);
                 loff += (uint32_t)(head + gb * kBatchVec * EPV);
             }
