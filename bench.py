@@ -830,6 +830,11 @@ def main():
                 "mean_accepted": float(accepted_h.mean()), "cache_selected_frac": float(select_h.mean()),
                 "kernel_us": kt, "roofline": roofline, "roofline_lookup": roofline_lookup,
                 "lookup_algorithmic_bytes": lookup_bytes,
+                # the whole step against the same peak: history bytes scanned + logits bytes read, per rank
+                "roofline_step": {"bound": "hbm", "algorithmic_bytes_per_step": lookup_bytes + verify_bytes,
+                                  "achieved": (lookup_bytes + verify_bytes) / (elapsed_ms / K_steps * 1e-3) / 1e9,
+                                  "peak": peak_gbs, "unit": "GB/s", "peak_kind": peak_kind,
+                                  "frac": (lookup_bytes + verify_bytes) / (elapsed_ms / K_steps * 1e-3) / 1e9 / peak_gbs},
                 "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": (4 if args.unfused else 3) * K_steps,
                 "clocks": sampler.summary(window)}
         print(json.dumps(line), flush=True)
