@@ -15,9 +15,15 @@
  * Conventions
  *  - Unless an argument is marked HOST, every pointer is a DEVICE pointer owned
  *    by the caller.  The library never frees caller memory and keeps no
- *    reference to it after the call returns.
+ *    reference to it after the call returns; the two registration calls
+ *    (hvd_set_corpus, hvd_set_token_classes) say so where they do.
  *  - Device entry points only enqueue work on `stream` (a cudaStream_t passed
- *    as void*, NULL = default stream) and never synchronise.
+ *    as void*, NULL = default stream) and never synchronise.  The set-up calls
+ *    (hvd_create, hvd_set_predictor*, hvd_set_corpus), hvd_step_host and the
+ *    first hvd_replay_labels call for a longer trace do wait, and say so.
+ *  - Variants of the three steps (two-layer and extended predictors, token
+ *    trees, frequency-weighted drafts, a shared warm-up corpus, vocabulary
+ *    shards, trace replay) are declared next to the step they vary.
  *  - Errors the host can see (NULL pointer, sizes outside the limits given at
  *    hvd_create, unknown dtype, misaligned base pointer) are returned at once
  *    and nothing is enqueued.  Data-dependent problems are reported per
