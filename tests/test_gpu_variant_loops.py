@@ -128,3 +128,52 @@ def test_variants_at_full_size(name):
     G.compare_lookup(g, lk)
     G.assert_equal("match_src", g["match_src"], lk.match_src)
     ctx.close()
+
+
+def test_variants_at_the_maximum_batch():
+    """8192 requests (the largest batch a context takes) with short histories through every variant entry
+    point: grids, per-request scratch and the 16-requests-per-cluster scoring at their limits."""
+    import torch
+    from tests.test_gpu_edge_cases import hand_requests, small
+    B = 8192
+    w = small(V=61, k_cap=8, hidden=256).scaled(B=B)
+    rng = np.random.default_rng(21)
+    hists = [rng.integers(0, 4, int(n)) for n in rng.integers(0, 90, B)]
+    rq = hand_requests(w, hists, rng.integers(0, 9, B))
+    ctx = G.make_ctx(w, rq)
+    batch = G.make_batch(ctx, w, rq)
+    args = (rq.hist, rq.hist_off, rq.hist_cap, rq.hist_len, rq.K)
+    kw = dict(k_cap=w.k_cap, l_max=w.l_max, min_match=w.min_match, nthreads=16)
+    # frequency-weighted lookup with selection
+    batch.lookup_freq(0.1, 128, 3.0)
+    g = batch.download()
+    fq = O.lookup_freq(*args, min_prob=0.1, max_occ=128, **kw)
+    G.compare_lookup(g, fq)
+    G.assert_equal("freq score bits", g["freq_score"].view(np.uint32), fq.score.view(np.uint32))
+    sel, sd, sl = O.freq_select(fq, 3.0, rq.model_draft, rq.model_len)
+    for k, v in (("select", sel), ("sel_draft", sd), ("sel_len", sl)):
+        G.assert_equal(k, g[k], v)
+    # corpus lookup
+    corpus = np.concatenate([rng.integers(0, 4, 3000), [-1], rng.integers(0, 4, 2000)]).astype(np.int32)
+    corpus_d = torch.as_tensor(corpus, device="cuda")
+    ctx.hvd_set_corpus(corpus_d)
+    batch.lookup_corpus()
+    g = batch.download()
+    lk = O.lookup_corpus(*args, corpus, **kw)
+    G.compare_lookup(g, lk)
+    G.assert_equal("match_src", g["match_src"], lk.match_src)
+    # extended features, two hidden layers (sixteen requests per cluster)
+    cls = rng.integers(0, 32, w.V).astype(np.uint8)
+    H = w.hidden
+    W1 = rng.normal(0, 0.1, (H, 14)).astype(f32); b1 = rng.normal(0, 0.1, H).astype(f32); W2 = rng.normal(0, 0.1, H).astype(f32)
+    Wh = rng.normal(0, 0.1, (H, H)).astype(f32); bh = rng.normal(0, 0.1, H).astype(f32)
+    cls_d = torch.as_tensor(cls, device="cuda")
+    ctx.hvd_set_token_classes(cls_d)
+    ctx.hvd_set_predictor_ext(W1, b1, W2, 6.0, 6.0, Wh, bh)
+    batch.score_select_ext(src=True)
+    g = batch.download()
+    sc = O.score_select_ext(rq.hist_len, rq.prompt_len, rq.state, rq.K, lk, None, cls, rq.model_draft, rq.model_len,
+                            k_cap=w.k_cap, W1=W1, b1=b1, W2=W2, b2=6.0, tau=6.0, Wh=Wh, bh=bh, nthreads=16, match_src=lk.match_src)
+    g["features"] = g["features_ext"]
+    G.compare_score(g, sc, 6.0)
+    ctx.close()
