@@ -93,7 +93,9 @@ struct hvd_ctx {
     int* dev_error;                  // device status word
     int vf_blocks_per_sm[2];         // per dtype
     // device staging of the host-buffer entry point (grown on demand)
-    bool use_pdl;  // programmatic dependent launch between the kernels of the path
+    bool use_pdl;     // programmatic dependent launch for every kernel of the library (HVD_ENABLE_PDL; experiments)
+    int pdl_mask;     // ... for the three kernels of a step: bit 0 commit, 1 lookup, 2 stream (default all)
+    bool pdl_commit;  // bit 0 of the mask
     char* host_ws;
     size_t host_ws_bytes;
 #ifdef HVD_TRACE

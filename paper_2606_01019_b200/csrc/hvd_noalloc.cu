@@ -59,6 +59,8 @@ hvd_status setup_device(int device, DeviceSetup** out, const char** why) {
             return HVD_ERR_UNSUPPORTED;
         }
         s.ctx.use_pdl = false;
+        s.ctx.pdl_commit = false;
+        s.ctx.pdl_mask = 0;
         s.ready = true;
     }
     *out = &s;

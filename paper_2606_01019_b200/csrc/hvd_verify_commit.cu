@@ -217,6 +217,7 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
         return;
     }
     const int m = q.nr - 1;
+    pdl_wait();  // everything above was the request's own data; the row keys come from the streaming kernel
     // rows lane, lane+32, lane+64 (at most 65 rows): target tokens from the row keys
     unsigned long long key[3];
 #pragma unroll
@@ -299,6 +300,7 @@ __device__ __forceinline__ void commit_tree_request(const VerifyArgs& a, int b, 
         return;
     }
     const int m = q.nr - 1;
+    pdl_wait();
     int tok[3];  // target tokens of rows lane, lane+32, lane+64
 #pragma unroll
     for (int k = 0; k < 3; ++k) {
@@ -357,12 +359,14 @@ constexpr int kCommitWarps = 4;
 __global__ void __launch_bounds__(kCommitWarps * 32) verify_commit_kernel(const VerifyArgs a) {
     const int b = blockIdx.x * kCommitWarps + (threadIdx.x >> 5);
     pdl_trigger();
-    pdl_wait();
-    if (b == 0 && (threadIdx.x & 31) < Q) a.next_unit[(threadIdx.x & 31) * kQueueStride] = 0u;  // zero at rest
+    // launched ahead of the streaming kernel's end when the launch allows it: the request's own data is
+    // fetched at once, the wait for the row keys sits inside the commit
     if (b < a.B) {
         if (a.parent) commit_tree_request(a, b, threadIdx.x & 31);
         else commit_request(a, b, threadIdx.x & 31);
     }
+    pdl_wait();
+    if (b == 0 && (threadIdx.x & 31) < Q) a.next_unit[(threadIdx.x & 31) * kQueueStride] = 0u;  // zero at rest
 }
 
 // Row keys of one vocabulary shard, for a reduction across ranks: indices become global (v_offset),
@@ -426,8 +430,10 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
     constexpr int EPV = Tracker<E>::kPerVec;
     constexpr int ESZ = 16 / EPV;
     TR(unsigned long long t_enter = gtime(); unsigned long long acc_wait = 0, acc_str = 0, acc_close = 0, n_b = 0;)
-    pdl_trigger();
+    // wait first, then let the commit kernel in: it reads the selection before its own wait, so it must not
+    // start before the kernel that wrote the selection (this kernel's predecessor) is known to be complete
     pdl_wait();
+    pdl_trigger();
 
     // Unit u belongs to queue u % Q.  The first unit of a warp is the one with its own number
     // (queue warp % Q); the next one is requested now and its answer is looked at after the first
@@ -636,11 +642,11 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
         return fail(ctx, HVD_ERR_UNSUPPORTED, "hvd_verify_commit: too many batches");
     const size_t smem = verify_dyn_smem(a.B);
     if (dtype == HVD_F32)
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_stream_kernel<float>, grid, T, smem, stream, a));
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 4), verify_stream_kernel<float>, grid, T, smem, stream, a));
     else
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_stream_kernel<__nv_bfloat16>, grid, T, smem, stream, a));
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 4), verify_stream_kernel<__nv_bfloat16>, grid, T, smem, stream, a));
     if (with_commit)
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || ctx->pdl_commit, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
                                         kCommitWarps * 32, 0, stream, a));
     return HVD_OK;
 }
