@@ -100,9 +100,10 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->has_predictor_ext = false;
     c->two_layer = false;
     c->score2_ready = false;
-    // programmatic dependent launch of the three kernels of a step (bit 0 commit, 1 lookup, 2 stream): the next
-    // kernel's CTAs are resident and past their prologue when the previous one ends; HVD_PDL_MASK=0 turns it off
-    c->pdl_mask = getenv("HVD_PDL_MASK") ? atoi(getenv("HVD_PDL_MASK")) : 7;
+    // programmatic dependent launch of the kernels of a step (bit 0 commit, 1 lookup, 2 stream, 3 one-layer
+    // scoring): the next kernel's CTAs are resident and past their prologue when the previous one ends;
+    // HVD_PDL_MASK=0 turns it off
+    c->pdl_mask = getenv("HVD_PDL_MASK") ? atoi(getenv("HVD_PDL_MASK")) : 15;
     c->pdl_commit = (c->pdl_mask & 1) != 0;
     c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // measured: no gain on this path, off unless asked for
     c->host_ws = nullptr;

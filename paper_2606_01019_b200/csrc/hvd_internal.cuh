@@ -94,7 +94,7 @@ struct hvd_ctx {
     int vf_blocks_per_sm[2];         // per dtype
     // device staging of the host-buffer entry point (grown on demand)
     bool use_pdl;     // programmatic dependent launch for every kernel of the library (HVD_ENABLE_PDL; experiments)
-    int pdl_mask;     // ... for the three kernels of a step: bit 0 commit, 1 lookup, 2 stream (default all)
+    int pdl_mask;     // ... for the three kernels of a step: bit 0 commit, 1 lookup, 2 stream, 3 one-layer scoring (default all)
     bool pdl_commit;  // bit 0 of the mask
     char* host_ws;
     size_t host_ws_bytes;
