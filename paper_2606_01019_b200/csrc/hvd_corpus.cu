@@ -151,6 +151,7 @@ struct CorpusArgs {
 __device__ __forceinline__ void corpus_merge_request(const CorpusArgs& a, int b, int lane) {
     const int32_t* __restrict__ corpus = a.corpus;
     const int m = a.m;
+    pdl_wait();  // the history lookup's result is needed from here on
     __threadfence();
     const unsigned long long key = __ldcg(a.key + b);
     int Lc = (int)(key >> 32);
@@ -200,8 +201,10 @@ __global__ void __launch_bounds__(kProbeThreads) corpus_probe_kernel(const Corpu
     const int lane = tid & 31;
     const int warp = tid >> 5;
     const int32_t* __restrict__ corpus = a.corpus;
+    // Launched behind the history lookup, this kernel does not wait for it until the merge: the search of the
+    // corpus reads only what was there before that lookup started (histories, lengths, the index), so the two
+    // searches run side by side.
     pdl_trigger();
-    pdl_wait();
     int n = a.hist_len[b];
     if (n < 0 || n > a.hist_cap[b] || n > a.n_max) n = 0;
     if (tid < HVD_MAX_L) s_q[tid] = (tid < n) ? a.hist[a.hist_off[b] + n - 1 - tid] : -1;
@@ -330,7 +333,7 @@ hvd_status launch_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, co
                                 int32_t* draft, int32_t* draft_len, int32_t* match_len, int32_t* match_pos,
                                 int32_t* match_src, int32_t* match_cnt, cudaStream_t stream) {
     const hvd_status r = launch_lookup(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, draft, draft_len,
-                                       match_len, match_pos, match_cnt, nullptr, stream);
+                                       match_len, match_pos, match_cnt, nullptr, stream, ctx->cp_start != nullptr);
     if (r != HVD_OK) return r;
     if (ctx->cp_start == nullptr) {
         HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, corpus_none_kernel, dim3((unsigned)((B + 255) / 256)), 256, 0,
@@ -349,7 +352,7 @@ hvd_status launch_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, co
     a.draft = draft; a.draft_len = draft_len; a.match_len = match_len; a.match_pos = match_pos;
     a.match_src = match_src; a.match_cnt = match_cnt;
     a.key = ctx->cp_key; a.cnt = ctx->cp_cnt; a.arrived = ctx->cp_arrived;
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, corpus_probe_kernel, dim3((unsigned)a.slices, (unsigned)B),
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || ctx->pdl_mask != 0, corpus_probe_kernel, dim3((unsigned)a.slices, (unsigned)B),
                                     kProbeThreads, 0, stream, a));
     return HVD_OK;
 }

@@ -150,7 +150,8 @@ struct ScoreArgs;  // hvd_score.cuh
 hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
                          const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
                          int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
-                         int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream);
+                         int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream,
+                         bool successor_works_ahead = false);
 
 ScoreArgs make_score_args(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
                           const hvd_req_state* state, const int32_t* K, const int32_t* draft,

@@ -30,6 +30,7 @@ struct LookupArgs {
     int32_t max_chunks;
     int32_t k_cap, l_max, min_match;
     float spec_factor, spec_offset;
+    bool successor_works_ahead;
 };
 
 struct Best {
@@ -74,8 +75,13 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    pdl_trigger();
+    // The next kernel may come in at once when it does nothing ahead of its own wait.  A successor that does
+    // (the corpus probe reads the histories there) must not start before this kernel's predecessor, which may
+    // have written them, is known to be complete: then the wait comes first.
+    const bool late = !FUSED && a.successor_works_ahead;  // the fused form is never followed by such a kernel
+    if (!late) pdl_trigger();
     pdl_wait();
+    if (late) pdl_trigger();
 
     // the request's scalars are fetched together, before any of them is looked at: the kernel is a chain
     // of dependent round trips and this keeps them to one
@@ -239,8 +245,10 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
 hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int64_t* hist_off,
                          const int32_t* hist_cap, const int32_t* hist_len, const int32_t* K,
                          int32_t n_max, int32_t* draft, int32_t* draft_len, int32_t* match_len,
-                         int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream) {
+                         int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream,
+                         bool successor_works_ahead) {
     LookupArgs a;
+    a.successor_works_ahead = successor_works_ahead;
     a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.K = K;
     a.n_max = n_max;
     a.draft = draft; a.draft_len = draft_len; a.match_len = match_len; a.match_pos = match_pos;
