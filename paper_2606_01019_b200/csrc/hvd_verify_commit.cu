@@ -620,7 +620,7 @@ hvd_status launch_verify_keys(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, long 
     const hvd_status r = launch_verify(ctx, a, dtype, stream, false);
     if (r != HVD_OK) return r;
     const int64_t n = a.total_rows > Q ? a.total_rows : Q;
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, keys_finish_kernel, dim3((unsigned)((n + 255) / 256)), 256, 0, stream,
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || ctx->pdl_mask != 0, keys_finish_kernel, dim3((unsigned)((n + 255) / 256)), 256, 0, stream,
                                     a.row_key, keys, a.total_rows, v_offset, a.next_unit));
     return HVD_OK;
 }
