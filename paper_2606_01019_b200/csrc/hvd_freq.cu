@@ -16,7 +16,7 @@
 //            occurrences that continue with that token.
 // Requests with more occurrences than the list holds follow the latest occurrence only (every
 // token then has probability 1), exactly like the plain lookup.
-#include "hvd_internal.cuh"
+#include "hvd_scan.cuh"
 
 namespace hvd {
 namespace {
@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(kCollectThreads) freq_collect_kernel(const Fre
 #pragma unroll
     for (int i = 0; i < kCollectIter; ++i) {
         const int v = v0 + i * kCollectThreads + tid;
-        x[i] = (4 * v < g_end) ? __ldg(vbase + v) : make_int4(0, 0, 0, 0);
+        x[i] = (4 * v < g_end) ? ld_hist(vbase + v) : make_int4(0, 0, 0, 0);
     }
     const int32_t q0 = slab[n - 1];
     const int32_t qa = (1 + lane <= n - 1) ? slab[n - 2 - lane] : 0;
@@ -94,40 +94,12 @@ __global__ void __launch_bounds__(kCollectThreads) freq_collect_kernel(const Fre
 #pragma unroll
     for (int i = 0; i < kCollectIter; ++i) {
         const int p0 = 4 * (v0 + i * kCollectThreads + tid) - mis;
-        uint32_t m = 0;
-        m |= (x[i].x == q0 && p0 + 0 >= 0 && p0 + 0 <= n - 2) ? 1u : 0u;
-        m |= (x[i].y == q0 && p0 + 1 >= 0 && p0 + 1 <= n - 2) ? 2u : 0u;
-        m |= (x[i].z == q0 && p0 + 2 >= 0 && p0 + 2 <= n - 2) ? 4u : 0u;
-        m |= (x[i].w == q0 && p0 + 3 >= 0 && p0 + 3 <= n - 2) ? 8u : 0u;
-        uint32_t hits = __ballot_sync(0xffffffffu, m != 0);
-        while (hits) {
-            const int src = __ffs(hits) - 1;
-            hits &= hits - 1;
-            uint32_t ms = __shfl_sync(0xffffffffu, m, src);
-            const int ps = __shfl_sync(0xffffffffu, p0, src);
-            while (ms) {
-                const int k = __ffs(ms) - 1;
-                ms &= ms - 1;
-                const int p = ps + k;  // last token of the matched copy; the continuation starts at p + 1
-                const int cap = min(a.l_max, p + 1);
-                int l = lane + 1;
-                bool eq = (l < cap) && (slab[p - l] == qa);
-                uint32_t mm = __ballot_sync(0xffffffffu, !eq);
-                int L;
-                if (mm != 0) {
-                    L = __ffs(mm);
-                } else {
-                    l = lane + 33;
-                    eq = (l < cap) && (slab[p - l] == qb);
-                    mm = __ballot_sync(0xffffffffu, !eq);
-                    L = 32 + __ffs(mm);
-                }
-                if (L == Lstar && lane == 0) {
-                    const uint32_t idx = atomicAdd(a.occ_cnt + b, 1u);
-                    if (idx < (uint32_t)HVD_FREQ_MAX_OCC) a.occ[(int64_t)b * HVD_FREQ_MAX_OCC + idx] = p + 1;
-                }
+        scan_vector(x[i], p0, n, slab, q0, qa, qb, a.l_max, lane, [&](int L, int p) {
+            if (L == Lstar && lane == 0) {  // the continuation of the copy that ends at p starts at p + 1
+                const uint32_t idx = atomicAdd(a.occ_cnt + b, 1u);
+                if (idx < (uint32_t)HVD_FREQ_MAX_OCC) a.occ[(int64_t)b * HVD_FREQ_MAX_OCC + idx] = p + 1;
             }
-        }
+        });
     }
 }
 

@@ -8,6 +8,7 @@
 // minimum-length and draft-length rules and copies the draft -- and, in the fused form, goes
 // straight on to the payoff features, the predictor and the draft selection of that request
 // (one kernel and one global round trip less per decoding step).  No CTA waits for another.
+#include "hvd_scan.cuh"
 #include "hvd_score.cuh"
 
 namespace hvd {
@@ -56,14 +57,6 @@ __device__ __forceinline__ Best warp_combine(Best v) {
         o.cnt = __shfl_xor_sync(0xffffffffu, v.cnt, off);
         v = combine(v, o);
     }
-    return v;
-}
-
-__device__ __forceinline__ int4 ld_hist(const int4* p) {
-    int4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
     return v;
 }
 
@@ -132,41 +125,12 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
 #pragma unroll
     for (int i = 0; i < ITER; ++i) {
         const int p0 = 4 * (v0 + i * THREADS + tid) - mis;  // position of x[i].x
-        uint32_t m = 0;
-        m |= (x[i].x == q0 && p0 + 0 >= 0 && p0 + 0 <= n - 2) ? 1u : 0u;
-        m |= (x[i].y == q0 && p0 + 1 >= 0 && p0 + 1 <= n - 2) ? 2u : 0u;
-        m |= (x[i].z == q0 && p0 + 2 >= 0 && p0 + 2 <= n - 2) ? 4u : 0u;
-        m |= (x[i].w == q0 && p0 + 3 >= 0 && p0 + 3 <= n - 2) ? 8u : 0u;
-        uint32_t hits = __ballot_sync(0xffffffffu, m != 0);
-        while (hits) {
-            const int src = __ffs(hits) - 1;
-            hits &= hits - 1;
-            uint32_t ms = __shfl_sync(0xffffffffu, m, src);
-            const int ps = __shfl_sync(0xffffffffu, p0, src);
-            while (ms) {
-                const int k = __ffs(ms) - 1;
-                ms &= ms - 1;
-                const int p = ps + k;
-                // match length of the copy ending at p (>= 1 already); limit: l_max and the slab start
-                const int cap = min(a.l_max, p + 1);
-                int l = lane + 1;
-                bool eq = (l < cap) && (slab[p - l] == qa);
-                uint32_t mm = __ballot_sync(0xffffffffu, !eq);
-                int L;
-                if (mm != 0) {
-                    L = __ffs(mm);  // first failing lane j: lengths 1..j hold, so L = 1 + j
-                } else {
-                    l = lane + 33;
-                    eq = (l < cap) && (slab[p - l] == qb);
-                    mm = __ballot_sync(0xffffffffu, !eq);  // lane 31 (l = 64) always fails
-                    L = 32 + __ffs(mm);
-                }
-                Best c;
-                c.key = ((unsigned long long)(uint32_t)L << 32) | (uint32_t)(p + 1);
-                c.cnt = 1;
-                best = combine(best, c);
-            }
-        }
+        scan_vector(x[i], p0, n, slab, q0, qa, qb, a.l_max, lane, [&](int L, int p) {
+            Best c;
+            c.key = ((unsigned long long)(uint32_t)L << 32) | (uint32_t)(p + 1);
+            c.cnt = 1;
+            best = combine(best, c);
+        });
     }
 
     __shared__ unsigned long long s_key[THREADS / 32];

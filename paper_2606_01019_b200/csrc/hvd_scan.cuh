@@ -1,0 +1,61 @@
+// The inner step of the history scan, shared by the lookup kernel and by the kernel that collects the
+// occurrences of the longest match: one 128-bit vector of history tokens per lane, candidates are the
+// positions that hold the history's last token, and the warp that finds one extends the match backwards
+// together (lane j compares the token j + 1 back; ballot + find-first-set gives the length, a second
+// round covers lengths 33 to 64).
+#pragma once
+
+#include "hvd_internal.cuh"
+
+namespace hvd {
+
+__device__ __forceinline__ int4 ld_hist(const int4* p) {
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// x: this lane's four tokens at positions p0 .. p0 + 3 of a history of n tokens (slab); q0 its last token,
+// qa / qb the tokens 1 + lane and 33 + lane back.  Calls on_match(L, p), in every lane of the warp with the
+// same arguments, for every candidate p in [0, n - 2] of the warp's 32 vectors: p holds q0 and L >= 1 is the
+// match length of the copy that ends there (capped at l_max and at the slab start).
+template <class OnMatch>
+__device__ __forceinline__ void scan_vector(const int4 x, int p0, int n, const int32_t* __restrict__ slab, int32_t q0,
+                                            int32_t qa, int32_t qb, int l_max, int lane, OnMatch&& on_match) {
+    uint32_t m = 0;
+    m |= (x.x == q0 && p0 + 0 >= 0 && p0 + 0 <= n - 2) ? 1u : 0u;
+    m |= (x.y == q0 && p0 + 1 >= 0 && p0 + 1 <= n - 2) ? 2u : 0u;
+    m |= (x.z == q0 && p0 + 2 >= 0 && p0 + 2 <= n - 2) ? 4u : 0u;
+    m |= (x.w == q0 && p0 + 3 >= 0 && p0 + 3 <= n - 2) ? 8u : 0u;
+    uint32_t hits = __ballot_sync(0xffffffffu, m != 0);
+    while (hits) {
+        const int src = __ffs(hits) - 1;
+        hits &= hits - 1;
+        uint32_t ms = __shfl_sync(0xffffffffu, m, src);
+        const int ps = __shfl_sync(0xffffffffu, p0, src);
+        while (ms) {
+            const int k = __ffs(ms) - 1;
+            ms &= ms - 1;
+            const int p = ps + k;
+            // match length of the copy ending at p (>= 1 already); limit: l_max and the slab start
+            const int cap = min(l_max, p + 1);
+            int l = lane + 1;
+            bool eq = (l < cap) && (slab[p - l] == qa);
+            uint32_t mm = __ballot_sync(0xffffffffu, !eq);
+            int L;
+            if (mm != 0) {
+                L = __ffs(mm);  // first failing lane j: lengths 1..j hold, so L = 1 + j
+            } else {
+                l = lane + 33;
+                eq = (l < cap) && (slab[p - l] == qb);
+                mm = __ballot_sync(0xffffffffu, !eq);  // lane 31 (l = 64) always fails
+                L = 32 + __ffs(mm);
+            }
+            on_match(L, p);
+        }
+    }
+}
+
+}  // namespace hvd
