@@ -167,13 +167,7 @@ __device__ __forceinline__ void corpus_merge_request(const CorpusArgs& a, int b,
     } else if (Lc == Lh) {  // the history comes first; the corpus occurrences are counted
         if (lane == 0) { a.match_src[b] = 0; a.match_cnt[b] = a.match_cnt[b] + cc; }
     } else {
-        int K = max(0, min(a.K[b], a.k_cap));
-        int lim = K;
-        if (a.spec_factor > 0.0f) {
-            const float f = __fadd_rn(__fmul_rn(a.spec_factor, (float)Lc), a.spec_offset);
-            lim = max(0, (int)floorf(f));
-        }
-        int d = min(min(K, lim), m - ec);
+        int d = min(draft_limit(a.K[b], a.k_cap, Lc, a.spec_factor, a.spec_offset), m - ec);
         int tok0 = lane < d ? corpus[ec + lane] : 0;
         int tok1 = lane + 32 < d ? corpus[ec + lane + 32] : 0;
         // a separator ends the draft

@@ -235,14 +235,7 @@ __global__ void __launch_bounds__(kWalkThreads) freq_walk_kernel(const FreqArgs 
     const int cnt = a.match_cnt[b];
     const int32_t* __restrict__ slab = a.hist + a.hist_off[b];
 
-    int limit = 0;
-    if (L > 0) {
-        limit = max(0, min(a.K[b], kc));
-        if (a.spec_factor > 0.0f) {
-            const float f = __fadd_rn(__fmul_rn(a.spec_factor, (float)L), a.spec_offset);
-            limit = min(limit, max(0, (int)floorf(f)));
-        }
-    }
+    const int limit = L > 0 ? draft_limit(a.K[b], kc, L, a.spec_factor, a.spec_offset) : 0;
     // 2 .. max_occ occurrences are merged; one occurrence, or too many, is the lookup's own draft
     const bool merged = (L > 0) && (cnt >= 2) && (cnt <= a.max_occ);
     const int c = merged ? min(cnt, HVD_FREQ_MAX_OCC) : 0;

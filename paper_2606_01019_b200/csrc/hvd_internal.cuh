@@ -130,6 +130,18 @@ inline hvd_status cuda_fail(hvd_ctx* ctx, cudaError_t e, const char* where) {
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Draft-length limit of a match of length L (App. A drafting table: draft cap, speculative factor and
+// offset): min(K, floor(factor * L + offset)) with K clamped to [0, k_cap]; the product and the sum are two
+// separately rounded fp32 operations; a factor <= 0 disables the second limit.
+__device__ __forceinline__ int draft_limit(int K, int k_cap, int L, float spec_factor, float spec_offset) {
+    int lim = max(0, min(K, k_cap));
+    if (spec_factor > 0.0f) {
+        const float f = __fadd_rn(__fmul_rn(spec_factor, (float)L), spec_offset);
+        lim = min(lim, max(0, (int)floorf(f)));
+    }
+    return lim;
+}
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                                  cudaStream_t stream, Args&&... args) {

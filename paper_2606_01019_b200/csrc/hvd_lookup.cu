@@ -180,14 +180,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
     if (L < a.min_match || L == 0) {
         L = 0; e = -1; cnt = 0;
     } else {
-        const int K = max(0, min(K_b, a.k_cap));
-        int lim = K;
-        if (a.spec_factor > 0.0f) {
-            // two separately rounded operations, as written: multiply, then add
-            const float f = __fadd_rn(__fmul_rn(a.spec_factor, (float)L), a.spec_offset);
-            lim = max(0, (int)floorf(f));
-        }
-        d = min(min(K, lim), n - e);
+        d = min(draft_limit(K_b, a.k_cap, L, a.spec_factor, a.spec_offset), n - e);
     }
     const int tok0 = lane < d ? slab[e + lane] : -1;
     const int tok1 = lane + 32 < d ? slab[e + lane + 32] : -1;

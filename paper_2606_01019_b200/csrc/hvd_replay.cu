@@ -112,12 +112,7 @@ __global__ void __launch_bounds__(256) replay_finish_kernel(const ReplayArgs a) 
         if (L < a.min_match || L == 0) {
             L = 0; e = -1; cnt = 0;
         } else {
-            int lim = a.K;
-            if (a.spec_factor > 0.0f) {
-                const float f = __fadd_rn(__fmul_rn(a.spec_factor, (float)L), a.spec_offset);
-                lim = max(0, (int)floorf(f));
-            }
-            d = min(min(a.K, lim), t - e);
+            d = min(draft_limit(a.K, a.K, L, a.spec_factor, a.spec_offset), t - e);
             // label: draft tokens x[e .. e+d) that the trace's continuation x[t ..) confirms
             while (y < d && t + y < a.n && x[e + y] == x[t + y]) ++y;
         }
