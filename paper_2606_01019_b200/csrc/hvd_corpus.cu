@@ -16,7 +16,7 @@
 // corpus wins and clears the scratch.  No CTA waits for another.
 #include <algorithm>
 
-#include "hvd_internal.cuh"
+#include "hvd_scan.cuh"
 
 namespace hvd {
 namespace {
@@ -204,8 +204,8 @@ __global__ void __launch_bounds__(kProbeThreads) corpus_probe_kernel(const Corpu
     if (tid < HVD_MAX_L) s_q[tid] = (tid < n) ? a.hist[a.hist_off[b] + n - 1 - tid] : -1;
     __syncthreads();
 
-    unsigned long long best_key = 0;
-    uint32_t best_cnt = 0;
+    Best best;  // this thread's candidates
+    best.key = 0; best.cnt = 0;
     const int g = a.g;
     const int32_t q0 = s_q[0], q1 = (g == 2) ? s_q[1] : 0;
     if (n >= g && q0 >= 0 && q1 >= 0) {
@@ -221,41 +221,32 @@ __global__ void __launch_bounds__(kProbeThreads) corpus_probe_kernel(const Corpu
                 int32_t c[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) c[k] = (L + k < cap) ? corpus[p - L - k] : -1;
-                int k = 0;
+                uint32_t fail = 0;  // bit j: the token L + j back does not continue the match
 #pragma unroll
-                for (int j = 7; j >= 0; --j)
-                    if (!(L + j < cap && c[j] >= 0 && c[j] == s_q[L + j])) k = j;  // ends as the first failing j
-                bool all = true;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) all = all && (L + j < cap && c[j] >= 0 && c[j] == s_q[L + j]);
-                if (all) { L += 8; } else { L += k; break; }
+                for (int j = 0; j < 8; ++j)
+                    if (!(L + j < cap && c[j] >= 0 && c[j] == s_q[L + j])) fail |= 1u << j;
+                if (fail == 0) { L += 8; } else { L += __ffs(fail) - 1; break; }
             }
-            const unsigned long long key = ((unsigned long long)(uint32_t)L << 32) | (uint32_t)(p + 1);
-            const uint32_t bl = (uint32_t)(best_key >> 32);
-            if ((uint32_t)L > bl) { best_key = key; best_cnt = 1; }
-            else if ((uint32_t)L == bl) { best_key = key > best_key ? key : best_key; ++best_cnt; }
+            Best c;
+            c.key = ((unsigned long long)(uint32_t)L << 32) | (uint32_t)(p + 1);
+            c.cnt = 1;
+            best = combine(best, c);
         }
     }
     // warp, then CTA: longest length, then latest position; counts add up at equal length
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const unsigned long long k2 = __shfl_xor_sync(0xffffffffu, best_key, off);
-        const uint32_t c2 = __shfl_xor_sync(0xffffffffu, best_cnt, off);
-        const uint32_t l1 = (uint32_t)(best_key >> 32), l2 = (uint32_t)(k2 >> 32);
-        if (l2 > l1) { best_key = k2; best_cnt = c2; }
-        else if (l2 == l1) { best_key = k2 > best_key ? k2 : best_key; best_cnt += c2; }
-    }
-    if (lane == 0) { s_key[warp] = best_key; s_cntL[warp] = best_cnt; }
+    best = warp_combine(best);
+    if (lane == 0) { s_key[warp] = best.key; s_cntL[warp] = best.cnt; }
     __syncthreads();
     if (tid == 0) {
-        unsigned long long key = 0;
-        uint32_t cnt = 0;
+        Best r;
+        r.key = 0; r.cnt = 0;
         for (int w = 0; w < kProbeWarps; ++w) {
-            const unsigned long long k2 = s_key[w];
-            const uint32_t l1 = (uint32_t)(key >> 32), l2 = (uint32_t)(k2 >> 32);
-            if (l2 > l1) { key = k2; cnt = s_cntL[w]; }
-            else if (l2 == l1 && l2 != 0) { key = k2 > key ? k2 : key; cnt += s_cntL[w]; }
+            Best o;
+            o.key = s_key[w]; o.cnt = s_cntL[w];
+            r = combine(r, o);
         }
+        const unsigned long long key = r.key;
+        const uint32_t cnt = r.cnt;
         if (key != 0) {
             atomicMax(a.key + b, key);
             atomicAdd(a.cnt + (int64_t)b * kCntStride + (key >> 32), cnt);

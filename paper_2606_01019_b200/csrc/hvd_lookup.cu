@@ -34,32 +34,6 @@ struct LookupArgs {
     bool successor_works_ahead;
 };
 
-struct Best {
-    unsigned long long key;  // (L << 32) | e ; 0 = nothing found
-    uint32_t cnt;
-};
-
-__device__ __forceinline__ Best combine(Best a, Best b) {
-    const uint32_t la = (uint32_t)(a.key >> 32), lb = (uint32_t)(b.key >> 32);
-    if (la > lb) return a;
-    if (lb > la) return b;
-    Best r;
-    r.key = a.key > b.key ? a.key : b.key;
-    r.cnt = a.cnt + b.cnt;
-    return r;
-}
-
-__device__ __forceinline__ Best warp_combine(Best v) {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        Best o;
-        o.key = __shfl_xor_sync(0xffffffffu, v.key, off);
-        o.cnt = __shfl_xor_sync(0xffffffffu, v.cnt, off);
-        v = combine(v, o);
-    }
-    return v;
-}
-
 template <int THREADS, int ITER, bool FUSED>
 __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 512 ? 2 : 4))) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
     __shared__ float s_hid[FUSED ? HVD_MAX_HIDDEN : 1];

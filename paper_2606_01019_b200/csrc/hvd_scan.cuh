@@ -9,6 +9,34 @@
 
 namespace hvd {
 
+// Best match seen so far: the longest length, then the latest position; the count is the number of
+// positions that reach that length.
+struct Best {
+    unsigned long long key;  // (L << 32) | e ; 0 = nothing found
+    uint32_t cnt;
+};
+
+__device__ __forceinline__ Best combine(Best a, Best b) {
+    const uint32_t la = (uint32_t)(a.key >> 32), lb = (uint32_t)(b.key >> 32);
+    if (la > lb) return a;
+    if (lb > la) return b;
+    Best r;
+    r.key = a.key > b.key ? a.key : b.key;
+    r.cnt = a.cnt + b.cnt;
+    return r;
+}
+
+__device__ __forceinline__ Best warp_combine(Best v) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        Best o;
+        o.key = __shfl_xor_sync(0xffffffffu, v.key, off);
+        o.cnt = __shfl_xor_sync(0xffffffffu, v.cnt, off);
+        v = combine(v, o);
+    }
+    return v;
+}
+
 __device__ __forceinline__ int4 ld_hist(const int4* p) {
     int4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
