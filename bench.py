@@ -34,7 +34,7 @@ L2_BYTES = 126 * 2**20
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one verify_commit launch on this workload, from
 # the ncu capture summarised under profiles/ (None until captured for a workload)
-NCU_VERIFY_TRAFFIC_BYTES = {"C2": 261588736}  # profiles/verify_stream_kernel_c2_ncu.txt, mean of two launches
+NCU_VERIFY_TRAFFIC_BYTES = {"C2": 261772928}  # profiles/verify_stream_kernel_c2_ncu.txt, mean of two launches
 
 
 def parse_args():
