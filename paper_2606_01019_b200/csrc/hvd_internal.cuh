@@ -37,7 +37,7 @@ constexpr int kVerifyUnroll = HVD_VERIFY_UNROLL;      // 128-bit loads in flight
 #endif
 constexpr int kVerifyUnitBatches = HVD_VERIFY_UNIT_BATCHES;  // 4 KB batches per unit drawn by a warp
 #ifndef HVD_VERIFY_ENDGAME_SHIFT
-#define HVD_VERIFY_ENDGAME_SHIFT 3
+#define HVD_VERIFY_ENDGAME_SHIFT 6
 #endif
 #ifndef HVD_VERIFY_QUEUES
 #define HVD_VERIFY_QUEUES 8
