@@ -539,22 +539,21 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
             const uint4* ptr = vrow + (int64_t)gb * kBatchVec + lane;
 
             uint32_t lord = 0u, loff = 0xffffffffu;  // this lane's maximum and its element index in the row
-            if (left >= kBatchVec) {
+            // Every load of the batch is issued before any is used, in a full batch and in the ragged last
+            // batch of a row alike (there the loads beyond the row are left out).  One code path with a
+            // warp-uniform switch: two paths with a register array each spilled, and a ragged path that
+            // loaded and folded in turn cost 2 us per C2 launch (one batch in 63 is ragged there).
+            const bool full = left >= kBatchVec;
+            if (full || lane < left) {
                 uint4 x[U];
 #pragma unroll
-                for (int u = 0; u < U; ++u) x[u] = ld_stream(ptr + u * 32, pol);
+                for (int u = 0; u < U; ++u)
+                    if (full || u * 32 + lane < left) x[u] = ld_stream(ptr + u * 32, pol);
                 Tracker<E> t;
                 t.init(x[0]);
 #pragma unroll
-                for (int u = 1; u < U; ++u) t.fold(x[u], u);
-                t.best(lane, lord, loff);
-                loff += (uint32_t)(head + gb * kBatchVec * EPV);
-            } else if (lane < left) {  // ragged last batch of the row
-                Tracker<E> t;
-                t.init(ld_stream(ptr, pol));
-#pragma unroll
                 for (int u = 1; u < U; ++u)
-                    if (u * 32 + lane < left) t.fold(ld_stream(ptr + u * 32, pol), u);
+                    if (full || u * 32 + lane < left) t.fold(x[u], u);
                 t.best(lane, lord, loff);
                 loff += (uint32_t)(head + gb * kBatchVec * EPV);
             }
