@@ -1,5 +1,7 @@
 """Pins for the oracle's frequency-weighted continuation and suffix score (merged occurrences of the
 longest match; draft limits and minimum token probability from the paper's drafting table)."""
+import os
+
 import numpy as np
 
 from oracle import hvd_oracle as O
@@ -117,3 +119,20 @@ def test_freq_select_hand_cases():
     sel, sd, sl = O.freq_select(out, 0.0)               # no model draft: empty selection when not chosen
     assert list(sel) == [1, 1, 0, 1] and list(sl) == [2, 1, 0, 3]
     assert sd[2].tolist() == [-1, -1, -1]
+
+
+def test_hand_worked_fixture():
+    path = os.path.join(os.path.dirname(__file__), "golden", "frequency_walk_cases.txt")
+    rows = [r for r in open(path) if r.strip() and not r.startswith("#")]
+    assert len(rows) >= 7
+    for r in rows:
+        f = [x.strip() for x in r.rstrip("\n").split("|")]
+        h = [int(x) for x in f[0].split()]
+        K, sf, mp, mo, L, cnt = int(f[1]), float(f[2]), float(f[3]), int(f[4]), int(f[5]), int(f[6])
+        want_d = [int(x) for x in f[7].split()]
+        want_sc = f32(0)
+        for t in f[8].split():
+            a, b = t.split("/")
+            want_sc = f32(want_sc + f32(a) / f32(b))
+        d, sc, out = run_one(h, K, spec_factor=sf, min_prob=mp, max_occ=mo)
+        assert (int(out.match_len[0]), int(out.match_cnt[0]), d, sc) == (L, cnt, want_d, want_sc), r
