@@ -24,6 +24,8 @@
 // No warp waits for another.
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "hvd_internal.cuh"
 
 namespace hvd {
@@ -617,10 +619,16 @@ hvd_status launch_commit_keys(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream) {
 
 hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit) {
     const int per_sm = ctx->vf_blocks_per_sm[dtype == HVD_F32 ? 0 : 1];
-    const int grid = ctx->num_sms * (per_sm > 0 ? per_sm : 1);
+    int grid = ctx->num_sms * (per_sm > 0 ? per_sm : 1);
     const int64_t esz = dtype == HVD_F32 ? 4 : 2;
     a.n_batch_row = (int32_t)((a.V * esz / 16 + kBatchVec - 1) / kBatchVec);
     if (a.n_batch_row < 1) a.n_batch_row = 1;
+    // a small call gets no more warps than it can have units, but at least one CTA for every second SM
+    // (measured on 36 rows of 32 000 floats: 74 to 96 CTAs 6.5 us, the full 592 CTAs 7.5 us, 72 CTAs 7.3 us,
+    // 37 CTAs 9.4 us)
+    const int64_t units_upper = (a.total_rows * (int64_t)a.n_batch_row + UB - 1) / UB;
+    const int64_t want = std::max<int64_t>((units_upper + NW - 1) / NW, (ctx->num_sms + 1) / 2);
+    if (want < grid) grid = (int)want;
     // unit numbers are 32-bit
     if (a.total_rows * (int64_t)a.n_batch_row / UB + 4 * (int64_t)grid * NW >= 0x7fffffffLL)
         return fail(ctx, HVD_ERR_UNSUPPORTED, "hvd_verify_commit: too many batches");
