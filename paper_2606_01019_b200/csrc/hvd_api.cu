@@ -105,7 +105,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     // HVD_PDL_MASK=0 turns it off
     c->pdl_mask = getenv("HVD_PDL_MASK") ? atoi(getenv("HVD_PDL_MASK")) : 15;
     c->pdl_commit = (c->pdl_mask & 1) != 0;
-    c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // measured: no gain on this path, off unless asked for
+    c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // every kernel of the library, the cluster kernel included: for experiments
     c->host_ws = nullptr;
     c->host_ws_bytes = 0;
 #ifdef HVD_TRACE
