@@ -132,3 +132,42 @@ def test_host_buffer_entry_point():
             G.assert_equal("acc_ring", rq_g.state["acc_ring"], rq_o.state["acc_ring"])
             G.assert_equal("sel_bits", rq_g.state["sel_bits"], rq_o.state["sel_bits"])
         ctx.close()
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_chained_steps_without_host_synchronisation(fused):
+    """Six steps enqueued back to back on one stream (no host synchronisation in between, so the kernels of
+    consecutive steps overlap as far as programmatic dependent launch lets them): the final histories,
+    lengths, states and the last step's outputs must equal the oracle's chain."""
+    import torch
+    w = W.CONFIGS["C2"].scaled(B=24, n=3000, V=5003)
+    inp = P.prepare(w, device="cuda")
+    S = 6
+    # the oracle's chain first: it fixes the logits of every step (each agrees with that step's selected draft)
+    rq_o = inp.rq.copy()
+    logits_dev, outs = [], []
+    for s in range(S):
+        lk = P.lookup(w, rq_o, 8)
+        sc = P.score_select(w, rq_o, lk, inp.W1, inp.b1, inp.W2, inp.b2, inp.tau, 8, inp.Wh, inp.bh)
+        A = W.make_agreement(w, sc.sel_len)
+        lg = W.make_logits(w, int(rq_o.row_off[-1]), device="cuda", salt=300 + s)
+        W.plant_agreement(w, lg, rq_o.row_off, sc.sel_draft, sc.sel_len, A, salt=300 + s)
+        vf = P.verify_commit(w, rq_o, sc, W.logits_to_numpy(lg), 8)
+        logits_dev.append(lg)
+        outs.append((lk, sc, vf))
+    # the same chain on the GPU, enqueued in one go
+    rq_g = inp.rq.copy()
+    ctx = G.make_ctx(w, rq_g)
+    G.set_predictor(ctx, inp)
+    batch = G.make_batch(ctx, w, rq_g)
+    torch.cuda.synchronize()
+    for s in range(S):
+        batch.step(logits_dev[s], fused=fused)
+    g = batch.download()
+    lk, sc, vf = outs[-1]
+    G.compare_lookup(g, lk)
+    same = G.compare_score(g, sc, inp.tau)
+    assert same.all()
+    G.compare_verify(g, vf, rq_o)
+    assert (rq_o.hist_len > inp.rq.hist_len).all()
+    ctx.close()
