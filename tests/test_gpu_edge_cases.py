@@ -232,3 +232,18 @@ def test_host_side_argument_errors():
     with pytest.raises(H.HvdError):
         H.Context(max_batch=4, k_cap=65, max_hist_len=10, max_rows=10, max_vocab=10)
     ctx.close()
+
+
+def test_parity_with_plain_launches():
+    """The same parity cases with programmatic dependent launch switched off (every kernel starts after
+    its predecessor has completed): a result must not depend on how far consecutive kernels overlap."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, HVD_PDL_MASK="0")
+    cmd = [sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", "tests/test_gpu_parity.py",
+           "-k", "c1_full or fused_lookup or multi_step or chained or switching"]
+    res = subprocess.run(cmd, cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
+    assert " passed" in res.stdout
