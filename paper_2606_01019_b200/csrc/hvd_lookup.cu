@@ -1,9 +1,10 @@
 // Cache-draft lookup (Sec. 3.2): longest match of the history's own suffix inside the history.
 //
-// One CTA scans a request's history (histories longer than 32 K tokens are cut into chunks, one
-// CTA each) with 128-bit loads, all issued up front, looking for the last token of the history.  Every hit is a candidate end position; the warp that found it
-// extends the match backwards cooperatively (one compared token per lane, ballot + find-first-set
-// gives the match length).  Each CTA leaves one partial (best length, latest position, count) in
+// One CTA scans a request's history (histories longer than 32 K tokens are cut into chunks of 8 K
+// tokens, one CTA each) with 128-bit loads, all issued up front, looking for the last token of the
+// history.  Every hit is a candidate end position; the warp that found it extends the match
+// backwards cooperatively (one compared token per lane, ballot + find-first-set gives the match
+// length).  Each CTA leaves one partial (best length, latest position, count) in
 // the context's scratch; the CTA that arrives last for a request combines the partials, applies the
 // minimum-length and draft-length rules and copies the draft -- and, in the fused form, goes
 // straight on to the payoff features, the predictor and the draft selection of that request
