@@ -80,6 +80,8 @@ typedef struct {
 } hvd_req_state;
 
 enum { HVD_N_FEATURES = 8, HVD_MAX_K = 64, HVD_MAX_L = 64, HVD_MAX_HIDDEN = 256 };
+/* Longest history a context accepts: positions and the rounded-up scan range stay inside int32. */
+enum { HVD_MAX_HIST_LEN = 0x7fffffff - (1 << 20) };
 enum { HVD_N_TOKEN_CLASSES = 5, HVD_N_FEATURES_EXT = 14 };
 
 typedef struct {
@@ -90,7 +92,7 @@ typedef struct {
     float spec_factor;    /* draft_len <= floor(spec_factor*match_len + spec_offset); <= 0 disables the limit */
     float spec_offset;    /* ("maximum speculative factor / offset" of the suffix cache: 1.0 / 0.0) */
     int32_t hidden;       /* hidden units of the payoff MLP, 1..256 */
-    int32_t max_hist_len; /* largest hist_len of any request */
+    int32_t max_hist_len; /* largest hist_len of any request, in [1, HVD_MAX_HIST_LEN] */
     int64_t max_rows;     /* largest total number of logits rows of any call */
     int64_t max_vocab;    /* largest V of any call */
 } hvd_config;

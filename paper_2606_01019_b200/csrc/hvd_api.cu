@@ -57,7 +57,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     if (cfg->l_max < 1 || cfg->l_max > HVD_MAX_L) return HVD_ERR_INVALID_ARG;
     if (cfg->min_match < 1) return HVD_ERR_INVALID_ARG;
     if (cfg->hidden < 1 || cfg->hidden > HVD_MAX_HIDDEN) return HVD_ERR_INVALID_ARG;
-    if (cfg->max_hist_len < 1) return HVD_ERR_INVALID_ARG;
+    if (cfg->max_hist_len < 1 || cfg->max_hist_len > HVD_MAX_HIST_LEN) return HVD_ERR_INVALID_ARG;
     if (cfg->max_rows < 1 || cfg->max_vocab < 1 || cfg->max_vocab > 0x7fffffffLL) return HVD_ERR_INVALID_ARG;
     if (!(cfg->spec_factor == cfg->spec_factor) || !(cfg->spec_offset == cfg->spec_offset)) return HVD_ERR_INVALID_ARG;
 

@@ -33,13 +33,16 @@ struct LookupArgs {
     int32_t k_cap, l_max, min_match;
     float spec_factor, spec_offset;
     bool successor_works_ahead;
+    bool chunks_on_x;
 };
 
 template <int THREADS, int ITER, bool FUSED>
 __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 512 ? 2 : 4))) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
     __shared__ float s_hid[FUSED ? HVD_MAX_HIDDEN : 1];
-    const int b = blockIdx.y;
-    const int chunk = blockIdx.x;
+    // requests run fastest: with ragged lengths the CTAs of the low chunks, which every request has, are
+    // dispatched first and the empty ones come last (chunks move to x when they outgrow the y range)
+    const int b = a.chunks_on_x ? blockIdx.y : blockIdx.x;
+    const int chunk = a.chunks_on_x ? blockIdx.x : blockIdx.y;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
@@ -208,7 +211,8 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
     const int64_t chunk = (int64_t)shapes[pick].threads * kLookupTokPerVec * shapes[pick].iter;
     const int64_t chunks = (span + chunk - 1) / chunk;
     if (chunks > ctx->lk_max_chunks) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_lookup: n_max exceeds max_hist_len");
-    dim3 grid((unsigned)chunks, (unsigned)B);
+    a.chunks_on_x = chunks > 65535;
+    const dim3 grid = a.chunks_on_x ? dim3((unsigned)chunks, (unsigned)B) : dim3((unsigned)B, (unsigned)chunks);
     cudaError_t e;
     const ScoreArgs sa = fused ? *fused : ScoreArgs();
 #define HVD_LAUNCH_LOOKUP(TH, I)                                                                       \

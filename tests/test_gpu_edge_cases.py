@@ -231,6 +231,34 @@ def test_host_side_argument_errors():
         H.Context(max_batch=0, k_cap=8, max_hist_len=10, max_rows=10, max_vocab=10)
     with pytest.raises(H.HvdError):
         H.Context(max_batch=4, k_cap=65, max_hist_len=10, max_rows=10, max_vocab=10)
+    with pytest.raises(H.HvdError):
+        H.Context(max_batch=4, k_cap=8, max_hist_len=2**31 - 1, max_rows=10, max_vocab=10)
+    ctx.close()
+
+
+def test_history_of_more_than_65535_chunks():
+    """A history so long that its chunks outgrow the y range of a grid (the launch then puts the chunks
+    on x): 537 M tokens in one request, the longest match planted far inside."""
+    import torch
+    w = small(k_cap=16)
+    n = 65536 * 8192 + 4321
+    rng = np.random.default_rng(21)
+    h = rng.integers(0, 1 << 30, n, dtype=np.int32)
+    tail = h[n - 24:].copy()
+    h[400_000_000:400_000_024] = tail            # the copy the lookup has to find, in a far chunk
+    h[123_456_789 - 9:123_456_789] = tail[-9:]   # a shorter one
+    rq = hand_requests(w, [h], [16])
+    del h
+    lk = P.lookup(w, rq, nthreads=1)
+    assert lk.match_len[0] == 24 and lk.match_pos[0] == 400_000_024 and lk.draft_len[0] == 16
+    ctx = G.make_ctx(w, rq)
+    b = G.make_batch(ctx, w, rq)
+    b.lookup()
+    torch.cuda.synchronize()
+    assert ctx.hvd_device_status() == 0
+    got = dict(draft=b.draft, draft_len=b.draft_len, match_len=b.match_len, match_pos=b.match_pos,
+               match_cnt=b.match_cnt)
+    G.compare_lookup({k: v.cpu().numpy() for k, v in got.items()}, lk)
     ctx.close()
 
 
