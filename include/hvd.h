@@ -35,6 +35,15 @@
  *  - Token histories are ragged: request b owns the slab
  *    hist[hist_off[b] .. hist_off[b] + hist_cap[b]) of which the first
  *    hist_len[b] tokens are valid (prompt followed by committed tokens).
+ *  - Consecutive kernels of a context are joined by programmatic dependent
+ *    launch: a kernel may be resident while its predecessor on the stream
+ *    still runs, and waits on the device before it reads anything the
+ *    predecessor writes.  Results do not depend on it.  Two environment
+ *    variables, read once by hvd_create, change it: HVD_PDL_MASK (a bit per
+ *    kernel pair: 1 commit, 2 lookup, 4 verify stream, 8 scoring; default 15,
+ *    0 = plain launches) and HVD_ENABLE_PDL (any value: the launch attribute
+ *    on every kernel of the library).  Nothing else is read from the
+ *    environment by the product path.
  */
 #ifndef HVD_H
 #define HVD_H
