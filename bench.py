@@ -586,9 +586,12 @@ def main():
         hist_len_steps.copy_(hist_len_pristine)
         state_steps.copy_(state_pristine)
 
-    def step(slot, events=None, with_verify=True, lookup_only=False, verify_only=False):
+    def step(slot, events=None, with_verify=True, lookup_only=False, verify_only=False, probe_only=False):
         r = slot % R
         hl, st = hist_len_steps[slot], state_steps[slot]
+        if probe_only:    # plain read loop over the same logits buffer: the part's read-only speed
+            ctx.hvd_read_probe(logits[r], logits[r].numel() * logits[r].element_size())
+            return
         if lookup_only:
             lookup(hists[r], hl)
             return
@@ -616,12 +619,12 @@ def main():
     mode = args.mode
     stream = torch.cuda.Stream(device=dev)
 
-    def capture(events=None, with_verify=True, lookup_only=False, verify_only=False):
+    def capture(events=None, with_verify=True, lookup_only=False, verify_only=False, probe_only=False):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
             g.capture_begin()
             for s in range(K_steps):
-                step(W_steps + s, events[s] if events else None, with_verify, lookup_only, verify_only)
+                step(W_steps + s, events[s] if events else None, with_verify, lookup_only, verify_only, probe_only)
             g.capture_end()
         torch.cuda.synchronize()
         with torch.cuda.stream(stream):
@@ -700,6 +703,8 @@ def main():
                 g_vo = capture(None, verify_only=True)
                 restore()
                 t_vo = timed(g_vo.replay)
+                g_pr = capture(None, probe_only=True)
+                t_pr = timed(g_pr.replay)
             else:
                 t_ev = timed(lambda: [step(W_steps + s, evs[s]) for s in range(K_steps)])
                 restore()
@@ -707,6 +712,7 @@ def main():
                 t_lk = timed(lambda: [step(W_steps + s, None, False, True) for s in range(K_steps)])
                 restore()
                 t_vo = timed(lambda: [step(W_steps + s, None, True, False, True) for s in range(K_steps)])
+                t_pr = timed(lambda: [step(W_steps + s, probe_only=True) for s in range(K_steps)])
             restore()
             d = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(2)] for e in evs])
             kt = {"lookup_plus_score_select_us": 1e3 * float(d[:, 0].mean()),
@@ -717,6 +723,7 @@ def main():
                   "lookup_only_us": 1e3 * t_lk / K_steps,
                   "verify_commit_us_by_difference": 1e3 * (elapsed_ms - t_nv) / K_steps,
                   "verify_commit_us_back_to_back": 1e3 * t_vo / K_steps,
+                  "read_probe_us": 1e3 * t_pr / K_steps,
                   "note": "event-bracketed times include the serialisation the event records add; "
                           "the headline region has no records in it"}
         except Exception as e:  # pragma: no cover
@@ -744,6 +751,12 @@ def main():
         roofline["achieved_with_event_records_in_graph"] = verify_bytes / (kt["verify_commit_us"] * 1e-6) / 1e9
         roofline_lookup["achieved"] = lookup_bytes / (kt["lookup_only_us"] * 1e-6) / 1e9
         roofline_lookup["frac"] = roofline_lookup["achieved"] / peak_gbs
+        probe_bytes = logits[0].numel() * logits[0].element_size()
+        roofline["read_only_kernel"] = {"achieved": probe_bytes / (kt["read_probe_us"] * 1e-6) / 1e9, "unit": "GB/s",
+                                        "bytes_per_launch": probe_bytes,
+                                        "what": "hvd_read_probe: a plain grid-stride read of the whole logits buffer, "
+                                                "timed like the verify call (K launches back to back on the rotating copies)"}
+        roofline["frac_of_read_only_kernel"] = roofline["achieved"] / roofline["read_only_kernel"]["achieved"]
         roofline["timing"] = ("CUDA events around a graph of the same K hvd_verify_commit launches back to back "
                               "(both kernels of the call, launch gaps included), on rotating inputs larger than L2")
 

@@ -420,6 +420,14 @@ HVD_API hvd_status hvd_commit_keys(hvd_ctx* ctx, int32_t B, const int64_t* keys,
                                    int32_t* target_tok, int32_t* status, void* stream);
 
 /*
+ * Measurement aid, not a step of the method: reads the first bytes / 16 * 16 bytes of buf (DEVICE,
+ * 16-byte aligned) once with a plain grid-stride loop of 128-bit loads and keeps only their maximum
+ * in context scratch.  Timed over the same buffers as hvd_verify_commit it gives the read-only
+ * speed of the part, the practical ceiling of the streaming kernel.  Enqueues one kernel.
+ */
+HVD_API hvd_status hvd_read_probe(hvd_ctx* ctx, const void* buf, int64_t bytes, void* stream);
+
+/*
  * Greedy verification and commit without a context and without any allocation.  (The paper has
  * no counterpart: this is a packaging variant of hvd_verify_commit.)
  *

@@ -19,7 +19,7 @@ void release(hvd_ctx* c) {
     cudaFree(c->cp_key); cudaFree(c->cp_cnt); cudaFree(c->cp_arrived);
     cudaFree(c->cp_start); cudaFree(c->cp_pos);
     cudaFree(c->rp_key); cudaFree(c->rp_cnt);
-    cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
+    cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->probe_sink); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
     delete c;
 }
@@ -89,6 +89,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->vf_row_key, (size_t)cfg->max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_next_unit, (size_t)kVerifyQueues * 32 * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->dev_error, sizeof(int)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->probe_sink, sizeof(unsigned long long)) == cudaSuccess;
     if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); release(c); return HVD_ERR_ALLOC; }
 
@@ -284,6 +285,14 @@ hvd_status hvd_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist, const i
     return launch_lookup_freq(ctx, B, hist, hist_off, hist_cap, hist_len, K, n_max, min_prob, max_occ, threshold,
                               model_draft, model_len, draft, draft_len, score, match_len, match_pos, match_cnt,
                               select, sel_draft, sel_len, static_cast<cudaStream_t>(stream));
+}
+
+hvd_status hvd_read_probe(hvd_ctx* ctx, const void* buf, int64_t bytes, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (!buf) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_read_probe: NULL pointer");
+    if (bytes < 0) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_read_probe: negative size");
+    if (reinterpret_cast<uintptr_t>(buf) & 15) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_read_probe: buf not 16-byte aligned");
+    return launch_read_probe(ctx, buf, bytes, static_cast<cudaStream_t>(stream));
 }
 
 hvd_status hvd_replay_labels(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label,

@@ -91,6 +91,7 @@ struct hvd_ctx {
     unsigned long long* vf_row_key;  // [max_rows], zero at rest
     uint32_t* vf_next_unit;          // zero at rest
     int* dev_error;                  // device status word
+    unsigned long long* probe_sink;  // result word of the read-only probe
     int vf_blocks_per_sm[2];         // per dtype
     // device staging of the host-buffer entry point (grown on demand)
     bool use_pdl;     // programmatic dependent launch for every kernel of the library (HVD_ENABLE_PDL; experiments)
@@ -186,6 +187,7 @@ hvd_status launch_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_
                                    const int32_t* model_draft, const int32_t* model_len, float* features, float* score,
                                    int32_t* select, int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream);
 
+hvd_status launch_read_probe(hvd_ctx* ctx, const void* buf, int64_t bytes, cudaStream_t stream);
 hvd_status launch_replay(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label, int32_t* draft_len,
                          int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream);
 

@@ -262,6 +262,26 @@ def test_history_of_more_than_65535_chunks():
     ctx.close()
 
 
+def test_read_probe_runs_and_checks_its_arguments():
+    """The read-only probe of the benchmark: any size (whole vectors, a ragged tail, nothing), and the
+    host-side argument checks."""
+    import torch
+    import paper_2606_01019_b200 as H
+    ctx = H.Context(max_batch=1, k_cap=8, max_hist_len=16, max_rows=1, max_vocab=16)
+    buf = torch.randint(0, 2**31 - 1, (1 << 20,), dtype=torch.int32, device="cuda")
+    for nbytes in (0, 16, 4096, 4 * (1 << 20) - 4, 4 * (1 << 20)):
+        ctx.hvd_read_probe(buf, nbytes)
+    torch.cuda.synchronize()
+    assert ctx.hvd_device_status() == 0
+    with pytest.raises(H.HvdError, match="NULL"):
+        ctx.hvd_read_probe(None, 16)
+    with pytest.raises(H.HvdError, match="negative"):
+        ctx.hvd_read_probe(buf, -1)
+    with pytest.raises(H.HvdError, match="aligned"):
+        ctx.hvd_read_probe(buf[1:], 16)
+    ctx.close()
+
+
 def test_parity_with_plain_launches():
     """The same parity cases with programmatic dependent launch switched off (every kernel starts after
     its predecessor has completed): a result must not depend on how far consecutive kernels overlap."""
