@@ -559,6 +559,19 @@ def main():
         ctx.hvd_verify_commit(B, logits, dtype, w.V, row_off, 0, total_rows, sel_draft, sel_len, select, hist,
                               hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, None, status)
 
+    # the commit and the next cycle's lookup + selection in one call; the next selection goes to arrays of its
+    # own, so that every timed step verifies the same (pristine) selection
+    select_n, sel_draft_n, sel_len_n = i32(B), i32(B, kc), i32(B)
+    n_max_next = min(int(rq.hist_cap.max()), n_max + kc + 1)
+
+    def cycle(logits, hist, hist_len, state):
+        ctx.hvd_verify_commit_next(B, logits, dtype, w.V, row_off, 0, total_rows, sel_draft, sel_len, select, hist,
+                                   hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, None, status,
+                                   K=Kt, n_max=n_max_next, prompt_len=prompt_len, model_draft=model_draft,
+                                   model_len=model_len, draft=draft, draft_len=draft_len, match_len=match_len,
+                                   match_pos=match_pos, match_cnt=match_cnt, features=None, score=score,
+                                   next_select=select_n, next_sel_draft=sel_draft_n, next_sel_len=sel_len_n)
+
     lookup(hist0, hist_len0)
     score_select(hist_len0, state0)
     if w.calibrate_cache_frac is not None:
@@ -586,9 +599,13 @@ def main():
         hist_len_steps.copy_(hist_len_pristine)
         state_steps.copy_(state_pristine)
 
-    def step(slot, events=None, with_verify=True, lookup_only=False, verify_only=False, probe_only=False):
+    def step(slot, events=None, with_verify=True, lookup_only=False, verify_only=False, probe_only=False,
+             cycle_only=False):
         r = slot % R
         hl, st = hist_len_steps[slot], state_steps[slot]
+        if cycle_only:    # verify + commit + the next cycle's lookup and selection: two kernels per step
+            cycle(logits[r], hists[r], hl, st)
+            return
         if probe_only:    # plain read loop over the same logits buffer: the part's read-only speed
             ctx.hvd_read_probe(logits[r], logits[r].numel() * logits[r].element_size())
             return
@@ -619,12 +636,14 @@ def main():
     mode = args.mode
     stream = torch.cuda.Stream(device=dev)
 
-    def capture(events=None, with_verify=True, lookup_only=False, verify_only=False, probe_only=False):
+    def capture(events=None, with_verify=True, lookup_only=False, verify_only=False, probe_only=False,
+                cycle_only=False):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
             g.capture_begin()
             for s in range(K_steps):
-                step(W_steps + s, events[s] if events else None, with_verify, lookup_only, verify_only, probe_only)
+                step(W_steps + s, events[s] if events else None, with_verify, lookup_only, verify_only, probe_only,
+                     cycle_only)
             g.capture_end()
         torch.cuda.synchronize()
         with torch.cuda.stream(stream):
@@ -705,6 +724,10 @@ def main():
                 t_vo = timed(g_vo.replay)
                 g_pr = capture(None, probe_only=True)
                 t_pr = timed(g_pr.replay)
+                restore()
+                g_cy = capture(None, cycle_only=True)
+                restore()
+                t_cy = timed(g_cy.replay)
             else:
                 t_ev = timed(lambda: [step(W_steps + s, evs[s]) for s in range(K_steps)])
                 restore()
@@ -713,6 +736,8 @@ def main():
                 restore()
                 t_vo = timed(lambda: [step(W_steps + s, None, True, False, True) for s in range(K_steps)])
                 t_pr = timed(lambda: [step(W_steps + s, probe_only=True) for s in range(K_steps)])
+                restore()
+                t_cy = timed(lambda: [step(W_steps + s, cycle_only=True) for s in range(K_steps)])
             restore()
             d = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(2)] for e in evs])
             kt = {"lookup_plus_score_select_us": 1e3 * float(d[:, 0].mean()),
@@ -724,6 +749,7 @@ def main():
                   "verify_commit_us_by_difference": 1e3 * (elapsed_ms - t_nv) / K_steps,
                   "verify_commit_us_back_to_back": 1e3 * t_vo / K_steps,
                   "read_probe_us": 1e3 * t_pr / K_steps,
+                  "step_us_commit_fused_with_next_lookup": 1e3 * t_cy / K_steps,
                   "note": "event-bracketed times include the serialisation the event records add; "
                           "the headline region has no records in it"}
         except Exception as e:  # pragma: no cover

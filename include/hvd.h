@@ -327,6 +327,47 @@ HVD_API hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits
                              int32_t* status, void* stream);
 
 /*
+ * hvd_verify_commit, then at once the NEXT cycle's hvd_lookup_score_select on the histories it has just
+ * extended (Algorithm 1: the end of one iteration and the start of the next).  In a decoding loop the two
+ * are adjacent, and one kernel does the commit and the lookup: a launch and two dependent global round
+ * trips less per cycle.  Results are exactly those of the two calls one after the other.
+ * The verification arguments are hvd_verify_commit's.  `next` (a HOST struct of DEVICE pointers, read
+ * before the call returns) holds hvd_lookup_score_select's remaining arguments:
+ *   K, prompt_len, model_draft, model_len (or both NULL)   inputs of the next cycle
+ *   n_max            HOST value: upper bound on hist_len[b] AFTER this commit (<= max_hist_len)
+ *   draft .. match_cnt, features (or NULL), score          outputs as in hvd_lookup / hvd_score_select
+ *   select, sel_draft, sel_len                             the next selection; these may be the very
+ *                    arrays the commit reads (a request's old entries are read before its new ones are written)
+ * hist, hist_off, hist_cap, hist_len and state are the ones of the verification.  The one-kernel form
+ * needs n_max + 2 <= 32768 and the one-layer predictor; otherwise the call enqueues the same kernels
+ * as the two separate calls.  Needs hvd_set_predictor first.
+ */
+typedef struct {
+    const int32_t* K;
+    int32_t n_max;
+    const int32_t* prompt_len;
+    const int32_t* model_draft;
+    const int32_t* model_len;
+    int32_t* draft;
+    int32_t* draft_len;
+    int32_t* match_len;
+    int32_t* match_pos;
+    int32_t* match_cnt;
+    float* features;
+    float* score;
+    int32_t* select;
+    int32_t* sel_draft;
+    int32_t* sel_len;
+} hvd_next_cycle;
+HVD_API hvd_status hvd_verify_commit_next(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                                          const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                                          const int32_t* sel_draft, const int32_t* sel_len, const int32_t* select,
+                                          int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                                          int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                                          int32_t* committed, int32_t* n_commit, int32_t* target_tok,
+                                          int32_t* status, const hvd_next_cycle* next, void* stream);
+
+/*
  * Greedy verification of a token TREE and commit.  The paper's model drafter (EAGLE3) proposes a
  * tree (App. A "Drafting configuration": 32 draft tokens, depth 8, top-k 4); the verification rule is
  * unchanged (Sec. 3.1, Sec. 3.4).  Node i of request b has token sel_draft[b, i] and parent

@@ -30,6 +30,13 @@ class HvdConfig(C.Structure):
                 ("max_hist_len", _i32), ("max_rows", _i64), ("max_vocab", _i64)]
 
 
+class NextCycle(C.Structure):
+    """hvd_next_cycle: the next cycle's lookup / score / select arguments of hvd_verify_commit_next."""
+    _fields_ = [("K", _vp), ("n_max", _i32), ("prompt_len", _vp), ("model_draft", _vp), ("model_len", _vp),
+                ("draft", _vp), ("draft_len", _vp), ("match_len", _vp), ("match_pos", _vp), ("match_cnt", _vp),
+                ("features", _vp), ("score", _vp), ("select", _vp), ("sel_draft", _vp), ("sel_len", _vp)]
+
+
 class HvdHostStepArgs(C.Structure):
     _fields_ = [("B", _i32), ("n_max", _i32), ("hist_words", _i64), ("hist", _vp), ("hist_off", _vp),
                 ("hist_cap", _vp), ("hist_len", _vp), ("K", _vp), ("prompt_len", _vp), ("state", _vp),
@@ -59,6 +66,7 @@ _SIGNATURES = {
     "hvd_replay_labels": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
+    "hvd_verify_commit_next": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp, _vp]),
     "hvd_verify_commit_tree": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 14 + [_vp]),
     "hvd_verify_keys": (_i32, [_vp, _i32, _vp, _i32, _i64, _i64, _vp, _i32, _i64, _vp, _vp, _vp, _vp, _vp]),
     "hvd_commit_keys": (_i32, [_vp, _i32, _vp, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
@@ -289,6 +297,22 @@ class Context:
                                                 _ptr(committed), _ptr(n_commit), _ptr(target_tok),
                                                 _ptr(status), _stream()),
                     "hvd_verify_commit")
+
+    def hvd_verify_commit_next(self, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
+                               select, hist, hist_off, hist_cap, hist_len, state, accepted, committed,
+                               n_commit, target_tok, status, *, K, n_max, prompt_len, model_draft, model_len,
+                               draft, draft_len, match_len, match_pos, match_cnt, features, score,
+                               next_select, next_sel_draft, next_sel_len):
+        nxt = NextCycle(_ptr(K), int(n_max), _ptr(prompt_len), _ptr(model_draft), _ptr(model_len), _ptr(draft),
+                        _ptr(draft_len), _ptr(match_len), _ptr(match_pos), _ptr(match_cnt), _ptr(features),
+                        _ptr(score), _ptr(next_select), _ptr(next_sel_draft), _ptr(next_sel_len))
+        self._check(self._lib.hvd_verify_commit_next(self._h, B, _ptr(logits), dtype, V, _ptr(row_off),
+                                                     k_uniform, total_rows, _ptr(sel_draft), _ptr(sel_len),
+                                                     _ptr(select), _ptr(hist), _ptr(hist_off), _ptr(hist_cap),
+                                                     _ptr(hist_len), _ptr(state), _ptr(accepted),
+                                                     _ptr(committed), _ptr(n_commit), _ptr(target_tok),
+                                                     _ptr(status), C.byref(nxt), _stream()),
+                    "hvd_verify_commit_next")
 
     def hvd_verify_keys(self, B, logits, dtype, V_shard, v_offset, row_off, k_uniform, total_rows, sel_len, hist_len,
                         hist_cap, keys):

@@ -391,7 +391,7 @@ static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits
                              int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
                              int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
                              int32_t* committed, int32_t* n_commit, int32_t* target_tok,
-                             int32_t* status, void* stream) {
+                             int32_t* status, void* stream, const hvd_next_cycle* next = nullptr) {
     if (!ctx) return HVD_ERR_INVALID_ARG;
     if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: B outside [1, max_batch]");
     if (dtype != HVD_F32 && dtype != HVD_BF16) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: unknown dtype");
@@ -423,7 +423,34 @@ static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits
 #endif
     a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error;
     a.row_key = ctx->vf_row_key; a.total_rows = total_rows; a.ext_keys = nullptr;
-    return launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
+    if (!next) return launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
+
+    // with the next cycle's lookup and scoring behind the commit
+    if (!ctx->has_predictor) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_next: call hvd_set_predictor first");
+    if (!next->K || !next->prompt_len || !next->draft || !next->draft_len || !next->match_len || !next->match_pos ||
+        !next->match_cnt || !next->score || !next->select || !next->sel_draft || !next->sel_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_next: NULL pointer in next");
+    if ((next->model_draft == nullptr) != (next->model_len == nullptr))
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_next: model_draft and model_len go together");
+    if (!aligned(hist, 16)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_next: hist must be 16-byte aligned");
+    if (next->n_max < 0 || next->n_max > ctx->cfg.max_hist_len)
+        return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_next: n_max outside [0, max_hist_len]");
+    if (ctx->two_layer || !cycle_fits_one_cta(next->n_max)) {
+        const hvd_status r = launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
+        if (r != HVD_OK) return r;
+        return hvd_lookup_score_select(ctx, B, hist, hist_off, hist_cap, hist_len, next->K, next->n_max, next->prompt_len,
+                                       state, next->model_draft, next->model_len, next->draft, next->draft_len,
+                                       next->match_len, next->match_pos, next->match_cnt, next->features, next->score,
+                                       next->select, next->sel_draft, next->sel_len, stream);
+    }
+    const hvd_status r = launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream), false);
+    if (r != HVD_OK) return r;
+    const ScoreArgs sa = make_score_args(ctx, B, hist_len, next->prompt_len, state, next->K, next->draft, next->draft_len,
+                                         next->match_len, next->match_pos, next->match_cnt, next->model_draft,
+                                         next->model_len, next->features, next->score, next->select, next->sel_draft,
+                                         next->sel_len);
+    return launch_commit_lookup(ctx, a, next->K, next->n_max, next->draft, next->draft_len, next->match_len,
+                                next->match_pos, next->match_cnt, sa, static_cast<cudaStream_t>(stream));
 }
 
 hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
@@ -436,6 +463,20 @@ hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dt
     return verify_commit_impl(ctx, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len, nullptr,
                               select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
                               target_tok, status, stream);
+}
+
+hvd_status hvd_verify_commit_next(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                                  const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                                  const int32_t* sel_draft, const int32_t* sel_len, const int32_t* select,
+                                  int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                                  int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                                  int32_t* committed, int32_t* n_commit, int32_t* target_tok,
+                                  int32_t* status, const hvd_next_cycle* next, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (!next) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_next: NULL pointer");
+    return verify_commit_impl(ctx, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len, nullptr,
+                              select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
+                              target_tok, status, stream, next);
 }
 
 hvd_status hvd_verify_commit_tree(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,

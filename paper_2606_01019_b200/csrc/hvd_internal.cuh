@@ -43,6 +43,7 @@ constexpr int kVerifyUnitBatches = HVD_VERIFY_UNIT_BATCHES;  // 4 KB batches per
 #define HVD_VERIFY_QUEUES 8
 #endif
 constexpr int kVerifyQueues = HVD_VERIFY_QUEUES;  // unit counters
+constexpr int kVerifyQueueStride = 32;           // ... on separate 128-byte lines (in 32-bit words)
 
 
 }  // namespace hvd
@@ -240,6 +241,11 @@ struct VerifyArgs {
 };
 
 hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit = true);
+// commit and the next cycle's lookup + scoring in one kernel (after launch_verify without its commit)
+bool cycle_fits_one_cta(int32_t n_max);
+hvd_status launch_commit_lookup(hvd_ctx* ctx, const VerifyArgs& va, const int32_t* K, int32_t n_max, int32_t* draft,
+                                int32_t* draft_len, int32_t* match_len, int32_t* match_pos, int32_t* match_cnt,
+                                const ScoreArgs& sa, cudaStream_t stream);
 hvd_status launch_verify_keys(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, long long* keys, int64_t v_offset,
                               cudaStream_t stream);
 hvd_status launch_commit_keys(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream);

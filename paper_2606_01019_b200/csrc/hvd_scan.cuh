@@ -49,7 +49,9 @@ __device__ __forceinline__ int4 ld_hist(const int4* p) {
 // qa / qb the tokens 1 + lane and 33 + lane back.  Calls on_match(L, p), in every lane of the warp with the
 // same arguments, for every candidate p in [0, n - 2] of the warp's 32 vectors: p holds q0 and L >= 1 is the
 // match length of the copy that ends there (capped at l_max and at the slab start).
-template <class OnMatch>
+// COHERENT: the tokens compared during the extension are read through the L2 (for a kernel that has itself
+// appended to the history it scans).
+template <bool COHERENT = false, class OnMatch>
 __device__ __forceinline__ void scan_vector(const int4 x, int p0, int n, const int32_t* __restrict__ slab, int32_t q0,
                                             int32_t qa, int32_t qb, int l_max, int lane, OnMatch&& on_match) {
     uint32_t m = 0;
@@ -70,14 +72,14 @@ __device__ __forceinline__ void scan_vector(const int4 x, int p0, int n, const i
             // match length of the copy ending at p (>= 1 already); limit: l_max and the slab start
             const int cap = min(l_max, p + 1);
             int l = lane + 1;
-            bool eq = (l < cap) && (slab[p - l] == qa);
+            bool eq = (l < cap) && ((COHERENT ? __ldcg(slab + p - l) : slab[p - l]) == qa);
             uint32_t mm = __ballot_sync(0xffffffffu, !eq);
             int L;
             if (mm != 0) {
                 L = __ffs(mm);  // first failing lane j: lengths 1..j hold, so L = 1 + j
             } else {
                 l = lane + 33;
-                eq = (l < cap) && (slab[p - l] == qb);
+                eq = (l < cap) && ((COHERENT ? __ldcg(slab + p - l) : slab[p - l]) == qb);
                 mm = __ballot_sync(0xffffffffu, !eq);  // lane 31 (l = 64) always fails
                 L = 32 + __ffs(mm);
             }

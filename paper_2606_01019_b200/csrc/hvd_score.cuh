@@ -48,13 +48,17 @@ __device__ __forceinline__ int bit_width(uint32_t x) { return 32 - __clz((int)x)
 // integer->float conversion or one correctly rounded IEEE operation).
 template <int N>
 __device__ __forceinline__ void payoff_features(const ScoreArgs& a, int b, int n, int d, int L, int pos, int cnt,
-                                                float (&phi)[N]) {
+                                                float (&phi)[N], const hvd_req_state* state_now = nullptr) {
     n = max(n, 0);
     // read-only inputs go through the non-coherent path so that the compiler may issue them early
     const int P = max(__ldg(a.prompt_len + b), 0);
     hvd_req_state st;
-    st.sel_bits = __ldg(&a.state[b].sel_bits);
-    st.acc_ring = __ldg(reinterpret_cast<const unsigned long long*>(&a.state[b].acc_ring));
+    if (state_now) {  // the caller has just updated the summary itself
+        st = *state_now;
+    } else {
+        st.sel_bits = __ldg(&a.state[b].sel_bits);
+        st.acc_ring = __ldg(reinterpret_cast<const unsigned long long*>(&a.state[b].acc_ring));
+    }
     cnt = max(cnt, 0);
     phi[0] = (float)L;
     phi[1] = (float)d;
@@ -175,11 +179,12 @@ __device__ __forceinline__ void select_draft(const ScoreArgs& a, int b, int lane
 template <bool EXT = false>
 __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, int lane, float* s_hid, int n,
                                                      int d, int L, int pos, int cnt, int tok0, int tok1,
-                                                     const ModelDraft* fetched = nullptr) {
+                                                     const ModelDraft* fetched = nullptr,
+                                                     const hvd_req_state* state_now = nullptr) {
     constexpr int N = NFeat<EXT>::value;
     d = max(0, min(d, a.k_cap));
     float phi[N];
-    payoff_features(a, b, n, d, L, pos, cnt, phi);
+    payoff_features(a, b, n, d, L, pos, cnt, phi, state_now);
     if constexpr (EXT) structure_features(a, b, lane, d, tok0, tok1, phi);
     if (a.features && lane < N) {
         float v = phi[0];

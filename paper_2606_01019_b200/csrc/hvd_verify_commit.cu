@@ -26,7 +26,7 @@
 
 #include <algorithm>
 
-#include "hvd_internal.cuh"
+#include "hvd_commit.cuh"
 
 namespace hvd {
 namespace {
@@ -36,7 +36,7 @@ constexpr int NW = T / 32;
 constexpr int U = kVerifyUnroll;
 constexpr int UB = kVerifyUnitBatches;
 constexpr int Q = kVerifyQueues;
-constexpr int kQueueStride = 32;  // counters sit on separate 128-byte lines
+constexpr int kQueueStride = kVerifyQueueStride;
 static_assert(NW % Q == 0, "every CTA must serve every queue equally");
 constexpr int kBatchVec = 32 * U;  // vectors a warp loads per batch
 constexpr uint32_t kFull = 0xffffffffu;
@@ -162,116 +162,6 @@ struct Tracker<__nv_bfloat16> {
         off = ((b16 >> 3) * 32u + (uint32_t)lane) * 8u + (b16 & 7u);
     }
 };
-
-struct Req {
-    int64_t r0, r1;  // logits rows of the request
-    int nr;          // rows needed = sel_len + 1 (0: request skipped)
-};
-
-__device__ __forceinline__ Req load_req(const VerifyArgs& a, int b) {
-    Req q;
-    if (a.row_off) { q.r0 = a.row_off[b]; q.r1 = a.row_off[b + 1]; }
-    else { q.r0 = (int64_t)b * (a.k_uniform + 1); q.r1 = q.r0 + a.k_uniform + 1; }
-    // every input is fetched before any is looked at: one round trip, not a chain of three
-    const int n = a.hist_len[b];
-    const int cap = a.hist_cap[b];
-    const int sl = a.sel_len[b];
-    q.nr = 0;
-    if (n >= 0 && n <= cap && q.r1 > q.r0) {
-        int m = max(0, min(sl, a.k_cap));
-        if ((int64_t)m > q.r1 - q.r0 - 1) m = (int)(q.r1 - q.r0 - 1);
-        q.nr = m + 1;
-    }
-    return q;
-}
-
-constexpr unsigned long long kKeySign = 0x8000000000000000ull;
-
-// The (value, ~index) key of a logits row.  Context scratch is put back to zero as it is read; keys
-// handed in by the caller (hvd_commit_keys) are in signed order and are left alone.
-__device__ __forceinline__ unsigned long long read_row_key(const VerifyArgs& a, int64_t r) {
-    if (a.ext_keys) return (unsigned long long)a.ext_keys[r] ^ kKeySign;  // "row not read" becomes 0
-    const unsigned long long key = a.row_key[r];
-    a.row_key[r] = 0ull;  // scratch is zero at rest
-    return key;
-}
-
-// Commit of one request by one warp, after all its needed rows are folded into the row keys.
-// Every load that does not depend on another is issued up front: the kernel is a short chain of
-// global round trips at the end of every decoding step.
-__device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int lane) {
-    const int kc = a.k_cap;
-    const int32_t* d = a.sel_draft + (int64_t)b * kc;
-    const int d0 = lane < kc ? d[lane] : -1;            // draft tokens lane, lane+32 (k_cap <= 64)
-    const int d1 = lane + 32 < kc ? d[lane + 32] : -1;
-    const int64_t hoff = a.hist_off[b];
-    const int sel = a.select[b];
-    hvd_req_state st = a.state[b];
-    const int n = a.hist_len[b];
-    const int cap = a.hist_cap[b];
-    const Req q = load_req(a, b);
-    int32_t* z = a.committed + (int64_t)b * (kc + 1);
-    if (q.nr == 0) {
-        // skipped request: neutral outputs, nothing else touched
-        for (int j = lane; j <= kc; j += 32) z[j] = -1;
-        if (a.target_tok) for (int64_t r = q.r0 + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
-        if (lane == 0) { a.accepted[b] = 0; a.n_commit[b] = 0; a.status[b] = HVD_REQ_BAD_LEN; }
-        return;
-    }
-    const int m = q.nr - 1;
-    pdl_wait();  // everything above was the request's own data; the row keys come from the streaming kernel
-    // rows lane, lane+32, lane+64 (at most 65 rows): target tokens from the row keys
-    unsigned long long key[3];
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-        const int i = lane + 32 * k;
-        key[k] = 0ull;
-        if (i <= m) {
-            key[k] = read_row_key(a, q.r0 + i);
-        }
-    }
-    int acc = -1;
-    int t_acc = 0;
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-        const int i = lane + 32 * k;
-        int t = (int)(~(uint32_t)(key[k] & 0xffffffffu));
-        t = (int)min((int64_t)max(t, 0), a.V - 1);  // inside the vocabulary whatever the data
-        bool stop = true;
-        if (i <= m) {
-            if (a.target_tok) a.target_tok[q.r0 + i] = t;
-            const int di = k == 0 ? d0 : (k == 1 ? d1 : -1);
-            stop = (i >= m) || (di != t);
-        }
-        const uint32_t stops = __ballot_sync(kFull, stop);
-        if (acc < 0 && stops != 0 && 32 * k <= m) {
-            const int j = __ffs(stops) - 1;
-            acc = 32 * k + j;
-            t_acc = __shfl_sync(kFull, t, j);
-        }
-    }
-    // acc <= m always (row m stops).  Rows beyond m were not read.
-    if (a.target_tok)
-        for (int64_t r = q.r0 + q.nr + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
-    const int room = cap - n;
-    const int w = min(acc + 1, room);
-    int32_t* h = a.hist + hoff;
-    for (int j = lane; j <= kc; j += 32) {
-        const int dj = j < 32 ? d0 : d1;
-        const int tok = (j < acc) ? dj : (j == acc ? t_acc : -1);
-        z[j] = tok;
-        if (j < w) h[n + j] = tok;
-    }
-    if (lane == 0) {
-        a.hist_len[b] = n + w;
-        a.n_commit[b] = w;
-        a.accepted[b] = acc;
-        a.status[b] = (w < acc + 1) ? HVD_REQ_CAPACITY : HVD_REQ_OK;
-        st.sel_bits = (st.sel_bits << 1) | (sel ? 1u : 0u);
-        st.acc_ring = (st.acc_ring << 8) | (unsigned long long)(acc & 0xff);
-        a.state[b] = st;
-    }
-}
 
 // Commit of one request whose draft is a token TREE (node i: token sel_draft[i], parent[i] in
 // {-1, 0..i-1}; logits row 0 follows the prefix, row i+1 follows node i), by one warp.  The walk

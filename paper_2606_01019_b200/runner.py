@@ -98,6 +98,25 @@ class DeviceBatch:
                                    self.target_tok if target_tok else None, self.status)
         self.n_max = min(self.cap_max, self.n_max + self.ctx.k_cap + 1)
 
+    def verify_commit_next(self, logits, target_tok=True, K=None, model_draft=None, model_len=None):
+        """Verification and commit of this cycle, then the next cycle's lookup, score and selection (on the
+        histories just extended) in the same call.  K / model_draft / model_len: the next cycle's inputs
+        (default: this cycle's arrays)."""
+        n_max = min(self.cap_max, self.n_max + self.ctx.k_cap + 1)
+        self.ctx.hvd_verify_commit_next(self.B, logits, self.dtype, self.V, self.row_off, self.k_uniform,
+                                        self.total_rows, self.sel_draft, self.sel_len, self.select, self.hist,
+                                        self.hist_off, self.hist_cap, self.hist_len, self.state,
+                                        self.accepted, self.committed, self.n_commit,
+                                        self.target_tok if target_tok else None, self.status,
+                                        K=self.K if K is None else K, n_max=n_max, prompt_len=self.prompt_len,
+                                        model_draft=self.model_draft if model_draft is None else model_draft,
+                                        model_len=self.model_len if model_len is None else model_len,
+                                        draft=self.draft, draft_len=self.draft_len, match_len=self.match_len,
+                                        match_pos=self.match_pos, match_cnt=self.match_cnt,
+                                        features=self.features, score=self.score, next_select=self.select,
+                                        next_sel_draft=self.sel_draft, next_sel_len=self.sel_len)
+        self.n_max = n_max
+
     def step(self, logits, target_tok=True, fused=False):
         if fused:
             self.lookup_score_select()
