@@ -141,3 +141,45 @@ def test_commit_next_equals_the_two_calls():
         if k in ("freq_score", "match_src", "features_ext"):
             continue
         assert np.array_equal(a.view(np.uint8), b.view(np.uint8)), k
+
+
+def test_host_side_argument_errors():
+    import paper_2606_01019_b200 as H
+    w = small()
+    rng = np.random.default_rng(46)
+    rq = hand_requests(w, [rng.integers(0, 4, 200) for _ in range(3)], [8] * 3)
+    inp = P.prepare(w.scaled(B=3), device="cuda", rq=rq)
+    ctx = G.make_ctx(w, rq)
+    b = G.make_batch(ctx, w, rq)
+    with pytest.raises(H.HvdError, match="hvd_set_predictor first"):
+        b.verify_commit_next(inp.logits)
+    G.set_predictor(ctx, inp)
+    b.lookup_score_select()
+    with pytest.raises(H.HvdError, match="go together"):
+        b.ctx.hvd_verify_commit_next(b.B, inp.logits, b.dtype, b.V, b.row_off, b.k_uniform, b.total_rows, b.sel_draft,
+                                     b.sel_len, b.select, b.hist, b.hist_off, b.hist_cap, b.hist_len, b.state,
+                                     b.accepted, b.committed, b.n_commit, None, b.status, K=b.K, n_max=b.n_max,
+                                     prompt_len=b.prompt_len, model_draft=b.model_draft, model_len=None,
+                                     draft=b.draft, draft_len=b.draft_len, match_len=b.match_len,
+                                     match_pos=b.match_pos, match_cnt=b.match_cnt, features=None, score=b.score,
+                                     next_select=b.select, next_sel_draft=b.sel_draft, next_sel_len=b.sel_len)
+    with pytest.raises(H.HvdError, match="NULL pointer in next"):
+        b.ctx.hvd_verify_commit_next(b.B, inp.logits, b.dtype, b.V, b.row_off, b.k_uniform, b.total_rows, b.sel_draft,
+                                     b.sel_len, b.select, b.hist, b.hist_off, b.hist_cap, b.hist_len, b.state,
+                                     b.accepted, b.committed, b.n_commit, None, b.status, K=b.K, n_max=b.n_max,
+                                     prompt_len=b.prompt_len, model_draft=None, model_len=None,
+                                     draft=b.draft, draft_len=b.draft_len, match_len=b.match_len,
+                                     match_pos=b.match_pos, match_cnt=b.match_cnt, features=None, score=None,
+                                     next_select=b.select, next_sel_draft=b.sel_draft, next_sel_len=b.sel_len)
+    with pytest.raises(H.HvdError, match="n_max"):
+        b.ctx.hvd_verify_commit_next(b.B, inp.logits, b.dtype, b.V, b.row_off, b.k_uniform, b.total_rows, b.sel_draft,
+                                     b.sel_len, b.select, b.hist, b.hist_off, b.hist_cap, b.hist_len, b.state,
+                                     b.accepted, b.committed, b.n_commit, None, b.status, K=b.K, n_max=10**7,
+                                     prompt_len=b.prompt_len, model_draft=None, model_len=None,
+                                     draft=b.draft, draft_len=b.draft_len, match_len=b.match_len,
+                                     match_pos=b.match_pos, match_cnt=b.match_cnt, features=None, score=b.score,
+                                     next_select=b.select, next_sel_draft=b.sel_draft, next_sel_len=b.sel_len)
+    import torch
+    torch.cuda.synchronize()
+    assert ctx.hvd_device_status() == 0
+    ctx.close()
