@@ -72,6 +72,13 @@ def test_chain_of_cycles(name, kw):
     assert grew.any()
 
 
+def test_full_size_c2():
+    """The benchmark's workload at full size (64 histories of 16 384 tokens, vocabulary 128 256)."""
+    inp = P.prepare(W.CONFIGS["C2"], device="cuda")
+    grew = run_chain(inp, inp.rq, 3)
+    assert grew.all()
+
+
 def test_chain_without_host_synchronisation():
     inp = P.prepare(W.CONFIGS["C2"].scaled(B=24, n=3000, V=5003), device="cuda")
     run_chain(inp, inp.rq, 6, check_every_cycle=False)
