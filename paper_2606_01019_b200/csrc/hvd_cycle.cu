@@ -9,7 +9,8 @@
 // with the new tail as the query; only the vectors that overlap the appended tokens are read again
 // (through the L2, where warp 0's stores are).  One launch and two dependent global round trips less
 // per decoding cycle.  Requests must fit one CTA (32 K tokens); the caller falls back to the two
-// separate launches otherwise.
+// separate launches otherwise.  Up to 18 K tokens the CTA has 512 threads, which fit on an SM beside the
+// streaming kernel's CTAs: the loads ahead of the wait then run while the logits still stream.
 #include "hvd_commit.cuh"
 #include "hvd_scan.cuh"
 #include "hvd_score.cuh"
@@ -173,10 +174,13 @@ hvd_status launch_commit_lookup(hvd_ctx* ctx, const VerifyArgs& va, const int32_
     a.n_queues = kVerifyQueues; a.queue_stride = kVerifyQueueStride;
     // one CTA per request: the smallest shape whose aligned grid covers n_max - 1 candidates plus up to
     // 3 tokens of misalignment (the same shapes as the lookup kernel's)
+    // CTAs of at most 512 threads and 64 registers fit on an SM beside the streaming kernel's CTAs, so that
+    // the loads ahead of the wait really run while the logits are still streaming; only the longest histories
+    // take a 1024-thread CTA
     struct Shape { int threads, iter; };
-    static const Shape shapes[] = {{256, 1}, {256, 2}, {512, 2}, {1024, 2}, {1024, 4}, {1024, 8}};
+    static const Shape shapes[] = {{256, 1}, {256, 2}, {512, 2}, {512, 4}, {512, 6}, {512, 8}, {512, 9}, {1024, 8}};
     int pick = -1;
-    for (int k = 0; k < 6; ++k)
+    for (int k = 0; k < 8; ++k)
         if ((int64_t)shapes[k].threads * kLookupTokPerVec * shapes[k].iter >= (int64_t)n_max + 2) { pick = k; break; }
     if (pick < 0) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_next: history too long for one CTA");
     const bool pdl = ctx->use_pdl || ctx->pdl_commit;
@@ -187,8 +191,10 @@ hvd_status launch_commit_lookup(hvd_ctx* ctx, const VerifyArgs& va, const int32_
         case 0: e = HVD_LAUNCH_CYCLE(256, 1); break;
         case 1: e = HVD_LAUNCH_CYCLE(256, 2); break;
         case 2: e = HVD_LAUNCH_CYCLE(512, 2); break;
-        case 3: e = HVD_LAUNCH_CYCLE(1024, 2); break;
-        case 4: e = HVD_LAUNCH_CYCLE(1024, 4); break;
+        case 3: e = HVD_LAUNCH_CYCLE(512, 4); break;
+        case 4: e = HVD_LAUNCH_CYCLE(512, 6); break;
+        case 5: e = HVD_LAUNCH_CYCLE(512, 8); break;
+        case 6: e = HVD_LAUNCH_CYCLE(512, 9); break;
         default: e = HVD_LAUNCH_CYCLE(1024, 8); break;
     }
 #undef HVD_LAUNCH_CYCLE
