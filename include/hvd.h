@@ -42,8 +42,13 @@
  *    variables, read once by hvd_create, change it: HVD_PDL_MASK (a bit per
  *    kernel pair: 1 commit, 2 lookup, 4 verify stream, 8 scoring; default 15,
  *    0 = plain launches) and HVD_ENABLE_PDL (any value: the launch attribute
- *    on every kernel of the library).  Nothing else is read from the
- *    environment by the product path.
+ *    on every kernel of the library).
+ *  - hvd_verify_commit and its variants stream the logits with one of two
+ *    kernels, chosen by the size of the logits: one warp per 4 KB batch of a
+ *    row up to 160 MB, a persistent kernel with work queues beyond that.
+ *    HVD_VERIFY_SMALL_BYTES (read once by hvd_create) moves the limit, 0 =
+ *    always the persistent kernel.  Results do not depend on it.  Nothing
+ *    else is read from the environment by the product path.
  */
 #ifndef HVD_H
 #define HVD_H

@@ -106,6 +106,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     // HVD_PDL_MASK=0 turns it off
     c->pdl_mask = getenv("HVD_PDL_MASK") ? atoi(getenv("HVD_PDL_MASK")) : 15;
     c->pdl_commit = (c->pdl_mask & 1) != 0;
+    c->vf_small_bytes = getenv("HVD_VERIFY_SMALL_BYTES") ? atoll(getenv("HVD_VERIFY_SMALL_BYTES")) : kVerifySmallBytes;
     c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // every kernel of the library, the cluster kernel included: for experiments
     c->host_ws = nullptr;
     c->host_ws_bytes = 0;

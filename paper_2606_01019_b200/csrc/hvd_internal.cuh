@@ -44,6 +44,8 @@ constexpr int kVerifyUnitBatches = HVD_VERIFY_UNIT_BATCHES;  // 4 KB batches per
 #endif
 constexpr int kVerifyQueues = HVD_VERIFY_QUEUES;  // unit counters
 constexpr int kVerifyQueueStride = 32;           // ... on separate 128-byte lines (in 32-bit words)
+constexpr long long kVerifySmallBytes = 160LL << 20;  // logits up to this size: one warp per 4 KB batch
+constexpr long long kVerifySpecBytes = 8LL << 20;     // ... and up to this size: loads before the need is known
 
 
 }  // namespace hvd
@@ -94,6 +96,7 @@ struct hvd_ctx {
     int* dev_error;                  // device status word
     unsigned long long* probe_sink;  // result word of the read-only probe
     int vf_blocks_per_sm[2];         // per dtype
+    long long vf_small_bytes;        // size limit of the warp-per-batch kernels (HVD_VERIFY_SMALL_BYTES; 0 = never)
     // device staging of the host-buffer entry point (grown on demand)
     bool use_pdl;     // programmatic dependent launch for every kernel of the library (HVD_ENABLE_PDL; experiments)
     int pdl_mask;     // ... for the three kernels of a step: bit 0 commit, 1 lookup, 2 stream, 3 one-layer scoring (default all)

@@ -61,6 +61,7 @@ hvd_status setup_device(int device, DeviceSetup** out, const char** why) {
         s.ctx.use_pdl = false;
         s.ctx.pdl_commit = false;
         s.ctx.pdl_mask = 0;
+        s.ctx.vf_small_bytes = kVerifySmallBytes;
         s.ready = true;
     }
     *out = &s;

@@ -21,6 +21,7 @@
 // verify_commit_kernel: one warp per request reads the row keys (the kernel boundary orders them
 // after every atomic), turns them into target tokens, compares them with the draft, commits, and
 // puts the scratch back to zero.
+// verify_small_kernel: the streaming kernel for logits of up to 160 MB (one warp per batch, no queues).
 // No warp waits for another.
 #include <cuda_bf16.h>
 
@@ -472,6 +473,96 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
 
 }  // namespace
 
+// Small calls (a few requests, a few MB of logits): the time of the streaming kernel above is then its chain
+// of dependent round trips (unit counters, per-request prefix, logits, atomic), not bandwidth.  Here one warp
+// takes one 4 KB batch of one logits row, known from its block and warp number alone, and issues its loads at
+// once; whether the row is needed at all (row <= sel_len of its request) is looked up while they are in
+// flight, and only needed rows publish their maximum.  Rows beyond the selected draft are read in vain,
+// which at these sizes costs less than finding out first.  Same keys, same result as the kernel above.
+constexpr int kSmallWarps = 4;
+constexpr int kSmallMaxBatch = 32;  // the request of a row is found by one warp-wide look at row_off
+
+template <typename E, bool SPEC>
+__global__ void __launch_bounds__(kSmallWarps * 32) verify_small_kernel(const VerifyArgs a) {
+    constexpr int EPV = Tracker<E>::kPerVec;
+    constexpr int ESZ = 16 / EPV;
+    const int lane = threadIdx.x & 31;
+    const int gb = blockIdx.x * kSmallWarps + (threadIdx.x >> 5);  // batch inside the row
+    const int64_t r = blockIdx.y;                                  // logits row
+    // wait first, then let the commit kernel in (it reads the selection before its own wait)
+    pdl_wait();
+    pdl_trigger();
+    if (gb >= a.n_batch_row) return;
+
+    const char* row = static_cast<const char*>(a.logits) + r * a.V * ESZ;
+    const int head_bytes = (int)((16 - (reinterpret_cast<uintptr_t>(row) & 15)) & 15);
+    const int head = (int)min((int64_t)(head_bytes / ESZ), a.V);
+    const int n_vec = (int)((a.V - head) / EPV);
+    const int tail = (int)(a.V - head - (int64_t)n_vec * EPV);
+    const uint4* vrow = reinterpret_cast<const uint4*>(row + (int64_t)head * ESZ);
+    const int left = n_vec - gb * kBatchVec;
+    const uint4* ptr = vrow + (int64_t)gb * kBatchVec + lane;
+    const unsigned long long pol = stream_policy();
+
+    uint32_t lord = 0u, loff = 0xffffffffu;
+    const bool full = left >= kBatchVec;
+    uint4 x[U];
+    if (SPEC && (full || lane < left)) {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (full || u * 32 + lane < left) x[u] = ld_stream(ptr + u * 32, pol);
+    }
+    // the row's request (with SPEC: while the loads are in flight)
+    int b;
+    if (a.row_off && a.B <= 32) {
+        const int64_t lo = lane < a.B ? a.row_off[lane] : 0;
+        const int64_t hi = lane < a.B ? a.row_off[lane + 1] : 0;
+        const uint32_t mine = __ballot_sync(kFull, lane < a.B && lo <= r && r < hi);
+        b = mine ? __ffs(mine) - 1 : -1;
+    } else if (a.row_off) {
+        int lo = 0, hi = a.B;  // largest b with row_off[b] <= r
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (a.row_off[mid] <= r) lo = mid; else hi = mid;
+        }
+        b = (a.row_off[lo] <= r && r < a.row_off[lo + 1]) ? lo : -1;
+    } else {
+        b = (int)(r / (a.k_uniform + 1));
+        if (b >= a.B) b = -1;
+    }
+    bool needed = false;
+    if (b >= 0) {
+        const Req q = load_req(a, b);
+        needed = r - q.r0 < q.nr;
+    }
+    if (!SPEC) {
+        if (!needed) return;  // warp-uniform
+        if (full || lane < left) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (full || u * 32 + lane < left) x[u] = ld_stream(ptr + u * 32, pol);
+        }
+    }
+    if (full || lane < left) {
+        Tracker<E> t;
+        t.init(x[0]);
+#pragma unroll
+        for (int u = 1; u < U; ++u)
+            if (full || u * 32 + lane < left) t.fold(x[u], u);
+        t.best(lane, lord, loff);
+        loff += (uint32_t)(head + gb * kBatchVec * EPV);
+    }
+    if (gb == 0 && lane < head + tail) {  // the ragged edges of the row ride along with batch 0
+        const int idx = lane < head ? lane : head + n_vec * EPV + (lane - head);
+        const uint32_t eord = ord32(Tracker<E>::scalar(row, idx));
+        if (eord > lord || (eord == lord && (uint32_t)idx < loff)) { lord = eord; loff = (uint32_t)idx; }
+    }
+    const uint32_t word = __reduce_max_sync(kFull, lord);
+    const uint32_t widx = __reduce_min_sync(kFull, lord == word ? loff : 0xffffffffu);
+    if (needed && lane == 0 && word != 0u && widx != 0xffffffffu)
+        atomicMax(a.row_key + r, ((unsigned long long)word << 32) | (uint32_t)(~widx));
+}
+
 size_t verify_dyn_smem(int32_t B) { return (size_t)B * 8 + (size_t)(B + 1) * 4; }
 
 int verify_occupancy(hvd_dtype dtype, size_t dyn_smem) {
@@ -523,7 +614,26 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
     if (a.total_rows * (int64_t)a.n_batch_row / UB + 4 * (int64_t)grid * NW >= 0x7fffffffLL)
         return fail(ctx, HVD_ERR_UNSUPPORTED, "hvd_verify_commit: too many batches");
     const size_t smem = verify_dyn_smem(a.B);
-    if (dtype == HVD_F32)
+    // By the full size of the logits (the needed part is only known on the device): up to 8 MB one warp per
+    // batch with loads issued before the row is known to be needed, up to vf_small_bytes (160 MB) one warp
+    // per batch that checks first, beyond that the persistent streaming kernel.  Measured, verify call with
+    // half the rows needed, bf16 rows of 128 256: 4.4 MB 6.3 / 4.0 / 4.4 us (streaming / loads first / check
+    // first), 17 MB 7.5 / 6.6 / 6.3, 70 MB 12.3 / 14.2 / 10.6, 140 MB 17.7 / 24.0 / 16.0, 279 MB 26.9 / 50.8 / 31.0.
+    const int64_t full_bytes = a.total_rows * a.V * esz;
+    const bool small = a.total_rows <= 65535 && full_bytes <= ctx->vf_small_bytes;
+    const bool spec = full_bytes <= kVerifySpecBytes;
+    if (small) {
+        const dim3 sgrid((unsigned)((a.n_batch_row + kSmallWarps - 1) / kSmallWarps), (unsigned)a.total_rows);
+        const bool pdl = ctx->use_pdl || (ctx->pdl_mask & 4);
+        cudaError_t e;
+        if (dtype == HVD_F32)
+            e = spec ? launch_kernel(pdl, verify_small_kernel<float, true>, sgrid, kSmallWarps * 32, 0, stream, a)
+                     : launch_kernel(pdl, verify_small_kernel<float, false>, sgrid, kSmallWarps * 32, 0, stream, a);
+        else
+            e = spec ? launch_kernel(pdl, verify_small_kernel<__nv_bfloat16, true>, sgrid, kSmallWarps * 32, 0, stream, a)
+                     : launch_kernel(pdl, verify_small_kernel<__nv_bfloat16, false>, sgrid, kSmallWarps * 32, 0, stream, a);
+        HVD_CUDA_TRY(ctx, e);
+    } else if (dtype == HVD_F32)
         HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 4), verify_stream_kernel<float>, grid, T, smem, stream, a));
     else
         HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 4), verify_stream_kernel<__nv_bfloat16>, grid, T, smem, stream, a));

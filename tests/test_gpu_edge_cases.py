@@ -295,3 +295,27 @@ def test_parity_with_plain_launches():
     res = subprocess.run(cmd, cwd=root, env=env, capture_output=True, text=True, timeout=900)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
     assert " passed" in res.stdout
+
+
+def _rerun(env_over, files, select):
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    cmd = [sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", *files, "-k", select]
+    res = subprocess.run(cmd, cwd=root, env=dict(os.environ, **env_over), capture_output=True, text=True, timeout=1200)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
+    assert " passed" in res.stdout
+
+
+def test_parity_with_the_persistent_streaming_kernel_only():
+    """Logits of up to 160 MB are streamed by the warp-per-batch kernels, so most cases of this suite never
+    reach the persistent kernel: the shape, alignment, tie and multi-step cases once more with the limit at 0."""
+    _rerun({"HVD_VERIFY_SMALL_BYTES": "0"}, ["tests/test_gpu_parity.py", "tests/test_gpu_edge_cases.py"],
+           "not full_size and not plain_launches and not kernel_only and not 65535 and not read_probe")
+
+
+def test_parity_with_the_warp_per_batch_kernel_on_a_large_call():
+    """... and the other way round: the full-size C2 and C5 workloads (279 MB and 2.5 GB of logits, uniform and
+    ragged rows) through the warp-per-batch kernel that checks the need first."""
+    _rerun({"HVD_VERIFY_SMALL_BYTES": str(1 << 40)}, ["tests/test_gpu_parity.py"], "full_size and (C2 or C5)")
