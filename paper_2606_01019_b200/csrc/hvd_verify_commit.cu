@@ -512,28 +512,54 @@ __global__ void __launch_bounds__(kSmallWarps * 32) verify_small_kernel(const Ve
         for (int u = 0; u < U; ++u)
             if (full || u * 32 + lane < left) x[u] = ld_stream(ptr + u * 32, pol);
     }
-    // the row's request (with SPEC: while the loads are in flight)
-    int b;
-    if (a.row_off && a.B <= 32) {
-        const int64_t lo = lane < a.B ? a.row_off[lane] : 0;
-        const int64_t hi = lane < a.B ? a.row_off[lane + 1] : 0;
-        const uint32_t mine = __ballot_sync(kFull, lane < a.B && lo <= r && r < hi);
-        b = mine ? __ffs(mine) - 1 : -1;
-    } else if (a.row_off) {
-        int lo = 0, hi = a.B;  // largest b with row_off[b] <= r
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (a.row_off[mid] <= r) lo = mid; else hi = mid;
-        }
-        b = (a.row_off[lo] <= r && r < a.row_off[lo + 1]) ? lo : -1;
-    } else {
-        b = (int)(r / (a.k_uniform + 1));
-        if (b >= a.B) b = -1;
-    }
+    // the row's request and whether it needs the row (with SPEC: while the loads are in flight)
     bool needed = false;
-    if (b >= 0) {
-        const Req q = load_req(a, b);
-        needed = r - q.r0 < q.nr;
+    if (a.row_off && a.B <= 1024) {
+        // Lane j fetches everything about request base + j in one round trip and the lane whose request owns
+        // the row decides.  With more than 32 requests a first round trip over 32 evenly spaced entries of
+        // row_off finds the block of (B + 31) / 32 <= 32 requests, from `base` on, that holds the row's owner.
+        int base = 0;
+        if (a.B > 32) {
+            const int stride = (a.B + 31) / 32;
+            const int j = min(lane * stride, a.B);
+            const uint32_t below = __ballot_sync(kFull, a.row_off[j] <= r);  // lanes 0..s (row_off is sorted)
+            base = below ? (31 - __clz((int)below)) * stride : 0;  // the owner is one of the next `stride` requests
+        }
+        const int jb = base + lane;
+        const bool in = jb < a.B && lane < ((a.B > 32) ? (a.B + 31) / 32 : 32);
+        const int64_t lo = in ? a.row_off[jb] : 0;
+        const int64_t hi = in ? a.row_off[jb + 1] : 0;
+        const int n = in ? a.hist_len[jb] : -1;
+        const int cap = in ? a.hist_cap[jb] : 0;
+        const int sl = in ? a.sel_len[jb] : 0;
+        bool mine = in && lo <= r && r < hi;
+        if (mine) {
+            int nr = 0;
+            if (n >= 0 && n <= cap) {  // the rule of load_req
+                int m = max(0, min(sl, a.k_cap));
+                if ((int64_t)m > hi - lo - 1) m = (int)(hi - lo - 1);
+                nr = m + 1;
+            }
+            mine = r - lo < nr;
+        }
+        needed = __any_sync(kFull, mine);
+    } else {
+        int b;
+        if (a.row_off) {
+            int lo = 0, hi = a.B;  // largest b with row_off[b] <= r
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (a.row_off[mid] <= r) lo = mid; else hi = mid;
+            }
+            b = (a.row_off[lo] <= r && r < a.row_off[lo + 1]) ? lo : -1;
+        } else {
+            b = (int)(r / (a.k_uniform + 1));
+            if (b >= a.B) b = -1;
+        }
+        if (b >= 0) {
+            const Req q = load_req(a, b);
+            needed = r - q.r0 < q.nr;
+        }
     }
     if (!SPEC) {
         if (!needed) return;  // warp-uniform
@@ -617,8 +643,9 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
     // By the full size of the logits (the needed part is only known on the device): up to 8 MB one warp per
     // batch with loads issued before the row is known to be needed, up to vf_small_bytes (160 MB) one warp
     // per batch that checks first, beyond that the persistent streaming kernel.  Measured, verify call with
-    // half the rows needed, bf16 rows of 128 256: 4.4 MB 6.3 / 4.0 / 4.4 us (streaming / loads first / check
-    // first), 17 MB 7.5 / 6.6 / 6.3, 70 MB 12.3 / 14.2 / 10.6, 140 MB 17.7 / 24.0 / 16.0, 279 MB 26.9 / 50.8 / 31.0.
+    // half the rows needed, bf16 rows of 128 256 (streaming / loads first / check first): 4.4 MB 6.3 / 3.8 /
+    // 4.2 us, 17 MB 7.5 / - / 5.8, 70 MB 12.3 / - / 10.0, 140 MB 17.7 / - / 14.9, 279 MB 26.9 / - / 26.4; with
+    // (nearly) all rows needed the persistent kernel is ahead from about 150 MB on (279 MB: 41.7 against 50.7 us).
     const int64_t full_bytes = a.total_rows * a.V * esz;
     const bool small = a.total_rows <= 65535 && full_bytes <= ctx->vf_small_bytes;
     const bool spec = full_bytes <= kVerifySpecBytes;
