@@ -480,7 +480,6 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
 // flight, and only needed rows publish their maximum.  Rows beyond the selected draft are read in vain,
 // which at these sizes costs less than finding out first.  Same keys, same result as the kernel above.
 constexpr int kSmallWarps = 4;
-constexpr int kSmallMaxBatch = 32;  // the request of a row is found by one warp-wide look at row_off
 
 template <typename E, bool SPEC>
 __global__ void __launch_bounds__(kSmallWarps * 32) verify_small_kernel(const VerifyArgs a) {
