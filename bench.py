@@ -57,6 +57,8 @@ def parse_args():
     ap.add_argument("--vocab-shards", action="store_true",
                     help="variant of the verify step: one rank's share under a vocabulary-parallel output layer "
                          "(hvd_verify_keys on a 1/S slice of every row + hvd_commit_keys), S = 2, 4, 8")
+    ap.add_argument("--verify-sweep", action="store_true",
+                    help="the verify call over batch sizes 1..64 (C2's rows), with both streaming kernels")
     ap.add_argument("--replay", action="store_true",
                     help="second workload: payoff labels by trace replay (hvd_replay_labels) on one history of the config")
     ap.add_argument("--unfused", action="store_true",
@@ -383,20 +385,29 @@ def run_vocab_shards(args):
     import hvd_workloads as W
     import paper_2606_01019_b200 as H
     from paper_2606_01019_b200.runner import DeviceBatch
-    from oracle import pipeline as P
     torch.cuda.set_device(0)
     w = W.CONFIGS[args.config]
-    inp = P.prepare(w, device="cuda")
-    rq = inp.rq
+    # inputs as in the main arm: the selection comes from the CUDA path itself, the logits are planted on it
+    rq = W.make_requests(w)
+    W1, b1, W2, b2, tau = W.make_predictor(w)
     B, rows = rq.B, int(rq.row_off[-1])
     ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=rows, max_vocab=w.V,
                     l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
-    ctx.hvd_set_predictor(inp.W1, inp.b1, inp.W2, inp.b2, inp.tau)
+    ctx.hvd_set_predictor(W1, b1, W2, b2, tau)
     batch = DeviceBatch(ctx, hist=rq.hist, hist_off=rq.hist_off, hist_cap=rq.hist_cap, hist_len=rq.hist_len, K=rq.K,
                         prompt_len=rq.prompt_len, state=rq.state, model_draft=rq.model_draft, model_len=rq.model_len,
                         row_off=rq.row_off, V=w.V, dtype=w.dtype)
     batch.lookup_score_select()
-    full = inp.logits.reshape(-1)[: rows * w.V].reshape(rows, w.V)
+    if w.calibrate_cache_frac is not None:
+        torch.cuda.synchronize()
+        tau = W.calibrate_tau(batch.score.cpu().numpy(), batch.draft_len.cpu().numpy() > 0, w.calibrate_cache_frac)
+        ctx.hvd_set_predictor(W1, b1, W2, b2, tau)
+        batch.lookup_score_select()
+    torch.cuda.synchronize()
+    sel_len_h, sel_draft_h = batch.sel_len.cpu().numpy(), batch.sel_draft.cpu().numpy()
+    logits = W.make_logits(w, rows, device="cuda")
+    W.plant_agreement(w, logits, rq.row_off, sel_draft_h, sel_len_h, W.make_agreement(w, sel_len_h))
+    full = logits.reshape(-1)[: rows * w.V].reshape(rows, w.V)
     needed = int((batch.sel_len.cpu().numpy().astype(np.int64) + 1).sum())
     hist_len0, state0 = batch.hist_len.clone(), batch.state.clone()
     reps = max(3, min(args.steps, 50))
@@ -453,6 +464,87 @@ def run_vocab_shards(args):
     ctx.close()
 
 
+# ----------------------------------------------------------------------------------------------
+# the verify call from one request to a full batch: which streaming kernel serves which size
+# ----------------------------------------------------------------------------------------------
+def run_verify_sweep(args):
+    """hvd_verify_commit on 1..64 requests with C2's logits rows (K + 1 = 17 rows of 128 256 bf16 per request),
+    selected draft lengths uniform in 0..K (about half the rows needed), timed with the persistent streaming
+    kernel only (HVD_VERIFY_SMALL_BYTES=0) and with the library's own choice.  Inputs are random: nothing is
+    checked here (the parity tests do that), only timed."""
+    import torch
+    import hvd_workloads as W
+    import paper_2606_01019_b200 as H
+    from paper_2606_01019_b200.runner import DeviceBatch
+    torch.cuda.set_device(0)
+    reps = max(3, min(args.steps, 40))
+    cases = []
+    for B in (1, 2, 4, 8, 16, 32, 64):
+        w = W.CONFIGS["C2"].scaled(B=B, n=2048)
+        rq = W.make_requests(w)
+        rows = int(rq.row_off[-1])
+        full_bytes = rows * w.V * w.elt
+        R = int(max(2, min(40, -(-4 * L2_BYTES // full_bytes))))
+        logits = [W.make_logits(w, rows, device="cuda", salt=r) for r in range(R)]
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(1000 + B)
+        sel_len = torch.randint(0, w.K + 1, (B,), generator=gen, device="cuda", dtype=torch.int32)
+        sel_draft = torch.randint(0, w.V, (B, w.k_cap), generator=gen, device="cuda", dtype=torch.int32)
+        needed_bytes = int((sel_len.cpu().numpy().astype(np.int64) + 1).sum()) * w.V * w.elt
+        us = {}
+        for kind, env in (("persistent", "0"), ("default", None)):
+            old = os.environ.pop("HVD_VERIFY_SMALL_BYTES", None)
+            if env is not None:
+                os.environ["HVD_VERIFY_SMALL_BYTES"] = env
+            ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=rows,
+                            max_vocab=w.V, l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
+            os.environ.pop("HVD_VERIFY_SMALL_BYTES", None)
+            if old is not None:
+                os.environ["HVD_VERIFY_SMALL_BYTES"] = old
+            b = DeviceBatch(ctx, hist=rq.hist, hist_off=rq.hist_off, hist_cap=rq.hist_cap, hist_len=rq.hist_len, K=rq.K,
+                            prompt_len=rq.prompt_len, state=rq.state, model_draft=rq.model_draft,
+                            model_len=rq.model_len, row_off=rq.row_off, V=w.V, dtype=w.dtype)
+            b.sel_len.copy_(sel_len); b.sel_draft.copy_(sel_draft); b.select.zero_()
+            hl0, st0 = b.hist_len.clone(), b.state.clone()
+
+            def body(i, with_call):
+                b.hist_len.copy_(hl0); b.state.copy_(st0)
+                if with_call:
+                    b.verify_commit(logits[i % R], target_tok=False)
+
+            for i in range(3):
+                body(i, True)
+            torch.cuda.synchronize()
+            stream = torch.cuda.Stream()
+            t = []
+            for with_call in (True, False):   # the same graph with and without the call
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(stream):
+                    g.capture_begin()
+                    for i in range(reps):
+                        body(i, with_call)
+                    g.capture_end()
+                torch.cuda.synchronize()
+                with torch.cuda.stream(stream):
+                    g.replay()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(); g.replay(); e1.record()
+                torch.cuda.synchronize()
+                t.append(e0.elapsed_time(e1))
+            us[kind] = (t[0] - t[1]) / reps * 1e3
+            ctx.close()
+        cases.append({"requests": B, "logits_bytes": full_bytes, "needed_bytes": needed_bytes,
+                      "us_persistent_kernel": us["persistent"], "us_library_choice": us["default"],
+                      "gbs_library_choice": needed_bytes / (us["default"] * 1e-6) / 1e9})
+    line = {"metric": "hvd_verify_commit call over batch sizes", "value": cases[0]["us_library_choice"], "unit": "us",
+            "n_gpus": 1, "steps": reps, "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "C2's logits rows (17 rows of 128256 bf16 per request), 1..64 requests, selected draft "
+                                   "lengths uniform in 0..16; calls in a CUDA graph on rotating logits copies larger than "
+                                   "L2 in total; time = graph with the calls minus the same graph without them"},
+            "cases": cases}
+    print(json.dumps(line), flush=True)
+
+
 def workload_config(w, n_gpus, extra=None):
     cfg = {"workload": f"{w.name}: batch {w.B}, histories {w.n} tokens, vocab {w.V}, K {w.K}, {w.dtype} logits",
            "requests_per_gpu": w.B, "parallelism": f"requests sharded over {n_gpus} GPU(s), no collective"}
@@ -477,6 +569,9 @@ def main():
         return
     if args.vocab_shards:
         run_vocab_shards(args)
+        return
+    if args.verify_sweep:
+        run_verify_sweep(args)
         return
     if args.replay:
         run_replay(args)

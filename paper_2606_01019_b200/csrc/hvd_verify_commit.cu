@@ -642,9 +642,9 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
     // By the full size of the logits (the needed part is only known on the device): up to 8 MB one warp per
     // batch with loads issued before the row is known to be needed, up to vf_small_bytes (160 MB) one warp
     // per batch that checks first, beyond that the persistent streaming kernel.  Measured, verify call with
-    // half the rows needed, bf16 rows of 128 256 (streaming / loads first / check first): 4.4 MB 6.3 / 3.8 /
-    // 4.2 us, 17 MB 7.5 / - / 5.8, 70 MB 12.3 / - / 10.0, 140 MB 17.7 / - / 14.9, 279 MB 26.9 / - / 26.4; with
-    // (nearly) all rows needed the persistent kernel is ahead from about 150 MB on (279 MB: 41.7 against 50.7 us).
+    // about half the rows needed, bf16 rows of 128 256 (persistent kernel -> warp per batch): 4.4 MB 6.3 -> 3.8 us,
+    // 17 MB 7.5 -> 5.5, 70 MB 11.2 -> 9.0, 140 MB 17.6 -> 14.5, 279 MB 27.8 -> 26.4; with (nearly) all rows
+    // needed the persistent kernel is ahead from about 150 MB on (279 MB: 41.7 against 50.7 us).
     const int64_t full_bytes = a.total_rows * a.V * esz;
     const bool small = a.total_rows <= 65535 && full_bytes <= ctx->vf_small_bytes;
     const bool spec = full_bytes <= kVerifySpecBytes;
