@@ -400,9 +400,11 @@ HVD_API hvd_status hvd_verify_commit_tree(hvd_ctx* ctx, int32_t B, const void* l
  * for the stream, and appends the committed tokens to the host histories.  Every pointer in the
  * struct is a HOST pointer (pinned memory makes the copies asynchronous and faster; pageable
  * memory works).  Arrays have the shapes documented at the three device entry points.
+ * Of the logits only the rows that verification reads (rows 0..sel_len of every valid request)
+ * are copied: the call waits for the selection in between, then copies those rows.
  * The context keeps a device staging area that it (re)allocates when a call needs more than any
  * earlier one (a synchronous cudaMalloc: not for use inside stream capture).  This entry point
- * synchronises `stream` before returning.
+ * synchronises `stream` twice (after the selection, and before returning).
  */
 typedef struct {
     int32_t B;

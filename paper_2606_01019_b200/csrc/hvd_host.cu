@@ -112,7 +112,6 @@ extern "C" hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args
         H2D(s.model_len, a.model_len, B * 4);
     }
     if (a.row_off) H2D(s.row_off, a.row_off, (B + 1) * 8);
-    H2D(s.logits, a.logits, (size_t)a.total_rows * (size_t)a.V * esz);
 
     hvd_status r = hvd_lookup(ctx, a.B, s.hist, s.hist_off, s.hist_cap, s.hist_len, s.K, a.n_max, s.draft,
                               s.draft_len, s.match_len, s.match_pos, s.match_cnt, st);
@@ -122,6 +121,32 @@ extern "C" hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args
                          a.model_draft ? s.model_len : nullptr, nullptr, s.score, s.select, s.sel_draft,
                          s.sel_len, st);
     if (r != HVD_OK) return r;
+
+    // The logits are the bulk of the bytes that cross the bus, and verification reads only rows 0..sel_len of
+    // a request: bring the selection back first and copy just those rows (adjacent ranges in one copy).
+    D2H(a.sel_len, s.sel_len, B * 4);
+    HVD_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+    {
+        const size_t row_bytes = (size_t)a.V * esz;
+        int64_t run0 = 0, run1 = 0;  // pending range of rows
+        for (int32_t b = 0; b <= a.B; ++b) {
+            int64_t r0 = 0, r1 = 0;
+            if (b < a.B) {
+                r0 = a.row_off ? a.row_off[b] : (int64_t)b * (a.k_uniform + 1);
+                const int64_t rend = a.row_off ? a.row_off[b + 1] : r0 + a.k_uniform + 1;
+                const bool ok = a.hist_len[b] >= 0 && a.hist_len[b] <= a.hist_cap[b] && rend > r0 && r0 >= 0 &&
+                                rend <= a.total_rows;
+                int64_t m = a.sel_len[b] < 0 ? 0 : (a.sel_len[b] > kc ? kc : a.sel_len[b]);
+                if (m > rend - r0 - 1) m = rend - r0 - 1;
+                r1 = ok ? r0 + m + 1 : r0;
+            }
+            if (b < a.B && r1 > r0 && r0 == run1 && run1 > run0) { run1 = r1; continue; }  // extends the pending range
+            if (run1 > run0)
+                H2D(s.logits + (size_t)run0 * row_bytes, static_cast<const char*>(a.logits) + (size_t)run0 * row_bytes,
+                    (size_t)(run1 - run0) * row_bytes);
+            run0 = r0; run1 = r1;
+        }
+    }
     r = hvd_verify_commit(ctx, a.B, s.logits, (hvd_dtype)a.dtype, a.V, a.row_off ? s.row_off : nullptr,
                           a.k_uniform, a.total_rows, s.sel_draft, s.sel_len, s.select, s.hist, s.hist_off,
                           s.hist_cap, s.hist_len, s.state, s.accepted, s.committed, s.n_commit, nullptr,
@@ -131,7 +156,6 @@ extern "C" hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args
     D2H(a.score, s.score, B * 4);
     D2H(a.select, s.select, B * 4);
     D2H(a.sel_draft, s.sel_draft, B * kc * 4);
-    D2H(a.sel_len, s.sel_len, B * 4);
     D2H(a.accepted, s.accepted, B * 4);
     D2H(a.committed, s.committed, B * (kc + 1) * 4);
     D2H(a.n_commit, s.n_commit, B * 4);
