@@ -26,6 +26,31 @@ def test_library_exports_every_declared_symbol():
     assert lib.hvd_status_string(0) == b"HVD_OK" and lib.hvd_status_string(3) == b"HVD_ERR_UNSUPPORTED"
 
 
+def test_binding_structs_have_the_layout_of_the_header(tmp_path):
+    """The ctypes mirrors of the header's structs (sizes and the offset of every field) against what a C
+    compiler makes of include/hvd.h."""
+    import ctypes as C
+    from paper_2606_01019_b200 import binding as b
+    pairs = [("hvd_config", b.HvdConfig), ("hvd_host_step_args", b.HvdHostStepArgs), ("hvd_next_cycle", b.NextCycle)]
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "hvd.h"', 'int main(void) {']
+    for cname, cls in pairs:
+        lines.append(f'  printf("{cname} %zu", sizeof({cname}));')
+        for field, _ in cls._fields_:
+            lines.append(f'  printf(" %zu", offsetof({cname}, {field}));')
+        lines.append('  printf("\\n");')
+    lines += ['  return 0;', '}']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.strip().splitlines()
+    assert len(out) == len(pairs)
+    for line, (cname, cls) in zip(out, pairs):
+        got = line.split()
+        want = [cname, str(C.sizeof(cls))] + [str(getattr(cls, f).offset) for f, _ in cls._fields_]
+        assert got == want, (cname, got, want)
+
+
 def test_no_cpu_fallback_without_a_device():
     import torch
     import pytest
