@@ -40,7 +40,7 @@ struct ScoreArgs {
 
 constexpr int kW1StrideExt = 16;  // row stride of the first layer's weights for the extended vector
 template <bool EXT>
-struct NFeat { static constexpr int value = EXT ? HVD_N_FEATURES_EXT : HVD_N_FEATURES; };
+struct NFeat { static constexpr int value = EXT ? (int)HVD_N_FEATURES_EXT : (int)HVD_N_FEATURES; };
 
 __device__ __forceinline__ int bit_width(uint32_t x) { return 32 - __clz((int)x); }
 
