@@ -976,6 +976,13 @@ def main():
                                   "frac": (lookup_bytes + verify_bytes) / (elapsed_ms / K_steps * 1e-3) / 1e9 / peak_gbs},
                 "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": (4 if args.unfused else 3) * K_steps,
                 "clocks": sampler.summary(window)}
+        if kt:
+            # the same K steps with hvd_verify_commit_next (commit + next cycle's lookup and selection in one
+            # kernel: two launches per step), single rank's figure; the headline keeps the separate entry points
+            line["variant_commit_fused_with_next_lookup"] = {
+                "value": 1.0 / (kt["step_us_commit_fused_with_next_lookup"] * 1e-6), "unit": UNIT,
+                "us_per_step": kt["step_us_commit_fused_with_next_lookup"],
+                "entry_points": "hvd_verify_commit_next (after one hvd_lookup_score_select)"}
         print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:
