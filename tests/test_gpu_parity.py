@@ -104,9 +104,17 @@ def test_multi_step_loop_and_scratch_reuse():
 def test_host_buffer_entry_point():
     """hvd_step_host: same step with host arrays in and out (copies inside the call)."""
     import paper_2606_01019_b200 as H
-    for name, kw in (("C1", {}), ("C5", dict(B=24, n=(64, 3000), V=20011))):
-        w = W.CONFIGS[name].scaled(**kw)
-        inp = P.prepare(w, device="cpu")
+    from tests.test_gpu_edge_cases import hand_requests, small
+    rng = np.random.default_rng(77)
+    we = small()
+    hists = [rng.integers(0, 3, n) for n in (0, 1, 5, 300, 301, 302, 1500, 1501, 2000)]
+    lens = [len(h) for h in hists]
+    lens[6], lens[7] = -2, len(hists[7]) + 500             # lengths outside the slab: no logits rows are copied
+    rq_e = hand_requests(we, hists, [8] * len(hists), cap_extra=[36, 36, 36, 0, 1, 3, 36, 36, 36], hist_len=lens)
+    cases = [(W.CONFIGS["C1"], None, False), (W.CONFIGS["C5"].scaled(B=24, n=(64, 3000), V=20011), None, False),
+             (we.scaled(B=rq_e.B), rq_e, False), (we.scaled(B=rq_e.B), rq_e, True)]
+    for w, rq_given, uniform in cases:
+        inp = P.prepare(w, device="cpu", rq=rq_given)
         rq_g, rq_o = inp.rq.copy(), inp.rq.copy()
         ctx = G.make_ctx(w, rq_g)
         ctx.hvd_set_predictor(inp.W1, inp.b1, inp.W2, inp.b2, inp.tau)
@@ -120,7 +128,8 @@ def test_host_buffer_entry_point():
                               hist_cap=rq_g.hist_cap, hist_len=rq_g.hist_len, K=rq_g.K, prompt_len=rq_g.prompt_len,
                               state=rq_g.state, model_draft=rq_g.model_draft, model_len=rq_g.model_len,
                               logits=inp.logits_np, dtype=H.F32 if w.dtype == "f32" else H.BF16, V=w.V,
-                              row_off=rq_g.row_off, k_uniform=0, total_rows=int(rq_g.row_off[-1]), **o)
+                              row_off=None if uniform else rq_g.row_off, k_uniform=w.k_cap if uniform else 0,
+                              total_rows=int(rq_g.row_off[-1]), **o)
             out = P.step(inp, rq_o)
             G.assert_equal("score", o["score"], out.sc.score)
             for k in ("select", "sel_draft", "sel_len"):
