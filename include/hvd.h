@@ -84,6 +84,13 @@ typedef enum {
     HVD_REQ_BAD_LEN = 2   /* hist_len outside [0, hist_cap] or no logits rows: request skipped */
 } hvd_req_status;
 
+/* values of the device status word (hvd_device_status) */
+typedef enum {
+    HVD_DEV_OK = 0,
+    HVD_DEV_WAIT_EXPIRED = 1, /* a kernel gave up a bounded wait for its own copies: outputs incomplete */
+    HVD_DEV_OUT_OF_BOUNDS = 2 /* bounds-checked builds only: an index left its array; the access was skipped */
+} hvd_dev_status;
+
 /* Recent-history summary h of one request (Sec. 3.3; Algorithm 1 "update C and h").
    bit j of sel_bits = 1 if the cache draft was verified j steps ago;
    byte j of acc_ring = accepted length j steps ago. */

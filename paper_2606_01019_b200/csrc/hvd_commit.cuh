@@ -20,6 +20,9 @@ __device__ __forceinline__ Req load_req(const VerifyArgs& a, int b) {
     const int cap = a.hist_cap[b];
     const int sl = a.sel_len[b];
     q.nr = 0;
+    // rows outside the logits array (a row_off entry below 0 or beyond total_rows): the request is skipped and
+    // its row range emptied, so that neither the logits nor the row keys nor target_tok are touched there
+    if (q.r0 < 0 || q.r1 > a.total_rows || q.r1 < q.r0) { q.r0 = 0; q.r1 = 0; }
     if (n >= 0 && n <= cap && q.r1 > q.r0) {
         int m = max(0, min(sl, a.k_cap));
         if ((int64_t)m > q.r1 - q.r0 - 1) m = (int)(q.r1 - q.r0 - 1);

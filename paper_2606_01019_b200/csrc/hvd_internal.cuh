@@ -170,6 +170,7 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
                          int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream,
                          bool successor_works_ahead = false);
 
+
 ScoreArgs make_score_args(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
                           const hvd_req_state* state, const int32_t* K, const int32_t* draft,
                           const int32_t* draft_len, const int32_t* match_len, const int32_t* match_pos,

@@ -15,27 +15,6 @@
 namespace hvd {
 namespace {
 
-struct LookupArgs {
-    const int32_t* hist;
-    const int64_t* hist_off;
-    const int32_t* hist_cap;
-    const int32_t* hist_len;
-    const int32_t* K;
-    int32_t n_max;
-    int32_t* draft;
-    int32_t* draft_len;
-    int32_t* match_len;
-    int32_t* match_pos;
-    int32_t* match_cnt;
-    LookupPartial* partial;
-    uint32_t* req_cnt;
-    int32_t max_chunks;
-    int32_t k_cap, l_max, min_match;
-    float spec_factor, spec_offset;
-    bool successor_works_ahead;
-    bool chunks_on_x;
-};
-
 template <int THREADS, int ITER, bool FUSED>
 __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 512 ? 2 : 4))) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
     __shared__ float s_hid[FUSED ? HVD_MAX_HIDDEN : 1];
@@ -183,6 +162,8 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
                          int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream,
                          bool successor_works_ahead) {
     LookupArgs a;
+    a.B = B;
+    a.dev_error = ctx->dev_error;
     a.successor_works_ahead = successor_works_ahead;
     a.hist = hist; a.hist_off = hist_off; a.hist_cap = hist_cap; a.hist_len = hist_len; a.K = K;
     a.n_max = n_max;

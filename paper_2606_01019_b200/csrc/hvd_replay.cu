@@ -145,6 +145,9 @@ hvd_status launch_replay(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t 
         }
         ctx->rp_states = n;
     }
+    // the walk puts one segment of kSegStates states on every grid row
+    if ((int64_t)n > 65535LL * kSegStates)
+        return fail(ctx, HVD_ERR_UNSUPPORTED, "hvd_replay_labels: traces beyond 65535 * 256 positions are not supported");
     ReplayArgs a;
     a.x = trace; a.n = n; a.K = K; a.l_max = ctx->cfg.l_max; a.min_match = ctx->cfg.min_match;
     a.spec_factor = ctx->cfg.spec_factor; a.spec_offset = ctx->cfg.spec_offset;

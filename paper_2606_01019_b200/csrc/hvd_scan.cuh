@@ -9,6 +9,30 @@
 
 namespace hvd {
 
+// Arguments of the lookup kernels (the one-CTA / chunk form and the tiled form).
+struct LookupArgs {
+    int32_t B;
+    const int32_t* hist;
+    const int64_t* hist_off;
+    const int32_t* hist_cap;
+    const int32_t* hist_len;
+    const int32_t* K;
+    int32_t n_max;
+    int32_t* draft;
+    int32_t* draft_len;
+    int32_t* match_len;
+    int32_t* match_pos;
+    int32_t* match_cnt;
+    LookupPartial* partial;
+    uint32_t* req_cnt;
+    int32_t max_chunks;
+    int32_t k_cap, l_max, min_match;
+    float spec_factor, spec_offset;
+    bool successor_works_ahead;
+    bool chunks_on_x;
+    int* dev_error;   // device status word of the context (set when a bounded wait runs out)
+};
+
 // Best match seen so far: the longest length, then the latest position; the count is the number of
 // positions that reach that length.
 struct Best {

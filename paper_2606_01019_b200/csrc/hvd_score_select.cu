@@ -74,6 +74,9 @@ score_select2_kernel(const ScoreArgs a) {
     const int nreq = min(REQ, a.B - b0);
     const int kc = a.k_cap;
     const int H = a.hidden;
+    // "this CTA runs": matched by the wait in front of the stores into CTA 0's shared memory, which may only be
+    // touched once every CTA of the cluster is known to have started (the arrival overlaps the slab copy)
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     // the weights do not depend on the previous kernel: this CTA's slab is requested at once
     {
         const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(s_w);
@@ -164,6 +167,7 @@ score_select2_kernel(const ScoreArgs a) {
 #pragma unroll
             for (int g = 0; g < G; ++g) acc[g] = __fmaf_rn(wv, s_h1[i][r4 + kReqPerGroup * g], acc[g]);
         }
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // every CTA of the cluster has started
         float* dst = cluster.map_shared_rank(&s_h2[0][0], 0);  // CTA 0's copy
 #pragma unroll
         for (int g = 0; g < G; ++g) {

@@ -534,7 +534,7 @@ __global__ void __launch_bounds__(kSmallWarps * 32) verify_small_kernel(const Ve
         bool mine = in && lo <= r && r < hi;
         if (mine) {
             int nr = 0;
-            if (n >= 0 && n <= cap) {  // the rule of load_req
+            if (n >= 0 && n <= cap && lo >= 0 && hi <= a.total_rows) {  // the rule of load_req
                 int m = max(0, min(sl, a.k_cap));
                 if ((int64_t)m > hi - lo - 1) m = (int)(hi - lo - 1);
                 nr = m + 1;
@@ -593,9 +593,13 @@ size_t verify_dyn_smem(int32_t B) { return (size_t)B * 8 + (size_t)(B + 1) * 4; 
 int verify_occupancy(hvd_dtype dtype, size_t dyn_smem) {
     int n = 0;
     cudaError_t e = cudaSuccess;
-    if (dyn_smem > 48 * 1024) {  // large batches: the per-request tables need the opt-in shared memory size
-        e = dtype == HVD_F32 ? cudaFuncSetAttribute(verify_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem)
-                             : cudaFuncSetAttribute(verify_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem);
+    {
+        // Large batches need the opt-in shared memory size for the per-request tables.  The attribute belongs to
+        // the device, not to a context: always opt in to the size of the largest batch a context can have, so
+        // that a later context (or the allocation-free entry point) never lowers what an earlier one relies on.
+        const int most = (int)verify_dyn_smem(8192);
+        e = dtype == HVD_F32 ? cudaFuncSetAttribute(verify_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, most)
+                             : cudaFuncSetAttribute(verify_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return 0; }
     }
     if (dtype == HVD_F32)

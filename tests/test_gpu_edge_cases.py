@@ -110,6 +110,52 @@ def test_capacity_edges_and_bad_lengths():
     assert (out.vf.status == O.REQ_CAPACITY).sum() >= 1
 
 
+@pytest.mark.parametrize("small_bytes", [None, "0"])
+def test_row_offsets_outside_the_logits(small_bytes, monkeypatch):
+    """A row_off entry below 0 or beyond total_rows: the request is skipped with HVD_REQ_BAD_LEN, nothing is read
+    or written outside the logits, the row keys or target_tok, and the other requests are verified as usual
+    (with the warp-per-batch kernel and with the persistent one)."""
+    if small_bytes is not None:
+        monkeypatch.setenv("HVD_VERIFY_SMALL_BYTES", small_bytes)
+    w = small()
+    rng = np.random.default_rng(21)
+    hists = [rng.integers(0, 3, 400 + 10 * i) for i in range(9)]
+    rq = hand_requests(w, hists, [8, 3, 8, 0, 5, 8, 8, 2, 8])
+    inp = P.prepare(w.scaled(B=rq.B), device="cuda", rq=rq)
+    good = rq.copy()
+    (g0, out, _) = G.run_and_compare(inp, rq=good)            # the reference results, with valid offsets
+    ctx = G.make_ctx(w, rq)
+    G.set_predictor(ctx, inp)
+    batch = G.make_batch(ctx, w, rq.copy())
+    import torch
+    bad = rq.row_off.copy()
+    bad[0] = -3                      # request 0 starts before the array
+    bad[-1] = rq.row_off[-1] + 5     # the last request ends beyond it
+    batch.row_off = torch.as_tensor(bad, device="cuda")
+    batch.step(inp.logits if inp.logits.device.type == "cuda" else inp.logits.cuda())
+    g = batch.download()
+    assert ctx.hvd_device_status() == 0
+    ctx.close()
+    B = rq.B
+    skipped = np.zeros(B, bool); skipped[[0, B - 1]] = True
+    assert (g["status"][skipped] == O.REQ_BAD_LEN).all()
+    assert (g["accepted"][skipped] == 0).all() and (g["n_commit"][skipped] == 0).all()
+    assert (g["committed"][skipped] == -1).all()
+    assert (g["hist_len"][skipped] == rq.hist_len[skipped]).all()
+    for k in ("accepted", "committed", "n_commit", "status", "hist_len"):
+        G.assert_equal(k, g[k][~skipped], (g0[k])[~skipped])
+    rows_ok = np.zeros(int(rq.row_off[-1]), bool)
+    rows_ok[rq.row_off[1]:rq.row_off[B - 1]] = True
+    G.assert_equal("target_tok", g["target_tok"][rows_ok], g0["target_tok"][rows_ok])
+    assert (g["target_tok"][~rows_ok] == -12345).all()        # rows of the skipped requests: never written
+    # histories: the skipped requests' slabs as before the call, the others as the reference run left them
+    want = good.hist.copy()
+    for b in (0, B - 1):
+        o, c = int(rq.hist_off[b]), int(rq.hist_cap[b])
+        want[o:o + c] = rq.hist[o:o + c]
+    G.assert_equal("hist (all slabs and guard words)", g["hist"], want)
+
+
 def test_model_draft_clamp_and_out_of_vocab_tokens():
     w = small(k_cap=16)
     rng = np.random.default_rng(8)

@@ -1,7 +1,8 @@
 """hvd_verify_commit_noalloc: the verification entry point for callers that cannot allocate
 (its scratch memory is a static array inside the library).  Called through the C ABI and checked
-against hvd_verify_commit on the same inputs, for two calls in a row, so that whatever the first
-call leaves in the shared array must not disturb the second.  Collected last on purpose."""
+against hvd_verify_commit on the same inputs and, in the first round, against the CPU oracle's
+verification of the same selection, for two calls in a row, so that whatever the first call leaves
+in the shared array must not disturb the second.  Collected last on purpose."""
 import numpy as np
 import pytest
 
@@ -35,6 +36,13 @@ def run_both(w, rounds=2):
                                     new.committed, new.n_commit, new.target_tok, new.status)
         torch.cuda.synchronize()
         a, b = ref.download(), new.download()
+        if r == 0:
+            # the oracle on the other side as well: its verification of the selection the kernels made
+            # (the selection itself is compared with the oracle's in the parity tests)
+            rq_o = inp.rq.copy()
+            sel = type("Sel", (), dict(sel_draft=b["sel_draft"], sel_len=b["sel_len"], select=b["select"]))
+            vf = P.verify_commit(w, rq_o, sel, inp.logits_np, nthreads=P.host_threads())
+            G.compare_verify(b, vf, rq_o)
         for k in OUTPUTS:                          # integer results: bit-exact, as in the other tests
             G.assert_equal(f"round {r}: {k}", b[k], a[k])
         G.assert_equal(f"round {r}: acc_ring", b["state"]["acc_ring"], a["state"]["acc_ring"])
@@ -49,6 +57,12 @@ def test_noalloc_matches_context_entry_point_fp32():
 
 def test_noalloc_matches_context_entry_point_bf16_ragged():
     run_both(W.CONFIGS["C5"].scaled(B=40, n=(64, 3000), V=32003))
+
+
+def test_noalloc_with_the_persistent_streaming_kernel():
+    """More than 160 MB of logits (816 rows of 128 256 bf16: 209 MB): the persistent kernel, its unit counters and
+    their reset run on the static array too."""
+    run_both(W.CONFIGS["C2"].scaled(B=48, n=1024))
 
 
 def test_noalloc_rejects_sizes_beyond_the_static_array():
