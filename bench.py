@@ -1,21 +1,26 @@
 #!/usr/bin/env python
 """Benchmark of the HVD per-step path (lookup -> score/select -> verify/commit) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--impl b200|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C3] [--impl b200|reference]
 
-One step = one pass of the whole path over one batch of seeded synthetic input.  Prints ONE JSON
-line.  With N > 1 (launched by torch.distributed.run) every rank runs its own copy of the batch:
-requests are independent, so the path shards with no collective on the data path ("weak" scaling);
-only the timing is reduced (max over ranks).
+One step = one pass of the whole path over one batch of seeded synthetic input.  Prints ONE JSON line:
+the headline workload (C3, the largest of the five that is a single uniform batch) at the top level and,
+at N = 1, every workload C1-C5 under `per_config` (same fields: step time, roofline of the verify kernel
+and of the lookup kernel, oracle baseline, end-to-end figure, clocks).  With N > 1 (launched by
+torch.distributed.run) every rank runs its own copy of the batch: requests are independent, so the path
+shards with no collective on the data path ("weak" scaling); only the timing is reduced (max over ranks).
 
-Timed region: K steps captured in one CUDA graph (3 kernel launches per step), bracketed by a
-barrier + synchronize, timed with CUDA events on the launching stream.  Consecutive steps use
-rotating copies of the big inputs (histories, logits) so that nothing a step reads is left in L2
-by an earlier step, and every step gets pristine per-step lengths/state.
+Timing protocol: the K steps are captured in one CUDA graph (3 kernel launches per step); after W eager
+warm-up steps and 3 untimed replays the graph is replayed 20 times, each replay between two CUDA events on
+the launching stream with a barrier + synchronize around the series; `value` is K / median replay time, the
+best replay is reported beside it.  Cold inputs: consecutive steps use rotating copies of the histories and
+logits whose total exceeds twice the L2, and every step gets pristine per-step lengths / state; the `warm`
+figure (same buffers every step) is reported separately and labelled.
 """
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
 import sys
@@ -32,39 +37,31 @@ METRIC = "HVD select+verify steps/s"
 UNIT = "steps/s"
 L2_BYTES = 126 * 2**20
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one verify_commit launch on this workload, from
-# the ncu capture summarised under profiles/ (None until captured for a workload)
-NCU_VERIFY_TRAFFIC_BYTES = {"C2": 261772928}  # profiles/verify_stream_kernel_c2_ncu.txt, mean of two launches
+HEADLINE = "C3"
+ALL_CONFIGS = ("C1", "C2", "C3", "C4", "C5")
+REPLAYS = 20          # timed replays of the K-step graph (median and best reported)
+UNTIMED_REPLAYS = 3
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the kernel on the workload, from the ncu captures
+# summarised under profiles/ (per launch, like the algorithmic bytes; absent = not captured)
+NCU_VERIFY_TRAFFIC_BYTES = {"C2": 261772928}   # profiles/verify_stream_kernel_c2_ncu.txt, mean of two launches
+NCU_LOOKUP_TRAFFIC_BYTES = {"C2": 4242048}     # profiles/lookup_kernel_c2_ncu.txt
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", default="C2")
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default=HEADLINE, help="headline workload of the line (default: C3)")
+    ap.add_argument("--only", action="store_true", help="measure the headline workload only (no per_config map)")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--mode", default="graph", choices=["graph", "stream"])
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--predictor", default="config", choices=["config", "2x256"],
                     help="2x256: the paper's predictor shape (two hidden layers of 256 units) instead of the config's")
-    ap.add_argument("--freq", action="store_true",
-                    help="variant of the lookup step: frequency-weighted draft and score (hvd_lookup_freq) on the config's requests")
-    ap.add_argument("--corpus", action="store_true",
-                    help="variant of the lookup step: shared warm-up corpus scanned with the history (hvd_lookup_corpus)")
-    ap.add_argument("--vocab-shards", action="store_true",
-                    help="variant of the verify step: one rank's share under a vocabulary-parallel output layer "
-                         "(hvd_verify_keys on a 1/S slice of every row + hvd_commit_keys), S = 2, 4, 8")
-    ap.add_argument("--verify-sweep", action="store_true",
-                    help="the verify call over batch sizes 1..64 (C2's rows), with both streaming kernels")
-    ap.add_argument("--replay", action="store_true",
-                    help="second workload: payoff labels by trace replay (hvd_replay_labels) on one history of the config")
     ap.add_argument("--unfused", action="store_true",
                     help="call hvd_lookup and hvd_score_select separately instead of hvd_lookup_score_select")
-    ap.add_argument("--no-kernel-events", action="store_true",
-                    help="leave the per-kernel event records out of the timed graph")
     return ap.parse_args()
 
 
@@ -139,6 +136,14 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(self.reasons), "samples": len(self.samples), "window": window}
 
 
+def workload_config(w, n_gpus, extra=None):
+    cfg = {"workload": f"{w.name}: batch {w.B}, histories {w.n} tokens, vocab {w.V}, K {w.K}, {w.dtype} logits",
+           "requests_per_gpu": w.B, "parallelism": f"requests sharded over {n_gpus} GPU(s), no collective"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
 # ----------------------------------------------------------------------------------------------
 # reference arm: the CPU oracle, as it stands, on the host cores
 # ----------------------------------------------------------------------------------------------
@@ -194,431 +199,67 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------------------------
-# second workload: trace-replay labels (training-data path)
+# the benchmark's own read-only probe kernel (libbench_probe.so, built from bench_probe.cu)
 # ----------------------------------------------------------------------------------------------
-def run_replay(args):
-    import torch
+class ReadProbe:
+    def __init__(self, torch, dev):
+        from paper_2606_01019_b200 import build
+        self.lib = ctypes.CDLL(build.build_bench_probe())
+        self.lib.bench_read_probe.restype = ctypes.c_int
+        self.lib.bench_read_probe.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+        self.sink = torch.zeros(1, dtype=torch.int64, device=dev)
+        self.grid = 8 * torch.cuda.get_device_properties(dev).multi_processor_count
+        self.torch = torch
+
+    def __call__(self, t):
+        st = self.torch.cuda.current_stream().cuda_stream
+        rc = self.lib.bench_read_probe(t.data_ptr(), t.numel() * t.element_size(), self.sink.data_ptr(), self.grid, st)
+        if rc != 0:
+            raise RuntimeError(f"bench_read_probe failed ({rc})")
+
+
+# ----------------------------------------------------------------------------------------------
+# one workload through the CUDA path
+# ----------------------------------------------------------------------------------------------
+def run_config(name, args, env, cpu_seconds):
+    """Everything measured on one workload; returns the dict that becomes the line (headline) or an entry of
+    per_config.  `env`: torch, dist, dev, rank, world, local, peak (GB/s), peak_kind, barrier, max_over_ranks."""
+    torch, dev, rank, world = env["torch"], env["dev"], env["rank"], env["world"]
+    barrier, peak_gbs, peak_kind = env["barrier"], env["peak"], env["peak_kind"]
     import hvd_workloads as W
     import paper_2606_01019_b200 as H
-    torch.cuda.set_device(0)
-    w = W.CONFIGS[args.config]
-    rq = W.make_requests(w.scaled(B=min(w.B, 4)))
-    x = np.ascontiguousarray(rq.history(0), np.int32)
-    n, K = len(x), int(rq.K[0])
-    ctx = H.Context(max_batch=4096, k_cap=w.k_cap, max_hist_len=n, max_rows=1, max_vocab=1, l_max=w.l_max,
-                    min_match=w.min_match)
-    xd = torch.as_tensor(x, device="cuda")
-    outs = [torch.zeros(n, dtype=torch.int32, device="cuda") for _ in range(5)]
-    for _ in range(max(3, args.warmup)):
-        ctx.hvd_replay_labels(xd, n, K, *outs)
-    torch.cuda.synchronize()
-    reps = max(1, min(args.steps, 50))
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        ctx.hvd_replay_labels(xd, n, K, *outs)
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / reps
-    label = outs[0].cpu().numpy()
-    from oracle import hvd_oracle as O
-    from oracle import pipeline as P
-    cores = P.host_threads()
-    t0 = time.perf_counter()
-    ref = O.replay_labels(x, K, k_cap=w.k_cap, l_max=w.l_max, min_match=w.min_match, nthreads=cores)
-    cpu_s = time.perf_counter() - t0
-    line = {"metric": "trace-replay labelled positions/s", "value": n / (ms * 1e-3), "unit": "positions/s",
-            "n_gpus": 1, "steps": reps, "ms_per_trace": ms, "higher_is_better": True, "dtype": "int32",
-            "data": "synthetic", "config": {"workload": f"replay of one {w.name} history: {n} positions, K {K}",
-                                            "launches_per_trace": 2},
-            "prefix_tokens_scanned_per_trace": int(n) * (int(n) + 1) // 2,
-            "scan_rate_gtokens_per_s": int(n) * (int(n) + 1) / 2 / (ms * 1e-3) / 1e9,
-            "mean_label": float(label.mean()), "labels_ge_6_frac": float((label >= 6).mean()),
-            "cpu_baseline": {"value": n / cpu_s, "unit": "positions/s", "cores": cores, "kind": "oracle",
-                             "sample": "the same whole trace, once", "agrees_with_gpu": bool((ref.label == label).all())}}
-    print(json.dumps(line), flush=True)
-    ctx.close()
 
-
-# ----------------------------------------------------------------------------------------------
-# variant of the lookup step: frequency-weighted draft and suffix score
-# ----------------------------------------------------------------------------------------------
-def run_freq(args):
-    import torch
-    import hvd_workloads as W
-    import paper_2606_01019_b200 as H
-    torch.cuda.set_device(0)
-    w = W.CONFIGS[args.config]
-    rq = W.make_requests(w)
-    B, n_max = rq.B, int(rq.hist_len.max())
-    dev = lambda a: torch.as_tensor(np.ascontiguousarray(a), device="cuda")
-    hist, off, cap, ln, K = dev(rq.hist), dev(rq.hist_off), dev(rq.hist_cap), dev(rq.hist_len), dev(rq.K)
-    i32 = lambda *shape: torch.zeros(shape, dtype=torch.int32, device="cuda")
-    draft, dlen, mlen, mpos, mcnt = i32(B, w.k_cap), i32(B), i32(B), i32(B), i32(B)
-    score = torch.zeros(B, device="cuda")
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    from oracle import hvd_oracle as O
-    from oracle import pipeline as P
-    cores = P.host_threads()
-    reps = max(3, min(args.steps, 50))
-    cases = []
-    for l_max in (w.l_max, 2):   # the configured maximum match length, and a short one (many occurrences per request)
-        ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=1, max_vocab=1,
-                        l_max=l_max, min_match=min(w.min_match, l_max), spec_factor=8.0)
-        calls = {"hvd_lookup": lambda: ctx.hvd_lookup(B, hist, off, cap, ln, K, n_max, draft, dlen, mlen, mpos, mcnt),
-                 "hvd_lookup_freq": lambda: ctx.hvd_lookup_freq(B, hist, off, cap, ln, K, n_max, 0.1, H.FREQ_MAX_OCC, 0.0,
-                                                                None, None, draft, dlen, score, mlen, mpos, mcnt)}
-        us = {}
-        for name, call in calls.items():
-            for _ in range(max(3, args.warmup)):
-                call()
-            evs = []
-            for _ in range(reps):   # all enqueued ahead: the fills hide the host's launch latency
-                flush.fill_(1)      # L2 flush between timed calls
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(); call(); e1.record()
-                evs.append((e0, e1))
-            torch.cuda.synchronize()
-            us[name] = sum(a.elapsed_time(b) for a, b in evs) / reps * 1e3
-        t0 = time.perf_counter()
-        ref = O.lookup_freq(rq.hist, rq.hist_off, rq.hist_cap, rq.hist_len, rq.K, k_cap=w.k_cap, l_max=l_max,
-                            min_match=min(w.min_match, l_max), spec_factor=8.0, min_prob=0.1, max_occ=H.FREQ_MAX_OCC,
-                            nthreads=cores)
-        cpu_s = time.perf_counter() - t0
-        agrees = bool((ref.draft == draft.cpu().numpy()).all() and
-                      (ref.score.view(np.uint32) == score.cpu().numpy().view(np.uint32)).all())
-        cases.append({"l_max": l_max, "us_lookup": us["hvd_lookup"], "us_lookup_freq": us["hvd_lookup_freq"],
-                      "mean_occurrences": float(ref.match_cnt.mean()), "max_occurrences": int(ref.match_cnt.max()),
-                      "merged_requests": int(((ref.match_cnt > 0) & (ref.match_cnt <= H.FREQ_MAX_OCC)).sum()),
-                      "mean_draft_len": float(ref.draft_len.mean()), "mean_score": float(ref.score.mean()),
-                      "oracle_ms": cpu_s * 1e3, "agrees_with_oracle": agrees})
-        ctx.close()
-    hist_bytes = int(rq.hist_len.sum()) * 4
-    c0 = cases[0]
-    line = {"metric": "frequency-weighted lookups/s", "value": B / (c0["us_lookup_freq"] * 1e-6), "unit": "requests/s",
-            "n_gpus": 1, "steps": reps, "higher_is_better": True, "dtype": "int32 (fp32 score)", "data": "synthetic",
-            "config": {"workload": f"{w.name}: batch {B}, histories {w.n} tokens; 3 launches per call, "
-                                   "L2 flushed between calls", "history_bytes": hist_bytes},
-            "history_scan_gbs": 2 * hist_bytes / (c0["us_lookup_freq"] * 1e-6) / 1e9,
-            "cases": cases,
-            "cpu_baseline": {"value": B / (c0["oracle_ms"] * 1e-3), "unit": "requests/s", "cores": cores, "kind": "oracle",
-                             "sample": "the same batch, once"}}
-    print(json.dumps(line), flush=True)
-
-
-# ----------------------------------------------------------------------------------------------
-# variant of the lookup step: shared warm-up corpus
-# ----------------------------------------------------------------------------------------------
-def run_corpus(args):
-    import torch
-    import hvd_workloads as W
-    import paper_2606_01019_b200 as H
-    torch.cuda.set_device(0)
-    w = W.CONFIGS[args.config]
-    rq = W.make_requests(w)
-    B, n_max = rq.B, int(rq.hist_len.max())
-    dev = lambda a: torch.as_tensor(np.ascontiguousarray(a), device="cuda")
-    hist, off, cap, ln, K = dev(rq.hist), dev(rq.hist_off), dev(rq.hist_cap), dev(rq.hist_len), dev(rq.K)
-    i32 = lambda *shape: torch.zeros(shape, dtype=torch.int32, device="cuda")
-    draft, dlen, mlen, mpos, msrc, mcnt = i32(B, w.k_cap), i32(B), i32(B), i32(B), i32(B), i32(B)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    from oracle import hvd_oracle as O
-    from oracle import pipeline as P
-    cores = P.host_threads()
-    reps = max(3, min(args.steps, 50))
-    ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=1, max_vocab=1,
-                    l_max=w.l_max, min_match=w.min_match)
-
-    def timed(call, cold):
-        for _ in range(max(3, args.warmup)):
-            call()
-        evs = []
-        for _ in range(reps):   # all enqueued ahead: the fills hide the host's launch latency
-            if cold:
-                flush.fill_(1)  # L2 flush between timed calls
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(); call(); e1.record()
-            evs.append((e0, e1))
-        torch.cuda.synchronize()
-        return sum(a.elapsed_time(b) for a, b in evs) / reps * 1e3
-
-    plain = lambda: ctx.hvd_lookup(B, hist, off, cap, ln, K, n_max, draft, dlen, mlen, mpos, mcnt)
-    both = lambda: ctx.hvd_lookup_corpus(B, hist, off, cap, ln, K, n_max, draft, dlen, mlen, mpos, msrc, mcnt)
-    us_plain = timed(plain, True)
-    cases = []
-    for n_traces in (16, 64, 256):
-        corpus = W.make_corpus(w, n_traces=n_traces)
-        cd = dev(corpus)
-        ctx.hvd_set_corpus(cd)
-        us_cold, us_warm = timed(both, True), timed(both, False)
-        t0 = time.perf_counter()
-        ref = O.lookup_corpus(rq.hist, rq.hist_off, rq.hist_cap, rq.hist_len, rq.K, corpus, k_cap=w.k_cap,
-                              l_max=w.l_max, min_match=w.min_match, nthreads=cores)
-        cpu_s = time.perf_counter() - t0
-        agrees = all(bool((getattr(ref, k) == t.cpu().numpy()).all()) for k, t in
-                     (("draft", draft), ("draft_len", dlen), ("match_len", mlen), ("match_pos", mpos),
-                      ("match_src", msrc), ("match_cnt", mcnt)))
-        m = len(corpus)
-        cases.append({"corpus_tokens": m, "us_lookup_corpus_cold": us_cold, "us_lookup_corpus_corpus_in_l2": us_warm,
-                      "token_compares_per_s": float(B) * m / (us_warm * 1e-6),
-                      "requests_matched_in_corpus": int(ref.match_src.sum()), "oracle_ms": cpu_s * 1e3,
-                      "agrees_with_oracle": agrees})
-    c = cases[1]
-    line = {"metric": "lookups over corpus and history per second", "value": B / (c["us_lookup_corpus_cold"] * 1e-6),
-            "unit": "requests/s", "n_gpus": 1, "steps": reps, "higher_is_better": True, "dtype": "int32",
-            "data": "synthetic",
-            "config": {"workload": f"{w.name}: batch {B}, histories {w.n} tokens, warm-up corpus of {c['corpus_tokens']} "
-                                   "tokens (64 traces); 2 launches per call, L2 flushed between calls"},
-            "us_lookup_history_only": us_plain, "cases": cases,
-            "cpu_baseline": {"value": B / (c["oracle_ms"] * 1e-3), "unit": "requests/s", "cores": cores, "kind": "oracle",
-                             "sample": "the same batch and corpus, once"}}
-    print(json.dumps(line), flush=True)
-    ctx.close()
-
-
-# ----------------------------------------------------------------------------------------------
-# variant of the verify step: vocabulary shards (one rank's work; the 8-bytes-per-row MAX all-reduce
-# between the two calls needs the other ranks and is not part of this single-GPU timing)
-# ----------------------------------------------------------------------------------------------
-def run_vocab_shards(args):
-    import torch
-    import hvd_workloads as W
-    import paper_2606_01019_b200 as H
-    from paper_2606_01019_b200.runner import DeviceBatch
-    torch.cuda.set_device(0)
-    w = W.CONFIGS[args.config]
-    # inputs as in the main arm: the selection comes from the CUDA path itself, the logits are planted on it
-    rq = W.make_requests(w)
-    W1, b1, W2, b2, tau = W.make_predictor(w)
-    B, rows = rq.B, int(rq.row_off[-1])
-    ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=rows, max_vocab=w.V,
-                    l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
-    ctx.hvd_set_predictor(W1, b1, W2, b2, tau)
-    batch = DeviceBatch(ctx, hist=rq.hist, hist_off=rq.hist_off, hist_cap=rq.hist_cap, hist_len=rq.hist_len, K=rq.K,
-                        prompt_len=rq.prompt_len, state=rq.state, model_draft=rq.model_draft, model_len=rq.model_len,
-                        row_off=rq.row_off, V=w.V, dtype=w.dtype)
-    batch.lookup_score_select()
-    if w.calibrate_cache_frac is not None:
-        torch.cuda.synchronize()
-        tau = W.calibrate_tau(batch.score.cpu().numpy(), batch.draft_len.cpu().numpy() > 0, w.calibrate_cache_frac)
-        ctx.hvd_set_predictor(W1, b1, W2, b2, tau)
-        batch.lookup_score_select()
-    torch.cuda.synchronize()
-    sel_len_h, sel_draft_h = batch.sel_len.cpu().numpy(), batch.sel_draft.cpu().numpy()
-    logits = W.make_logits(w, rows, device="cuda")
-    W.plant_agreement(w, logits, rq.row_off, sel_draft_h, sel_len_h, W.make_agreement(w, sel_len_h))
-    full = logits.reshape(-1)[: rows * w.V].reshape(rows, w.V)
-    needed = int((batch.sel_len.cpu().numpy().astype(np.int64) + 1).sum())
-    hist_len0, state0 = batch.hist_len.clone(), batch.state.clone()
-    reps = max(3, min(args.steps, 50))
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    cases = []
-    for S in (1, 2, 4, 8):
-        Vs = w.V // S
-        copies = [full[:, :Vs].contiguous() for _ in range(2 if S > 1 else 1)]
-        keys = torch.zeros(rows, dtype=torch.int64, device="cuda")
-
-        def call(i):
-            ctx.hvd_verify_keys(B, copies[i % len(copies)], batch.dtype, Vs, 0, batch.row_off, 0, rows, batch.sel_len,
-                                batch.hist_len, batch.hist_cap, keys)
-            ctx.hvd_commit_keys(B, keys, w.V, batch.row_off, 0, rows, batch.sel_draft, batch.sel_len, batch.select,
-                                batch.hist, batch.hist_off, batch.hist_cap, batch.hist_len, batch.state, batch.accepted,
-                                batch.committed, batch.n_commit, None, batch.status)
-
-        def body(i, with_call):
-            batch.hist_len.copy_(hist_len0); batch.state.copy_(state0)
-            flush.fill_(1)   # L2 flush between calls
-            if with_call:
-                call(i)
-
-        for i in range(3):
-            body(i, True)
-        torch.cuda.synchronize()
-        stream = torch.cuda.Stream()
-        times = []
-        for with_call in (True, False):   # the same graph with and without the calls: the difference is the calls
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.stream(stream):
-                g.capture_begin()
-                for i in range(reps):
-                    body(i, with_call)
-                g.capture_end()
-            torch.cuda.synchronize()
-            with torch.cuda.stream(stream):
-                g.replay()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(); g.replay(); e1.record()
-            torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1))
-        us = (times[0] - times[1]) / reps * 1e3
-        shard_bytes = needed * Vs * w.elt
-        cases.append({"shards": S, "us_per_rank": us, "shard_bytes": shard_bytes, "gbs": shard_bytes / (us * 1e-6) / 1e9,
-                      "allreduce_bytes_per_rank": rows * 8, "logits_allgather_bytes_avoided": needed * (w.V - Vs) * w.elt})
-    line = {"metric": "verify+commit per rank under vocabulary shards", "value": cases[-1]["us_per_rank"], "unit": "us",
-            "n_gpus": 1, "steps": reps, "higher_is_better": False, "dtype": w.dtype, "data": "synthetic",
-            "config": {"workload": f"{w.name}: batch {B}, {rows} logits rows, vocab {w.V} in S slices; one rank's "
-                                   "hvd_verify_keys + hvd_commit_keys (4 kernels) in a CUDA graph, L2 flushed between calls; "
-                                   "time = graph with the calls minus the same graph without them"},
-            "cases": cases}
-    print(json.dumps(line), flush=True)
-    ctx.close()
-
-
-# ----------------------------------------------------------------------------------------------
-# the verify call from one request to a full batch: which streaming kernel serves which size
-# ----------------------------------------------------------------------------------------------
-def run_verify_sweep(args):
-    """hvd_verify_commit on 1..64 requests with C2's logits rows (K + 1 = 17 rows of 128 256 bf16 per request),
-    selected draft lengths uniform in 0..K (about half the rows needed), timed with the persistent streaming
-    kernel only (HVD_VERIFY_SMALL_BYTES=0) and with the library's own choice.  Inputs are random: nothing is
-    checked here (the parity tests do that), only timed."""
-    import torch
-    import hvd_workloads as W
-    import paper_2606_01019_b200 as H
-    from paper_2606_01019_b200.runner import DeviceBatch
-    torch.cuda.set_device(0)
-    reps = max(3, min(args.steps, 40))
-    cases = []
-    for B in (1, 2, 4, 8, 16, 32, 64):
-        w = W.CONFIGS["C2"].scaled(B=B, n=2048)
-        rq = W.make_requests(w)
-        rows = int(rq.row_off[-1])
-        full_bytes = rows * w.V * w.elt
-        R = int(max(2, min(40, -(-4 * L2_BYTES // full_bytes))))
-        logits = [W.make_logits(w, rows, device="cuda", salt=r) for r in range(R)]
-        gen = torch.Generator(device="cuda")
-        gen.manual_seed(1000 + B)
-        sel_len = torch.randint(0, w.K + 1, (B,), generator=gen, device="cuda", dtype=torch.int32)
-        sel_draft = torch.randint(0, w.V, (B, w.k_cap), generator=gen, device="cuda", dtype=torch.int32)
-        needed_bytes = int((sel_len.cpu().numpy().astype(np.int64) + 1).sum()) * w.V * w.elt
-        us = {}
-        for kind, env in (("persistent", "0"), ("default", None)):
-            old = os.environ.pop("HVD_VERIFY_SMALL_BYTES", None)
-            if env is not None:
-                os.environ["HVD_VERIFY_SMALL_BYTES"] = env
-            ctx = H.Context(max_batch=B, k_cap=w.k_cap, max_hist_len=int(rq.hist_cap.max()), max_rows=rows,
-                            max_vocab=w.V, l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
-            os.environ.pop("HVD_VERIFY_SMALL_BYTES", None)
-            if old is not None:
-                os.environ["HVD_VERIFY_SMALL_BYTES"] = old
-            b = DeviceBatch(ctx, hist=rq.hist, hist_off=rq.hist_off, hist_cap=rq.hist_cap, hist_len=rq.hist_len, K=rq.K,
-                            prompt_len=rq.prompt_len, state=rq.state, model_draft=rq.model_draft,
-                            model_len=rq.model_len, row_off=rq.row_off, V=w.V, dtype=w.dtype)
-            b.sel_len.copy_(sel_len); b.sel_draft.copy_(sel_draft); b.select.zero_()
-            hl0, st0 = b.hist_len.clone(), b.state.clone()
-
-            def body(i, with_call):
-                b.hist_len.copy_(hl0); b.state.copy_(st0)
-                if with_call:
-                    b.verify_commit(logits[i % R], target_tok=False)
-
-            for i in range(3):
-                body(i, True)
-            torch.cuda.synchronize()
-            stream = torch.cuda.Stream()
-            t = []
-            for with_call in (True, False):   # the same graph with and without the call
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.stream(stream):
-                    g.capture_begin()
-                    for i in range(reps):
-                        body(i, with_call)
-                    g.capture_end()
-                torch.cuda.synchronize()
-                with torch.cuda.stream(stream):
-                    g.replay()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record(); g.replay(); e1.record()
-                torch.cuda.synchronize()
-                t.append(e0.elapsed_time(e1))
-            us[kind] = (t[0] - t[1]) / reps * 1e3
-            ctx.close()
-        cases.append({"requests": B, "logits_bytes": full_bytes, "needed_bytes": needed_bytes,
-                      "us_persistent_kernel": us["persistent"], "us_library_choice": us["default"],
-                      "gbs_library_choice": needed_bytes / (us["default"] * 1e-6) / 1e9})
-    line = {"metric": "hvd_verify_commit call over batch sizes", "value": cases[0]["us_library_choice"], "unit": "us",
-            "n_gpus": 1, "steps": reps, "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "C2's logits rows (17 rows of 128256 bf16 per request), 1..64 requests, selected draft "
-                                   "lengths uniform in 0..16; calls in a CUDA graph on rotating logits copies larger than "
-                                   "L2 in total; time = graph with the calls minus the same graph without them"},
-            "cases": cases}
-    print(json.dumps(line), flush=True)
-
-
-def workload_config(w, n_gpus, extra=None):
-    cfg = {"workload": f"{w.name}: batch {w.B}, histories {w.n} tokens, vocab {w.V}, K {w.K}, {w.dtype} logits",
-           "requests_per_gpu": w.B, "parallelism": f"requests sharded over {n_gpus} GPU(s), no collective"}
-    if extra:
-        cfg.update(extra)
-    return cfg
-
-
-# ----------------------------------------------------------------------------------------------
-# the CUDA path
-# ----------------------------------------------------------------------------------------------
-def main():
-    args = parse_args()
-    if args.impl == "reference":
-        run_reference(args)
-        return
-    if args.freq:
-        run_freq(args)
-        return
-    if args.corpus:
-        run_corpus(args)
-        return
-    if args.vocab_shards:
-        run_vocab_shards(args)
-        return
-    if args.verify_sweep:
-        run_verify_sweep(args)
-        return
-    if args.replay:
-        run_replay(args)
-        return
-
-    import torch
-    import torch.distributed as dist
-    import hvd_workloads as W
-    import paper_2606_01019_b200 as H
-    from paper_2606_01019_b200.sharding import max_over_ranks
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device; the HVD path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    w = W.CONFIGS[args.config]
+    w = W.CONFIGS[name]
     if args.predictor == "2x256":
         w = w.scaled(hidden=256, hidden_layers=2)
     K_steps, W_steps = args.steps, args.warmup
     n_slots = K_steps + W_steps
-    peak_gbs, peak_kind = measured_peak()
 
     # ---- inputs: the product path itself produces the drafts the logits are planted on ----------
     rq = W.make_requests(w)
     W1, b1, W2, b2, tau = W.make_predictor(w)
     B, kc = rq.B, w.k_cap
     total_rows = int(rq.row_off[-1])
-    ctx = H.Context(max_batch=B, k_cap=kc, max_hist_len=int(rq.hist_cap.max()), max_rows=total_rows,
-                    max_vocab=w.V, l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
+    ctx_kw = dict(max_batch=B, k_cap=kc, max_hist_len=int(rq.hist_cap.max()), max_rows=total_rows,
+                  max_vocab=w.V, l_max=w.l_max, min_match=w.min_match, hidden=w.hidden)
+    ctx = H.Context(**ctx_kw)
+    # the same library with plain launches (no programmatic dependent launch): a call measured with nothing of its
+    # neighbours overlapping it
+    old_mask = os.environ.get("HVD_PDL_MASK")
+    os.environ["HVD_PDL_MASK"] = "0"
+    ctx_plain = H.Context(**ctx_kw)
+    if old_mask is None:
+        del os.environ["HVD_PDL_MASK"]
+    else:
+        os.environ["HVD_PDL_MASK"] = old_mask
     Wh, bh = W.make_second_layer(w) if w.hidden_layers == 2 else (None, None)
 
     def set_predictor(t):
-        if Wh is not None:
-            ctx.hvd_set_predictor2(W1, b1, Wh, bh, W2, b2, t)
-        else:
-            ctx.hvd_set_predictor(W1, b1, W2, b2, t)
+        for c in (ctx, ctx_plain):
+            if Wh is not None:
+                c.hvd_set_predictor2(W1, b1, Wh, bh, W2, b2, t)
+            else:
+                c.hvd_set_predictor(W1, b1, W2, b2, t)
 
     set_predictor(tau)
     up = lambda a, dt: torch.as_tensor(np.ascontiguousarray(a, dt), device=dev)
@@ -634,10 +275,10 @@ def main():
     score = torch.zeros(B, dtype=torch.float32, device=dev)
     select, sel_draft, sel_len = i32(B), i32(B, kc), i32(B)
     accepted, committed, n_commit, status = i32(B), i32(B, kc + 1), i32(B), i32(B)
+    dtype = H.F32 if w.dtype == "f32" else H.BF16
 
-    def lookup(hist, hist_len):
-        ctx.hvd_lookup(B, hist, hist_off, hist_cap, hist_len, Kt, n_max, draft, draft_len, match_len,
-                       match_pos, match_cnt)
+    def lookup(hist, hist_len, c=ctx):
+        c.hvd_lookup(B, hist, hist_off, hist_cap, hist_len, Kt, n_max, draft, draft_len, match_len, match_pos, match_cnt)
 
     def score_select(hist_len, state):
         ctx.hvd_score_select(B, hist_len, prompt_len, state, Kt, draft, draft_len, match_len, match_pos,
@@ -648,11 +289,9 @@ def main():
                                     model_draft, model_len, draft, draft_len, match_len, match_pos, match_cnt,
                                     None, score, select, sel_draft, sel_len)
 
-    dtype = H.F32 if w.dtype == "f32" else H.BF16
-
-    def verify(logits, hist, hist_len, state):
-        ctx.hvd_verify_commit(B, logits, dtype, w.V, row_off, 0, total_rows, sel_draft, sel_len, select, hist,
-                              hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, None, status)
+    def verify(logits, hist, hist_len, state, c=ctx):
+        c.hvd_verify_commit(B, logits, dtype, w.V, row_off, 0, total_rows, sel_draft, sel_len, select, hist,
+                            hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, None, status)
 
     # the commit and the next cycle's lookup + selection in one call; the next selection goes to arrays of its
     # own, so that every timed step verifies the same (pristine) selection
@@ -682,204 +321,172 @@ def main():
     W.plant_agreement(w, logits0, rq.row_off, sel_draft_h, sel_len_h, A)
 
     # ---- rotating copies of the big inputs, pristine per-step small arrays ------------------------
-    foot = hist0.numel() * 4 + logits0.numel() * logits0.element_size()
-    R = int(max(2, -(-4 * L2_BYTES // foot)))
-    hists = [hist0] + [hist0.clone() for _ in range(R - 1)]
+    hist_bytes_alloc = hist0.numel() * 4
+    logits_bytes_alloc = logits0.numel() * logits0.element_size()
+    R = int(max(2, -(-4 * L2_BYTES // (hist_bytes_alloc + logits_bytes_alloc))))
+    # the histories alone rotate over enough copies to leave the L2 between two uses (at most 64 copies)
+    RH = int(max(R, min(64, -(-4 * L2_BYTES // hist_bytes_alloc))))
+    hist_cold = RH * hist_bytes_alloc >= 2 * L2_BYTES
+    hists = [hist0] + [hist0.clone() for _ in range(RH - 1)]
     logits = [logits0] + [logits0.clone() for _ in range(R - 1)]
     hist_len_steps = hist_len0.repeat(n_slots, 1).contiguous()
     state_steps = state0.repeat(n_slots, 1, 1).contiguous()
     hist_len_pristine, state_pristine = hist_len_steps.clone(), state_steps.clone()
+    probe = ReadProbe(torch, dev)
+
+    stream = torch.cuda.Stream(device=dev)   # everything after the eager warm-up runs on this stream
 
     def restore():
-        hist_len_steps.copy_(hist_len_pristine)
-        state_steps.copy_(state_pristine)
+        with torch.cuda.stream(stream):
+            hist_len_steps.copy_(hist_len_pristine)
+            state_steps.copy_(state_pristine)
 
-    def step(slot, events=None, with_verify=True, lookup_only=False, verify_only=False, probe_only=False,
-             cycle_only=False):
-        r = slot % R
+    def step(slot, what="step", warm=False):
+        rl, rh = (0, 0) if warm else (slot % R, slot % RH)
         hl, st = hist_len_steps[slot], state_steps[slot]
-        if cycle_only:    # verify + commit + the next cycle's lookup and selection: two kernels per step
-            cycle(logits[r], hists[r], hl, st)
-            return
-        if probe_only:    # plain read loop over the same logits buffer: the part's read-only speed
-            ctx.hvd_read_probe(logits[r], logits[r].numel() * logits[r].element_size())
-            return
-        if lookup_only:
-            lookup(hists[r], hl)
-            return
-        if verify_only:   # the selection of the last lookup is still in place: every step starts from the same state
-            verify(logits[r], hists[r], hl, st)
-            return
-        if events is not None:
-            events[0].record()
-        if args.unfused:
-            lookup(hists[r], hl)
-            score_select(hl, st)
+        if what == "cycle":       # verify + commit + the next cycle's lookup and selection: two kernels per step
+            cycle(logits[rl], hists[rh], hl, st)
+        elif what == "probe":     # plain read loop over the same logits buffer: the part's read-only speed
+            probe(logits[rl])
+        elif what == "lookup":
+            lookup(hists[rh], hl)
+        elif what == "lookup_plain":
+            lookup(hists[rh], hl, ctx_plain)
+        elif what == "verify":    # the selection of the last lookup is still in place: every step starts from the same state
+            verify(logits[rl], hists[rh], hl, st)
+        elif what == "verify_plain":
+            verify(logits[rl], hists[rh], hl, st, ctx_plain)
         else:
-            lookup_score_select(hists[r], hl, st)
-        if events is not None:
-            events[1].record()
-        if with_verify:
-            verify(logits[r], hists[r], hl, st)
-        if events is not None:
-            events[2].record()
+            if args.unfused:
+                lookup(hists[rh], hl)
+                score_select(hl, st)
+            else:
+                lookup_score_select(hists[rh], hl, st)
+            if what == "step":
+                verify(logits[rl], hists[rh], hl, st)
 
-    # ---- warm-up (eager), then the timed K steps --------------------------------------------------
+    # ---- warm-up (eager), then graphs of the K steps ------------------------------------------------
     for s in range(W_steps):
         step(s)
     torch.cuda.synchronize()
-    mode = args.mode
-    stream = torch.cuda.Stream(device=dev)
 
-    def capture(events=None, with_verify=True, lookup_only=False, verify_only=False, probe_only=False,
-                cycle_only=False):
+    def capture(what="step", warm=False):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
             g.capture_begin()
             for s in range(K_steps):
-                step(W_steps + s, events[s] if events else None, with_verify, lookup_only, verify_only, probe_only,
-                     cycle_only)
+                step(W_steps + s, what, warm)
             g.capture_end()
         torch.cuda.synchronize()
-        with torch.cuda.stream(stream):
-            g.replay()               # untimed: instantiation and upload costs
-        torch.cuda.synchronize()
-        restore()
         return g
 
-    graph = None
-    if mode == "graph":
-        try:
-            graph = capture()
-        except Exception as e:  # pragma: no cover
-            sys.stderr.write(f"bench.py: graph capture failed ({e!r}); timing plain stream launches\n")
-            mode, graph = "stream", None
-            torch.cuda.synchronize()
+    def timed_replays(g, replays=REPLAYS, untimed=UNTIMED_REPLAYS, sampler=None):
+        """Device times (ms) of `replays` replays of g, after `untimed` ones; barrier + synchronize around the series,
+        every replay between two events on the launching stream, pristine lengths and state before each."""
+        for _ in range(untimed):
             restore()
-
-    def timed(run):
-        """Device time of run() on `stream`, bracketed by barrier + synchronize on both sides."""
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(stream):
+                g.replay()
+        torch.cuda.synchronize()
+        evs = []
         barrier()
+        if sampler is not None:
+            sampler.start()
         with torch.cuda.stream(stream):
-            e0.record()
-            run()
-            e1.record()
+            for _ in range(replays):
+                restore()                      # on the same stream, outside the two events
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); g.replay(); e1.record()
+                evs.append((e0, e1))
         barrier()
-        return e0.elapsed_time(e1)
+        ms = np.array([a.elapsed_time(b) for a, b in evs])
+        restore()
+        return ms
 
-    # ---- the timed region: K steps, nothing but the path's kernels between the two events -------------
-    sampler = ClockSampler(local)
-    sampler.start()
-    if graph is not None:
-        elapsed_ms = timed(graph.replay)
-    else:
-        elapsed_ms = timed(lambda: [step(W_steps + s) for s in range(K_steps)])
-    window = "timed region"
+    sampler = ClockSampler(env["local"])
+    g_step = capture("step")
+    ms_step = timed_replays(g_step, sampler=sampler)
+    window = "the 20 timed replays"
     # results of the timed steps (every step does the same work on identical copies)
     n_commit_h = n_commit.cpu().numpy()
     accepted_h = accepted.cpu().numpy()
     select_h = select.cpu().numpy()
     status_h = status.cpu().numpy()
     sel_len_after = sel_len.cpu().numpy()
-    if len(sampler.samples) < 5 and graph is not None:
+    if len(sampler.samples) < 5:
         # region too short for the sampler: keep the same graph running, untimed, while sampling
-        window = "timed region + untimed repeats of the same graph"
+        window = "the 20 timed replays + untimed repeats of the same graph"
         t_end = time.time() + 0.3
         while time.time() < t_end:
             restore()
             with torch.cuda.stream(stream):
-                graph.replay()
+                g_step.replay()
             torch.cuda.synchronize()
     sampler.stop_flag.set()
     sampler.join(timeout=2)
+    clocks = sampler.summary(window)
+    ms_step = env["max_over_ranks_vec"](ms_step)
+    med_ms, best_ms = float(np.median(ms_step)), float(ms_step.min())
+    del g_step
 
-    # ---- per-kernel times: the same K steps again, (a) with event records around the verify call
-    # inside the graph (each record is a graph node of its own and costs a few microseconds of
-    # serialisation, so these are upper bounds), (b) without the verify call (difference to the
-    # timed region = what verify adds to a step) ------------------------------------------------------
-    kt = None
-    if not args.no_kernel_events:
-        try:
-            restore()
-            ext = graph is not None
-            evs = [[torch.cuda.Event(enable_timing=True, external=ext) for _ in range(3)] for _ in range(K_steps)]
-            if graph is not None:
-                g_ev = capture(evs)
-                t_ev = timed(g_ev.replay)
-                restore()
-                g_nv = capture(None, with_verify=False)
-                restore()
-                t_nv = timed(g_nv.replay)
-                g_lk = capture(None, lookup_only=True)
-                t_lk = timed(g_lk.replay)
-                restore()
-                g_vo = capture(None, verify_only=True)
-                restore()
-                t_vo = timed(g_vo.replay)
-                g_pr = capture(None, probe_only=True)
-                t_pr = timed(g_pr.replay)
-                restore()
-                g_cy = capture(None, cycle_only=True)
-                restore()
-                t_cy = timed(g_cy.replay)
-            else:
-                t_ev = timed(lambda: [step(W_steps + s, evs[s]) for s in range(K_steps)])
-                restore()
-                t_nv = timed(lambda: [step(W_steps + s, None, False) for s in range(K_steps)])
-                t_lk = timed(lambda: [step(W_steps + s, None, False, True) for s in range(K_steps)])
-                restore()
-                t_vo = timed(lambda: [step(W_steps + s, None, True, False, True) for s in range(K_steps)])
-                t_pr = timed(lambda: [step(W_steps + s, probe_only=True) for s in range(K_steps)])
-                restore()
-                t_cy = timed(lambda: [step(W_steps + s, cycle_only=True) for s in range(K_steps)])
-            restore()
-            d = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(2)] for e in evs])
-            kt = {"lookup_plus_score_select_us": 1e3 * float(d[:, 0].mean()),
-                  "verify_commit_us": 1e3 * float(d[:, 1].mean()),
-                  "verify_commit_us_median": 1e3 * float(np.median(d[:, 1])),
-                  "step_us_with_event_records": 1e3 * t_ev / K_steps,
-                  "step_us_without_verify": 1e3 * t_nv / K_steps,
-                  "lookup_only_us": 1e3 * t_lk / K_steps,
-                  "verify_commit_us_by_difference": 1e3 * (elapsed_ms - t_nv) / K_steps,
-                  "verify_commit_us_back_to_back": 1e3 * t_vo / K_steps,
-                  "read_probe_us": 1e3 * t_pr / K_steps,
-                  "step_us_commit_fused_with_next_lookup": 1e3 * t_cy / K_steps,
-                  "note": "event-bracketed times include the serialisation the event records add; "
-                          "the headline region has no records in it"}
-        except Exception as e:  # pragma: no cover
-            sys.stderr.write(f"bench.py: per-kernel events unavailable ({e!r})\n")
+    def us_per_step(what, warm=False, replays=REPLAYS):
+        g = capture(what, warm)
+        ms = timed_replays(g, replays=replays, untimed=2)
+        del g
+        return 1e3 * float(np.median(ms)) / K_steps, 1e3 * float(ms.min()) / K_steps
 
-    elapsed_ms = max_over_ranks(elapsed_ms, dev)
-    steps_per_s = world * K_steps / (elapsed_ms * 1e-3)
+    kt = {}
+    kt["step_us_warm"], kt["step_us_warm_best"] = us_per_step("step", warm=True)
+    kt["step_us_without_verify"], _ = us_per_step("noverify")
+    kt["lookup_us"], kt["lookup_us_best"] = us_per_step("lookup")
+    kt["lookup_us_plain_launches"], _ = us_per_step("lookup_plain")
+    kt["lookup_us_warm"], _ = us_per_step("lookup", warm=True)
+    kt["verify_commit_us_back_to_back"], _ = us_per_step("verify")
+    kt["verify_commit_us_isolated"], kt["verify_commit_us_isolated_best"] = us_per_step("verify_plain")
+    kt["verify_commit_us_by_difference"] = 1e3 * med_ms / K_steps - kt["step_us_without_verify"]
+    kt["read_probe_us"], _ = us_per_step("probe")
+    kt["step_us_commit_fused_with_next_lookup"], _ = us_per_step("cycle")
+
+    steps_per_s = world * K_steps / (med_ms * 1e-3)
     tokens_per_step = int(n_commit_h.sum())
     assert (status_h == 0).all(), "a request reported a capacity or length problem"
+    step_us = 1e3 * med_ms / K_steps
 
-    # ---- roofline of the dominant kernel (verify/commit): algorithmic bytes = needed rows x V x elt ----
+    # ---- rooflines: algorithmic bytes = needed rows x V x elt (verify), 4 bytes per history token (lookup) ----
     verify_bytes = int((sel_len_after.astype(np.int64) + 1).sum()) * w.V * w.elt
     lookup_bytes = int(rq.hist_len.astype(np.int64).sum()) * 4
-    roofline = {"bound": "hbm", "kernel": "verify_stream_kernel (+ verify_commit_kernel)", "achieved": None, "peak": peak_gbs, "unit": "GB/s",
-                "frac": None, "traffic": NCU_VERIFY_TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind,
-                "algorithmic_bytes_per_launch": verify_bytes}
-    roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel (hvd_lookup alone, back to back in one graph)",
-                       "achieved": None, "peak": peak_gbs, "unit": "GB/s", "frac": None, "traffic": None,
-                       "peak_kind": peak_kind, "algorithmic_bytes_per_launch": lookup_bytes}
-    if kt:
-        roofline["achieved"] = verify_bytes / (kt["verify_commit_us_back_to_back"] * 1e-6) / 1e9
-        roofline["frac"] = roofline["achieved"] / peak_gbs
-        roofline["frac_of_8000_nominal"] = roofline["achieved"] / 8000.0
-        roofline["achieved_by_difference"] = verify_bytes / (kt["verify_commit_us_by_difference"] * 1e-6) / 1e9
-        roofline["achieved_with_event_records_in_graph"] = verify_bytes / (kt["verify_commit_us"] * 1e-6) / 1e9
-        roofline_lookup["achieved"] = lookup_bytes / (kt["lookup_only_us"] * 1e-6) / 1e9
-        roofline_lookup["frac"] = roofline_lookup["achieved"] / peak_gbs
-        probe_bytes = logits[0].numel() * logits[0].element_size()
-        roofline["read_only_kernel"] = {"achieved": probe_bytes / (kt["read_probe_us"] * 1e-6) / 1e9, "unit": "GB/s",
-                                        "bytes_per_launch": probe_bytes,
-                                        "what": "hvd_read_probe: a plain grid-stride read of the whole logits buffer, "
-                                                "timed like the verify call (K launches back to back on the rotating copies)"}
-        roofline["frac_of_read_only_kernel"] = roofline["achieved"] / roofline["read_only_kernel"]["achieved"]
-        roofline["timing"] = ("CUDA events around a graph of the same K hvd_verify_commit launches back to back "
-                              "(both kernels of the call, launch gaps included), on rotating inputs larger than L2")
+    gbs = lambda nbytes, us: nbytes / (us * 1e-6) / 1e9
+    v_iso, v_b2b = gbs(verify_bytes, kt["verify_commit_us_isolated"]), gbs(verify_bytes, kt["verify_commit_us_back_to_back"])
+    probe_bytes = logits0.numel() * logits0.element_size()
+    probe_gbs = gbs(probe_bytes, kt["read_probe_us"])
+    roofline = {"bound": "hbm", "kernel": "verify_stream_kernel (+ verify_commit_kernel)" if logits_bytes_alloc > 160 * 2**20
+                else "verify_small_kernel (+ verify_commit_kernel)",
+                "achieved": v_iso, "peak": peak_gbs, "unit": "GB/s", "frac": v_iso / peak_gbs,
+                "traffic": NCU_VERIFY_TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind,
+                "algorithmic_bytes_per_launch": verify_bytes,
+                "frac_of_8000_nominal": v_iso / 8000.0,
+                "achieved_back_to_back": v_b2b, "frac_back_to_back": v_b2b / peak_gbs,
+                "achieved_by_difference": gbs(verify_bytes, kt["verify_commit_us_by_difference"]),
+                "read_only_kernel": {"achieved": probe_gbs, "unit": "GB/s", "bytes_per_launch": probe_bytes,
+                                     "what": "bench_probe.cu: a plain grid-stride read of the whole logits buffer, K launches "
+                                             "back to back on the rotating copies"},
+                "frac_of_read_only_kernel": v_iso / probe_gbs,
+                "timing": "CUDA events around a graph of K hvd_verify_commit calls (both kernels of the call) on rotating "
+                          "inputs larger than L2; `achieved` = isolated: plain launches, every kernel starts after its "
+                          "predecessor has completed; `achieved_back_to_back` = with programmatic dependent launch, the "
+                          "next call's start-up hidden under this call's tail (as inside a step)"}
+    l_b2b = gbs(lookup_bytes, kt["lookup_us"])
+    roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel (hvd_lookup alone, K calls back to back in one graph)",
+                       "achieved": l_b2b, "peak": peak_gbs, "unit": "GB/s", "frac": l_b2b / peak_gbs,
+                       "traffic": NCU_LOOKUP_TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind,
+                       "algorithmic_bytes_per_launch": lookup_bytes,
+                       "cold": bool(hist_cold), "history_copies": RH,
+                       "achieved_plain_launches": gbs(lookup_bytes, kt["lookup_us_plain_launches"]),
+                       "achieved_warm_l2_resident": gbs(lookup_bytes, kt["lookup_us_warm"]),
+                       "traffic_floor_us_at_peak": lookup_bytes / peak_gbs / 1e3}
+    roofline_step = {"bound": "hbm", "algorithmic_bytes_per_step": lookup_bytes + verify_bytes,
+                     "achieved": gbs(lookup_bytes + verify_bytes, step_us), "peak": peak_gbs, "unit": "GB/s",
+                     "peak_kind": peak_kind, "frac": gbs(lookup_bytes + verify_bytes, step_us) / peak_gbs}
 
     # ---- end to end through the host-buffer entry point --------------------------------------------
     e2e = None
@@ -914,7 +521,7 @@ def main():
             host_step()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        dt = max_over_ranks(dt, dev)
+        dt = env["max_over_ranks"](dt)
         assert (o_acc.numpy() == accepted_h).all() and (o_nc.numpy() == n_commit_h).all()
         small = B * (8 + 4 * 5 + 16) + (B + 1) * 8 + B * kc * 4
         # of the logits the call copies the rows verification reads (rows 0..sel_len of every request)
@@ -927,6 +534,7 @@ def main():
                "logits_bytes_on_host": int(h_logits.numel() * h_logits.element_size()),
                "note": "histories, per-request arrays and the logits rows that verification reads cross the bus "
                        "every step (the rows beyond a request's selected draft are not copied)"}
+        del h_logits, h_hist
 
     # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ----------
     cpu_baseline = None
@@ -937,7 +545,7 @@ def main():
         inp = P.Inputs(w, rq, W1, b1, W2, b2, tau, Wh=Wh, bh=bh, A=A, strict=np.ones(B, bool), logits_np=logits_np)
         times, out = [], None
         t_begin = time.perf_counter()
-        while len(times) < 5 or (time.perf_counter() - t_begin < 10.0 and len(times) < 200):
+        while len(times) < 3 or (time.perf_counter() - t_begin < cpu_seconds and len(times) < 200):
             rq_c = rq.copy()
             t0 = time.perf_counter()
             out = P.step(inp, rq_c, nthreads=cores)
@@ -950,41 +558,100 @@ def main():
                                   f"median of {len(times)} repetitions",
                         "ms_per_step": 1e3 * med, "tokens_per_s": tokens_per_step / med,
                         "agrees_with_gpu_step": same}
+        del logits_np, inp
 
-    if rank == 0:
-        line = {"metric": METRIC, "value": steps_per_s, "unit": UNIT, "n_gpus": world, "steps": K_steps,
-                "warmup": W_steps, "ms_per_step": elapsed_ms / K_steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
-                "config": workload_config(w, world, {
-                    "cold_cache": f"{R} rotating copies of histories+logits ({foot / 2**20:.0f} MiB each, "
-                                  f"L2 is 126 MiB); inputs per step exceed L2",
-                    "launch": f"{mode}: {K_steps} steps x {4 if args.unfused else 3} kernels in one CUDA graph"
-                              if graph is not None else f"stream: {4 if args.unfused else 3} kernel launches per step",
-                    "entry_points": "hvd_lookup + hvd_score_select + hvd_verify_commit" if args.unfused
-                                    else "hvd_lookup_score_select + hvd_verify_commit",
-                    "kernel_events_in_timed_region": False, "tau": tau,
-                    "predictor": f"8->{w.hidden}" + (f"->{w.hidden}" if w.hidden_layers == 2 else "") + "->1 fp32"}),
-                "tokens_per_s": world * K_steps * tokens_per_step / (elapsed_ms * 1e-3),
-                "tokens_per_step": tokens_per_step,
-                "mean_accepted": float(accepted_h.mean()), "cache_selected_frac": float(select_h.mean()),
-                "kernel_us": kt, "roofline": roofline, "roofline_lookup": roofline_lookup,
-                "lookup_algorithmic_bytes": lookup_bytes,
-                # the whole step against the same peak: history bytes scanned + logits bytes read, per rank
-                "roofline_step": {"bound": "hbm", "algorithmic_bytes_per_step": lookup_bytes + verify_bytes,
-                                  "achieved": (lookup_bytes + verify_bytes) / (elapsed_ms / K_steps * 1e-3) / 1e9,
-                                  "peak": peak_gbs, "unit": "GB/s", "peak_kind": peak_kind,
-                                  "frac": (lookup_bytes + verify_bytes) / (elapsed_ms / K_steps * 1e-3) / 1e9 / peak_gbs},
-                "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": (4 if args.unfused else 3) * K_steps,
-                "clocks": sampler.summary(window)}
-        if kt:
-            # the same K steps with hvd_verify_commit_next (commit + next cycle's lookup and selection in one
-            # kernel: two launches per step), single rank's figure; the headline keeps the separate entry points
-            line["variant_commit_fused_with_next_lookup"] = {
-                "value": 1.0 / (kt["step_us_commit_fused_with_next_lookup"] * 1e-6), "unit": UNIT,
-                "us_per_step": kt["step_us_commit_fused_with_next_lookup"],
-                "entry_points": "hvd_verify_commit_next (after one hvd_lookup_score_select)"}
-        print(json.dumps(line), flush=True)
+    launches = 4 if args.unfused else 3
+    res = {"metric": METRIC, "value": steps_per_s, "unit": UNIT, "n_gpus": world, "steps": K_steps,
+           "warmup": W_steps, "ms_per_step": med_ms / K_steps, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+           "config": workload_config(w, world, {
+               "cold_cache": f"{R} rotating copies of the logits ({logits_bytes_alloc / 2**20:.0f} MiB each) and {RH} of the "
+                             f"histories ({hist_bytes_alloc / 2**20:.1f} MiB each); L2 is 126 MiB; "
+                             + ("inputs per step exceed L2 and no copy is reused within 2x L2 of traffic"
+                                if hist_cold else "the histories of the whole batch are too small to leave the L2"),
+               "launch": f"graph: {K_steps} steps x {launches} kernels in one CUDA graph, replayed {REPLAYS} times "
+                         f"after {UNTIMED_REPLAYS} untimed replays; value = K / median replay time",
+               "entry_points": "hvd_lookup + hvd_score_select + hvd_verify_commit" if args.unfused
+                               else "hvd_lookup_score_select + hvd_verify_commit",
+               "tau": tau,
+               "predictor": f"8->{w.hidden}" + (f"->{w.hidden}" if w.hidden_layers == 2 else "") + "->1 fp32"}),
+           "replays": REPLAYS, "us_per_step": step_us, "us_per_step_best": 1e3 * best_ms / K_steps,
+           "steps_per_s_best": world * K_steps / (best_ms * 1e-3),
+           "tokens_per_s": world * K_steps * tokens_per_step / (med_ms * 1e-3),
+           "tokens_per_step": tokens_per_step,
+           "mean_accepted": float(accepted_h.mean()), "cache_selected_frac": float(select_h.mean()),
+           "warm": {"us_per_step": kt["step_us_warm"], "us_per_step_best": kt["step_us_warm_best"],
+                    "steps_per_s": 1.0 / (kt["step_us_warm"] * 1e-6),
+                    "what": "the same K steps on ONE copy of the histories and logits (every step re-reads the buffers the "
+                            "previous step read: L2-resident as far as they fit 126 MiB); per rank"},
+           "kernel_us": kt, "roofline": roofline, "roofline_lookup": roofline_lookup, "roofline_step": roofline_step,
+           "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches * K_steps * REPLAYS,
+           "clocks": clocks,
+           "us_per_step_x_sm_ghz": step_us * (clocks["sm_mhz"] or 0) / 1e3,
+           # the same K steps with hvd_verify_commit_next (commit + next cycle's lookup and selection in one kernel:
+           # two launches per step), single rank's figure; the headline keeps the separate entry points
+           "variant_commit_fused_with_next_lookup": {
+               "value": 1.0 / (kt["step_us_commit_fused_with_next_lookup"] * 1e-6), "unit": UNIT,
+               "us_per_step": kt["step_us_commit_fused_with_next_lookup"],
+               "entry_points": "hvd_verify_commit_next (after one hvd_lookup_score_select)"}}
     ctx.close()
+    ctx_plain.close()
+    del hists, logits, logits0, hist0
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    return res
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2606_01019_b200.sharding import max_over_ranks
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the HVD path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_vec(ms):
+        if world == 1:
+            return ms
+        t = torch.as_tensor(ms, dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return t.cpu().numpy()
+
+    peak_gbs, peak_kind = measured_peak()
+    env = {"torch": torch, "dev": dev, "rank": rank, "world": world, "local": local, "peak": peak_gbs,
+           "peak_kind": peak_kind, "barrier": barrier, "max_over_ranks": lambda x: max_over_ranks(x, dev),
+           "max_over_ranks_vec": max_vec}
+    line = run_config(args.config, args, env, cpu_seconds=10.0)
+    if world == 1 and not args.only:
+        # every workload in the same line; the oracle leg is capped at a few seconds per workload
+        keep = ("us_per_step", "us_per_step_best", "value", "steps_per_s_best", "tokens_per_s", "tokens_per_step",
+                "mean_accepted", "cache_selected_frac", "warm", "kernel_us", "roofline", "roofline_lookup",
+                "roofline_step", "cpu_baseline", "e2e", "clocks", "us_per_step_x_sm_ghz", "dtype", "config")
+        per = {}
+        for name in ALL_CONFIGS:
+            r = line if name == args.config else run_config(name, args, env, cpu_seconds=4.0)
+            per[name] = {k: r[k] for k in keep}
+            per[name]["steps_per_s"] = per[name].pop("value")
+        line["per_config"] = per
+    if rank == 0:
+        print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 

@@ -1,10 +1,10 @@
-// Read-only streaming probe: the speed at which this GPU reads a buffer once with nothing else to do.
-// Not a step of the method: the benchmark runs it over the same logits buffers as the verification
-// kernel, so that the kernel's GB/s can be read against what a plain read loop reaches on the same
-// part, next to the copy bandwidth and the nominal figure.
-#include "hvd_internal.cuh"
+// Read-only streaming probe of bench.py: the speed at which this GPU reads a buffer once with nothing else to
+// do.  Not part of the HVD library and not a step of the method: the benchmark runs it over the same logits
+// buffers as the verification kernel, so that the kernel's GB/s can be read against what a plain read loop
+// reaches on the same part, next to the copy bandwidth and the nominal figure.
+#include <cuda_runtime.h>
+#include <stdint.h>
 
-namespace hvd {
 namespace {
 
 constexpr int kProbeThreads = 256;
@@ -35,12 +35,13 @@ __global__ void __launch_bounds__(kProbeThreads) read_probe_kernel(const uint4* 
 
 }  // namespace
 
-hvd_status launch_read_probe(hvd_ctx* ctx, const void* buf, int64_t bytes, cudaStream_t stream) {
-    const size_t n_vec = (size_t)bytes / 16;
-    const int grid = ctx->num_sms * 8;
-    read_probe_kernel<<<grid, kProbeThreads, 0, stream>>>(static_cast<const uint4*>(buf), n_vec, ctx->probe_sink);
-    HVD_CUDA_TRY(ctx, cudaGetLastError());
-    return HVD_OK;
+// Reads the first bytes / 16 * 16 bytes of buf (DEVICE, 16-byte aligned) once and leaves their maximum word in
+// *sink (DEVICE, 8 bytes).  Enqueues one kernel on `stream` (a cudaStream_t) with `grid` CTAs; returns the CUDA
+// error code of the launch (0 = success), -1 for a bad argument.
+extern "C" __attribute__((visibility("default"))) int bench_read_probe(const void* buf, int64_t bytes, void* sink,
+                                                                        int grid, void* stream) {
+    if (!buf || !sink || bytes < 0 || grid < 1 || (reinterpret_cast<uintptr_t>(buf) & 15)) return -1;
+    read_probe_kernel<<<grid, kProbeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(buf), (size_t)bytes / 16, static_cast<unsigned long long*>(sink));
+    return (int)cudaGetLastError();
 }
-
-}  // namespace hvd

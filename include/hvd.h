@@ -38,16 +38,17 @@
  *  - Consecutive kernels of a context are joined by programmatic dependent
  *    launch: a kernel may be resident while its predecessor on the stream
  *    still runs, and waits on the device before it reads anything the
- *    predecessor writes.  Results do not depend on it.  Two environment
- *    variables, read once by hvd_create, change it: HVD_PDL_MASK (a bit per
+ *    predecessor writes.  Results do not depend on it.  One environment
+ *    variable, read once by hvd_create, changes it: HVD_PDL_MASK (a bit per
  *    kernel pair: 1 commit, 2 lookup, 4 verify stream, 8 scoring; default 15,
- *    0 = plain launches) and HVD_ENABLE_PDL (any value: the launch attribute
- *    on every kernel of the library).
+ *    0 = plain launches).  It exists for the tests, which run the parity
+ *    cases with and without the overlap.
  *  - hvd_verify_commit and its variants stream the logits with one of two
  *    kernels, chosen by the size of the logits: one warp per 4 KB batch of a
  *    row up to 160 MB, a persistent kernel with work queues beyond that.
  *    HVD_VERIFY_SMALL_BYTES (read once by hvd_create) moves the limit, 0 =
- *    always the persistent kernel.  Results do not depend on it.  Nothing
+ *    always the persistent kernel: it exists for the tests, which run both
+ *    kernels over the same cases.  Results do not depend on it.  Nothing
  *    else is read from the environment by the product path.
  */
 #ifndef HVD_H
@@ -473,14 +474,6 @@ HVD_API hvd_status hvd_commit_keys(hvd_ctx* ctx, int32_t B, const int64_t* keys,
                                    const int64_t* hist_off, const int32_t* hist_cap, int32_t* hist_len,
                                    hvd_req_state* state, int32_t* accepted, int32_t* committed, int32_t* n_commit,
                                    int32_t* target_tok, int32_t* status, void* stream);
-
-/*
- * Measurement aid, not a step of the method: reads the first bytes / 16 * 16 bytes of buf (DEVICE,
- * 16-byte aligned) once with a plain grid-stride loop of 128-bit loads and keeps only their maximum
- * in context scratch.  Timed over the same buffers as hvd_verify_commit it gives the read-only
- * speed of the part, the practical ceiling of the streaming kernel.  Enqueues one kernel.
- */
-HVD_API hvd_status hvd_read_probe(hvd_ctx* ctx, const void* buf, int64_t bytes, void* stream);
 
 /*
  * Greedy verification and commit without a context and without any allocation.  (The paper has

@@ -62,7 +62,6 @@ _SIGNATURES = {
     "hvd_set_corpus": (_i32, [_vp, _vp, _i64]),
     "hvd_lookup_corpus": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_lookup_freq": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _f32, _i32, _f32] + [_vp] * 11 + [_vp]),
-    "hvd_read_probe": (_i32, [_vp, _vp, _i64, _vp]),
     "hvd_replay_labels": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
@@ -269,9 +268,6 @@ class Context:
             max_occ, threshold, _ptr(model_draft), _ptr(model_len), _ptr(draft), _ptr(draft_len), _ptr(score),
             _ptr(match_len), _ptr(match_pos), _ptr(match_cnt), _ptr(select), _ptr(sel_draft), _ptr(sel_len),
             _stream()), "hvd_lookup_freq")
-
-    def hvd_read_probe(self, buf, nbytes):
-        self._check(self._lib.hvd_read_probe(self._h, _ptr(buf), int(nbytes), _stream()), "hvd_read_probe")
 
     def hvd_replay_labels(self, trace, n, K, label, draft_len, match_len, match_pos, match_cnt):
         self._check(self._lib.hvd_replay_labels(self._h, _ptr(trace), n, K, _ptr(label), _ptr(draft_len),

@@ -47,5 +47,22 @@ def build(force: bool = False, verbose: bool = False, defines=()) -> str:
     return LIB
 
 
+PROBE_SRC = os.path.join(ROOT, "bench_probe.cu")
+PROBE_LIB = os.path.join(ROOT, "libbench_probe.so")
+
+
+def build_bench_probe(force: bool = False) -> str:
+    """The benchmark's read-only probe kernel (bench_probe.cu beside bench.py): a library of its own, so that
+    the product library exports only the method."""
+    if not force and os.path.exists(PROBE_LIB) and os.path.getmtime(PROBE_LIB) >= os.path.getmtime(PROBE_SRC):
+        return PROBE_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    res = subprocess.run([nvcc, *NVCC_FLAGS, "-o", PROBE_LIB, PROBE_SRC], capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed building libbench_probe.so")
+    return PROBE_LIB
+
+
 if __name__ == "__main__":
     print(build(force=True, verbose="-v" in sys.argv))

@@ -19,7 +19,7 @@ void release(hvd_ctx* c) {
     cudaFree(c->cp_key); cudaFree(c->cp_cnt); cudaFree(c->cp_arrived);
     cudaFree(c->cp_start); cudaFree(c->cp_pos);
     cudaFree(c->rp_key); cudaFree(c->rp_cnt);
-    cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->probe_sink); cudaFree(c->vf_row_key);
+    cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
     cudaFree(c->host_ws);
     delete c;
 }
@@ -89,7 +89,6 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->vf_row_key, (size_t)cfg->max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_next_unit, (size_t)kVerifyQueues * 32 * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->dev_error, sizeof(int)) == cudaSuccess;
-    ok = ok && alloc_zero(&c->probe_sink, sizeof(unsigned long long)) == cudaSuccess;
     if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); release(c); return HVD_ERR_ALLOC; }
 
@@ -107,29 +106,14 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->pdl_mask = getenv("HVD_PDL_MASK") ? atoi(getenv("HVD_PDL_MASK")) : 15;
     c->pdl_commit = (c->pdl_mask & 1) != 0;
     c->vf_small_bytes = getenv("HVD_VERIFY_SMALL_BYTES") ? atoll(getenv("HVD_VERIFY_SMALL_BYTES")) : kVerifySmallBytes;
-    c->use_pdl = getenv("HVD_ENABLE_PDL") != nullptr;  // every kernel of the library, the cluster kernel included: for experiments
     c->host_ws = nullptr;
     c->host_ws_bytes = 0;
-#ifdef HVD_TRACE
-    c->trace_words = (size_t)c->num_sms * 64 * 8;
-    alloc_zero(&c->trace, c->trace_words * 8);
-#endif
     *out = c;
     return HVD_OK;
 }
 
 hvd_status hvd_destroy(hvd_ctx* ctx) {
     if (!ctx) return HVD_ERR_INVALID_ARG;
-#ifdef HVD_TRACE
-    if (const char* path = getenv("HVD_TRACE_FILE")) {
-        unsigned long long* h = (unsigned long long*)malloc(ctx->trace_words * 8);
-        cudaDeviceSynchronize();
-        cudaMemcpy(h, ctx->trace, ctx->trace_words * 8, cudaMemcpyDeviceToHost);
-        if (FILE* f = fopen(path, "wb")) { fwrite(h, 8, ctx->trace_words, f); fclose(f); }
-        free(h);
-    }
-    cudaFree(ctx->trace);
-#endif
     release(ctx);
     return HVD_OK;
 }
@@ -288,14 +272,6 @@ hvd_status hvd_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist, const i
                               select, sel_draft, sel_len, static_cast<cudaStream_t>(stream));
 }
 
-hvd_status hvd_read_probe(hvd_ctx* ctx, const void* buf, int64_t bytes, void* stream) {
-    if (!ctx) return HVD_ERR_INVALID_ARG;
-    if (!buf) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_read_probe: NULL pointer");
-    if (bytes < 0) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_read_probe: negative size");
-    if (reinterpret_cast<uintptr_t>(buf) & 15) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_read_probe: buf not 16-byte aligned");
-    return launch_read_probe(ctx, buf, bytes, static_cast<cudaStream_t>(stream));
-}
-
 hvd_status hvd_replay_labels(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label,
                              int32_t* draft_len, int32_t* match_len, int32_t* match_pos, int32_t* match_cnt,
                              void* stream) {
@@ -419,9 +395,6 @@ static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits
     a.accepted = accepted; a.committed = committed; a.n_commit = n_commit; a.target_tok = target_tok;
     a.status = status; a.k_cap = ctx->cfg.k_cap;
     
-#ifdef HVD_TRACE
-    a.trace = ctx->trace;
-#endif
     a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error;
     a.row_key = ctx->vf_row_key; a.total_rows = total_rows; a.ext_keys = nullptr;
     if (!next) return launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
@@ -525,9 +498,6 @@ hvd_status hvd_verify_keys(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtyp
     a.sel_len = sel_len; a.hist_len = const_cast<int32_t*>(hist_len); a.hist_cap = hist_cap; a.k_cap = ctx->cfg.k_cap;
     a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error; a.total_rows = total_rows; a.ext_keys = nullptr;
     a.row_key = ctx->vf_row_key;
-#ifdef HVD_TRACE
-    a.trace = ctx->trace;
-#endif
     return launch_verify_keys(ctx, a, dtype, reinterpret_cast<long long*>(keys), v_offset, static_cast<cudaStream_t>(stream));
 }
 

@@ -321,7 +321,7 @@ hvd_status launch_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, co
                                        match_len, match_pos, match_cnt, nullptr, stream, ctx->cp_start != nullptr);
     if (r != HVD_OK) return r;
     if (ctx->cp_start == nullptr) {
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, corpus_none_kernel, dim3((unsigned)((B + 255) / 256)), 256, 0,
+        HVD_CUDA_TRY(ctx, launch_kernel(false, corpus_none_kernel, dim3((unsigned)((B + 255) / 256)), 256, 0,
                                         stream, B, match_src));
         return HVD_OK;
     }
@@ -337,7 +337,7 @@ hvd_status launch_lookup_corpus(hvd_ctx* ctx, int32_t B, const int32_t* hist, co
     a.draft = draft; a.draft_len = draft_len; a.match_len = match_len; a.match_pos = match_pos;
     a.match_src = match_src; a.match_cnt = match_cnt;
     a.key = ctx->cp_key; a.cnt = ctx->cp_cnt; a.arrived = ctx->cp_arrived;
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || ctx->pdl_mask != 0, corpus_probe_kernel, dim3((unsigned)a.slices, (unsigned)B),
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_mask != 0, corpus_probe_kernel, dim3((unsigned)a.slices, (unsigned)B),
                                     kProbeThreads, 0, stream, a));
     return HVD_OK;
 }

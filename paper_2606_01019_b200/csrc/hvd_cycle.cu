@@ -183,7 +183,7 @@ hvd_status launch_commit_lookup(hvd_ctx* ctx, const VerifyArgs& va, const int32_
     for (int k = 0; k < 8; ++k)
         if ((int64_t)shapes[k].threads * kLookupTokPerVec * shapes[k].iter >= (int64_t)n_max + 2) { pick = k; break; }
     if (pick < 0) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_next: history too long for one CTA");
-    const bool pdl = ctx->use_pdl || ctx->pdl_commit;
+    const bool pdl = ctx->pdl_commit;
     const dim3 grid((unsigned)va.B);
     cudaError_t e;
 #define HVD_LAUNCH_CYCLE(TH, I) launch_kernel(pdl, commit_lookup_kernel<TH, I>, grid, TH, 0, stream, va, a, sa)

@@ -312,9 +312,9 @@ hvd_status launch_lookup_freq(hvd_ctx* ctx, int32_t B, const int32_t* hist, cons
     a.occ = ctx->fq_occ; a.occ_cnt = ctx->fq_cnt;
     const int64_t span = (int64_t)(n_max > 1 ? n_max - 1 : 1) + 3;
     const unsigned chunks = (unsigned)((span + kCollectChunk - 1) / kCollectChunk);
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || ctx->pdl_mask != 0, freq_collect_kernel, dim3(chunks, (unsigned)B), kCollectThreads, 0,
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_mask != 0, freq_collect_kernel, dim3(chunks, (unsigned)B), kCollectThreads, 0,
                                     stream, a));
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || ctx->pdl_mask != 0, freq_walk_kernel, dim3((unsigned)B), kWalkThreads, 0, stream, a));
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_mask != 0, freq_walk_kernel, dim3((unsigned)B), kWalkThreads, 0, stream, a));
     return HVD_OK;
 }
 

@@ -94,19 +94,13 @@ struct hvd_ctx {
     unsigned long long* vf_row_key;  // [max_rows], zero at rest
     uint32_t* vf_next_unit;          // zero at rest
     int* dev_error;                  // device status word
-    unsigned long long* probe_sink;  // result word of the read-only probe
     int vf_blocks_per_sm[2];         // per dtype
     long long vf_small_bytes;        // size limit of the warp-per-batch kernels (HVD_VERIFY_SMALL_BYTES; 0 = never)
     // device staging of the host-buffer entry point (grown on demand)
-    bool use_pdl;     // programmatic dependent launch for every kernel of the library (HVD_ENABLE_PDL; experiments)
     int pdl_mask;     // ... for the three kernels of a step: bit 0 commit, 1 lookup, 2 stream, 3 one-layer scoring (default all)
     bool pdl_commit;  // bit 0 of the mask
     char* host_ws;
     size_t host_ws_bytes;
-#ifdef HVD_TRACE
-    unsigned long long* trace;  // [num_sms * 64 warps * 8] last verify launch, dumped by hvd_destroy
-    size_t trace_words;
-#endif
     char last_error[256];
 };
 
@@ -192,7 +186,6 @@ hvd_status launch_score_select_ext(hvd_ctx* ctx, int32_t B, const int32_t* hist_
                                    const int32_t* model_draft, const int32_t* model_len, float* features, float* score,
                                    int32_t* select, int32_t* sel_draft, int32_t* sel_len, cudaStream_t stream);
 
-hvd_status launch_read_probe(hvd_ctx* ctx, const void* buf, int64_t bytes, cudaStream_t stream);
 hvd_status launch_replay(hvd_ctx* ctx, const int32_t* trace, int32_t n, int32_t K, int32_t* label, int32_t* draft_len,
                          int32_t* match_len, int32_t* match_pos, int32_t* match_cnt, cudaStream_t stream);
 
@@ -239,9 +232,6 @@ struct VerifyArgs {
     uint32_t* next_unit;   // unit counter, zero at rest
     int* dev_error;        // device status word (no kernel sets it at present)
     int32_t n_batch_row;   // 4 KB batches per row
-#ifdef HVD_TRACE
-    unsigned long long* trace;  // per-warp timeline (debug builds only)
-#endif
 };
 
 hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit = true);

@@ -197,8 +197,8 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
     cudaError_t e;
     const ScoreArgs sa = fused ? *fused : ScoreArgs();
 #define HVD_LAUNCH_LOOKUP(TH, I)                                                                       \
-    (fused ? launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 2), lookup_kernel<TH, I, true>, grid, TH, 0, stream, a, sa)      \
-           : launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 2), lookup_kernel<TH, I, false>, grid, TH, 0, stream, a, sa))
+    (fused ? launch_kernel((ctx->pdl_mask & 2), lookup_kernel<TH, I, true>, grid, TH, 0, stream, a, sa)      \
+           : launch_kernel((ctx->pdl_mask & 2), lookup_kernel<TH, I, false>, grid, TH, 0, stream, a, sa))
     switch (pick) {
         case 0: e = HVD_LAUNCH_LOOKUP(256, 1); break;
         case 1: e = HVD_LAUNCH_LOOKUP(256, 2); break;

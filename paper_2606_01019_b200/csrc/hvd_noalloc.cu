@@ -58,7 +58,6 @@ hvd_status setup_device(int device, DeviceSetup** out, const char** why) {
             *why = "the verify kernels do not fit this device";
             return HVD_ERR_UNSUPPORTED;
         }
-        s.ctx.use_pdl = false;
         s.ctx.pdl_commit = false;
         s.ctx.pdl_mask = 0;
         s.ctx.vf_small_bytes = kVerifySmallBytes;
@@ -138,9 +137,6 @@ hvd_status hvd_verify_commit_noalloc(int32_t B, int32_t k_cap, const void* logit
     a.status = status; a.k_cap = k_cap;
     a.next_unit = counters; a.dev_error = nullptr;
     a.row_key = row_key; a.total_rows = total_rows; a.ext_keys = nullptr;
-#ifdef HVD_TRACE
-    a.trace = nullptr;
-#endif
     hvd_ctx call_ctx = s->ctx;  // private copy: the error text of a failed launch lands here
     call_ctx.cfg.k_cap = k_cap;
     const hvd_status r = launch_verify(&call_ctx, a, dtype, cs);

@@ -234,7 +234,7 @@ static hvd_status launch_score_kernels(hvd_ctx* ctx, const ScoreArgs& a, int32_t
         return HVD_OK;
     }
     const int blocks = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 8), score_select_kernel<EXT>, blocks, kWarpsPerBlock * 32, 0, stream, a));
+    HVD_CUDA_TRY(ctx, launch_kernel((ctx->pdl_mask & 8), score_select_kernel<EXT>, blocks, kWarpsPerBlock * 32, 0, stream, a));
     return HVD_OK;
 }
 

@@ -299,16 +299,6 @@ struct Smem {
     }
 };
 
-#ifdef HVD_TRACE
-__device__ __forceinline__ unsigned long long gtime() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define TR(...) __VA_ARGS__
-#else
-#define TR(...)
-#endif
 
 template <typename E>
 __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel(const VerifyArgs a) {
@@ -322,7 +312,6 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
     const int warp = tid >> 5;
     constexpr int EPV = Tracker<E>::kPerVec;
     constexpr int ESZ = 16 / EPV;
-    TR(unsigned long long t_enter = gtime(); unsigned long long acc_wait = 0, acc_str = 0, acc_close = 0, n_b = 0;)
     // wait first, then let the commit kernel in: it reads the selection before its own wait, so it must not
     // start before the kernel that wrote the selection (this kernel's predecessor) is known to be complete
     pdl_wait();
@@ -376,11 +365,9 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
     const uint32_t n_units = n_big + (uint32_t)(total - (int64_t)n_big * UB);
     const char* base_ptr = static_cast<const char*>(a.logits);
     const unsigned long long pol = stream_policy();
-    TR(unsigned long long t_loop = gtime();)
 
     // ---- phase 1: units of batches -------------------------------------------------------------------
     while (cur < n_units) {
-        TR(unsigned long long tw0 = gtime();)
         // `nxt` was requested a unit ago; the one after it is requested now, a whole unit before it is
         // needed (in the end game too: holding one single-batch unit back costs less than waiting for every
         // answer: measured 1.3 us per C2 launch, 17 us on C3)
@@ -394,7 +381,6 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
         }
         if (nxt < n_units) { if (lane == 0) nn = fetch(queue); }
         else nn = nxt;  // nothing left, stays so
-        TR(acc_wait += gtime() - tw0;)
 
         const int64_t c0 = cur < n_big ? (int64_t)cur * UB : (int64_t)n_big * UB + (cur - n_big);
         const int64_t c1 = cur < n_big ? c0 + UB : c0 + 1;
@@ -409,7 +395,6 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
         int geom_r = -1;
 #pragma unroll 1
         for (int64_t p = c0; p < c1; ++p, ++gb) {
-            TR(unsigned long long ts0 = gtime();)
             if (gb >= nbr) { gb -= nbr; ++r; }
             if (r != geom_r) {
                 if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + grow, ukey);
@@ -462,13 +447,11 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
                 const unsigned long long key = ((unsigned long long)word << 32) | (uint32_t)(~widx);
                 ukey = key > ukey ? key : ukey;
             }
-            TR(acc_str += gtime() - ts0; ++n_b;)
         }
         if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + grow, ukey);
         cur = nxt;
         nxt = nn;
     }
-    TR(if (a.trace && lane == 0) { unsigned long long* tr = a.trace + ((size_t)blockIdx.x * NW + warp) * 8; tr[0] = t_enter; tr[1] = t_loop; tr[2] = gtime(); tr[3] = acc_wait; tr[4] = acc_str; tr[5] = acc_close; tr[6] = 0; tr[7] = n_b; })
 }
 
 }  // namespace
@@ -616,13 +599,13 @@ hvd_status launch_verify_keys(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, long 
     const hvd_status r = launch_verify(ctx, a, dtype, stream, false);
     if (r != HVD_OK) return r;
     const int64_t n = a.total_rows > Q ? a.total_rows : Q;
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || ctx->pdl_mask != 0, keys_finish_kernel, dim3((unsigned)((n + 255) / 256)), 256, 0, stream,
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_mask != 0, keys_finish_kernel, dim3((unsigned)((n + 255) / 256)), 256, 0, stream,
                                     a.row_key, keys, a.total_rows, v_offset, a.next_unit));
     return HVD_OK;
 }
 
 hvd_status launch_commit_keys(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream) {
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl, commit_keys_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+    HVD_CUDA_TRY(ctx, launch_kernel(false, commit_keys_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
                                     kCommitWarps * 32, 0, stream, a));
     return HVD_OK;
 }
@@ -654,7 +637,7 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
     const bool spec = full_bytes <= kVerifySpecBytes;
     if (small) {
         const dim3 sgrid((unsigned)((a.n_batch_row + kSmallWarps - 1) / kSmallWarps), (unsigned)a.total_rows);
-        const bool pdl = ctx->use_pdl || (ctx->pdl_mask & 4);
+        const bool pdl = (ctx->pdl_mask & 4);
         cudaError_t e;
         if (dtype == HVD_F32)
             e = spec ? launch_kernel(pdl, verify_small_kernel<float, true>, sgrid, kSmallWarps * 32, 0, stream, a)
@@ -664,11 +647,11 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
                      : launch_kernel(pdl, verify_small_kernel<__nv_bfloat16, false>, sgrid, kSmallWarps * 32, 0, stream, a);
         HVD_CUDA_TRY(ctx, e);
     } else if (dtype == HVD_F32)
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 4), verify_stream_kernel<float>, grid, T, smem, stream, a));
+        HVD_CUDA_TRY(ctx, launch_kernel((ctx->pdl_mask & 4), verify_stream_kernel<float>, grid, T, smem, stream, a));
     else
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || (ctx->pdl_mask & 4), verify_stream_kernel<__nv_bfloat16>, grid, T, smem, stream, a));
+        HVD_CUDA_TRY(ctx, launch_kernel((ctx->pdl_mask & 4), verify_stream_kernel<__nv_bfloat16>, grid, T, smem, stream, a));
     if (with_commit)
-        HVD_CUDA_TRY(ctx, launch_kernel(ctx->use_pdl || ctx->pdl_commit, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_commit, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
                                         kCommitWarps * 32, 0, stream, a));
     return HVD_OK;
 }

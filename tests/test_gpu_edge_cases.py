@@ -308,26 +308,6 @@ def test_history_of_more_than_65535_chunks():
     ctx.close()
 
 
-def test_read_probe_runs_and_checks_its_arguments():
-    """The read-only probe of the benchmark: any size (whole vectors, a ragged tail, nothing), and the
-    host-side argument checks."""
-    import torch
-    import paper_2606_01019_b200 as H
-    ctx = H.Context(max_batch=1, k_cap=8, max_hist_len=16, max_rows=1, max_vocab=16)
-    buf = torch.randint(0, 2**31 - 1, (1 << 20,), dtype=torch.int32, device="cuda")
-    for nbytes in (0, 16, 4096, 4 * (1 << 20) - 4, 4 * (1 << 20)):
-        ctx.hvd_read_probe(buf, nbytes)
-    torch.cuda.synchronize()
-    assert ctx.hvd_device_status() == 0
-    with pytest.raises(H.HvdError, match="NULL"):
-        ctx.hvd_read_probe(None, 16)
-    with pytest.raises(H.HvdError, match="negative"):
-        ctx.hvd_read_probe(buf, -1)
-    with pytest.raises(H.HvdError, match="aligned"):
-        ctx.hvd_read_probe(buf[1:], 16)
-    ctx.close()
-
-
 def test_parity_with_plain_launches():
     """The same parity cases with programmatic dependent launch switched off (every kernel starts after
     its predecessor has completed): a result must not depend on how far consecutive kernels overlap."""
@@ -358,7 +338,7 @@ def test_parity_with_the_persistent_streaming_kernel_only():
     """Logits of up to 160 MB are streamed by the warp-per-batch kernels, so most cases of this suite never
     reach the persistent kernel: the shape, alignment, tie and multi-step cases once more with the limit at 0."""
     _rerun({"HVD_VERIFY_SMALL_BYTES": "0"}, ["tests/test_gpu_parity.py", "tests/test_gpu_edge_cases.py"],
-           "not full_size and not plain_launches and not kernel_only and not 65535 and not read_probe")
+           "not full_size and not plain_launches and not kernel_only and not 65535")
 
 
 def test_parity_with_the_warp_per_batch_kernel_on_a_large_call():
