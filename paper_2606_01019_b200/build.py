@@ -47,6 +47,27 @@ def build(force: bool = False, verbose: bool = False, defines=()) -> str:
     return LIB
 
 
+BOUNDS_LIB = os.path.join(PKG, "libhvd_b200_bounds.so")
+
+
+def build_bounds_checked(force: bool = False) -> str:
+    """The same sources with -DHVD_DEBUG_BOUNDS: every index of the lookup, commit and streaming kernels is tested
+    before the access, a violation lands in the device status word (hvd_device_status) and the access is
+    skipped.  The tests run the edge cases against this library (HVD_B200_LIB selects it)."""
+    if not force and os.path.exists(BOUNDS_LIB):
+        t = os.path.getmtime(BOUNDS_LIB)
+        deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
+        if all(os.path.getmtime(d) <= t for d in deps):
+            return BOUNDS_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    cmd = [nvcc, *NVCC_FLAGS, "-DHVD_DEBUG_BOUNDS", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", BOUNDS_LIB, *sources()]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed building libhvd_b200_bounds.so")
+    return BOUNDS_LIB
+
+
 PROBE_SRC = os.path.join(ROOT, "bench_probe.cu")
 PROBE_LIB = os.path.join(ROOT, "libbench_probe.so")
 

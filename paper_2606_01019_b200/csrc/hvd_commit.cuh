@@ -36,6 +36,7 @@ constexpr unsigned long long kKeySign = 0x8000000000000000ull;
 // The (value, ~index) key of a logits row.  Context scratch is put back to zero as it is read; keys
 // handed in by the caller (hvd_commit_keys) are in signed order and are left alone.
 __device__ __forceinline__ unsigned long long read_row_key(const VerifyArgs& a, int64_t r) {
+    if (!HVD_IN_BOUNDS(a.dev_error, r, 0, a.total_rows)) return 0ull;
     if (a.ext_keys) return (unsigned long long)a.ext_keys[r] ^ kKeySign;  // "row not read" becomes 0
     const unsigned long long key = a.row_key[r];
     a.row_key[r] = 0ull;  // scratch is zero at rest
@@ -67,7 +68,9 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
     if (q.nr == 0) {
         // skipped request: neutral outputs, nothing else touched
         for (int j = lane; j <= kc; j += 32) z[j] = -1;
-        if (a.target_tok) for (int64_t r = q.r0 + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
+        if (a.target_tok)
+            for (int64_t r = q.r0 + lane; r < q.r1; r += 32)
+                if (HVD_IN_BOUNDS(a.dev_error, r, 0, a.total_rows)) a.target_tok[r] = -1;
         if (lane == 0) { a.accepted[b] = 0; a.n_commit[b] = 0; a.status[b] = HVD_REQ_BAD_LEN; }
         if (out) { out->n = n; out->st = st; }
         return;
@@ -93,7 +96,7 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
         t = (int)min((int64_t)max(t, 0), a.V - 1);  // inside the vocabulary whatever the data
         bool stop = true;
         if (i <= m) {
-            if (a.target_tok) a.target_tok[q.r0 + i] = t;
+            if (a.target_tok && HVD_IN_BOUNDS(a.dev_error, q.r0 + i, 0, a.total_rows)) a.target_tok[q.r0 + i] = t;
             const int di = k == 0 ? d0 : (k == 1 ? d1 : -1);
             stop = (i >= m) || (di != t);
         }
@@ -106,7 +109,8 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
     }
     // acc <= m always (row m stops).  Rows beyond m were not read.
     if (a.target_tok)
-        for (int64_t r = q.r0 + q.nr + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
+        for (int64_t r = q.r0 + q.nr + lane; r < q.r1; r += 32)
+            if (HVD_IN_BOUNDS(a.dev_error, r, 0, a.total_rows)) a.target_tok[r] = -1;
     const int room = cap - n;
     const int w = min(acc + 1, room);
     int32_t* h = a.hist + hoff;
@@ -114,7 +118,7 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
         const int dj = j < 32 ? d0 : d1;
         const int tok = (j < acc) ? dj : (j == acc ? t_acc : -1);
         z[j] = tok;
-        if (j < w) h[n + j] = tok;
+        if (j < w && HVD_IN_BOUNDS(a.dev_error, n + j, 0, cap)) h[n + j] = tok;
     }
     st.sel_bits = (st.sel_bits << 1) | (sel ? 1u : 0u);
     st.acc_ring = (st.acc_ring << 8) | (unsigned long long)(acc & 0xff);

@@ -122,6 +122,21 @@ inline hvd_status cuda_fail(hvd_ctx* ctx, cudaError_t e, const char* where) {
         if (e_ != cudaSuccess) return hvd::cuda_fail((ctx), e_, #call);  \
     } while (0)
 
+// Bounds-checked builds (-DHVD_DEBUG_BOUNDS; the stand-in for a memory checker where none can be run): every
+// index into a history slab, the logits, the row keys and the per-row / per-request outputs is tested before
+// the access.  A violation sets the device status word to HVD_DEV_OUT_OF_BOUNDS and the access is skipped:
+// nothing traps.  In the normal build the test is the constant `true` and costs nothing.
+#if defined(__CUDACC__) && defined(HVD_DEBUG_BOUNDS)
+__device__ __forceinline__ bool index_in_bounds(int* status_word, long long i, long long lo, long long hi) {
+    if (i >= lo && i < hi) return true;
+    if (status_word) atomicExch(status_word, (int)HVD_DEV_OUT_OF_BOUNDS);
+    return false;
+}
+#define HVD_IN_BOUNDS(status_word, i, lo, hi) hvd::index_in_bounds((status_word), (long long)(i), (long long)(lo), (long long)(hi))
+#else
+#define HVD_IN_BOUNDS(status_word, i, lo, hi) true
+#endif
+
 // Programmatic dependent launch: every kernel of the path lets its successor in the stream be
 // scheduled early (pdl_trigger) and waits for its predecessor's memory (pdl_wait) before it reads
 // anything a predecessor wrote.  Both are no-ops for a launch without the attribute.

@@ -68,13 +68,14 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
 #pragma unroll
     for (int i = 0; i < ITER; ++i) {
         const int v = v0 + i * THREADS + tid;
-        if (4 * v < g_end) x[i] = ld_hist(vbase + v);
+        // (bounds-checked builds: an aligned vector may reach up to 3 tokens before the slab and past its end)
+        if (4 * v < g_end && HVD_IN_BOUNDS(a.dev_error, 4 * v - mis, -3, (int64_t)cap_b + 1)) x[i] = ld_hist(vbase + v);
         else x[i] = make_int4(0, 0, 0, 0);
     }
     // query: the history's own tail.  q0 = last token; lane j keeps the tokens 1+j and 33+j back.
-    const int32_t q0 = slab[n - 1];
-    const int32_t qa = (1 + lane <= n - 1) ? slab[n - 2 - lane] : 0;
-    const int32_t qb = (33 + lane <= n - 1) ? slab[n - 34 - lane] : 0;
+    const int32_t q0 = HVD_IN_BOUNDS(a.dev_error, n - 1, 0, cap_b) ? slab[n - 1] : 0;
+    const int32_t qa = (1 + lane <= n - 1 && HVD_IN_BOUNDS(a.dev_error, n - 2 - lane, 0, cap_b)) ? slab[n - 2 - lane] : 0;
+    const int32_t qb = (33 + lane <= n - 1 && HVD_IN_BOUNDS(a.dev_error, n - 34 - lane, 0, cap_b)) ? slab[n - 34 - lane] : 0;
 
     Best best;  // identical in all lanes of a warp
     best.key = 0; best.cnt = 0;
@@ -87,7 +88,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
             c.key = ((unsigned long long)(uint32_t)L << 32) | (uint32_t)(p + 1);
             c.cnt = 1;
             best = combine(best, c);
-        });
+        }, a.dev_error);
     }
 
     __shared__ unsigned long long s_key[THREADS / 32];
@@ -105,7 +106,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
     if (lane == 0) {
         if (n_chunks > 1) {
             LookupPartial* slot = a.partial + (int64_t)b * a.max_chunks + chunk;
-            slot->key = r.key; slot->cnt = r.cnt;
+            if (HVD_IN_BOUNDS(a.dev_error, chunk, 0, a.max_chunks)) { slot->key = r.key; slot->cnt = r.cnt; }
             __threadfence();
             const uint32_t old = atomicAdd(a.req_cnt + b, 1u);
             last = (old + 1 == (uint32_t)n_chunks) ? 1u : 0u;
@@ -139,8 +140,8 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
     } else {
         d = min(draft_limit(K_b, a.k_cap, L, a.spec_factor, a.spec_offset), n - e);
     }
-    const int tok0 = lane < d ? slab[e + lane] : -1;
-    const int tok1 = lane + 32 < d ? slab[e + lane + 32] : -1;
+    const int tok0 = (lane < d && HVD_IN_BOUNDS(a.dev_error, e + lane, 0, n)) ? slab[e + lane] : -1;
+    const int tok1 = (lane + 32 < d && HVD_IN_BOUNDS(a.dev_error, e + lane + 32, 0, n)) ? slab[e + lane + 32] : -1;
     if (FUSED) {
         // everything the scoring reads is requested before the lookup's own results are stored (a store
         // would hold back the loads behind it): draft tokens, decode state and model draft in one round trip

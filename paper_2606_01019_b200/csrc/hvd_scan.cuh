@@ -77,7 +77,8 @@ __device__ __forceinline__ int4 ld_hist(const int4* p) {
 // appended to the history it scans).
 template <bool COHERENT = false, class OnMatch>
 __device__ __forceinline__ void scan_vector(const int4 x, int p0, int n, const int32_t* __restrict__ slab, int32_t q0,
-                                            int32_t qa, int32_t qb, int l_max, int lane, OnMatch&& on_match) {
+                                            int32_t qa, int32_t qb, int l_max, int lane, OnMatch&& on_match,
+                                            int* status_word = nullptr) {
     uint32_t m = 0;
     m |= (x.x == q0 && p0 + 0 >= 0 && p0 + 0 <= n - 2) ? 1u : 0u;
     m |= (x.y == q0 && p0 + 1 >= 0 && p0 + 1 <= n - 2) ? 2u : 0u;
@@ -96,14 +97,14 @@ __device__ __forceinline__ void scan_vector(const int4 x, int p0, int n, const i
             // match length of the copy ending at p (>= 1 already); limit: l_max and the slab start
             const int cap = min(l_max, p + 1);
             int l = lane + 1;
-            bool eq = (l < cap) && ((COHERENT ? __ldcg(slab + p - l) : slab[p - l]) == qa);
+            bool eq = (l < cap) && HVD_IN_BOUNDS(status_word, p - l, 0, n) && ((COHERENT ? __ldcg(slab + p - l) : slab[p - l]) == qa);
             uint32_t mm = __ballot_sync(0xffffffffu, !eq);
             int L;
             if (mm != 0) {
                 L = __ffs(mm);  // first failing lane j: lengths 1..j hold, so L = 1 + j
             } else {
                 l = lane + 33;
-                eq = (l < cap) && ((COHERENT ? __ldcg(slab + p - l) : slab[p - l]) == qb);
+                eq = (l < cap) && HVD_IN_BOUNDS(status_word, p - l, 0, n) && ((COHERENT ? __ldcg(slab + p - l) : slab[p - l]) == qb);
                 mm = __ballot_sync(0xffffffffu, !eq);  // lane 31 (l = 64) always fails
                 L = 32 + __ffs(mm);
             }

@@ -188,7 +188,9 @@ __device__ __forceinline__ void commit_tree_request(const VerifyArgs& a, int b, 
     int32_t* z = a.committed + (int64_t)b * (kc + 1);
     if (q.nr == 0) {
         for (int j = lane; j <= kc; j += 32) z[j] = -1;
-        if (a.target_tok) for (int64_t r = q.r0 + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
+        if (a.target_tok)
+            for (int64_t r = q.r0 + lane; r < q.r1; r += 32)
+                if (HVD_IN_BOUNDS(a.dev_error, r, 0, a.total_rows)) a.target_tok[r] = -1;
         if (lane == 0) { a.accepted[b] = 0; a.n_commit[b] = 0; a.status[b] = HVD_REQ_BAD_LEN; }
         return;
     }
@@ -203,11 +205,12 @@ __device__ __forceinline__ void commit_tree_request(const VerifyArgs& a, int b, 
             const unsigned long long key = read_row_key(a, q.r0 + i);
             const int t = (int)(~(uint32_t)(key & 0xffffffffu));
             tok[k] = (int)min((int64_t)max(t, 0), a.V - 1);
-            if (a.target_tok) a.target_tok[q.r0 + i] = tok[k];
+            if (a.target_tok && HVD_IN_BOUNDS(a.dev_error, q.r0 + i, 0, a.total_rows)) a.target_tok[q.r0 + i] = tok[k];
         }
     }
     if (a.target_tok)
-        for (int64_t r = q.r0 + q.nr + lane; r < q.r1; r += 32) a.target_tok[r] = -1;
+        for (int64_t r = q.r0 + q.nr + lane; r < q.r1; r += 32)
+            if (HVD_IN_BOUNDS(a.dev_error, r, 0, a.total_rows)) a.target_tok[r] = -1;
     int zr[3] = {-1, -1, -1};  // committed tokens lane, lane+32, lane+64
     int acc = 0, cur = -1;
     for (;;) {
@@ -233,7 +236,7 @@ __device__ __forceinline__ void commit_tree_request(const VerifyArgs& a, int b, 
         if (j <= kc) {
             const int tk = j <= acc ? zr[k] : -1;
             z[j] = tk;
-            if (j < w) h[n + j] = tk;
+            if (j < w && HVD_IN_BOUNDS(a.dev_error, n + j, 0, cap)) h[n + j] = tk;
         }
     }
     if (lane == 0) {
@@ -397,7 +400,7 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
         for (int64_t p = c0; p < c1; ++p, ++gb) {
             if (gb >= nbr) { gb -= nbr; ++r; }
             if (r != geom_r) {
-                if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + grow, ukey);
+                if (lane == 0 && ukey != 0ull && grow >= 0) atomicMax(a.row_key + grow, ukey);
                 ukey = 0ull;
                 geom_r = r;
                 int lo = 0, hi = a.B;  // request of the row: largest b with pref[b] <= r
@@ -406,6 +409,7 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
                     if (sm.pref[mid] <= r) lo = mid; else hi = mid;
                 }
                 grow = sm.row0[lo] + (r - sm.pref[lo]);
+                if (!HVD_IN_BOUNDS(a.dev_error, grow, 0, a.total_rows)) { grow = -1; head = 0; n_vec = 0; tail = 0; continue; }
                 row = base_ptr + grow * a.V * ESZ;
                 const int head_bytes = (int)((16 - (reinterpret_cast<uintptr_t>(row) & 15)) & 15);
                 head = (int)min((int64_t)(head_bytes / ESZ), a.V);
@@ -448,7 +452,7 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
                 ukey = key > ukey ? key : ukey;
             }
         }
-        if (lane == 0 && ukey != 0ull) atomicMax(a.row_key + grow, ukey);
+        if (lane == 0 && ukey != 0ull && grow >= 0) atomicMax(a.row_key + grow, ukey);
         cur = nxt;
         nxt = nn;
     }
@@ -471,6 +475,7 @@ __global__ void __launch_bounds__(kSmallWarps * 32) verify_small_kernel(const Ve
     const int lane = threadIdx.x & 31;
     const int gb = blockIdx.x * kSmallWarps + (threadIdx.x >> 5);  // batch inside the row
     const int64_t r = blockIdx.y;                                  // logits row
+    if (!HVD_IN_BOUNDS(a.dev_error, r, 0, a.total_rows)) return;   // warp-uniform
     // wait first, then let the commit kernel in (it reads the selection before its own wait)
     pdl_wait();
     pdl_trigger();

@@ -24,3 +24,22 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _device_status_stays_clean(monkeypatch):
+    """With HVD_ASSERT_DEVICE_STATUS=1 (set by the test that reruns the edge cases against the bounds-checked
+    build of the library) every context must still report device status 0 when it is closed."""
+    if os.environ.get("HVD_ASSERT_DEVICE_STATUS") != "1":
+        yield
+        return
+    import paper_2606_01019_b200 as H
+    orig = H.Context.close
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            assert self.hvd_device_status() == 0, "a kernel of the bounds-checked build recorded an index out of range"
+        orig(self)
+
+    monkeypatch.setattr(H.Context, "close", close)
+    yield

@@ -345,3 +345,17 @@ def test_parity_with_the_warp_per_batch_kernel_on_a_large_call():
     """... and the other way round: the full-size C2 and C5 workloads (279 MB and 2.5 GB of logits, uniform and
     ragged rows) through the warp-per-batch kernel that checks the need first."""
     _rerun({"HVD_VERIFY_SMALL_BYTES": str(1 << 40)}, ["tests/test_gpu_parity.py"], "full_size and (C2 or C5)")
+
+
+def test_edge_cases_against_the_bounds_checked_build():
+    """The stand-in for a memory checker: the library built with -DHVD_DEBUG_BOUNDS tests every index of the
+    lookup, commit and streaming kernels before the access and records a violation in the device status word.
+    The edge, shape and random cases once more against that build (with both streaming kernels); every context
+    must close with status 0, and the results must still equal the oracle's."""
+    from paper_2606_01019_b200 import build
+    lib = build.build_bounds_checked()
+    sel = "not plain_launches and not kernel_only and not large_call and not bounds_checked and not full_size"
+    files = ["tests/test_gpu_edge_cases.py", "tests/test_gpu_parity.py", "tests/test_gpu_cycle.py", "tests/test_gpu_tree.py"]
+    _rerun({"HVD_B200_LIB": lib, "HVD_ASSERT_DEVICE_STATUS": "1"}, files, sel)
+    _rerun({"HVD_B200_LIB": lib, "HVD_ASSERT_DEVICE_STATUS": "1", "HVD_VERIFY_SMALL_BYTES": "0"},
+           ["tests/test_gpu_edge_cases.py"], sel)
