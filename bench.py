@@ -43,8 +43,18 @@ REPLAYS = 20          # timed replays of the K-step graph (median and best repor
 UNTIMED_REPLAYS = 3
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the kernel on the workload, from the ncu captures
 # summarised under profiles/ (per launch, like the algorithmic bytes; absent = not captured)
-NCU_VERIFY_TRAFFIC_BYTES = {"C2": 261772928}   # profiles/verify_stream_kernel_c2_ncu.txt, mean of two launches
-NCU_LOOKUP_TRAFFIC_BYTES = {"C2": 4242048}     # profiles/lookup_kernel_c2_ncu.txt
+NCU_VERIFY_TRAFFIC_BYTES = {
+    "C2": (261772928, "profiles/verify_stream_kernel_c2_ncu.txt"),
+    "C3": (2129576753, "profiles/verify_stream_kernel_c3_batch64_ncu.txt: captured at batch 64 (1.0060 x the algorithmic "
+                       "bytes), scaled to the full launch by the needed rows"),
+    "C4": (431484000, "profiles/verify_stream_kernel_c4_ncu.txt"),
+}
+NCU_LOOKUP_TRAFFIC_BYTES = {
+    "C2": (4239744, "profiles/lookup_kernel_c2_ncu.txt"),
+    "C3": (33662000, "profiles/lookup_kernel_c3_ncu.txt"),
+    "C4": (16845000, "profiles/lookup_kernel_c4_ncu.txt"),
+    "C5": (29784000, "profiles/lookup_kernel_c5_ncu.txt"),
+}
 
 
 def parse_args():
@@ -60,6 +70,13 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--predictor", default="config", choices=["config", "2x256"],
                     help="2x256: the paper's predictor shape (two hidden layers of 256 units) instead of the config's")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="scale the workload to this many requests (profiling a workload's shape at a smaller size)")
+    ap.add_argument("--profile", default=None, choices=["step", "lookup", "cycle"],
+                    help="profiling run, meant for ncu: W warm-up steps and K steps as plain stream launches on the "
+                         "rotating inputs and nothing else (no graphs, no oracle, no end-to-end leg); `lookup`: only the "
+                         "fused lookup + scoring kernel, and no logits are allocated; `cycle`: hvd_verify_commit_next "
+                         "(commit fused with the next lookup) in place of the step's three kernels")
     ap.add_argument("--unfused", action="store_true",
                     help="call hvd_lookup and hvd_score_select separately instead of hvd_lookup_score_select")
     return ap.parse_args()
@@ -232,6 +249,8 @@ def run_config(name, args, env, cpu_seconds):
     w = W.CONFIGS[name]
     if args.predictor == "2x256":
         w = w.scaled(hidden=256, hidden_layers=2)
+    if args.batch:
+        w = w.scaled(B=args.batch)
     K_steps, W_steps = args.steps, args.warmup
     n_slots = K_steps + W_steps
 
@@ -314,6 +333,16 @@ def run_config(name, args, env, cpu_seconds):
         set_predictor(tau)
         score_select(hist_len0, state0)
     torch.cuda.synchronize()
+    if args.profile == "lookup":
+        nb = rq.hist.nbytes
+        RH = int(max(2, min(64, -(-4 * L2_BYTES // nb))))
+        hists = [hist0] + [hist0.clone() for _ in range(RH - 1)]
+        for s in range(W_steps + K_steps):
+            lookup_score_select(hists[s % RH], hist_len0, state0)
+        torch.cuda.synchronize()
+        ctx.close(); ctx_plain.close()
+        return {"profile_run": "lookup", "config": workload_config(w, world), "steps": K_steps, "warmup": W_steps,
+                "history_copies": RH, "lookup_algorithmic_bytes_per_launch": int(rq.hist_len.astype(np.int64).sum()) * 4}
     sel_len_h = sel_len.cpu().numpy()
     sel_draft_h = sel_draft.cpu().numpy()
     A = W.make_agreement(w, sel_len_h)
@@ -369,6 +398,16 @@ def run_config(name, args, env, cpu_seconds):
     for s in range(W_steps):
         step(s)
     torch.cuda.synchronize()
+    if args.profile:
+        for s in range(K_steps):
+            step(W_steps + s, "cycle" if args.profile == "cycle" else "step")
+        torch.cuda.synchronize()
+        needed = int((sel_len.cpu().numpy().astype(np.int64) + 1).sum())
+        ctx.close(); ctx_plain.close()
+        return {"profile_run": True, "config": workload_config(w, world), "steps": K_steps, "warmup": W_steps,
+                "launches_per_step": 4 if args.unfused else 3, "needed_rows": needed,
+                "verify_algorithmic_bytes_per_launch": needed * w.V * w.elt,
+                "lookup_algorithmic_bytes_per_launch": int(rq.hist_len.astype(np.int64).sum()) * 4}
 
     def capture(what="step", warm=False):
         g = torch.cuda.CUDAGraph()
@@ -462,7 +501,8 @@ def run_config(name, args, env, cpu_seconds):
     roofline = {"bound": "hbm", "kernel": "verify_stream_kernel (+ verify_commit_kernel)" if logits_bytes_alloc > 160 * 2**20
                 else "verify_small_kernel (+ verify_commit_kernel)",
                 "achieved": v_iso, "peak": peak_gbs, "unit": "GB/s", "frac": v_iso / peak_gbs,
-                "traffic": NCU_VERIFY_TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind,
+                "traffic": NCU_VERIFY_TRAFFIC_BYTES.get(w.name, (None, None))[0] if not args.batch else None,
+                "traffic_source": NCU_VERIFY_TRAFFIC_BYTES.get(w.name, (None, "not captured"))[1], "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": verify_bytes,
                 "frac_of_8000_nominal": v_iso / 8000.0,
                 "achieved_back_to_back": v_b2b, "frac_back_to_back": v_b2b / peak_gbs,
@@ -478,7 +518,8 @@ def run_config(name, args, env, cpu_seconds):
     l_b2b = gbs(lookup_bytes, kt["lookup_us"])
     roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel (hvd_lookup alone, K calls back to back in one graph)",
                        "achieved": l_b2b, "peak": peak_gbs, "unit": "GB/s", "frac": l_b2b / peak_gbs,
-                       "traffic": NCU_LOOKUP_TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind,
+                       "traffic": NCU_LOOKUP_TRAFFIC_BYTES.get(w.name, (None, None))[0] if not args.batch else None,
+                       "traffic_source": NCU_LOOKUP_TRAFFIC_BYTES.get(w.name, (None, "not captured"))[1], "peak_kind": peak_kind,
                        "algorithmic_bytes_per_launch": lookup_bytes,
                        "cold": bool(hist_cold), "history_copies": RH,
                        "achieved_plain_launches": gbs(lookup_bytes, kt["lookup_us_plain_launches"]),
@@ -639,7 +680,7 @@ def main():
            "peak_kind": peak_kind, "barrier": barrier, "max_over_ranks": lambda x: max_over_ranks(x, dev),
            "max_over_ranks_vec": max_vec}
     line = run_config(args.config, args, env, cpu_seconds=10.0)
-    if world == 1 and not args.only:
+    if world == 1 and not args.only and not args.profile:
         # every workload in the same line; the oracle leg is capped at a few seconds per workload
         keep = ("us_per_step", "us_per_step_best", "value", "steps_per_s_best", "tokens_per_s", "tokens_per_step",
                 "mean_accepted", "cache_selected_frac", "warm", "kernel_us", "roofline", "roofline_lookup",
