@@ -48,8 +48,15 @@
  *    row up to 160 MB, a persistent kernel with work queues beyond that.
  *    HVD_VERIFY_SMALL_BYTES (read once by hvd_create) moves the limit, 0 =
  *    always the persistent kernel: it exists for the tests, which run both
- *    kernels over the same cases.  Results do not depend on it.  Nothing
- *    else is read from the environment by the product path.
+ *    kernels over the same cases.  Results do not depend on it.
+ *  - hvd_lookup and its variants scan a history that does not fit one CTA
+ *    in chunks of 8 K or 16 K tokens, one CTA each.  When every request's
+ *    chunk CTAs can be resident at once they form one thread-block cluster
+ *    per request and meet in distributed shared memory, else they meet
+ *    through the context's scratch.  HVD_LOOKUP_CLUSTER=0 (read once by
+ *    hvd_create) turns the cluster form off: it exists for the tests, which
+ *    run both.  Results do not depend on it.  Nothing else is read from the
+ *    environment by the product path.
  */
 #ifndef HVD_H
 #define HVD_H

@@ -96,6 +96,8 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->vf_blocks_per_sm[0] = verify_occupancy(HVD_F32, smem);
     c->vf_blocks_per_sm[1] = verify_occupancy(HVD_BF16, smem);
     if (c->vf_blocks_per_sm[0] < 1 || c->vf_blocks_per_sm[1] < 1) { release(c); return HVD_ERR_UNSUPPORTED; }
+    c->lk_cluster_mode = getenv("HVD_LOOKUP_CLUSTER") ? atoi(getenv("HVD_LOOKUP_CLUSTER")) : 1;
+    lookup_cluster_setup(c);
     c->has_predictor = false;
     c->has_predictor_ext = false;
     c->two_layer = false;

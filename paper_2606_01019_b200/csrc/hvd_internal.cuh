@@ -72,6 +72,8 @@ struct hvd_ctx {
     hvd::LookupPartial* lk_partial;  // [max_batch, lk_max_chunks]
     uint32_t* lk_cnt;                // [max_batch], zero at rest
     int lk_max_chunks;
+    int lk_clusters[2][4];           // clusters of 2, 4, 8, 16 CTAs of the cluster lookup kernel (256, 512 threads) resident together
+    int lk_cluster_mode;             // 0: never take the cluster form (HVD_LOOKUP_CLUSTER=0; tests run both forms)
     // occurrence lists of the frequency-weighted draft
     int32_t* fq_occ;    // [max_batch, HVD_FREQ_MAX_OCC]
     uint32_t* fq_cnt;   // [max_batch], zero at rest
@@ -179,6 +181,8 @@ hvd_status launch_lookup(hvd_ctx* ctx, int32_t B, const int32_t* hist, const int
                          int32_t* match_pos, int32_t* match_cnt, const ScoreArgs* fused, cudaStream_t stream,
                          bool successor_works_ahead = false);
 
+
+void lookup_cluster_setup(hvd_ctx* ctx);
 
 ScoreArgs make_score_args(hvd_ctx* ctx, int32_t B, const int32_t* hist_len, const int32_t* prompt_len,
                           const hvd_req_state* state, const int32_t* K, const int32_t* draft,

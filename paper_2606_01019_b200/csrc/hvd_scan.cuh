@@ -74,16 +74,18 @@ __device__ __forceinline__ int4 ld_hist(const int4* p) {
 // same arguments, for every candidate p in [0, n - 2] of the warp's 32 vectors: p holds q0 and L >= 1 is the
 // match length of the copy that ends there (capped at l_max and at the slab start).
 // COHERENT: the tokens compared during the extension are read through the L2 (for a kernel that has itself
-// appended to the history it scans).
+// appended to the history it scans).  p_last: candidates beyond this position are left to another call
+// (default: none are).
 template <bool COHERENT = false, class OnMatch>
 __device__ __forceinline__ void scan_vector(const int4 x, int p0, int n, const int32_t* __restrict__ slab, int32_t q0,
                                             int32_t qa, int32_t qb, int l_max, int lane, OnMatch&& on_match,
-                                            int* status_word = nullptr) {
+                                            int* status_word = nullptr, int p_last = 0x7fffffff) {
+    const int last = min(n - 2, p_last);
     uint32_t m = 0;
-    m |= (x.x == q0 && p0 + 0 >= 0 && p0 + 0 <= n - 2) ? 1u : 0u;
-    m |= (x.y == q0 && p0 + 1 >= 0 && p0 + 1 <= n - 2) ? 2u : 0u;
-    m |= (x.z == q0 && p0 + 2 >= 0 && p0 + 2 <= n - 2) ? 4u : 0u;
-    m |= (x.w == q0 && p0 + 3 >= 0 && p0 + 3 <= n - 2) ? 8u : 0u;
+    m |= (x.x == q0 && p0 + 0 >= 0 && p0 + 0 <= last) ? 1u : 0u;
+    m |= (x.y == q0 && p0 + 1 >= 0 && p0 + 1 <= last) ? 2u : 0u;
+    m |= (x.z == q0 && p0 + 2 >= 0 && p0 + 2 <= last) ? 4u : 0u;
+    m |= (x.w == q0 && p0 + 3 >= 0 && p0 + 3 <= last) ? 8u : 0u;
     uint32_t hits = __ballot_sync(0xffffffffu, m != 0);
     while (hits) {
         const int src = __ffs(hits) - 1;

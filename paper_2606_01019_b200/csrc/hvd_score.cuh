@@ -48,10 +48,11 @@ __device__ __forceinline__ int bit_width(uint32_t x) { return 32 - __clz((int)x)
 // integer->float conversion or one correctly rounded IEEE operation).
 template <int N>
 __device__ __forceinline__ void payoff_features(const ScoreArgs& a, int b, int n, int d, int L, int pos, int cnt,
-                                                float (&phi)[N], const hvd_req_state* state_now = nullptr) {
+                                                float (&phi)[N], const hvd_req_state* state_now = nullptr,
+                                                const int* prompt_now = nullptr) {
     n = max(n, 0);
     // read-only inputs go through the non-coherent path so that the compiler may issue them early
-    const int P = max(__ldg(a.prompt_len + b), 0);
+    const int P = max(prompt_now ? *prompt_now : __ldg(a.prompt_len + b), 0);
     hvd_req_state st;
     if (state_now) {  // the caller has just updated the summary itself
         st = *state_now;
@@ -180,11 +181,12 @@ template <bool EXT = false>
 __device__ __forceinline__ void score_select_request(const ScoreArgs& a, int b, int lane, float* s_hid, int n,
                                                      int d, int L, int pos, int cnt, int tok0, int tok1,
                                                      const ModelDraft* fetched = nullptr,
-                                                     const hvd_req_state* state_now = nullptr) {
+                                                     const hvd_req_state* state_now = nullptr,
+                                                     const int* prompt_now = nullptr) {
     constexpr int N = NFeat<EXT>::value;
     d = max(0, min(d, a.k_cap));
     float phi[N];
-    payoff_features(a, b, n, d, L, pos, cnt, phi, state_now);
+    payoff_features(a, b, n, d, L, pos, cnt, phi, state_now, prompt_now);
     if constexpr (EXT) structure_features(a, b, lane, d, tok0, tok1, phi);
     if (a.features && lane < N) {
         float v = phi[0];

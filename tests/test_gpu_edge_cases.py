@@ -338,13 +338,21 @@ def test_parity_with_the_persistent_streaming_kernel_only():
     """Logits of up to 160 MB are streamed by the warp-per-batch kernels, so most cases of this suite never
     reach the persistent kernel: the shape, alignment, tie and multi-step cases once more with the limit at 0."""
     _rerun({"HVD_VERIFY_SMALL_BYTES": "0"}, ["tests/test_gpu_parity.py", "tests/test_gpu_edge_cases.py"],
-           "not full_size and not plain_launches and not kernel_only and not 65535")
+           "not full_size and not plain_launches and not kernel_only and not 65535 and not chunk_lookup_only and not bounds_checked")
 
 
 def test_parity_with_the_warp_per_batch_kernel_on_a_large_call():
     """... and the other way round: the full-size C2 and C5 workloads (279 MB and 2.5 GB of logits, uniform and
     ragged rows) through the warp-per-batch kernel that checks the need first."""
     _rerun({"HVD_VERIFY_SMALL_BYTES": str(1 << 40)}, ["tests/test_gpu_parity.py"], "full_size and (C2 or C5)")
+
+
+def test_parity_with_the_chunk_lookup_only():
+    """Batches of long histories that fit the GPU in one wave take the cluster form of the lookup (a request's chunk
+    CTAs as one thread-block cluster); the same cases once more with the plain chunk kernel and its global
+    combine, which larger batches use."""
+    _rerun({"HVD_LOOKUP_CLUSTER": "0"}, ["tests/test_gpu_parity.py", "tests/test_gpu_random_sweep.py"],
+           "(full_size and C4) or random_batches")
 
 
 def test_edge_cases_against_the_bounds_checked_build():
@@ -354,7 +362,7 @@ def test_edge_cases_against_the_bounds_checked_build():
     must close with status 0, and the results must still equal the oracle's."""
     from paper_2606_01019_b200 import build
     lib = build.build_bounds_checked()
-    sel = "not plain_launches and not kernel_only and not large_call and not bounds_checked and not full_size"
+    sel = "not plain_launches and not kernel_only and not large_call and not bounds_checked and not full_size and not chunk_lookup_only"
     files = ["tests/test_gpu_edge_cases.py", "tests/test_gpu_parity.py", "tests/test_gpu_cycle.py", "tests/test_gpu_tree.py"]
     _rerun({"HVD_B200_LIB": lib, "HVD_ASSERT_DEVICE_STATUS": "1"}, files, sel)
     _rerun({"HVD_B200_LIB": lib, "HVD_ASSERT_DEVICE_STATUS": "1", "HVD_VERIFY_SMALL_BYTES": "0"},
