@@ -50,10 +50,10 @@ NCU_VERIFY_TRAFFIC_BYTES = {
     "C4": (431484000, "profiles/verify_stream_kernel_c4_ncu.txt"),
 }
 NCU_LOOKUP_TRAFFIC_BYTES = {
-    "C2": (4239744, "profiles/lookup_kernel_c2_ncu.txt"),
-    "C3": (33662000, "profiles/lookup_kernel_c3_ncu.txt"),
-    "C4": (16845000, "profiles/lookup_kernel_c4_ncu.txt"),
-    "C5": (29784000, "profiles/lookup_kernel_c5_ncu.txt"),
+    "C2": (4242000, "profiles/lookup_kernel_c2_ncu.txt"),
+    "C3": (33658000, "profiles/lookup_kernel_c3_ncu.txt"),
+    "C4": (16825600, "profiles/lookup_kernel_c4_ncu.txt"),
+    "C5": (29787000, "profiles/lookup_kernel_c5_ncu.txt"),
 }
 
 
@@ -516,7 +516,7 @@ def run_config(name, args, env, cpu_seconds):
                           "predecessor has completed; `achieved_back_to_back` = with programmatic dependent launch, the "
                           "next call's start-up hidden under this call's tail (as inside a step)"}
     l_b2b = gbs(lookup_bytes, kt["lookup_us"])
-    roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel (hvd_lookup alone, K calls back to back in one graph)",
+    roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel / lookup_cluster_kernel (hvd_lookup alone, K calls back to back in one graph)",
                        "achieved": l_b2b, "peak": peak_gbs, "unit": "GB/s", "frac": l_b2b / peak_gbs,
                        "traffic": NCU_LOOKUP_TRAFFIC_BYTES.get(w.name, (None, None))[0] if not args.batch else None,
                        "traffic_source": NCU_LOOKUP_TRAFFIC_BYTES.get(w.name, (None, "not captured"))[1], "peak_kind": peak_kind,
