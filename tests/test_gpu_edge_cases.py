@@ -282,6 +282,36 @@ def test_host_side_argument_errors():
     ctx.close()
 
 
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("B,n_top", [(60, 50000), (20, 100000), (33, 100000), (10, 200000), (40, 100000)])
+def test_long_histories_in_small_batches(B, n_top, fused):
+    """The lookup shapes for histories beyond 32 K tokens: a request's chunks as one thread-block cluster of 8 or 16
+    CTAs of 256 threads (60 x 50 000, 20 x 100 000), of 8 or 16 CTAs of 512 threads (33 x 100 000, 10 x 200 000), or
+    as plain CTAs that meet through global memory when the clusters do not all fit at once (40 x 100 000).  Ragged
+    on purpose: one request of full length, the others anywhere below it (empty chunks inside a cluster), lengths
+    at the chunk edges, slabs off the 16-byte grid, unusable lengths, and a small vocabulary so that every warp
+    has candidates to extend."""
+    w = small(V=211)
+    rng = np.random.default_rng(1000 * B + n_top // 1000)
+    lens = [n_top, 0, 1, 2, 8192, 8193, 8195, 16384, 16385, 32768, 32769, 32772, n_top - 1, n_top - 3]
+    lens = [min(x, n_top) for x in lens][:B]
+    lens += [int(x) for x in rng.integers(3, n_top + 1, B - len(lens))]
+    hists = []
+    for i, n in enumerate(lens):
+        h = rng.integers(0, 3 if i % 3 else w.V, n)
+        if n > 200 and i % 2 == 0:               # a long match planted somewhere inside, in whatever chunk
+            t = int(rng.integers(2, 100))
+            e0 = int(rng.integers(t, n - t))
+            h[e0 - t:e0] = h[n - t:]
+        hists.append(h)
+    hist_len = list(lens)
+    hist_len[5], hist_len[6] = -7, 2**31 - 1     # unusable lengths: skipped with neutral outputs
+    mis = [i % 4 for i in range(B)]
+    rq = hand_requests(w, hists, [int(k) for k in rng.integers(0, 9, B)], hist_len=hist_len, misalign=mis)
+    (g, out, _), _ = run(w, rq, fused=fused)
+    assert (out.lk.match_len >= 2).sum() >= (B - 5) // 2   # five requests are empty, too short or unusable
+
+
 def test_history_of_more_than_65535_chunks():
     """A history so long that its chunks outgrow the y range of a grid (the launch then puts the chunks
     on x): 537 M tokens in one request, the longest match planted far inside."""
