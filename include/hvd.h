@@ -38,7 +38,13 @@
  *  - Consecutive kernels of a context are joined by programmatic dependent
  *    launch: a kernel may be resident while its predecessor on the stream
  *    still runs, and waits on the device before it reads anything the
- *    predecessor writes.  Results do not depend on it.  One environment
+ *    predecessor writes.  What no call of this library writes (hist_off,
+ *    hist_cap, K, the predictor) may be read before that wait, and the
+ *    lookup asks the L2 for the history slabs there.  A caller's own kernel
+ *    that writes those arrays is complete before a kernel of the library
+ *    starts, unless it signals programmatic launch completion itself: then it
+ *    must have written them before it does.
+ *    Results do not depend on it.  One environment
  *    variable, read once by hvd_create, changes it: HVD_PDL_MASK (a bit per
  *    kernel pair: 1 commit, 2 lookup, 4 verify stream, 8 scoring; default 15,
  *    0 = plain launches).  It exists for the tests, which run the parity

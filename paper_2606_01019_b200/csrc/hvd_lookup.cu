@@ -30,23 +30,44 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
     // have written them, is known to be complete: then the wait comes first.
     const bool late = !FUSED && a.successor_works_ahead;  // the fused form is never followed by such a kernel
     if (!late) pdl_trigger();
-    pdl_wait();
-    if (late) pdl_trigger();
-
-    // the request's scalars are fetched together, before any of them is looked at: the kernel is a chain
-    // of dependent round trips and this keeps them to one
-    const int n_raw = a.hist_len[b];
-    const int cap_b = a.hist_cap[b];
-    const int64_t off_b = a.hist_off[b];
-    const int K_b = a.K[b];
-    int n = n_raw;
-    if (n < 0 || n > cap_b || n > a.n_max) n = 0;  // unusable length: empty history
+    constexpr int CHUNK = THREADS * kLookupTokPerVec * ITER;  // tokens of the aligned grid per CTA
+    // The request's scalars are fetched together, before any of them is looked at: the kernel is a chain of
+    // dependent round trips and this keeps them to one.  The shapes for one request per SM (8 K to 32 K tokens)
+    // split that round trip: where the slab lies and how long it can get is never written by a kernel of this
+    // library, so it is read ahead of the wait for the previous kernel, and the L2 is asked for the slab; when the
+    // previous kernel is still running, the scan finds its tokens in the L2 (step of 64 x 16 K tokens 47.1 -> 46.5 us, of
+    // 128 x 32 K tokens 159.0 -> 157.5 us).  When it is not, the second round trip costs up to 0.7 us; the shapes for
+    // short histories and for more than one request per SM gained nothing in a step and do not do this.
+    constexpr bool AHEAD = THREADS == 1024 && ITER >= 4;
+    int n_raw, cap_b, K_b;
+    int64_t off_b;
+    if constexpr (AHEAD) {
+        cap_b = a.hist_cap[b];
+        off_b = a.hist_off[b];
+        K_b = a.K[b];
+        if (warp == 0) {
+            const int32_t* first = a.hist + off_b;
+            const int skip = (int)((4 - ((reinterpret_cast<uintptr_t>(first) >> 2) & 3)) & 3);
+            prefetch_history_l2(first + skip + chunk * CHUNK, min(CHUNK, min(cap_b, a.n_max) - skip - chunk * CHUNK), lane);
+        }
+        pdl_wait();
+        if (late) pdl_trigger();
+        n_raw = a.hist_len[b];
+    } else {
+        pdl_wait();
+        if (late) pdl_trigger();
+        n_raw = a.hist_len[b];
+        cap_b = a.hist_cap[b];
+        off_b = a.hist_off[b];
+        K_b = a.K[b];
+    }
     const int32_t* __restrict__ slab = a.hist + off_b;
     // 128-bit loads run on the 16-byte grid, which starts at the first 16-byte boundary inside the slab: the
     // `head` (0 to 3) tokens in front of it are looked at one by one, by the first warp of the first chunk, so
     // that a history of 2^k tokens takes 2^k / CHUNK chunks whatever its alignment
     const int head = (int)((4 - ((reinterpret_cast<uintptr_t>(slab) >> 2) & 3)) & 3);
-    constexpr int CHUNK = THREADS * kLookupTokPerVec * ITER;  // tokens of the aligned grid per CTA
+    int n = n_raw;
+    if (n < 0 || n > cap_b || n > a.n_max) n = 0;  // unusable length: empty history
     // candidate positions p (index of the matched copy's last token) are 0 .. n-2; grid position g is p - head
     const int g_end = (n >= 2) ? max(n - 1 - head, 0) : 0;  // exclusive end on the aligned grid
     const int n_chunks = (n >= 2) ? max((g_end + CHUNK - 1) / CHUNK, 1) : 0;
@@ -211,17 +232,23 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 4 : 2) lookup_cluste
     cluster_arrive();  // "this CTA runs": matched by the wait in front of the store into the first CTA
     const bool late = !FUSED && a.successor_works_ahead;
     if (!late) pdl_trigger();
-    pdl_wait();
-    if (late) pdl_trigger();
-
-    const int n_raw = a.hist_len[b];
+    // where the slab lies and how long it can get is never written by a kernel of this library: read ahead of the
+    // wait for the previous kernel, and the L2 is asked for this CTA's part of the slab, so that the scan finds its
+    // tokens there when the previous kernel is still running (C4 step 72.8 -> 71.6 us; a call that does not
+    // overlap its predecessor pays 0.25 us for the second round trip)
     const int cap_b = a.hist_cap[b];
     const int64_t off_b = a.hist_off[b];
     const int K_b = a.K[b];
-    int n = n_raw;
-    if (n < 0 || n > cap_b || n > a.n_max) n = 0;  // unusable length: empty history
     const int32_t* __restrict__ slab = a.hist + off_b;
     const int head = (int)((4 - ((reinterpret_cast<uintptr_t>(slab) >> 2) & 3)) & 3);
+    constexpr int CHUNK_AHEAD = THREADS * kLookupTokPerVec * kClusterIter;
+    if (warp == 0)
+        prefetch_history_l2(slab + head + chunk * CHUNK_AHEAD, min(CHUNK_AHEAD, min(cap_b, a.n_max) - head - chunk * CHUNK_AHEAD), lane);
+    pdl_wait();
+    if (late) pdl_trigger();
+    const int n_raw = a.hist_len[b];
+    int n = n_raw;
+    if (n < 0 || n > cap_b || n > a.n_max) n = 0;  // unusable length: empty history
     const int g_end = (n >= 2) ? max(n - 1 - head, 0) : 0;
     const int n_chunks = (n >= 2) ? max((g_end + CHUNK - 1) / CHUNK, 1) : 0;
     const bool has_work = chunk < n_chunks;  // a CTA without work still goes through both barriers

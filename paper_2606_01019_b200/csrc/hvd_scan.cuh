@@ -69,6 +69,21 @@ __device__ __forceinline__ int4 ld_hist(const int4* p) {
     return v;
 }
 
+// Asks the L2 for `tokens` history tokens from p (16-byte aligned) on: 32 bulk prefetches, one per lane of the
+// calling warp.  Nothing is waited for and nothing arrives in the SM: a later load finds the line in the L2 or
+// on its way there.  Used ahead of the wait for the previous kernel: the L2 is the point of coherence, so a
+// line fetched early still shows what that kernel writes afterwards.
+__device__ __forceinline__ void prefetch_history_l2(const int32_t* p, int tokens, int lane) {
+    const int bytes = (tokens >> 2) << 4;
+    if (bytes <= 0) return;
+    const int seg = (((bytes + 31) >> 5) + 127) & ~127;
+    const int at = lane * seg;
+    if (at < bytes) {
+        const uint32_t size = (uint32_t)min(seg, bytes - at);
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char*>(p) + at), "r"(size) : "memory");
+    }
+}
+
 // x: this lane's four tokens at positions p0 .. p0 + 3 of a history of n tokens (slab); q0 its last token,
 // qa / qb the tokens 1 + lane and 33 + lane back.  Calls on_match(L, p), in every lane of the warp with the
 // same arguments, for every candidate p in [0, n - 2] of the warp's 32 vectors: p holds q0 and L >= 1 is the
