@@ -15,6 +15,14 @@
 namespace hvd {
 namespace {
 
+// How many tokens of a slab to ask the L2 for ahead of the wait for the previous kernel.  The length is read
+// while that kernel may still be about to raise it (a commit appends at most k_cap + 1 tokens), so it is only a hint:
+// it sizes a prefetch and nothing else, and whatever it holds, the range stays inside the slab.
+__device__ __forceinline__ int length_ahead(const LookupArgs& a, int b, int cap_b) {
+    const int hint = *reinterpret_cast<const volatile int32_t*>(a.hist_len + b);
+    return (int)min((int64_t)min(cap_b, a.n_max), (int64_t)max(hint, 0) + a.k_cap + 1);
+}
+
 template <int THREADS, int ITER, bool FUSED>
 __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 512 ? 2 : 4))) lookup_kernel(const LookupArgs a, const ScoreArgs sa) {
     __shared__ float s_hid[FUSED ? HVD_MAX_HIDDEN : 1];
@@ -48,7 +56,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS == 1024 ? 1 : (THREADS == 51
         if (warp == 0) {
             const int32_t* first = a.hist + off_b;
             const int skip = (int)((4 - ((reinterpret_cast<uintptr_t>(first) >> 2) & 3)) & 3);
-            prefetch_history_l2(first + skip + chunk * CHUNK, min(CHUNK, min(cap_b, a.n_max) - skip - chunk * CHUNK), lane);
+            prefetch_history_l2(first + skip + chunk * CHUNK, min(CHUNK, length_ahead(a, b, cap_b) - skip - chunk * CHUNK), lane);
         }
         pdl_wait();
         if (late) pdl_trigger();
@@ -243,7 +251,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 4 : 2) lookup_cluste
     const int head = (int)((4 - ((reinterpret_cast<uintptr_t>(slab) >> 2) & 3)) & 3);
     constexpr int CHUNK_AHEAD = THREADS * kLookupTokPerVec * kClusterIter;
     if (warp == 0)
-        prefetch_history_l2(slab + head + chunk * CHUNK_AHEAD, min(CHUNK_AHEAD, min(cap_b, a.n_max) - head - chunk * CHUNK_AHEAD), lane);
+        prefetch_history_l2(slab + head + chunk * CHUNK_AHEAD, min(CHUNK_AHEAD, length_ahead(a, b, cap_b) - head - chunk * CHUNK_AHEAD), lane);
     pdl_wait();
     if (late) pdl_trigger();
     const int n_raw = a.hist_len[b];
