@@ -50,10 +50,10 @@ NCU_VERIFY_TRAFFIC_BYTES = {
     "C4": (431484000, "profiles/verify_stream_kernel_c4_ncu.txt"),
 }
 NCU_LOOKUP_TRAFFIC_BYTES = {
-    "C2": (4242000, "profiles/lookup_kernel_c2_ncu.txt"),
-    "C3": (33658000, "profiles/lookup_kernel_c3_ncu.txt"),
-    "C4": (16825600, "profiles/lookup_kernel_c4_ncu.txt"),
-    "C5": (29787000, "profiles/lookup_kernel_c5_ncu.txt"),
+    "C2": (4242688, "profiles/lookup_kernel_c2_ncu.txt"),
+    "C3": (33657856, "profiles/lookup_kernel_c3_ncu.txt"),
+    "C4": (16831104, "profiles/lookup_kernel_c4_ncu.txt"),
+    "C5": (29786880, "profiles/lookup_kernel_c5_ncu.txt"),
 }
 
 
