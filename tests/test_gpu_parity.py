@@ -144,12 +144,15 @@ def test_host_buffer_entry_point():
 
 
 @pytest.mark.parametrize("fused", [True, False])
-def test_chained_steps_without_host_synchronisation(fused):
+@pytest.mark.parametrize("B,n", [(24, 3000), (24, 12000), (10, 30000), (6, 50000), (20, 70000)])
+def test_chained_steps_without_host_synchronisation(fused, B, n):
     """Six steps enqueued back to back on one stream (no host synchronisation in between, so the kernels of
     consecutive steps overlap as far as programmatic dependent launch lets them): the final histories,
-    lengths, states and the last step's outputs must equal the oracle's chain."""
+    lengths, states and the last step's outputs must equal the oracle's chain.  The longer histories take the
+    lookup shapes that read the slab layout and ask the L2 for the slab while the previous step's commit may
+    still be appending to it (one CTA of 1024 threads per request; clusters of 8 and 16 chunk CTAs)."""
     import torch
-    w = W.CONFIGS["C2"].scaled(B=24, n=3000, V=5003)
+    w = W.CONFIGS["C2"].scaled(B=B, n=n, V=5003)
     inp = P.prepare(w, device="cuda")
     S = 6
     # the oracle's chain first: it fixes the logits of every step (each agrees with that step's selected draft)
