@@ -393,7 +393,8 @@ def test_edge_cases_against_the_bounds_checked_build():
     from paper_2606_01019_b200 import build
     lib = build.build_bounds_checked()
     sel = "not plain_launches and not kernel_only and not large_call and not bounds_checked and not full_size and not chunk_lookup_only"
-    files = ["tests/test_gpu_edge_cases.py", "tests/test_gpu_parity.py", "tests/test_gpu_cycle.py", "tests/test_gpu_tree.py"]
+    files = ["tests/test_gpu_edge_cases.py", "tests/test_gpu_parity.py", "tests/test_gpu_cycle.py", "tests/test_gpu_tree.py",
+             "tests/test_gpu_random_sweep.py"]
     _rerun({"HVD_B200_LIB": lib, "HVD_ASSERT_DEVICE_STATUS": "1"}, files, sel)
     _rerun({"HVD_B200_LIB": lib, "HVD_ASSERT_DEVICE_STATUS": "1", "HVD_VERIFY_SMALL_BYTES": "0"},
            ["tests/test_gpu_edge_cases.py"], sel)
