@@ -353,6 +353,30 @@ HVD_API hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits
                              int32_t* status, void* stream);
 
 /*
+ * hvd_verify_commit without target_tok, reading the logits only as far as the result depends on them
+ * (Sec. 3.1: Verify returns the accepted length a and the tokens z; rows behind the first rejected draft
+ * token enter neither).  The needed rows of a request are streamed window by window, rows [0,2), [2,4),
+ * [4,8), [8,16), ... of its block (the last window ends at row k_cap), one streaming launch per window over
+ * all requests that are still alive: a request goes on to its next window only if every row so far carried
+ * its draft token and rows are left.  accepted, committed, n_commit, status, the histories and the state come
+ * out exactly as from hvd_verify_commit; a request reads at most twice the rows its result needs, plus two.
+ * It pays when accepted lengths are short against the drafts (the paper's runs: a few tokens on average,
+ * Sec. 5.4 execution breakdown) and the logits are large; with long accepted prefixes or small calls the
+ * windows' launches cost more than the rows they save, and hvd_verify_commit is the one to call.
+ * Chain drafts only (no token trees).
+ *
+ * rows_read  device uint64, 8-byte aligned, or NULL: the number of logits rows streamed is ADDED to it
+ * all else   as hvd_verify_commit
+ */
+HVD_API hvd_status hvd_verify_commit_prefix(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                                    const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                                    const int32_t* sel_draft, const int32_t* sel_len, const int32_t* select,
+                                    int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                                    int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                                    int32_t* committed, int32_t* n_commit, uint64_t* rows_read,
+                                    int32_t* status, void* stream);
+
+/*
  * hvd_verify_commit, then at once the NEXT cycle's hvd_lookup_score_select on the histories it has just
  * extended (Algorithm 1: the end of one iteration and the start of the next).  In a decoding loop the two
  * are adjacent, and one kernel does the commit and the lookup: a launch and two dependent global round

@@ -287,6 +287,75 @@ def verify_commit(logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, sele
     return out
 
 
+def prefix_windows(k_cap: int) -> list:
+    """Row windows of the prefix verification: needed rows [e[j], e[j+1]) of every request form window j.
+    Two rows, two rows, then doubling; the last window ends at row k_cap (a block has k_cap + 1 rows)."""
+    e, x = [0], 2
+    while x < k_cap:
+        e.append(x)
+        x *= 2
+    e.append(k_cap + 1)
+    return e
+
+
+@dataclass
+class PrefixOut:
+    accepted: np.ndarray
+    committed: np.ndarray
+    n_commit: np.ndarray
+    status: np.ndarray
+    rows_read: int          # logits rows looked at, whole windows counted
+    rows_needed: int        # rows the results depend on: sum of accepted + 1
+
+
+def verify_commit_prefix(logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, select, *, k_cap, hist,
+                         hist_off, hist_cap, hist_len, state) -> PrefixOut:
+    """Verify (Sec. 3.1) and commit (Sec. 3.4, Algorithm 1) of a chain draft, walking the rows of each request in
+    order and looking at no row behind the first rejected draft token: (a, z) depend on rows 0..a only.  Rows
+    are taken window by window (prefix_windows); a request goes on to its next window only if every row so far
+    carried its draft token and rows are left.  Plain Python over requests and rows; the argmax of a row is the
+    scalar first-maximum scan of the C oracle.  `hist`, `hist_len`, `state` are updated IN PLACE."""
+    B = len(hist_len)
+    edges = prefix_windows(k_cap)
+    out = PrefixOut(np.zeros(B, np.int32), np.full((B, k_cap + 1), -1, np.int32), np.zeros(B, np.int32),
+                    np.zeros(B, np.int32), 0, 0)
+    rows2d = logits.reshape(-1, V)
+    for b in range(B):
+        r0 = int(row_off[b]) if row_off is not None else b * (k_uniform + 1)
+        r1 = int(row_off[b + 1]) if row_off is not None else r0 + k_uniform + 1
+        n, cap = int(hist_len[b]), int(hist_cap[b])
+        if n < 0 or n > cap or r1 - r0 <= 0:
+            out.status[b] = REQ_BAD_LEN
+            continue
+        m = min(max(int(sel_len[b]), 0), k_cap, r1 - r0 - 1)
+        d = sel_draft[b]
+        a, t_a = None, None
+        for lo, hi in zip(edges[:-1], edges[1:]):
+            if lo > m:
+                break
+            top = min(hi, m + 1)
+            out.rows_read += top - lo                      # the whole window is looked at
+            for i in range(lo, top):
+                t = argmax_row(rows2d[r0 + i], dtype)
+                if a is None and (i == m or int(d[i]) != t):
+                    a, t_a = i, t                          # first rejected position (or the draft's end)
+            if a is not None:
+                break                                      # nothing behind this window is looked at
+        out.rows_needed += a + 1
+        z = [int(x) for x in d[:a]] + [t_a]
+        w = min(a + 1, cap - n)
+        out.committed[b, :a + 1] = z
+        o = int(hist_off[b])
+        hist[o + n:o + n + w] = z[:w]
+        hist_len[b] = n + w
+        out.n_commit[b] = w
+        out.accepted[b] = a
+        out.status[b] = REQ_CAPACITY if w < a + 1 else REQ_OK
+        state["sel_bits"][b] = np.uint32(((int(state["sel_bits"][b]) << 1) | (1 if select[b] else 0)) & 0xffffffff)
+        state["acc_ring"][b] = np.uint64(((int(state["acc_ring"][b]) << 8) | (a & 0xff)) & 0xffffffffffffffff)
+    return out
+
+
 def argmax_row(row: np.ndarray, dtype: int) -> int:
     row = np.ascontiguousarray(row)
     return int(lib().oracle_argmax_row(_p(row), C.c_int32(dtype), C.c_int64(row.size)))

@@ -65,6 +65,7 @@ _SIGNATURES = {
     "hvd_replay_labels": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "hvd_score_select": (_i32, [_vp, _i32] + [_vp] * 16 + [_vp]),
     "hvd_verify_commit": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
+    "hvd_verify_commit_prefix": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp]),
     "hvd_verify_commit_next": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 13 + [_vp, _vp]),
     "hvd_verify_commit_tree": (_i32, [_vp, _i32, _vp, _i32, _i64, _vp, _i32, _i64] + [_vp] * 14 + [_vp]),
     "hvd_verify_keys": (_i32, [_vp, _i32, _vp, _i32, _i64, _i64, _vp, _i32, _i64, _vp, _vp, _vp, _vp, _vp]),
@@ -293,6 +294,17 @@ class Context:
                                                 _ptr(committed), _ptr(n_commit), _ptr(target_tok),
                                                 _ptr(status), _stream()),
                     "hvd_verify_commit")
+
+    def hvd_verify_commit_prefix(self, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
+                                 select, hist, hist_off, hist_cap, hist_len, state, accepted, committed,
+                                 n_commit, rows_read, status):
+        self._check(self._lib.hvd_verify_commit_prefix(self._h, B, _ptr(logits), dtype, V, _ptr(row_off),
+                                                       k_uniform, total_rows, _ptr(sel_draft), _ptr(sel_len),
+                                                       _ptr(select), _ptr(hist), _ptr(hist_off), _ptr(hist_cap),
+                                                       _ptr(hist_len), _ptr(state), _ptr(accepted),
+                                                       _ptr(committed), _ptr(n_commit), _ptr(rows_read),
+                                                       _ptr(status), _stream()),
+                    "hvd_verify_commit_prefix")
 
     def hvd_verify_commit_next(self, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len,
                                select, hist, hist_off, hist_cap, hist_len, state, accepted, committed,

@@ -19,7 +19,7 @@ void release(hvd_ctx* c) {
     cudaFree(c->cp_key); cudaFree(c->cp_cnt); cudaFree(c->cp_arrived);
     cudaFree(c->cp_start); cudaFree(c->cp_pos);
     cudaFree(c->rp_key); cudaFree(c->rp_cnt);
-    cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key);
+    cudaFree(c->vf_next_unit); cudaFree(c->dev_error); cudaFree(c->vf_row_key); cudaFree(c->vf_alive);
     cudaFree(c->host_ws);
     delete c;
 }
@@ -88,6 +88,7 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     ok = ok && alloc_zero(&c->cp_arrived, (size_t)cfg->max_batch * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_row_key, (size_t)cfg->max_rows * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && alloc_zero(&c->vf_next_unit, (size_t)kVerifyQueues * 32 * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && alloc_zero(&c->vf_alive, (size_t)cfg->max_batch * sizeof(int32_t)) == cudaSuccess;
     ok = ok && alloc_zero(&c->dev_error, sizeof(int)) == cudaSuccess;
     if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) { (void)cudaGetLastError(); release(c); return HVD_ERR_ALLOC; }
@@ -370,7 +371,8 @@ static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits
                              int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
                              int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
                              int32_t* committed, int32_t* n_commit, int32_t* target_tok,
-                             int32_t* status, void* stream, const hvd_next_cycle* next = nullptr) {
+                             int32_t* status, void* stream, const hvd_next_cycle* next = nullptr, bool prefix = false,
+                             unsigned long long* rows_read = nullptr) {
     if (!ctx) return HVD_ERR_INVALID_ARG;
     if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: B outside [1, max_batch]");
     if (dtype != HVD_F32 && dtype != HVD_BF16) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: unknown dtype");
@@ -399,6 +401,10 @@ static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits
     
     a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error;
     a.row_key = ctx->vf_row_key; a.total_rows = total_rows; a.ext_keys = nullptr;
+    if (prefix) {
+        a.rows_read = rows_read;
+        return launch_verify_prefix(ctx, a, dtype, static_cast<cudaStream_t>(stream));
+    }
     if (!next) return launch_verify(ctx, a, dtype, static_cast<cudaStream_t>(stream));
 
     // with the next cycle's lookup and scoring behind the commit
@@ -439,6 +445,20 @@ hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dt
     return verify_commit_impl(ctx, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len, nullptr,
                               select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
                               target_tok, status, stream);
+}
+
+hvd_status hvd_verify_commit_prefix(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
+                                    const int64_t* row_off, int32_t k_uniform, int64_t total_rows,
+                                    const int32_t* sel_draft, const int32_t* sel_len, const int32_t* select,
+                                    int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                                    int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
+                                    int32_t* committed, int32_t* n_commit, uint64_t* rows_read,
+                                    int32_t* status, void* stream) {
+    if (!ctx) return HVD_ERR_INVALID_ARG;
+    if (rows_read && !aligned(rows_read, 8)) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit_prefix: rows_read must be 8-byte aligned");
+    return verify_commit_impl(ctx, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len, nullptr,
+                              select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
+                              nullptr, status, stream, nullptr, true, reinterpret_cast<unsigned long long*>(rows_read));
 }
 
 hvd_status hvd_verify_commit_next(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,

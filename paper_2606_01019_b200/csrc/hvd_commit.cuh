@@ -31,6 +31,16 @@ __device__ __forceinline__ Req load_req(const VerifyArgs& a, int b) {
     return q;
 }
 
+// The part of a request's needed rows that the current launch streams: all of them, or (prefix verification)
+// rows [win_lo, win_hi) of a request that is still alive.  Returns the number of rows, `first` = the first one.
+__device__ __forceinline__ int streamed_rows(const VerifyArgs& a, const Req& q, int b, int64_t& first) {
+    const int lo = min(a.win_lo, q.nr);
+    int hi = min(a.win_hi, q.nr);
+    if (a.alive && hi > lo && a.alive[b] == 0) hi = lo;
+    first = q.r0 + lo;
+    return hi - lo;
+}
+
 constexpr unsigned long long kKeySign = 0x8000000000000000ull;
 
 // The (value, ~index) key of a logits row.  Context scratch is put back to zero as it is read; keys

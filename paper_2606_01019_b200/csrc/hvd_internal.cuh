@@ -95,6 +95,7 @@ struct hvd_ctx {
     // verify scratch
     unsigned long long* vf_row_key;  // [max_rows], zero at rest
     uint32_t* vf_next_unit;          // zero at rest
+    int32_t* vf_alive;               // [max_batch] prefix verification: request still accepted through the last window
     int* dev_error;                  // device status word
     int vf_blocks_per_sm[2];         // per dtype
     long long vf_small_bytes;        // size limit of the warp-per-batch kernels (HVD_VERIFY_SMALL_BYTES; 0 = never)
@@ -251,9 +252,16 @@ struct VerifyArgs {
     uint32_t* next_unit;   // unit counter, zero at rest
     int* dev_error;        // device status word (no kernel sets it at present)
     int32_t n_batch_row;   // 4 KB batches per row
+    // prefix verification: only the needed rows [win_lo, win_hi) of a request are streamed, and only while the
+    // request is alive (alive == NULL: every request is); the defaults stream every needed row
+    int32_t win_lo = 0, win_hi = 0x7fffffff;
+    int32_t* alive = nullptr;
+    unsigned long long* rows_read = nullptr;  // optional: += logits rows streamed by the call
 };
 
 hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit = true);
+// the same result (without target tokens) from the rows up to the first rejected draft token only
+hvd_status launch_verify_prefix(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream);
 // commit and the next cycle's lookup + scoring in one kernel (after launch_verify without its commit)
 bool cycle_fits_one_cta(int32_t n_max);
 hvd_status launch_commit_lookup(hvd_ctx* ctx, const VerifyArgs& va, const int32_t* K, int32_t n_max, int32_t* draft,

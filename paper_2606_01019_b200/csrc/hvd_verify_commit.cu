@@ -293,6 +293,44 @@ __global__ void __launch_bounds__(kCommitWarps * 32) commit_keys_kernel(const Ve
     if (b < a.B) commit_request(a, b, threadIdx.x & 31);
 }
 
+// Prefix verification, between two streaming launches: one warp per request looks at the row keys of the window
+// that has just been streamed (they stay in place for the commit) and decides whether the request goes on: every
+// row of the window must carry its draft token, and rows must be left beyond the window.  A request that has
+// met its first rejected token, or has used up its draft, is dead for all later windows.
+__global__ void __launch_bounds__(kCommitWarps * 32) prefix_gate_kernel(const VerifyArgs a) {
+    const int b = blockIdx.x * kCommitWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    pdl_trigger();
+    bool go = false;
+    if (b < a.B) {
+        const Req q = load_req(a, b);
+        const int m = q.nr - 1;
+        const int lo = a.win_lo, hi = a.win_hi;
+        const int32_t* d = a.sel_draft + (int64_t)b * a.k_cap;
+        const int i0 = lo + lane, i1 = lo + lane + 32;  // a window has at most 64 rows
+        const int d0 = (i0 < hi && i0 < m) ? d[i0] : -1;
+        const int d1 = (i1 < hi && i1 < m) ? d[i1] : -1;
+        pdl_wait();  // the row keys come from the streaming kernel, the flags from the gate before it
+        const bool was = q.nr > 0 && hi <= m && (lo == 0 || a.alive[b] != 0);  // hi <= m: rows are left beyond the window
+        // the target's token of a row, exactly as the commit reads it (inside the vocabulary whatever the data)
+        auto token = [&](int i) {
+            if (!HVD_IN_BOUNDS(a.dev_error, q.r0 + i, 0, a.total_rows)) return -2;
+            const int t = (int)(~(uint32_t)(a.row_key[q.r0 + i] & 0xffffffffu));
+            return (int)min((int64_t)max(t, 0), a.V - 1);
+        };
+        bool ok = true;
+        if (was) {
+            if (i0 < hi) ok = ok && token(i0) == d0;
+            if (i1 < hi) ok = ok && token(i1) == d1;
+        }
+        go = was && __all_sync(0xffffffffu, ok);
+        if (lane == 0) a.alive[b] = go ? 1 : 0;
+    } else {
+        pdl_wait();
+    }
+    if (b == 0 && lane < Q) a.next_unit[lane * kQueueStride] = 0u;  // the next launch draws its units from zero
+}
+
 struct Smem {
     long long* row0;  // [B] first logits row of each request
     int* pref;        // [B+1] exclusive prefix of needed rows over requests
@@ -339,8 +377,9 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
         int nr = 0;
         if (b < a.B) {
             const Req q = load_req(a, b);
-            nr = q.nr;
-            sm.row0[b] = q.r0;
+            int64_t first;
+            nr = streamed_rows(a, q, b, first);
+            sm.row0[b] = first;
         }
         int v = nr;  // inclusive scan of nr over the tile
 #pragma unroll
@@ -362,6 +401,7 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
 
     const int nbr = a.n_batch_row;
     const int64_t total = (int64_t)sm.pref[a.B] * nbr;  // batches of all needed rows
+    if (a.rows_read && blockIdx.x == 0 && tid == 0) atomicAdd(a.rows_read, (unsigned long long)sm.pref[a.B]);
     // all but the last 1/2^HVD_VERIFY_ENDGAME_SHIFT (1/64) of the batches go out in units of UB, the rest one by one:
     // near the end a warp on a slow SM should not sit on more than it can finish quickly
     const uint32_t n_big = (uint32_t)((total - (total >> HVD_VERIFY_ENDGAME_SHIFT)) / UB);
@@ -615,6 +655,38 @@ hvd_status launch_commit_keys(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream) {
     return HVD_OK;
 }
 
+// Windows of prefix verification: needed rows [e[j], e[j+1]) are streamed by launch j.  Two rows, two rows, then
+// doubling: a request that is rejected early (the common case: the accepted length is geometric in the paper's
+// runs, a few tokens on average) costs two to four rows, and no request reads more than twice what it needs
+// plus two rows; a window of a single last row is merged into the one before it.
+static int prefix_edges(int k_cap, int* e) {
+    int n = 0;
+    e[n++] = 0;
+    for (int x = 2; x < k_cap; x *= 2) e[n++] = x;
+    e[n++] = k_cap + 1;
+    return n - 1;  // number of windows
+}
+
+hvd_status launch_verify_prefix(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream) {
+    int e[16];
+    const int n_win = prefix_edges(a.k_cap, e);
+    a.alive = ctx->vf_alive;
+    a.target_tok = nullptr;
+    const int cgrid = (a.B + kCommitWarps - 1) / kCommitWarps;
+    for (int j = 0; j < n_win; ++j) {
+        a.win_lo = e[j]; a.win_hi = e[j + 1];
+        const bool last = j + 1 == n_win;
+        VerifyArgs s = a;
+        if (j == 0) s.alive = nullptr;  // every request starts alive (the flags are written by the first gate)
+        const hvd_status r = launch_verify(ctx, s, dtype, stream, false);
+        if (r != HVD_OK) return r;
+        if (!last) HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_commit, prefix_gate_kernel, cgrid, kCommitWarps * 32, 0, stream, a));
+    }
+    a.win_lo = 0; a.win_hi = 0x7fffffff; a.alive = nullptr;
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_commit, verify_commit_kernel, cgrid, kCommitWarps * 32, 0, stream, a));
+    return HVD_OK;
+}
+
 hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit) {
     const int per_sm = ctx->vf_blocks_per_sm[dtype == HVD_F32 ? 0 : 1];
     int grid = ctx->num_sms * (per_sm > 0 ? per_sm : 1);
@@ -624,7 +696,9 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
     // a small call gets no more warps than it can have units, but at least one CTA for every second SM
     // (measured on 36 rows of 32 000 floats: 74 to 96 CTAs 6.5 us, the full 592 CTAs 7.5 us, 72 CTAs 7.3 us,
     // 37 CTAs 9.4 us)
-    const int64_t units_upper = (a.total_rows * (int64_t)a.n_batch_row + UB - 1) / UB;
+    const bool windowed = a.win_lo != 0 || a.win_hi != 0x7fffffff;
+    const int64_t rows_upper = windowed ? std::min<int64_t>(a.total_rows, (int64_t)a.B * (a.win_hi - a.win_lo)) : a.total_rows;
+    const int64_t units_upper = (rows_upper * (int64_t)a.n_batch_row + UB - 1) / UB;
     const int64_t want = std::max<int64_t>((units_upper + NW - 1) / NW, (ctx->num_sms + 1) / 2);
     if (want < grid) grid = (int)want;
     // unit numbers are 32-bit
@@ -638,7 +712,8 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
     // 17 MB 7.5 -> 5.5, 70 MB 11.2 -> 9.0, 140 MB 17.6 -> 14.5, 279 MB 27.8 -> 26.4; with (nearly) all rows
     // needed the persistent kernel is ahead from about 150 MB on (279 MB: 41.7 against 50.7 us).
     const int64_t full_bytes = a.total_rows * a.V * esz;
-    const bool small = a.total_rows <= 65535 && full_bytes <= ctx->vf_small_bytes;
+    // (a windowed launch takes the persistent kernel whatever its size: its work list leaves out dead requests)
+    const bool small = !windowed && a.total_rows <= 65535 && full_bytes <= ctx->vf_small_bytes;
     const bool spec = full_bytes <= kVerifySpecBytes;
     if (small) {
         const dim3 sgrid((unsigned)((a.n_batch_row + kSmallWarps - 1) / kSmallWarps), (unsigned)a.total_rows);

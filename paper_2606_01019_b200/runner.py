@@ -98,6 +98,15 @@ class DeviceBatch:
                                    self.target_tok if target_tok else None, self.status)
         self.n_max = min(self.cap_max, self.n_max + self.ctx.k_cap + 1)
 
+    def verify_commit_prefix(self, logits, rows_read=None):
+        """Verification and commit that read the logits only up to the first rejected draft token
+        (no target_tok); rows_read: optional uint64 device scalar that the rows streamed are added to."""
+        self.ctx.hvd_verify_commit_prefix(self.B, logits, self.dtype, self.V, self.row_off, self.k_uniform,
+                                          self.total_rows, self.sel_draft, self.sel_len, self.select, self.hist,
+                                          self.hist_off, self.hist_cap, self.hist_len, self.state,
+                                          self.accepted, self.committed, self.n_commit, rows_read, self.status)
+        self.n_max = min(self.cap_max, self.n_max + self.ctx.k_cap + 1)
+
     def verify_commit_next(self, logits, target_tok=True, K=None, model_draft=None, model_len=None):
         """Verification and commit of this cycle, then the next cycle's lookup, score and selection (on the
         histories just extended) in the same call.  K / model_draft / model_len: the next cycle's inputs

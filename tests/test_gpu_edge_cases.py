@@ -346,8 +346,8 @@ def test_parity_with_plain_launches():
     import sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     env = dict(os.environ, HVD_PDL_MASK="0")
-    cmd = [sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", "tests/test_gpu_parity.py",
-           "-k", "c1_full or fused_lookup or multi_step or chained or switching"]
+    cmd = [sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", "tests/test_gpu_parity.py", "tests/test_gpu_prefix.py",
+           "-k", "c1_full or fused_lookup or multi_step or chained or switching or scaled_workloads or every_accepted"]
     res = subprocess.run(cmd, cwd=root, env=env, capture_output=True, text=True, timeout=900)
     assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
     assert " passed" in res.stdout
@@ -394,7 +394,7 @@ def test_edge_cases_against_the_bounds_checked_build():
     lib = build.build_bounds_checked()
     sel = "not plain_launches and not kernel_only and not large_call and not bounds_checked and not full_size and not chunk_lookup_only"
     files = ["tests/test_gpu_edge_cases.py", "tests/test_gpu_parity.py", "tests/test_gpu_cycle.py", "tests/test_gpu_tree.py",
-             "tests/test_gpu_random_sweep.py"]
+             "tests/test_gpu_random_sweep.py", "tests/test_gpu_prefix.py"]
     _rerun({"HVD_B200_LIB": lib, "HVD_ASSERT_DEVICE_STATUS": "1"}, files, sel)
     _rerun({"HVD_B200_LIB": lib, "HVD_ASSERT_DEVICE_STATUS": "1", "HVD_VERIFY_SMALL_BYTES": "0"},
            ["tests/test_gpu_edge_cases.py"], sel)
