@@ -312,6 +312,13 @@ def run_config(name, args, env, cpu_seconds):
         c.hvd_verify_commit(B, logits, dtype, w.V, row_off, 0, total_rows, sel_draft, sel_len, select, hist,
                             hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, None, status)
 
+    rows_streamed = torch.zeros(1, dtype=torch.int64, device=dev)
+
+    def verify_prefix(logits, hist, hist_len, state):
+        ctx.hvd_verify_commit_prefix(B, logits, dtype, w.V, row_off, 0, total_rows, sel_draft, sel_len, select, hist,
+                                     hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, rows_streamed,
+                                     status)
+
     # the commit and the next cycle's lookup + selection in one call; the next selection goes to arrays of its
     # own, so that every timed step verifies the same (pristine) selection
     select_n, sel_draft_n, sel_len_n = i32(B), i32(B, kc), i32(B)
@@ -385,6 +392,11 @@ def run_config(name, args, env, cpu_seconds):
             verify(logits[rl], hists[rh], hl, st)
         elif what == "verify_plain":
             verify(logits[rl], hists[rh], hl, st, ctx_plain)
+        elif what == "verify_prefix":
+            verify_prefix(logits[rl], hists[rh], hl, st)
+        elif what == "step_prefix":
+            lookup_score_select(hists[rh], hl, st)
+            verify_prefix(logits[rl], hists[rh], hl, st)
         else:
             if args.unfused:
                 lookup(hists[rh], hl)
@@ -485,6 +497,18 @@ def run_config(name, args, env, cpu_seconds):
     kt["verify_commit_us_by_difference"] = 1e3 * med_ms / K_steps - kt["step_us_without_verify"]
     kt["read_probe_us"], _ = us_per_step("probe")
     kt["step_us_commit_fused_with_next_lookup"], _ = us_per_step("cycle")
+    # the same step with the verification that stops behind the first rejected draft token (same outputs: the
+    # timed steps ask for no target_tok).  Rows streamed: counted by the kernels over one eager call.
+    kt["step_us_prefix_verification"], kt["step_us_prefix_verification_best"] = us_per_step("step_prefix")
+    kt["verify_prefix_us_back_to_back"], _ = us_per_step("verify_prefix")
+    restore()
+    with torch.cuda.stream(stream):
+        rows_streamed.zero_()
+        step(W_steps, "verify_prefix")
+    torch.cuda.synchronize()
+    prefix_rows = int(rows_streamed.item())
+    prefix_same = bool((accepted.cpu().numpy() == accepted_h).all() and (n_commit.cpu().numpy() == n_commit_h).all())
+    restore()
 
     steps_per_s = world * K_steps / (med_ms * 1e-3)
     tokens_per_step = int(n_commit_h.sum())
@@ -515,6 +539,20 @@ def run_config(name, args, env, cpu_seconds):
                           "inputs larger than L2; `achieved` = isolated: plain launches, every kernel starts after its "
                           "predecessor has completed; `achieved_back_to_back` = with programmatic dependent launch, the "
                           "next call's start-up hidden under this call's tail (as inside a step)"}
+    rows_full = int((sel_len_after.astype(np.int64) + 1).sum())
+    rows_needed = int((accepted_h.astype(np.int64) + 1)[status_h != 2].sum())
+    prefix = {"entry_point": "hvd_lookup_score_select + hvd_verify_commit_prefix",
+              "us_per_step": kt["step_us_prefix_verification"], "us_per_step_best": kt["step_us_prefix_verification_best"],
+              "steps_per_s": world * 1e6 / kt["step_us_prefix_verification"],
+              "speedup_over_the_full_verification": step_us / kt["step_us_prefix_verification"],
+              "verify_us_back_to_back": kt["verify_prefix_us_back_to_back"],
+              "rows_streamed": prefix_rows, "rows_the_results_depend_on": rows_needed, "rows_of_the_full_verification": rows_full,
+              "bytes_streamed": prefix_rows * w.V * w.elt,
+              "achieved_on_streamed_bytes": gbs(prefix_rows * w.V * w.elt, kt["verify_prefix_us_back_to_back"]),
+              "frac_on_streamed_bytes": gbs(prefix_rows * w.V * w.elt, kt["verify_prefix_us_back_to_back"]) / peak_gbs,
+              "unit": "GB/s", "same_results_as_the_full_verification": prefix_same,
+              "what": "rows [0,2), [2,4), [4,8), ... of every request still accepted so far, one streaming launch per "
+                      "window; accepted, committed tokens, histories and state as from hvd_verify_commit"}
     l_b2b = gbs(lookup_bytes, kt["lookup_us"])
     roofline_lookup = {"bound": "hbm", "kernel": "lookup_kernel / lookup_cluster_kernel (hvd_lookup alone, K calls back to back in one graph)",
                        "achieved": l_b2b, "peak": peak_gbs, "unit": "GB/s", "frac": l_b2b / peak_gbs,
@@ -625,7 +663,7 @@ def run_config(name, args, env, cpu_seconds):
                     "steps_per_s": 1.0 / (kt["step_us_warm"] * 1e-6),
                     "what": "the same K steps on ONE copy of the histories and logits (every step re-reads the buffers the "
                             "previous step read: L2-resident as far as they fit 126 MiB); per rank"},
-           "kernel_us": kt, "roofline": roofline, "roofline_lookup": roofline_lookup, "roofline_step": roofline_step,
+           "kernel_us": kt, "prefix_verification": prefix, "roofline": roofline, "roofline_lookup": roofline_lookup, "roofline_step": roofline_step,
            "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches * K_steps * REPLAYS,
            "clocks": clocks,
            "us_per_step_x_sm_ghz": step_us * (clocks["sm_mhz"] or 0) / 1e3,
@@ -683,7 +721,7 @@ def main():
     if world == 1 and not args.only and not args.profile:
         # every workload in the same line; the oracle leg is capped at a few seconds per workload
         keep = ("us_per_step", "us_per_step_best", "value", "steps_per_s_best", "tokens_per_s", "tokens_per_step",
-                "mean_accepted", "cache_selected_frac", "warm", "kernel_us", "roofline", "roofline_lookup",
+                "mean_accepted", "cache_selected_frac", "warm", "kernel_us", "prefix_verification", "roofline", "roofline_lookup",
                 "roofline_step", "cpu_baseline", "e2e", "clocks", "us_per_step_x_sm_ghz", "dtype", "config")
         per = {}
         for name in ALL_CONFIGS:

@@ -61,8 +61,13 @@
  *    per request and meet in distributed shared memory, else they meet
  *    through the context's scratch.  HVD_LOOKUP_CLUSTER=0 (read once by
  *    hvd_create) turns the cluster form off: it exists for the tests, which
- *    run both.  Results do not depend on it.  Nothing else is read from the
- *    environment by the product path.
+ *    run both.  Results do not depend on it.
+ *  - hvd_verify_commit_prefix cuts the rows of a request into windows whose
+ *    sizes follow from the size of the call; HVD_PREFIX_BOUNDARY_BYTES (read
+ *    once by hvd_create; default 64 MiB, what one more streaming launch is
+ *    worth in streamed bytes) moves them: it exists for the tests, which set
+ *    it to 1 to get every window on small inputs.  Results do not depend on
+ *    it.  Nothing else is read from the environment by the product path.
  */
 #ifndef HVD_H
 #define HVD_H
@@ -355,17 +360,19 @@ HVD_API hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits
 /*
  * hvd_verify_commit without target_tok, reading the logits only as far as the result depends on them
  * (Sec. 3.1: Verify returns the accepted length a and the tokens z; rows behind the first rejected draft
- * token enter neither).  The needed rows of a request are streamed window by window, rows [0,2), [2,4),
- * [4,8), [8,16), ... of its block (the last window ends at row k_cap), one streaming launch per window over
- * all requests that are still alive: a request goes on to its next window only if every row so far carried
- * its draft token and rows are left.  accepted, committed, n_commit, status, the histories and the state come
- * out exactly as from hvd_verify_commit; a request reads at most twice the rows its result needs, plus two.
+ * token enter neither).  The needed rows of a request are streamed window by window, one streaming launch
+ * per window over all requests that are still alive: a request goes on to its next window only if every row
+ * so far carried its draft token and rows are left.  The first window holds at least 64 MiB of the batch
+ * (B * V * element size per row index) and at least two rows, the windows double from there, and no further
+ * boundary is set once the rows left, halved per window so far, weigh less than 128 MiB: on a large call
+ * rows [0,2), [2,4), [4,8), [8,16), [16, k_cap]; on a small one a single window, i.e. hvd_verify_commit.
+ * accepted, committed, n_commit, status, the histories and the state come out exactly as from
+ * hvd_verify_commit; a request reads at most twice the rows its result needs, plus the first window.
  * It pays when accepted lengths are short against the drafts (the paper's runs: a few tokens on average,
- * Sec. 5.4 execution breakdown) and the logits are large; with long accepted prefixes or small calls the
- * windows' launches cost more than the rows they save, and hvd_verify_commit is the one to call.
- * Chain drafts only (no token trees).
+ * Sec. 5.4 execution breakdown) and the logits are large; when most drafts are accepted to the end the
+ * extra launches are paid for nothing (8 to 10 us each).  Chain drafts only (no token trees).
  *
- * rows_read  device uint64, 8-byte aligned, or NULL: the number of logits rows streamed is ADDED to it
+ * rows_read  device uint64, 8-byte aligned, or NULL: the number of needed logits rows streamed is ADDED to it
  * all else   as hvd_verify_commit
  */
 HVD_API hvd_status hvd_verify_commit_prefix(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,

@@ -287,13 +287,23 @@ def verify_commit(logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, sele
     return out
 
 
-def prefix_windows(k_cap: int) -> list:
+PREFIX_BOUNDARY_BYTES = 64 << 20
+
+
+def prefix_windows(k_cap: int, bytes_per_row_index: int, boundary_bytes: int = PREFIX_BOUNDARY_BYTES) -> list:
     """Row windows of the prefix verification: needed rows [e[j], e[j+1]) of every request form window j.
-    Two rows, two rows, then doubling; the last window ends at row k_cap (a block has k_cap + 1 rows)."""
-    e, x = [0], 2
+    bytes_per_row_index = B * V * element size: what one row of every request weighs.  The first window holds at
+    least boundary_bytes (64 MiB) of the batch and at least two rows, windows double from there, and no boundary
+    is set once the rows left, halved once per window so far, weigh less than twice that; the last window ends
+    at row k_cap (a block has k_cap + 1 rows)."""
+    per_row = max(int(bytes_per_row_index), 1)
+    e, x, j = [0], max(2, -(-boundary_bytes // per_row)), 1
     while x < k_cap:
         e.append(x)
+        if ((k_cap + 1 - x) * per_row) // (1 << j) < 2 * boundary_bytes:
+            break
         x *= 2
+        j += 1
     e.append(k_cap + 1)
     return e
 
@@ -309,14 +319,14 @@ class PrefixOut:
 
 
 def verify_commit_prefix(logits, dtype, V, row_off, k_uniform, sel_draft, sel_len, select, *, k_cap, hist,
-                         hist_off, hist_cap, hist_len, state) -> PrefixOut:
+                         hist_off, hist_cap, hist_len, state, boundary_bytes=PREFIX_BOUNDARY_BYTES) -> PrefixOut:
     """Verify (Sec. 3.1) and commit (Sec. 3.4, Algorithm 1) of a chain draft, walking the rows of each request in
     order and looking at no row behind the first rejected draft token: (a, z) depend on rows 0..a only.  Rows
     are taken window by window (prefix_windows); a request goes on to its next window only if every row so far
     carried its draft token and rows are left.  Plain Python over requests and rows; the argmax of a row is the
     scalar first-maximum scan of the C oracle.  `hist`, `hist_len`, `state` are updated IN PLACE."""
     B = len(hist_len)
-    edges = prefix_windows(k_cap)
+    edges = prefix_windows(k_cap, B * V * (4 if dtype == F32 else 2), boundary_bytes)
     out = PrefixOut(np.zeros(B, np.int32), np.full((B, k_cap + 1), -1, np.int32), np.zeros(B, np.int32),
                     np.zeros(B, np.int32), 0, 0)
     rows2d = logits.reshape(-1, V)

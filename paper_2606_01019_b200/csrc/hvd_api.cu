@@ -109,6 +109,8 @@ hvd_status hvd_create(hvd_ctx** out, const hvd_config* cfg) {
     c->pdl_mask = getenv("HVD_PDL_MASK") ? atoi(getenv("HVD_PDL_MASK")) : 15;
     c->pdl_commit = (c->pdl_mask & 1) != 0;
     c->vf_small_bytes = getenv("HVD_VERIFY_SMALL_BYTES") ? atoll(getenv("HVD_VERIFY_SMALL_BYTES")) : kVerifySmallBytes;
+    c->vf_boundary_bytes = getenv("HVD_PREFIX_BOUNDARY_BYTES") ? atoll(getenv("HVD_PREFIX_BOUNDARY_BYTES")) : kPrefixBoundaryBytes;
+    if (c->vf_boundary_bytes < 1) c->vf_boundary_bytes = 1;
     c->host_ws = nullptr;
     c->host_ws_bytes = 0;
     *out = c;

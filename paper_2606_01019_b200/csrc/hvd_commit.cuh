@@ -86,6 +86,7 @@ __device__ __forceinline__ void commit_request(const VerifyArgs& a, int b, int l
         return;
     }
     const int m = q.nr - 1;
+    if (a.rows_in_commit && a.rows_read && lane == 0) atomicAdd(a.rows_read, (unsigned long long)q.nr);
     pdl_wait();  // everything above was the request's own data; the row keys come from the streaming kernel
     // rows lane, lane+32, lane+64 (at most 65 rows): target tokens from the row keys
     unsigned long long key[3];

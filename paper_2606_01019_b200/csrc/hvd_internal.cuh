@@ -45,6 +45,7 @@ constexpr int kVerifyUnitBatches = HVD_VERIFY_UNIT_BATCHES;  // 4 KB batches per
 constexpr int kVerifyQueues = HVD_VERIFY_QUEUES;  // unit counters
 constexpr int kVerifyQueueStride = 32;           // ... on separate 128-byte lines (in 32-bit words)
 constexpr long long kVerifySmallBytes = 160LL << 20;  // logits up to this size: one warp per 4 KB batch
+constexpr long long kPrefixBoundaryBytes = 64LL << 20;  // prefix verification: a window boundary costs what streaming this much costs
 constexpr long long kVerifySpecBytes = 8LL << 20;     // ... and up to this size: loads before the need is known
 
 
@@ -99,6 +100,7 @@ struct hvd_ctx {
     int* dev_error;                  // device status word
     int vf_blocks_per_sm[2];         // per dtype
     long long vf_small_bytes;        // size limit of the warp-per-batch kernels (HVD_VERIFY_SMALL_BYTES; 0 = never)
+    long long vf_boundary_bytes;     // prefix verification: streamed bytes that one window boundary is worth (HVD_PREFIX_BOUNDARY_BYTES)
     // device staging of the host-buffer entry point (grown on demand)
     int pdl_mask;     // ... for the three kernels of a step: bit 0 commit, 1 lookup, 2 stream, 3 one-layer scoring (default all)
     bool pdl_commit;  // bit 0 of the mask
@@ -257,6 +259,7 @@ struct VerifyArgs {
     int32_t win_lo = 0, win_hi = 0x7fffffff;
     int32_t* alive = nullptr;
     unsigned long long* rows_read = nullptr;  // optional: += logits rows streamed by the call
+    bool rows_in_commit = false;              // ... counted by the commit (one window: any streaming kernel) or by the streaming launches
 };
 
 hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit = true);

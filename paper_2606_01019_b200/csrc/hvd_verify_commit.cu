@@ -401,7 +401,7 @@ __global__ void __launch_bounds__(T, HVD_VERIFY_MIN_BLOCKS) verify_stream_kernel
 
     const int nbr = a.n_batch_row;
     const int64_t total = (int64_t)sm.pref[a.B] * nbr;  // batches of all needed rows
-    if (a.rows_read && blockIdx.x == 0 && tid == 0) atomicAdd(a.rows_read, (unsigned long long)sm.pref[a.B]);
+    if (a.rows_read && !a.rows_in_commit && blockIdx.x == 0 && tid == 0) atomicAdd(a.rows_read, (unsigned long long)sm.pref[a.B]);
     // all but the last 1/2^HVD_VERIFY_ENDGAME_SHIFT (1/64) of the batches go out in units of UB, the rest one by one:
     // near the end a warp on a slow SM should not sit on more than it can finish quickly
     const uint32_t n_big = (uint32_t)((total - (total >> HVD_VERIFY_ENDGAME_SHIFT)) / UB);
@@ -655,23 +655,35 @@ hvd_status launch_commit_keys(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream) {
     return HVD_OK;
 }
 
-// Windows of prefix verification: needed rows [e[j], e[j+1]) are streamed by launch j.  Two rows, two rows, then
-// doubling: a request that is rejected early (the common case: the accepted length is geometric in the paper's
-// runs, a few tokens on average) costs two to four rows, and no request reads more than twice what it needs
-// plus two rows; a window of a single last row is merged into the one before it.
-static int prefix_edges(int k_cap, int* e) {
+// Windows of prefix verification: needed rows [e[j], e[j+1]) are streamed by launch j.  A boundary between two
+// windows costs what about 64 MiB of streaming costs (the tail of one launch, the gate, the start of the next:
+// 8 to 10 us measured), so the first window takes at least that much of the batch (at least two rows), windows
+// double from there (no request reads more than twice what it needs plus the first window), and no further
+// boundary is set once what is left cannot repay it even if half of the requests die per window.  Small calls
+// end up with one window: the plain verification.
+static int prefix_edges(int k_cap, int64_t bytes_per_row_index, int64_t boundary, int* e) {
     int n = 0;
     e[n++] = 0;
-    for (int x = 2; x < k_cap; x *= 2) e[n++] = x;
+    const int64_t per_row = bytes_per_row_index > 0 ? bytes_per_row_index : 1;
+    const int64_t w0 = std::max<int64_t>(2, (boundary + per_row - 1) / per_row);
+    int j = 1;
+    for (int64_t x = w0; x < k_cap; x *= 2, ++j) {
+        e[n++] = (int)x;
+        if ((((int64_t)(k_cap + 1) - x) * per_row >> j) < 2 * boundary) break;
+    }
     e[n++] = k_cap + 1;
     return n - 1;  // number of windows
 }
 
 hvd_status launch_verify_prefix(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream) {
     int e[16];
-    const int n_win = prefix_edges(a.k_cap, e);
-    a.alive = ctx->vf_alive;
+    const int n_win = prefix_edges(a.k_cap, (int64_t)a.B * a.V * (dtype == HVD_F32 ? 4 : 2), ctx->vf_boundary_bytes, e);
     a.target_tok = nullptr;
+    if (n_win == 1) {  // the plain verification, whichever streaming kernel it takes; the commit counts the rows
+        a.rows_in_commit = true;
+        return launch_verify(ctx, a, dtype, stream, true);
+    }
+    a.alive = ctx->vf_alive;
     const int cgrid = (a.B + kCommitWarps - 1) / kCommitWarps;
     for (int j = 0; j < n_win; ++j) {
         a.win_lo = e[j]; a.win_hi = e[j + 1];

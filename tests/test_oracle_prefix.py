@@ -26,15 +26,28 @@ def one_request(draft, targets, k_cap, V=12, cap_extra=80, n0=5, select=1, poiso
     return logits, sd, [m], [select], kw
 
 
+BIG = 1 << 30    # a batch so heavy that every boundary pays: two rows, two rows, then doubling
+EVERY = dict(boundary_bytes=1)   # ... and the same windows for the small cases below
+
+
 def test_windows_by_hand():
-    assert O.prefix_windows(1) == [0, 2]
-    assert O.prefix_windows(2) == [0, 3]
-    assert O.prefix_windows(3) == [0, 2, 4]
-    assert O.prefix_windows(4) == [0, 2, 5]
-    assert O.prefix_windows(8) == [0, 2, 4, 9]
-    assert O.prefix_windows(16) == [0, 2, 4, 8, 17]
-    assert O.prefix_windows(32) == [0, 2, 4, 8, 16, 33]
-    assert O.prefix_windows(64) == [0, 2, 4, 8, 16, 32, 65]
+    assert O.prefix_windows(1, BIG) == [0, 2]
+    assert O.prefix_windows(2, BIG) == [0, 3]
+    assert O.prefix_windows(3, BIG) == [0, 2, 4]
+    assert O.prefix_windows(4, BIG) == [0, 2, 5]
+    assert O.prefix_windows(8, BIG) == [0, 2, 4, 9]
+    assert O.prefix_windows(16, BIG) == [0, 2, 4, 8, 17]
+    assert O.prefix_windows(32, BIG) == [0, 2, 4, 8, 16, 33]
+    assert O.prefix_windows(64, BIG) == [0, 2, 4, 8, 16, 32, 65]
+    # by size (worked by hand from the rule: first window >= 64 MiB, stop when rows left / 2^j < 128 MiB)
+    MiB = 1 << 20
+    assert O.prefix_windows(32, 256 * 151936 * 2) == [0, 2, 4, 8, 16, 33]     # 74.2 MiB per row index: 17 rows left / 16 = 79 MiB
+    assert O.prefix_windows(16, 64 * 128256 * 2) == [0, 5, 17]                # 15.7 MiB: first window 5 rows, 12 left / 2 = 94 MiB
+    assert O.prefix_windows(64, 32 * 128256 * 2) == [0, 9, 18, 65]            # 7.8 MiB: 9 rows, 56 left / 2 = 219, 47 left / 4 = 92
+    assert O.prefix_windows(32, 512 * 128256 * 2) == [0, 2, 4, 8, 16, 33]     # 125 MiB
+    assert O.prefix_windows(8, 4 * 32000 * 4) == [0, 9]                       # 0.5 MiB: one window, the plain verification
+    assert O.prefix_windows(64, 64 * MiB) == [0, 2, 4, 8, 16, 32, 65]         # 49 rows left * 64 / 16 = 196 MiB: on; 33 * 64 / 32 = 66: stop
+    assert O.prefix_windows(64, 1) == [0, 65]
 
 
 def test_hand_worked_fixture_and_rows_read_by_hand():
@@ -47,7 +60,7 @@ def test_hand_worked_fixture_and_rows_read_by_hand():
         draft = [int(x) for x in f[0].split()]; targets = [int(x) for x in f[1].split()]
         a = int(f[2]); z = [int(x) for x in f[3].split()]
         logits, sd, sl, sel, kw = one_request(draft, targets, k_cap=4, V=50)
-        out = O.verify_commit_prefix(logits, O.F32, 50, np.array([0, len(targets)]), 0, sd, sl, sel, **kw)
+        out = O.verify_commit_prefix(logits, O.F32, 50, np.array([0, len(targets)]), 0, sd, sl, sel, **kw, **EVERY)
         assert out.accepted[0] == a and list(out.committed[0, :a + 1]) == z and (out.committed[0, a + 1:] == -1).all(), line
         assert list(kw["hist"][5:5 + a + 1]) == z and kw["hist_len"][0] == 5 + a + 1
         assert kw["state"]["sel_bits"][0] == (0b1011 << 1 | 1) and kw["state"]["acc_ring"][0] == (0x0102 << 8 | a)
@@ -57,16 +70,16 @@ def test_hand_worked_fixture_and_rows_read_by_hand():
     for a, want in by_hand.items():
         targets = draft[:a] + [0] + [9] * (8 - a)            # row a carries 0 (never a draft token)
         logits, sd, sl, sel, kw = one_request(draft, targets, k_cap=8)
-        out = O.verify_commit_prefix(logits, O.F32, 12, np.array([0, 9]), 0, sd, sl, sel, **kw)
+        out = O.verify_commit_prefix(logits, O.F32, 12, np.array([0, 9]), 0, sd, sl, sel, **kw, **EVERY)
         assert out.accepted[0] == a and out.rows_read == want and out.rows_needed == a + 1, (a, out.rows_read)
     # a draft of 3 tokens, all accepted: rows 0..3, windows [0,2) and [2,4): 4 rows; of 2 tokens: 3 rows
     logits, sd, sl, sel, kw = one_request([1, 2, 3], [1, 2, 3, 7], k_cap=8)
-    assert O.verify_commit_prefix(logits, O.F32, 12, np.array([0, 4]), 0, sd, sl, sel, **kw).rows_read == 4
+    assert O.verify_commit_prefix(logits, O.F32, 12, np.array([0, 4]), 0, sd, sl, sel, **kw, **EVERY).rows_read == 4
     logits, sd, sl, sel, kw = one_request([1, 2], [1, 2, 7], k_cap=8)
-    assert O.verify_commit_prefix(logits, O.F32, 12, np.array([0, 3]), 0, sd, sl, sel, **kw).rows_read == 3
+    assert O.verify_commit_prefix(logits, O.F32, 12, np.array([0, 3]), 0, sd, sl, sel, **kw, **EVERY).rows_read == 3
     # an empty draft: one row
     logits, sd, sl, sel, kw = one_request([], [4], k_cap=8)
-    out = O.verify_commit_prefix(logits, O.F32, 12, np.array([0, 1]), 0, sd, sl, sel, **kw)
+    out = O.verify_commit_prefix(logits, O.F32, 12, np.array([0, 1]), 0, sd, sl, sel, **kw, **EVERY)
     assert out.rows_read == 1 and out.accepted[0] == 0 and out.committed[0, 0] == 4
 
 
@@ -75,7 +88,7 @@ def test_no_row_behind_the_stopping_window_is_looked_at(k_cap):
     """Every (draft length m, accepted length a): the rows behind the window in which the walk stops hold NaN,
     and the result is still that of the full verification of the clean logits; the rows looked at stay within
     twice the rows needed plus two."""
-    edges = O.prefix_windows(k_cap)
+    edges = O.prefix_windows(k_cap, 12 * 4, 1)
     rng = np.random.default_rng(k_cap)
     for m in range(0, k_cap + 1):
         for a in sorted(set([0, 1, 2, 3, m // 2, m - 1, m]) & set(range(0, m + 1))):
@@ -85,7 +98,7 @@ def test_no_row_behind_the_stopping_window_is_looked_at(k_cap):
             poison = list(range(min(stop_hi, m + 1), m + 1))
             logits, sd, sl, sel, kw = one_request(draft, targets, k_cap=k_cap, poison=poison)
             clean, sd2, sl2, sel2, kw2 = one_request(draft, targets, k_cap=k_cap)
-            got = O.verify_commit_prefix(logits, O.F32, 12, np.array([0, m + 1]), 0, sd, sl, sel, **kw)
+            got = O.verify_commit_prefix(logits, O.F32, 12, np.array([0, m + 1]), 0, sd, sl, sel, **kw, **EVERY)
             want = O.verify_commit(clean, O.F32, 12, np.array([0, m + 1], np.int64), 0, sd2, sl2, sel2, **kw2)
             assert got.accepted[0] == want.accepted[0] == a
             assert (got.committed == want.committed).all() and got.n_commit[0] == want.n_commit[0]
@@ -124,11 +137,14 @@ def test_equals_the_full_verification_on_random_batches():
         h2, l2, s2 = hist.copy(), n.copy(), state.copy()
         want = O.verify_commit(logits, dtype, V, row_off, 0, sd, sel_len, select, k_cap=k_cap, hist=h1, hist_off=hist_off,
                                hist_cap=cap, hist_len=l1, state=s1)
+        bb = int(rng.choice([1, 1, 40, 64 << 20]))
+        w0 = O.prefix_windows(k_cap, B * V * (4 if dtype == O.F32 else 2), bb)[1]
         got = O.verify_commit_prefix(logits, dtype, V, row_off, 0, sd, sel_len, select, k_cap=k_cap, hist=h2,
-                                     hist_off=hist_off, hist_cap=cap, hist_len=l2, state=s2)
+                                     hist_off=hist_off, hist_cap=cap, hist_len=l2, state=s2,
+                                     boundary_bytes=bb)
         for k in ("accepted", "committed", "n_commit", "status"):
             assert (getattr(got, k) == getattr(want, k)).all(), (it, k)
         assert (h1 == h2).all() and (l1 == l2).all() and (s1 == s2).all(), it
         valid = want.status != O.REQ_BAD_LEN
         assert got.rows_needed == int((want.accepted[valid] + 1).sum())
-        assert got.rows_needed <= got.rows_read <= 2 * got.rows_needed + 2 * int(valid.sum())
+        assert got.rows_needed <= got.rows_read <= 2 * got.rows_needed + w0 * int(valid.sum())   # twice the need plus the first window
