@@ -72,11 +72,12 @@ def parse_args():
                     help="2x256: the paper's predictor shape (two hidden layers of 256 units) instead of the config's")
     ap.add_argument("--batch", type=int, default=0,
                     help="scale the workload to this many requests (profiling a workload's shape at a smaller size)")
-    ap.add_argument("--profile", default=None, choices=["step", "lookup", "cycle"],
+    ap.add_argument("--profile", default=None, choices=["step", "lookup", "cycle", "prefix"],
                     help="profiling run, meant for ncu: W warm-up steps and K steps as plain stream launches on the "
                          "rotating inputs and nothing else (no graphs, no oracle, no end-to-end leg); `lookup`: only the "
                          "fused lookup + scoring kernel, and no logits are allocated; `cycle`: hvd_verify_commit_next "
-                         "(commit fused with the next lookup) in place of the step's three kernels")
+                         "(commit fused with the next lookup) in place of the step's three kernels; `prefix`: the step with "
+                         "hvd_verify_commit_prefix (one streaming launch and one gate per row window)")
     ap.add_argument("--unfused", action="store_true",
                     help="call hvd_lookup and hvd_score_select separately instead of hvd_lookup_score_select")
     return ap.parse_args()
@@ -412,7 +413,7 @@ def run_config(name, args, env, cpu_seconds):
     torch.cuda.synchronize()
     if args.profile:
         for s in range(K_steps):
-            step(W_steps + s, "cycle" if args.profile == "cycle" else "step")
+            step(W_steps + s, {"cycle": "cycle", "prefix": "step_prefix"}.get(args.profile, "step"))
         torch.cuda.synchronize()
         needed = int((sel_len.cpu().numpy().astype(np.int64) + 1).sum())
         ctx.close(); ctx_plain.close()
