@@ -604,8 +604,9 @@ def run_config(name, args, env, cpu_seconds):
         dt = env["max_over_ranks"](dt)
         assert (o_acc.numpy() == accepted_h).all() and (o_nc.numpy() == n_commit_h).all()
         small = B * (8 + 4 * 5 + 16) + (B + 1) * 8 + B * kc * 4
-        # of the logits the call copies the rows verification reads (rows 0..sel_len of every request)
-        logits_h2d = int((o_sl.numpy().astype(np.int64) + 1).sum()) * w.V * w.elt
+        # of the logits the call copies the rows its verification reads: window by window, as hvd_verify_commit_prefix
+        # does (the same rule on the same selection: the rows counted by the kernels above)
+        logits_h2d = prefix_rows * w.V * w.elt
         h2d = int(h_hist.numel() * 4 + logits_h2d + small)
         d2h = int(B * 4 * 7 + B * kc * 4 + B * (kc + 1) * 4 + B * 16)
         e2e = {"value": world * E / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -613,7 +614,8 @@ def run_config(name, args, env, cpu_seconds):
                "api": "hvd_step_host (pinned host buffers)",
                "logits_bytes_on_host": int(h_logits.numel() * h_logits.element_size()),
                "note": "histories, per-request arrays and the logits rows that verification reads cross the bus "
-                       "every step (the rows beyond a request's selected draft are not copied)"}
+                       "every step: rows window by window up to the window of a request's first rejected draft token "
+                       "(hvd_verify_commit_prefix's rule); h2d_bytes_per_step counts those rows"}
         del h_logits, h_hist
 
     # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ----------

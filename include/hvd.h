@@ -452,11 +452,15 @@ HVD_API hvd_status hvd_verify_commit_tree(hvd_ctx* ctx, int32_t B, const void* l
  * for the stream, and appends the committed tokens to the host histories.  Every pointer in the
  * struct is a HOST pointer (pinned memory makes the copies asynchronous and faster; pageable
  * memory works).  Arrays have the shapes documented at the three device entry points.
- * Of the logits only the rows that verification reads (rows 0..sel_len of every valid request)
- * are copied: the call waits for the selection in between, then copies those rows.
+ * Of the logits only rows that verification reads are copied, and verification reads as
+ * hvd_verify_commit_prefix does (there is no target_tok here): the call waits for the selection, then
+ * copies and verifies the needed rows window by window, waiting after every window but the last for the
+ * flags of which requests are still accepted so far; a small call (one window) copies rows 0..sel_len of
+ * every valid request at once.  The logits are the bulk of what crosses the bus, and with accepted
+ * lengths of a few tokens most of them stay on the host.
  * The context keeps a device staging area that it (re)allocates when a call needs more than any
  * earlier one (a synchronous cudaMalloc: not for use inside stream capture).  This entry point
- * synchronises `stream` twice (after the selection, and before returning).
+ * synchronises `stream` after the selection, after every window but the last, and before returning.
  */
 typedef struct {
     int32_t B;

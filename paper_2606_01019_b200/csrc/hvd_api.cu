@@ -374,7 +374,7 @@ static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits
                              int32_t* hist_len, hvd_req_state* state, int32_t* accepted,
                              int32_t* committed, int32_t* n_commit, int32_t* target_tok,
                              int32_t* status, void* stream, const hvd_next_cycle* next = nullptr, bool prefix = false,
-                             unsigned long long* rows_read = nullptr) {
+                             unsigned long long* rows_read = nullptr, VerifyArgs* args_only = nullptr) {
     if (!ctx) return HVD_ERR_INVALID_ARG;
     if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: B outside [1, max_batch]");
     if (dtype != HVD_F32 && dtype != HVD_BF16) return fail(ctx, HVD_ERR_INVALID_ARG, "hvd_verify_commit: unknown dtype");
@@ -403,6 +403,7 @@ static hvd_status verify_commit_impl(hvd_ctx* ctx, int32_t B, const void* logits
     
     a.next_unit = ctx->vf_next_unit; a.dev_error = ctx->dev_error;
     a.row_key = ctx->vf_row_key; a.total_rows = total_rows; a.ext_keys = nullptr;
+    if (args_only) { *args_only = a; return HVD_OK; }
     if (prefix) {
         a.rows_read = rows_read;
         return launch_verify_prefix(ctx, a, dtype, static_cast<cudaStream_t>(stream));
@@ -448,6 +449,20 @@ hvd_status hvd_verify_commit(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dt
                               select, hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit,
                               target_tok, status, stream);
 }
+
+extern "C++" {
+namespace hvd {
+hvd_status make_verify_args(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V, const int64_t* row_off,
+                            int32_t k_uniform, int64_t total_rows, const int32_t* sel_draft, const int32_t* sel_len,
+                            const int32_t* select, int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                            int32_t* hist_len, hvd_req_state* state, int32_t* accepted, int32_t* committed,
+                            int32_t* n_commit, int32_t* status, VerifyArgs* out) {
+    return verify_commit_impl(ctx, B, logits, dtype, V, row_off, k_uniform, total_rows, sel_draft, sel_len, nullptr, select,
+                              hist, hist_off, hist_cap, hist_len, state, accepted, committed, n_commit, nullptr, status,
+                              nullptr, nullptr, false, nullptr, out);
+}
+}  // namespace hvd
+}  // extern "C++"
 
 hvd_status hvd_verify_commit_prefix(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V,
                                     const int64_t* row_off, int32_t k_uniform, int64_t total_rows,

@@ -126,19 +126,22 @@ extern "C" hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args
     // a request: bring the selection back first and copy just those rows (adjacent ranges in one copy).
     D2H(a.sel_len, s.sel_len, B * 4);
     HVD_CUDA_TRY(ctx, cudaStreamSynchronize(st));
-    {
-        const size_t row_bytes = (size_t)a.V * esz;
+    const size_t row_bytes = (size_t)a.V * esz;
+    // rows [lo, hi) of the needed rows of every request that is alive, adjacent ranges in one copy each
+    auto copy_rows = [&](int lo, int hi, const int32_t* alive) -> hvd_status {
         int64_t run0 = 0, run1 = 0;  // pending range of rows
         for (int32_t b = 0; b <= a.B; ++b) {
             int64_t r0 = 0, r1 = 0;
             if (b < a.B) {
-                r0 = a.row_off ? a.row_off[b] : (int64_t)b * (a.k_uniform + 1);
-                const int64_t rend = a.row_off ? a.row_off[b + 1] : r0 + a.k_uniform + 1;
-                const bool ok = a.hist_len[b] >= 0 && a.hist_len[b] <= a.hist_cap[b] && rend > r0 && r0 >= 0 &&
-                                rend <= a.total_rows;
+                const int64_t first = a.row_off ? a.row_off[b] : (int64_t)b * (a.k_uniform + 1);
+                const int64_t rend = a.row_off ? a.row_off[b + 1] : first + a.k_uniform + 1;
+                const bool ok = a.hist_len[b] >= 0 && a.hist_len[b] <= a.hist_cap[b] && rend > first && first >= 0 &&
+                                rend <= a.total_rows && (!alive || alive[b] != 0);
                 int64_t m = a.sel_len[b] < 0 ? 0 : (a.sel_len[b] > kc ? kc : a.sel_len[b]);
-                if (m > rend - r0 - 1) m = rend - r0 - 1;
-                r1 = ok ? r0 + m + 1 : r0;
+                if (m > rend - first - 1) m = rend - first - 1;
+                const int64_t nr = ok ? m + 1 : 0;  // needed rows of the request
+                r0 = first + (lo < nr ? lo : nr);
+                r1 = first + (hi < nr ? hi : nr);
             }
             if (b < a.B && r1 > r0 && r0 == run1 && run1 > run0) { run1 = r1; continue; }  // extends the pending range
             if (run1 > run0)
@@ -146,12 +149,43 @@ extern "C" hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args
                     (size_t)(run1 - run0) * row_bytes);
             run0 = r0; run1 = r1;
         }
-    }
-    r = hvd_verify_commit(ctx, a.B, s.logits, (hvd_dtype)a.dtype, a.V, a.row_off ? s.row_off : nullptr,
-                          a.k_uniform, a.total_rows, s.sel_draft, s.sel_len, s.select, s.hist, s.hist_off,
-                          s.hist_cap, s.hist_len, s.state, s.accepted, s.committed, s.n_commit, nullptr,
-                          s.status, st);
+        return HVD_OK;
+    };
+    // Verification reads the logits window by window, and only of the requests that are still accepted through
+    // the window before (the rule of hvd_verify_commit_prefix): a window's rows are copied just before its
+    // streaming launch, and the flags of who is still alive come back to the host before the next window's
+    // copies.  This entry point has no target_tok, so nothing else would read the rows left out.
+    VerifyArgs va;
+    r = make_verify_args(ctx, a.B, s.logits, (hvd_dtype)a.dtype, a.V, a.row_off ? s.row_off : nullptr, a.k_uniform,
+                         a.total_rows, s.sel_draft, s.sel_len, s.select, s.hist, s.hist_off, s.hist_cap, s.hist_len,
+                         s.state, s.accepted, s.committed, s.n_commit, s.status, &va);
     if (r != HVD_OK) return r;
+    int edges[16];
+    const int n_win = prefix_window_edges(ctx, va, (hvd_dtype)a.dtype, edges);
+    if (n_win > 1) {
+        int32_t* alive = nullptr;  // host copy of the flags: the caller's `accepted` array serves until the results arrive
+        for (int j = 0; j < n_win; ++j) {
+            r = copy_rows(edges[j], edges[j + 1], alive);
+            if (r != HVD_OK) return r;
+            r = launch_prefix_window(ctx, va, (hvd_dtype)a.dtype, edges, j, n_win, st);
+            if (r != HVD_OK) return r;
+            if (j + 1 < n_win) {
+                alive = a.accepted;
+                D2H(alive, ctx->vf_alive, B * 4);
+                HVD_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+            }
+        }
+        r = launch_prefix_commit(ctx, va, st);
+        if (r != HVD_OK) return r;
+    } else {  // a small call: one window, all needed rows at once
+        r = copy_rows(0, 0x7fffffff, nullptr);
+        if (r != HVD_OK) return r;
+        r = hvd_verify_commit(ctx, a.B, s.logits, (hvd_dtype)a.dtype, a.V, a.row_off ? s.row_off : nullptr,
+                              a.k_uniform, a.total_rows, s.sel_draft, s.sel_len, s.select, s.hist, s.hist_off,
+                              s.hist_cap, s.hist_len, s.state, s.accepted, s.committed, s.n_commit, nullptr,
+                              s.status, st);
+        if (r != HVD_OK) return r;
+    }
 
     D2H(a.score, s.score, B * 4);
     D2H(a.select, s.select, B * 4);

@@ -265,6 +265,17 @@ struct VerifyArgs {
 hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit = true);
 // the same result (without target tokens) from the rows up to the first rejected draft token only
 hvd_status launch_verify_prefix(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream);
+// ... and its pieces, for the host-buffer entry point, which copies a window's rows between two launches:
+// the window edges e[0..n] (returns n), window j (streaming launch and gate), the commit
+int prefix_window_edges(const hvd_ctx* ctx, const VerifyArgs& a, hvd_dtype dtype, int* e);
+hvd_status launch_prefix_window(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, const int* e, int j, int n_win, cudaStream_t stream);
+hvd_status launch_prefix_commit(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream);
+// the checked arguments of a verification call (hvd_api.cu), without launching anything
+hvd_status make_verify_args(hvd_ctx* ctx, int32_t B, const void* logits, hvd_dtype dtype, int64_t V, const int64_t* row_off,
+                            int32_t k_uniform, int64_t total_rows, const int32_t* sel_draft, const int32_t* sel_len,
+                            const int32_t* select, int32_t* hist, const int64_t* hist_off, const int32_t* hist_cap,
+                            int32_t* hist_len, hvd_req_state* state, int32_t* accepted, int32_t* committed,
+                            int32_t* n_commit, int32_t* status, VerifyArgs* out);
 // commit and the next cycle's lookup + scoring in one kernel (after launch_verify without its commit)
 bool cycle_fits_one_cta(int32_t n_max);
 hvd_status launch_commit_lookup(hvd_ctx* ctx, const VerifyArgs& va, const int32_t* K, int32_t n_max, int32_t* draft,

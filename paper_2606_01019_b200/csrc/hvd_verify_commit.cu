@@ -675,28 +675,47 @@ static int prefix_edges(int k_cap, int64_t bytes_per_row_index, int64_t boundary
     return n - 1;  // number of windows
 }
 
+int prefix_window_edges(const hvd_ctx* ctx, const VerifyArgs& a, hvd_dtype dtype, int* e) {
+    return prefix_edges(a.k_cap, (int64_t)a.B * a.V * (dtype == HVD_F32 ? 4 : 2), ctx->vf_boundary_bytes, e);
+}
+
+// Window j of n_win: the streaming launch over rows [e[j], e[j+1]) of the requests still alive and, unless it is
+// the last window, the gate that decides who goes on (flags in the context's scratch).
+hvd_status launch_prefix_window(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, const int* e, int j, int n_win, cudaStream_t stream) {
+    a.target_tok = nullptr;
+    a.alive = ctx->vf_alive;
+    a.win_lo = e[j]; a.win_hi = e[j + 1];
+    VerifyArgs s = a;
+    if (j == 0) s.alive = nullptr;  // every request starts alive (the flags are written by the first gate)
+    const hvd_status r = launch_verify(ctx, s, dtype, stream, false);
+    if (r != HVD_OK) return r;
+    if (j + 1 < n_win)
+        HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_commit, prefix_gate_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+                                        kCommitWarps * 32, 0, stream, a));
+    return HVD_OK;
+}
+
+hvd_status launch_prefix_commit(hvd_ctx* ctx, VerifyArgs a, cudaStream_t stream) {
+    a.target_tok = nullptr;
+    a.win_lo = 0; a.win_hi = 0x7fffffff; a.alive = nullptr;
+    HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_commit, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+                                    kCommitWarps * 32, 0, stream, a));
+    return HVD_OK;
+}
+
 hvd_status launch_verify_prefix(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream) {
     int e[16];
-    const int n_win = prefix_edges(a.k_cap, (int64_t)a.B * a.V * (dtype == HVD_F32 ? 4 : 2), ctx->vf_boundary_bytes, e);
+    const int n_win = prefix_window_edges(ctx, a, dtype, e);
     a.target_tok = nullptr;
     if (n_win == 1) {  // the plain verification, whichever streaming kernel it takes; the commit counts the rows
         a.rows_in_commit = true;
         return launch_verify(ctx, a, dtype, stream, true);
     }
-    a.alive = ctx->vf_alive;
-    const int cgrid = (a.B + kCommitWarps - 1) / kCommitWarps;
     for (int j = 0; j < n_win; ++j) {
-        a.win_lo = e[j]; a.win_hi = e[j + 1];
-        const bool last = j + 1 == n_win;
-        VerifyArgs s = a;
-        if (j == 0) s.alive = nullptr;  // every request starts alive (the flags are written by the first gate)
-        const hvd_status r = launch_verify(ctx, s, dtype, stream, false);
+        const hvd_status r = launch_prefix_window(ctx, a, dtype, e, j, n_win, stream);
         if (r != HVD_OK) return r;
-        if (!last) HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_commit, prefix_gate_kernel, cgrid, kCommitWarps * 32, 0, stream, a));
     }
-    a.win_lo = 0; a.win_hi = 0x7fffffff; a.alive = nullptr;
-    HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_commit, verify_commit_kernel, cgrid, kCommitWarps * 32, 0, stream, a));
-    return HVD_OK;
+    return launch_prefix_commit(ctx, a, stream);
 }
 
 hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream_t stream, bool with_commit) {
