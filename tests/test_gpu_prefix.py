@@ -174,6 +174,43 @@ def test_prefix_and_full_calls_share_one_context():
     ctx.close()
 
 
+@pytest.mark.parametrize("B,n", [(24, 3000), (10, 30000), (6, 50000)])
+def test_chain_without_host_synchronisation(B, n):
+    """Six steps enqueued back to back on one stream, each verified by the prefix form (no host synchronisation
+    in between: the lookup of a step may be resident while the windows of the step before are still streaming):
+    final histories, lengths, states and the last step's outputs must equal the oracle's chain."""
+    import torch
+    w = W.CONFIGS["C2"].scaled(B=B, n=n, V=5003)
+    inp = P.prepare(w, device="cuda")
+    S = 6
+    rq_o = inp.rq.copy()
+    logits_dev, outs = [], []
+    for s in range(S):
+        lk = P.lookup(w, rq_o, 8)
+        sc = P.score_select(w, rq_o, lk, inp.W1, inp.b1, inp.W2, inp.b2, inp.tau, 8, inp.Wh, inp.bh)
+        lg = W.make_logits(w, int(rq_o.row_off[-1]), device="cuda", salt=300 + s)
+        W.plant_agreement(w, lg, rq_o.row_off, sc.sel_draft, sc.sel_len, W.make_agreement(w, sc.sel_len), salt=300 + s)
+        vf = P.verify_commit(w, rq_o, sc, W.logits_to_numpy(lg), 8)
+        logits_dev.append(lg)
+        outs.append((lk, sc, vf))
+    rq_g = inp.rq.copy()
+    ctx = G.make_ctx(w, rq_g)
+    G.set_predictor(ctx, inp)
+    batch = G.make_batch(ctx, w, rq_g)
+    rows = torch.zeros(1, dtype=torch.int64, device="cuda")
+    torch.cuda.synchronize()
+    for s in range(S):
+        batch.lookup_score_select()
+        batch.verify_commit_prefix(logits_dev[s], rows)
+    g = batch.download()
+    lk, sc, vf = outs[-1]
+    G.compare_lookup(g, lk)
+    assert G.compare_score(g, sc, inp.tau).all()
+    compare(g, vf, rq_o)
+    assert ctx.hvd_device_status() == 0 and int(rows.item()) > 0
+    ctx.close()
+
+
 def test_random_batches():
     from tests.test_gpu_random_sweep import draw_case
     for it in range(60):
