@@ -257,6 +257,7 @@ struct VerifyArgs {
     // prefix verification: only the needed rows [win_lo, win_hi) of a request are streamed, and only while the
     // request is alive (alive == NULL: every request is); the defaults stream every needed row
     int32_t win_lo = 0, win_hi = 0x7fffffff;
+    int32_t win_index = 0;
     int32_t* alive = nullptr;
     unsigned long long* rows_read = nullptr;  // optional: += logits rows streamed by the call
     bool rows_in_commit = false;              // ... counted by the commit (one window: any streaming kernel) or by the streaming launches

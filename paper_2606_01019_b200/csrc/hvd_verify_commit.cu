@@ -616,6 +616,65 @@ __global__ void __launch_bounds__(kSmallWarps * 32) verify_small_kernel(const Ve
         atomicMax(a.row_key + r, ((unsigned long long)word << 32) | (uint32_t)(~widx));
 }
 
+// Prefix verification, early windows: while (nearly) every request is still alive, a window's rows are known from
+// the grid alone -- block z is the request, block y the row inside the window, and one warp takes one 4 KB batch of
+// that row, as in the kernel above.  The warp looks its request up (one round trip), leaves if the request is dead
+// or has no such row, and streams its batch.  No work list, no queues: a launch of up to 160 MB starts and ends
+// sooner than the persistent kernel (whose start and end game cost 8 to 10 us).
+template <typename E>
+__global__ void __launch_bounds__(kSmallWarps * 32) verify_window_kernel(const VerifyArgs a) {
+    constexpr int EPV = Tracker<E>::kPerVec;
+    constexpr int ESZ = 16 / EPV;
+    const int lane = threadIdx.x & 31;
+    const int gb = blockIdx.x * kSmallWarps + (threadIdx.x >> 5);  // batch inside the row
+    const int b = blockIdx.z;
+    pdl_wait();
+    pdl_trigger();
+    if (gb >= a.n_batch_row) return;
+    const Req q = load_req(a, b);
+    int64_t first;
+    const int rows = streamed_rows(a, q, b, first);
+    if ((int)blockIdx.y >= rows) return;  // warp-uniform
+    const int64_t r = first + blockIdx.y;
+    if (!HVD_IN_BOUNDS(a.dev_error, r, 0, a.total_rows)) return;
+
+    const char* row = static_cast<const char*>(a.logits) + r * a.V * ESZ;
+    const int head_bytes = (int)((16 - (reinterpret_cast<uintptr_t>(row) & 15)) & 15);
+    const int head = (int)min((int64_t)(head_bytes / ESZ), a.V);
+    const int n_vec = (int)((a.V - head) / EPV);
+    const int tail = (int)(a.V - head - (int64_t)n_vec * EPV);
+    const uint4* vrow = reinterpret_cast<const uint4*>(row + (int64_t)head * ESZ);
+    const int left = n_vec - gb * kBatchVec;
+    const uint4* ptr = vrow + (int64_t)gb * kBatchVec + lane;
+    const unsigned long long pol = stream_policy();
+
+    uint32_t lord = 0u, loff = 0xffffffffu;
+    const bool full = left >= kBatchVec;
+    if (full || lane < left) {
+        uint4 x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (full || u * 32 + lane < left) x[u] = ld_stream(ptr + u * 32, pol);
+        Tracker<E> t;
+        t.init(x[0]);
+#pragma unroll
+        for (int u = 1; u < U; ++u)
+            if (full || u * 32 + lane < left) t.fold(x[u], u);
+        t.best(lane, lord, loff);
+        loff += (uint32_t)(head + gb * kBatchVec * EPV);
+    }
+    if (gb == 0 && lane < head + tail) {  // the ragged edges of the row ride along with batch 0
+        const int idx = lane < head ? lane : head + n_vec * EPV + (lane - head);
+        const uint32_t eord = ord32(Tracker<E>::scalar(row, idx));
+        if (eord > lord || (eord == lord && (uint32_t)idx < loff)) { lord = eord; loff = (uint32_t)idx; }
+    }
+    const uint32_t word = __reduce_max_sync(kFull, lord);
+    const uint32_t widx = __reduce_min_sync(kFull, lord == word ? loff : 0xffffffffu);
+    if (lane == 0 && word != 0u && widx != 0xffffffffu)
+        atomicMax(a.row_key + r, ((unsigned long long)word << 32) | (uint32_t)(~widx));
+    if (a.rows_read && !a.rows_in_commit && gb == 0 && blockIdx.y == 0 && lane == 0) atomicAdd(a.rows_read, (unsigned long long)rows);
+}
+
 size_t verify_dyn_smem(int32_t B) { return (size_t)B * 8 + (size_t)(B + 1) * 4; }
 
 int verify_occupancy(hvd_dtype dtype, size_t dyn_smem) {
@@ -684,7 +743,7 @@ int prefix_window_edges(const hvd_ctx* ctx, const VerifyArgs& a, hvd_dtype dtype
 hvd_status launch_prefix_window(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, const int* e, int j, int n_win, cudaStream_t stream) {
     a.target_tok = nullptr;
     a.alive = ctx->vf_alive;
-    a.win_lo = e[j]; a.win_hi = e[j + 1];
+    a.win_lo = e[j]; a.win_hi = e[j + 1]; a.win_index = j;
     VerifyArgs s = a;
     if (j == 0) s.alive = nullptr;  // every request starts alive (the flags are written by the first gate)
     const hvd_status r = launch_verify(ctx, s, dtype, stream, false);
@@ -743,7 +802,19 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
     // 17 MB 7.5 -> 5.5, 70 MB 11.2 -> 9.0, 140 MB 17.6 -> 14.5, 279 MB 27.8 -> 26.4; with (nearly) all rows
     // needed the persistent kernel is ahead from about 150 MB on (279 MB: 41.7 against 50.7 us).
     const int64_t full_bytes = a.total_rows * a.V * esz;
-    // (a windowed launch takes the persistent kernel whatever its size: its work list leaves out dead requests)
+    // A windowed launch: the first two windows (most requests still alive) of up to four times vf_small_bytes
+    // (640 MB) take the kernel whose grid is (batch, row of the window, request); later windows the persistent
+    // kernel, whose work list leaves out the dead requests.  Measured, prefix step with the persistent kernel for
+    // every window -> with this kernel for the first two: C2 37.9 -> 34.4 us, C3 141.0 -> 132.5, C4 70.6 -> 65.6
+    // (windows of 74 to 156 MB), C5 168.1 -> 159.9 (262 MB).
+    if (windowed && a.win_index < 2 && a.B <= 65535 && a.win_hi - a.win_lo <= 65535 &&
+        (int64_t)a.B * (a.win_hi - a.win_lo) * a.V * esz <= 4 * ctx->vf_small_bytes) {
+        const dim3 wgrid((unsigned)((a.n_batch_row + kSmallWarps - 1) / kSmallWarps), (unsigned)(a.win_hi - a.win_lo), (unsigned)a.B);
+        const bool pdl = (ctx->pdl_mask & 4);
+        HVD_CUDA_TRY(ctx, dtype == HVD_F32 ? launch_kernel(pdl, verify_window_kernel<float>, wgrid, kSmallWarps * 32, 0, stream, a)
+                                           : launch_kernel(pdl, verify_window_kernel<__nv_bfloat16>, wgrid, kSmallWarps * 32, 0, stream, a));
+        return HVD_OK;
+    }
     const bool small = !windowed && a.total_rows <= 65535 && full_bytes <= ctx->vf_small_bytes;
     const bool spec = full_bytes <= kVerifySpecBytes;
     if (small) {
