@@ -616,6 +616,8 @@ __global__ void __launch_bounds__(kSmallWarps * 32) verify_small_kernel(const Ve
         atomicMax(a.row_key + r, ((unsigned long long)word << 32) | (uint32_t)(~widx));
 }
 
+namespace {
+
 // Prefix verification, early windows: while (nearly) every request is still alive, a window's rows are known from
 // the grid alone -- block z is the request, block y the row inside the window, and one warp takes one 4 KB batch of
 // that row, as in the kernel above.  The warp looks its request up (one round trip), leaves if the request is dead
@@ -674,6 +676,8 @@ __global__ void __launch_bounds__(kSmallWarps * 32) verify_window_kernel(const V
         atomicMax(a.row_key + r, ((unsigned long long)word << 32) | (uint32_t)(~widx));
     if (a.rows_read && !a.rows_in_commit && gb == 0 && blockIdx.y == 0 && lane == 0) atomicAdd(a.rows_read, (unsigned long long)rows);
 }
+
+}  // namespace
 
 size_t verify_dyn_smem(int32_t B) { return (size_t)B * 8 + (size_t)(B + 1) * 4; }
 
