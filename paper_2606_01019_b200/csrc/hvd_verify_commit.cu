@@ -805,22 +805,42 @@ hvd_status launch_verify(hvd_ctx* ctx, VerifyArgs a, hvd_dtype dtype, cudaStream
     // about half the rows needed, bf16 rows of 128 256 (persistent kernel -> warp per batch): 4.4 MB 6.3 -> 3.8 us,
     // 17 MB 7.5 -> 5.5, 70 MB 11.2 -> 9.0, 140 MB 17.6 -> 14.5, 279 MB 27.8 -> 26.4; with (nearly) all rows
     // needed the persistent kernel is ahead from about 150 MB on (279 MB: 41.7 against 50.7 us).
+    // Between vf_small_bytes and four times that (160 to 640 MB), when the row blocks are of about equal height, a
+    // grid of (batch, row of the block, request) is hardly larger than the logits, and the kernel with that grid (a
+    // warp knows its request and row from its block numbers, looks the request up and streams its batch: no work
+    // list, no queues) starts and ends sooner than the persistent kernel.  Measured, step in us, persistent ->
+    // grid: 209 MB 38.0 -> 35.8, 257 MB (C2) 46.4 -> 45.3, 397 MB 66.5 -> 63.9, 428 MB with a fifth of the rows not
+    // needed (C4) 70.9 -> 71.1, 515 MB 81.8 -> 81.6; below 160 MB it equals the warp-per-batch kernels (17 MB 11.7 ->
+    // 11.6, 70 MB 19.5 -> 19.1, 140 MB 27.5 -> 27.5), at 2.1 GB the persistent kernel is 6 us ahead, and on ragged
+    // blocks the grid wastes its CTAs (C5: 345 against 321 us for the verify call).
+    // Prefix verification: the first two windows (most requests still alive) of up to 640 MB take the grid kernel
+    // over the window's rows; later windows the persistent kernel, whose work list leaves out the dead requests.
+    // Measured, prefix step with the persistent kernel for every window -> with the grid kernel for the first two:
+    // C2 37.9 -> 34.4 us, C3 141.0 -> 132.5, C4 70.6 -> 65.6 (windows of 74 to 156 MB), C5 168.1 -> 159.9 (262 MB).
     const int64_t full_bytes = a.total_rows * a.V * esz;
-    // A windowed launch: the first two windows (most requests still alive) of up to four times vf_small_bytes
-    // (640 MB) take the kernel whose grid is (batch, row of the window, request); later windows the persistent
-    // kernel, whose work list leaves out the dead requests.  Measured, prefix step with the persistent kernel for
-    // every window -> with this kernel for the first two: C2 37.9 -> 34.4 us, C3 141.0 -> 132.5, C4 70.6 -> 65.6
-    // (windows of 74 to 156 MB), C5 168.1 -> 159.9 (262 MB).
-    if (windowed && a.win_index < 2 && a.B <= 65535 && a.win_hi - a.win_lo <= 65535 &&
+    const bool spec = full_bytes <= kVerifySpecBytes;
+    bool by_grid = false;
+    if (windowed) {
+        by_grid = a.win_index < 2;
+    } else if (!spec) {
+        const int64_t block_rows = (a.row_off ? a.k_cap : a.k_uniform) + 1;  // rows of the tallest block
+        by_grid = (int64_t)a.B * block_rows * 4 <= a.total_rows * 5 &&      // grid rows <= 1.25 x the rows there are
+                  (int64_t)a.B * block_rows * a.V * esz > ctx->vf_small_bytes;
+        if (by_grid) { a.win_lo = 0; a.win_hi = (int32_t)block_rows; a.win_index = 0; a.alive = nullptr; }
+    }
+    if (by_grid && a.B <= 65535 && a.win_hi - a.win_lo <= 65535 &&
         (int64_t)a.B * (a.win_hi - a.win_lo) * a.V * esz <= 4 * ctx->vf_small_bytes) {
         const dim3 wgrid((unsigned)((a.n_batch_row + kSmallWarps - 1) / kSmallWarps), (unsigned)(a.win_hi - a.win_lo), (unsigned)a.B);
         const bool pdl = (ctx->pdl_mask & 4);
         HVD_CUDA_TRY(ctx, dtype == HVD_F32 ? launch_kernel(pdl, verify_window_kernel<float>, wgrid, kSmallWarps * 32, 0, stream, a)
                                            : launch_kernel(pdl, verify_window_kernel<__nv_bfloat16>, wgrid, kSmallWarps * 32, 0, stream, a));
+        if (with_commit)
+            HVD_CUDA_TRY(ctx, launch_kernel(ctx->pdl_commit, verify_commit_kernel, (a.B + kCommitWarps - 1) / kCommitWarps,
+                                            kCommitWarps * 32, 0, stream, a));
         return HVD_OK;
     }
+    if (!windowed) { a.win_lo = 0; a.win_hi = 0x7fffffff; }
     const bool small = !windowed && a.total_rows <= 65535 && full_bytes <= ctx->vf_small_bytes;
-    const bool spec = full_bytes <= kVerifySpecBytes;
     if (small) {
         const dim3 sgrid((unsigned)((a.n_batch_row + kSmallWarps - 1) / kSmallWarps), (unsigned)a.total_rows);
         const bool pdl = (ctx->pdl_mask & 4);

@@ -59,10 +59,14 @@ def test_noalloc_matches_context_entry_point_bf16_ragged():
     run_both(W.CONFIGS["C5"].scaled(B=40, n=(64, 3000), V=32003))
 
 
-def test_noalloc_with_the_persistent_streaming_kernel():
-    """More than 160 MB of logits (816 rows of 128 256 bf16: 209 MB): the persistent kernel, its unit counters and
-    their reset run on the static array too."""
+def test_noalloc_beyond_160_mb_of_logits():
+    """More than 160 MB of logits.  Row blocks of equal height (816 rows of 128 256 bf16: 209 MB): the kernel whose
+    grid is (batch, row of the block, request).  Ragged row blocks (48 requests with 5 to 33 rows, about 230 MB):
+    the persistent kernel, whose unit counters and their reset then run on the static array too."""
     run_both(W.CONFIGS["C2"].scaled(B=48, n=1024))
+    w = W.CONFIGS["C5"].scaled(B=48, n=(64, 3000))
+    assert int(W.make_requests(w).row_off[-1]) * w.V * w.elt > 160 * 2**20
+    run_both(w)
 
 
 def test_noalloc_rejects_sizes_beyond_the_static_array():
