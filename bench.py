@@ -44,10 +44,10 @@ UNTIMED_REPLAYS = 3
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the kernel on the workload, from the ncu captures
 # summarised under profiles/ (per launch, like the algorithmic bytes; absent = not captured)
 NCU_VERIFY_TRAFFIC_BYTES = {
-    "C2": (261772928, "profiles/verify_stream_kernel_c2_ncu.txt"),
-    "C3": (2129576753, "profiles/verify_stream_kernel_c3_batch64_ncu.txt: captured at batch 64 (1.0060 x the algorithmic "
+    "C2": (260997504, "profiles/verify_window_kernel_c2_ncu.txt"),
+    "C3": (2130413885, "profiles/verify_stream_kernel_c3_batch64_ncu.txt: captured at batch 64 (1.0064 x the algorithmic "
                        "bytes), scaled to the full launch by the needed rows"),
-    "C4": (431484000, "profiles/verify_stream_kernel_c4_ncu.txt"),
+    "C4": (431483136, "profiles/verify_window_kernel_c4_ncu.txt"),
 }
 NCU_LOOKUP_TRAFFIC_BYTES = {
     "C2": (4242688, "profiles/lookup_kernel_c2_ncu.txt"),
@@ -523,8 +523,15 @@ def run_config(name, args, env, cpu_seconds):
     v_iso, v_b2b = gbs(verify_bytes, kt["verify_commit_us_isolated"]), gbs(verify_bytes, kt["verify_commit_us_back_to_back"])
     probe_bytes = logits0.numel() * logits0.element_size()
     probe_gbs = gbs(probe_bytes, kt["read_probe_us"])
-    roofline = {"bound": "hbm", "kernel": "verify_stream_kernel (+ verify_commit_kernel)" if logits_bytes_alloc > 160 * 2**20
-                else "verify_small_kernel (+ verify_commit_kernel)",
+    # which streaming kernel hvd_verify_commit takes for this call (the rule of launch_verify in csrc/hvd_verify_commit.cu)
+    grid_bytes = B * (kc + 1) * w.V * w.elt
+    if 160 * 2**20 < grid_bytes <= 640 * 2**20 and B * (kc + 1) * 4 <= total_rows * 5:
+        stream_kernel = "verify_window_kernel"
+    elif logits_bytes_alloc > 160 * 2**20:
+        stream_kernel = "verify_stream_kernel"
+    else:
+        stream_kernel = "verify_small_kernel"
+    roofline = {"bound": "hbm", "kernel": stream_kernel + " (+ verify_commit_kernel)",
                 "achieved": v_iso, "peak": peak_gbs, "unit": "GB/s", "frac": v_iso / peak_gbs,
                 "traffic": NCU_VERIFY_TRAFFIC_BYTES.get(w.name, (None, None))[0] if not args.batch else None,
                 "traffic_source": NCU_VERIFY_TRAFFIC_BYTES.get(w.name, (None, "not captured"))[1], "peak_kind": peak_kind,
