@@ -452,15 +452,16 @@ HVD_API hvd_status hvd_verify_commit_tree(hvd_ctx* ctx, int32_t B, const void* l
  * for the stream, and appends the committed tokens to the host histories.  Every pointer in the
  * struct is a HOST pointer (pinned memory makes the copies asynchronous and faster; pageable
  * memory works).  Arrays have the shapes documented at the three device entry points.
- * Of the logits only rows that verification reads are copied, and verification reads as
- * hvd_verify_commit_prefix does (there is no target_tok here): the call waits for the selection, then
- * copies and verifies the needed rows window by window, waiting after every window but the last for the
- * flags of which requests are still accepted so far; a small call (one window) copies rows 0..sel_len of
- * every valid request at once.  The logits are the bulk of what crosses the bus, and with accepted
- * lengths of a few tokens most of them stay on the host.
+ * Of the logits only rows that verification reads cross the bus, and verification reads as
+ * hvd_verify_commit_prefix does (there is no target_tok here): with accepted lengths of a few tokens most
+ * of the logits stay on the host.  Logits in page-locked memory (cudaHostAlloc, cudaHostRegister, a pinned
+ * tensor) are read in place: the streaming kernels load the rows they need straight from the host buffer,
+ * nothing is staged, and the call waits for the stream once, before it returns.  Pageable logits are staged:
+ * the call waits for the selection, then copies and verifies the needed rows window by window, waiting after
+ * every window but the last for the flags of which requests are still accepted so far (a small call, one
+ * window, copies rows 0..sel_len of every valid request at once).
  * The context keeps a device staging area that it (re)allocates when a call needs more than any
- * earlier one (a synchronous cudaMalloc: not for use inside stream capture).  This entry point
- * synchronises `stream` after the selection, after every window but the last, and before returning.
+ * earlier one (a synchronous cudaMalloc: not for use inside stream capture).
  */
 typedef struct {
     int32_t B;

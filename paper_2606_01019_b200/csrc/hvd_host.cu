@@ -122,70 +122,85 @@ extern "C" hvd_status hvd_step_host(hvd_ctx* ctx, const hvd_host_step_args* args
                          s.sel_len, st);
     if (r != HVD_OK) return r;
 
-    // The logits are the bulk of the bytes that cross the bus, and verification reads only rows 0..sel_len of
-    // a request: bring the selection back first and copy just those rows (adjacent ranges in one copy).
+    // The logits are the bulk of the bytes that cross the bus, and verification reads as hvd_verify_commit_prefix
+    // does (this entry point has no target_tok): only rows up to the window of a request's first rejected draft
+    // token.
     D2H(a.sel_len, s.sel_len, B * 4);
-    HVD_CUDA_TRY(ctx, cudaStreamSynchronize(st));
-    const size_t row_bytes = (size_t)a.V * esz;
-    // rows [lo, hi) of the needed rows of every request that is alive, adjacent ranges in one copy each
-    auto copy_rows = [&](int lo, int hi, const int32_t* alive) -> hvd_status {
-        int64_t run0 = 0, run1 = 0;  // pending range of rows
-        for (int32_t b = 0; b <= a.B; ++b) {
-            int64_t r0 = 0, r1 = 0;
-            if (b < a.B) {
-                const int64_t first = a.row_off ? a.row_off[b] : (int64_t)b * (a.k_uniform + 1);
-                const int64_t rend = a.row_off ? a.row_off[b + 1] : first + a.k_uniform + 1;
-                const bool ok = a.hist_len[b] >= 0 && a.hist_len[b] <= a.hist_cap[b] && rend > first && first >= 0 &&
-                                rend <= a.total_rows && (!alive || alive[b] != 0);
-                int64_t m = a.sel_len[b] < 0 ? 0 : (a.sel_len[b] > kc ? kc : a.sel_len[b]);
-                if (m > rend - first - 1) m = rend - first - 1;
-                const int64_t nr = ok ? m + 1 : 0;  // needed rows of the request
-                r0 = first + (lo < nr ? lo : nr);
-                r1 = first + (hi < nr ? hi : nr);
-            }
-            if (b < a.B && r1 > r0 && r0 == run1 && run1 > run0) { run1 = r1; continue; }  // extends the pending range
-            if (run1 > run0)
-                H2D(s.logits + (size_t)run0 * row_bytes, static_cast<const char*>(a.logits) + (size_t)run0 * row_bytes,
-                    (size_t)(run1 - run0) * row_bytes);
-            run0 = r0; run1 = r1;
-        }
-        return HVD_OK;
+    const hvd_dtype dtype = (hvd_dtype)a.dtype;
+    auto verify_args = [&](const void* logits, VerifyArgs* va) {
+        return make_verify_args(ctx, a.B, logits, dtype, a.V, a.row_off ? s.row_off : nullptr, a.k_uniform, a.total_rows,
+                                s.sel_draft, s.sel_len, s.select, s.hist, s.hist_off, s.hist_cap, s.hist_len, s.state,
+                                s.accepted, s.committed, s.n_commit, s.status, va);
     };
-    // Verification reads the logits window by window, and only of the requests that are still accepted through
-    // the window before (the rule of hvd_verify_commit_prefix): a window's rows are copied just before its
-    // streaming launch, and the flags of who is still alive come back to the host before the next window's
-    // copies.  This entry point has no target_tok, so nothing else would read the rows left out.
-    VerifyArgs va;
-    r = make_verify_args(ctx, a.B, s.logits, (hvd_dtype)a.dtype, a.V, a.row_off ? s.row_off : nullptr, a.k_uniform,
-                         a.total_rows, s.sel_draft, s.sel_len, s.select, s.hist, s.hist_off, s.hist_cap, s.hist_len,
-                         s.state, s.accepted, s.committed, s.n_commit, s.status, &va);
-    if (r != HVD_OK) return r;
-    int edges[16];
-    const int n_win = prefix_window_edges(ctx, va, (hvd_dtype)a.dtype, edges);
-    if (n_win > 1) {
+
+    // Logits in page-locked host memory (cudaHostAlloc, cudaHostRegister, a pinned tensor) are read where they
+    // lie: the streaming kernels load every needed row once, straight over the bus; nothing is staged and the
+    // host waits for nothing in between.
+    auto verify_in_place = [&](const void* device_view) -> hvd_status {
+        VerifyArgs va;
+        const hvd_status e = verify_args(device_view, &va);
+        return e != HVD_OK ? e : launch_verify_prefix(ctx, va, dtype, st);
+    };
+
+    // Pageable logits: the selection comes back first, then the needed rows are copied and verified window by
+    // window (adjacent ranges in one copy each); the flags of who is still alive come back to the host after
+    // every window but the last and decide the next window's copies.
+    auto verify_staged = [&]() -> hvd_status {
+        HVD_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+        const size_t row_bytes = (size_t)a.V * esz;
+        auto copy_rows = [&](int lo, int hi, const int32_t* alive) -> hvd_status {  // rows [lo, hi) of the needed rows
+            int64_t run0 = 0, run1 = 0;  // pending range of rows
+            for (int32_t b = 0; b <= a.B; ++b) {
+                int64_t r0 = 0, r1 = 0;
+                if (b < a.B) {
+                    const int64_t first = a.row_off ? a.row_off[b] : (int64_t)b * (a.k_uniform + 1);
+                    const int64_t rend = a.row_off ? a.row_off[b + 1] : first + a.k_uniform + 1;
+                    const bool ok = a.hist_len[b] >= 0 && a.hist_len[b] <= a.hist_cap[b] && rend > first && first >= 0 &&
+                                    rend <= a.total_rows && (!alive || alive[b] != 0);
+                    int64_t m = a.sel_len[b] < 0 ? 0 : (a.sel_len[b] > kc ? kc : a.sel_len[b]);
+                    if (m > rend - first - 1) m = rend - first - 1;
+                    const int64_t nr = ok ? m + 1 : 0;  // needed rows of the request
+                    r0 = first + (lo < nr ? lo : nr);
+                    r1 = first + (hi < nr ? hi : nr);
+                }
+                if (b < a.B && r1 > r0 && r0 == run1 && run1 > run0) { run1 = r1; continue; }  // extends the pending range
+                if (run1 > run0)
+                    H2D(s.logits + (size_t)run0 * row_bytes, static_cast<const char*>(a.logits) + (size_t)run0 * row_bytes,
+                        (size_t)(run1 - run0) * row_bytes);
+                run0 = r0; run1 = r1;
+            }
+            return HVD_OK;
+        };
+        VerifyArgs va;
+        hvd_status e = verify_args(s.logits, &va);
+        if (e != HVD_OK) return e;
+        int edges[16];
+        const int n_win = prefix_window_edges(ctx, va, dtype, edges);
+        if (n_win == 1) {  // a small call: all needed rows at once
+            e = copy_rows(0, 0x7fffffff, nullptr);
+            return e != HVD_OK ? e : launch_verify_prefix(ctx, va, dtype, st);
+        }
         int32_t* alive = nullptr;  // host copy of the flags: the caller's `accepted` array serves until the results arrive
         for (int j = 0; j < n_win; ++j) {
-            r = copy_rows(edges[j], edges[j + 1], alive);
-            if (r != HVD_OK) return r;
-            r = launch_prefix_window(ctx, va, (hvd_dtype)a.dtype, edges, j, n_win, st);
-            if (r != HVD_OK) return r;
+            e = copy_rows(edges[j], edges[j + 1], alive);
+            if (e != HVD_OK) return e;
+            e = launch_prefix_window(ctx, va, dtype, edges, j, n_win, st);
+            if (e != HVD_OK) return e;
             if (j + 1 < n_win) {
                 alive = a.accepted;
                 D2H(alive, ctx->vf_alive, B * 4);
                 HVD_CUDA_TRY(ctx, cudaStreamSynchronize(st));
             }
         }
-        r = launch_prefix_commit(ctx, va, st);
-        if (r != HVD_OK) return r;
-    } else {  // a small call: one window, all needed rows at once
-        r = copy_rows(0, 0x7fffffff, nullptr);
-        if (r != HVD_OK) return r;
-        r = hvd_verify_commit(ctx, a.B, s.logits, (hvd_dtype)a.dtype, a.V, a.row_off ? s.row_off : nullptr,
-                              a.k_uniform, a.total_rows, s.sel_draft, s.sel_len, s.select, s.hist, s.hist_off,
-                              s.hist_cap, s.hist_len, s.state, s.accepted, s.committed, s.n_commit, nullptr,
-                              s.status, st);
-        if (r != HVD_OK) return r;
-    }
+        return launch_prefix_commit(ctx, va, st);
+    };
+
+    cudaPointerAttributes at;
+    const bool page_locked = cudaPointerGetAttributes(&at, a.logits) == cudaSuccess && at.type == cudaMemoryTypeHost &&
+                             at.devicePointer != nullptr;
+    if (!page_locked) (void)cudaGetLastError();
+    r = page_locked ? verify_in_place(at.devicePointer) : verify_staged();
+    if (r != HVD_OK) return r;
 
     D2H(a.score, s.score, B * 4);
     D2H(a.select, s.select, B * 4);

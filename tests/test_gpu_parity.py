@@ -101,12 +101,14 @@ def test_multi_step_loop_and_scratch_reuse():
         ctx.close()
 
 
+@pytest.mark.parametrize("pinned", [False, True])
 @pytest.mark.parametrize("boundary", [None, "1"])
-def test_host_buffer_entry_point(boundary, monkeypatch):
+def test_host_buffer_entry_point(boundary, pinned, monkeypatch):
     """hvd_step_host: same step with host arrays in and out (copies inside the call).  The logits are copied and
     verified window by window; small inputs have one window, so every case runs once more with a window boundary
     worth one byte (rows [0,2), [2,4), [4,9) for the draft cap of 8).  The second call gets other logits: a row
-    that this call leaves on the host must not be read from what an earlier call left in the staging area."""
+    that this call leaves on the host must not be read from what an earlier call left in the staging area.
+    Pageable logits are staged window by window; page-locked ones are read in place by the streaming kernels."""
     if boundary is not None:
         monkeypatch.setenv("HVD_PREFIX_BOUNDARY_BYTES", boundary)
     import paper_2606_01019_b200 as H
@@ -131,10 +133,14 @@ def test_host_buffer_entry_point(boundary, monkeypatch):
                  status=np.zeros(B, np.int32))
         for rep in range(2):       # second call: staging area reused, histories have grown
             lg_np = inp.logits_np if rep == 0 else np.ascontiguousarray(np.roll(inp.logits_np.reshape(-1, w.V), 1, axis=1))
+            lg_host = lg_np
+            if pinned:
+                import torch
+                lg_host = torch.from_numpy(lg_np.view(np.int16) if lg_np.dtype == np.uint16 else lg_np).pin_memory()
             ctx.hvd_step_host(B=B, n_max=int(rq_g.hist_cap.max()), hist=rq_g.hist, hist_off=rq_g.hist_off,
                               hist_cap=rq_g.hist_cap, hist_len=rq_g.hist_len, K=rq_g.K, prompt_len=rq_g.prompt_len,
                               state=rq_g.state, model_draft=rq_g.model_draft, model_len=rq_g.model_len,
-                              logits=lg_np, dtype=H.F32 if w.dtype == "f32" else H.BF16, V=w.V,
+                              logits=lg_host, dtype=H.F32 if w.dtype == "f32" else H.BF16, V=w.V,
                               row_off=None if uniform else rq_g.row_off, k_uniform=w.k_cap if uniform else 0,
                               total_rows=int(rq_g.row_off[-1]), **o)
             out = P.step(inp, rq_o, logits_np=lg_np)
