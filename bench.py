@@ -622,7 +622,8 @@ def run_config(name, args, env, cpu_seconds):
                "logits_bytes_on_host": int(h_logits.numel() * h_logits.element_size()),
                "note": "histories, per-request arrays and the logits rows that verification reads cross the bus "
                        "every step: rows window by window up to the window of a request's first rejected draft token "
-                       "(hvd_verify_commit_prefix's rule); h2d_bytes_per_step counts those rows"}
+                       "(hvd_verify_commit_prefix's rule), read in place from the pinned host buffer by the streaming "
+                       "kernels; h2d_bytes_per_step counts those rows"}
         del h_logits, h_hist
 
     # ---- CPU baseline: the oracle, as it stands, on this machine's host cores (rank 0, N = 1) ----------
